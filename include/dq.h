@@ -1,0 +1,162 @@
+/*
+ * dq.h -- C ABI of the D-Quant hot path for NVIDIA B200 (sm_100a).
+ *
+ * D-Quant ("D-Quant: Driftable Entropy Coding for KV Cache Quantization") stores the
+ * keys and values of every token in fixed-size, rANS-coded containers and decodes
+ * them inside the decode-step attention kernel.  This library holds that path:
+ *
+ *   dq_build_tables      normal-derived rANS tables             (Sec. 3.1, 4.2, 4.4)
+ *   dq_encode_tokens     K/V bf16 -> containers + window means  (Fig. 1, Algorithm 1)
+ *   dq_decode_attention  q, containers -> attention output      (Algorithm 2, App. A)
+ *   dq_decode_tokens     containers -> symbols / dequantised values (Algorithm 2; checks)
+ *   dq_bf16_decode_attention  plain bf16-cache decode attention (comparison baseline)
+ *
+ * Conventions
+ *   - A *stream* is the 128 values of one (token, KV head).  Its *record* is
+ *     rec_bytes = floor(bits_per_elem * 128 / 8) bytes:
+ *       [0:2) s fp16 LE | [2:4) o fp16 LE | [4:8) final rANS state u32 LE |
+ *       [8:8+k) renormalisation bytes in decode order | zero padding.
+ *     The container of Eq. (budget) is C = rec_bytes - 4 bytes, sigma = 32,
+ *     B = 8C - 32 bits; rANS precision p = 8, state in [2^23, 2^31), byte-wise
+ *     renormalisation.
+ *   - Containers live in pages of 16 tokens: uint8 [num_pages][Hkv][16][rec_bytes].
+ *     slot = page * 16 + index-in-page.  A record's address follows from (slot, head)
+ *     alone (fixed stride, Sec. 4.1).
+ *   - Key channel means: one per (sequence, window of 128 positions, KV head):
+ *     int8 [S][max_windows][Hkv][128] and float scale [S][max_windows][Hkv];
+ *     mean_j = scale * q_j, in the Hadamard-rotated domain.
+ *   - Every pointer named "device" must be device memory reachable from the current
+ *     device; the caller owns all of it, and the CUDA stream.  The library owns only
+ *     dq_tables (host memory).  Calls validate their arguments, enqueue kernels on the
+ *     given stream and return; 0 means "validated and enqueued".
+ *   - Errors are returned, never thrown; nothing is launched when validation fails;
+ *     no kernel traps or spins.
+ */
+#ifndef DQ_H_
+#define DQ_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define DQ_OK 0
+#define DQ_ERR_ARG (-1)          /* null / out-of-range argument                     */
+#define DQ_ERR_INFEASIBLE (-2)   /* the all-central stream does not fit the container */
+#define DQ_ERR_UNSUPPORTED (-3)  /* head_dim != 128, GQA group > 8, record too large  */
+#define DQ_ERR_WORKSPACE (-4)    /* workspace smaller than dq_decode_workspace_bytes  */
+#define DQ_ERR_CUDA (-5)         /* a CUDA runtime call failed (see dq_last_cuda_error) */
+
+#define DQ_MAX_LEVELS 16
+#define DQ_HEAD_DIM 128
+#define DQ_PAGE_TOKENS 16
+#define DQ_WINDOW_TOKENS 128
+#define DQ_MAX_REC_BYTES 160
+#define DQ_MAX_GROUP 8           /* query heads per KV head                           */
+
+#define DQ_MEAN_COMPUTE 0
+#define DQ_MEAN_REUSE 1
+
+typedef struct dq_tables dq_tables; /* opaque, immutable after build, host memory */
+
+typedef struct {
+    int head_dim;   /* must be 128 */
+    double alpha;   /* sharpening exponent p' ~ p^alpha (Sec. 4.4; paper: 1.4).  >= 0: used as
+                       given (0 = uniform table).  < 0: smallest of 1.4, 1.5, ..., 32.0 whose
+                       table has entropy <= B/128 and passes the feasibility test. */
+    int has_mean;   /* 1: streams had a window mean removed (keys); 0: values          */
+    int rotate;     /* 1: the library applies the per-head Hadamard rotation (Sec. 4.2) */
+} dq_table_opts;
+
+typedef struct {
+    int levels, head_dim, rec_bytes, container_bytes, budget_bits, mstar, has_mean, rotate;
+    double alpha;
+    int32_t f[DQ_MAX_LEVELS];      /* frequencies, sum 256            */
+    int32_t c[DQ_MAX_LEVELS + 1];  /* cumulative frequencies          */
+    float r[DQ_MAX_LEVELS];        /* -log2(f/256), bits (Algorithm 1) */
+    uint32_t R[DQ_MAX_LEVELS];     /* ceil(r * 65536)                  */
+    uint32_t lut[256];             /* (fp16 bits of level) << 16 | f << 8 | (z - c) */
+} dq_table_info;
+
+/* Probability model and rANS tables of one tensor kind (Sec. 3.1 "Entropy Coding",
+ * Sec. 4.2 last paragraph, Sec. 4.4 "Distribution sharpening").  The probability of level
+ * m is the N(0,1) mass of its cell on an M-level grid spanning +-E[max of 128 normals];
+ * frequencies are integers summing to 256.  Host only; needs no GPU.
+ * Returns DQ_ERR_INFEASIBLE when 128 * R[mstar] > 65536 * B.  *out is set only on DQ_OK. */
+int dq_build_tables(int levels, double bits_per_elem, const dq_table_opts *opts, dq_tables **out);
+void dq_free_tables(dq_tables *t);
+int dq_tables_info(const dq_tables *t, dq_table_info *out);
+
+/* Encoder (Fig. 1; Algorithm 1; Sec. 4.5 "Encoding"): Hadamard rotation, windowed channel
+ * mean removal (keys), min-max affine grid, drift, least-squares refit, fp16 metadata,
+ * second drift, rANS.  One warp per stream.
+ *   tk / tv          tables for keys / values; either may be NULL to skip that tensor
+ *   k_bf16, v_bf16   device, bf16 [T][Hkv][128]
+ *   seq_id, pos      device int32 [T]: sequence and position of each token
+ *   slot             device int32 [T]: physical slot; distinct per token
+ *   k_cont, v_cont   device, containers as laid out above; only the T records written
+ *   k_mean_q/scale   device, mean arrays as laid out above (keys with has_mean only)
+ *   mean_mode        DQ_MEAN_COMPUTE: every maximal run of consecutive call tokens with the
+ *                    same (seq_id, pos / 128) defines that window's mean (the tokens of a
+ *                    window must be contiguous and ascending in pos).  DQ_MEAN_REUSE: stored
+ *                    means are used; a token with pos % 128 == 0 first copies the previous
+ *                    window's mean into its own window (window 0: zero); at most one such
+ *                    token per sequence per call.
+ *   status           device uint32[4], nullable, accumulated (not cleared): [0] streams that
+ *                    fell back to the all-central assignment, [1] constant streams,
+ *                    [2] rejected refits, [3] max record bytes used (atomicMax).
+ * Errors: DQ_ERR_ARG for null / negative arguments, DQ_ERR_CUDA on launch failure. */
+int dq_encode_tokens(const dq_tables *tk, const dq_tables *tv, const void *k_bf16,
+                     const void *v_bf16, int T, int Hkv, const int32_t *seq_id,
+                     const int32_t *pos, const int32_t *slot, uint8_t *k_cont, uint8_t *v_cont,
+                     int8_t *k_mean_q, float *k_mean_scale, int max_windows, int mean_mode,
+                     uint32_t *status, void *cuda_stream);
+
+/* Bytes of scratch dq_decode_attention needs (split-K partials and a work counter). */
+size_t dq_decode_workspace_bytes(int B, int Hq, int max_pages);
+
+/* Decode-step attention over the compressed cache (Sec. 4.5 "Decoding"; Algorithm 2;
+ * Appendix A fold-key / fold-value): every record is rANS-decoded in shared memory, the
+ * levels feed tensor-core contractions, the affine terms are applied after them, softmax
+ * is online, token ranges are split over CTAs and merged by log-sum-exp.
+ *   q_bf16      device bf16 [B][Hq][128]; the library rotates it when keys are rotated
+ *   page_table  device int32 [B][max_pages]: physical page of tokens 16 i .. 16 i + 15
+ *   seq_lens    device int32 [B]; 0 gives a zero output row; must be <= 16 * max_pages
+ *   out_bf16    device bf16 [B][Hq][128] (nullable if out_f32 is given)
+ *   out_f32     device float [B][Hq][128], nullable: the result before bf16 rounding
+ *   workspace   device, >= dq_decode_workspace_bytes(B, Hq, max_pages), 16-byte aligned
+ * Hq must be a multiple of Hkv with Hq / Hkv <= 8 (else DQ_ERR_UNSUPPORTED). */
+int dq_decode_attention(const dq_tables *tk, const dq_tables *tv, const void *q_bf16,
+                        const uint8_t *k_cont, const uint8_t *v_cont, const int8_t *k_mean_q,
+                        const float *k_mean_scale, int max_windows, const int32_t *page_table,
+                        int max_pages, const int32_t *seq_lens, int B, int Hq, int Hkv,
+                        float sm_scale, void *out_bf16, float *out_f32, void *workspace,
+                        size_t workspace_bytes, void *cuda_stream);
+
+/* Check/debug export of Algorithm 2: decode T * Hkv records to symbols and to dequantised
+ * values in the rotated domain, xhat = fma(m, s, o) (+ mean for keys).
+ *   symbols  device uint8 [T][Hkv][128], nullable;  dequant  device float, same shape, nullable
+ *   mean arrays may be NULL when t has no mean. */
+int dq_decode_tokens(const dq_tables *t, const uint8_t *cont, const int8_t *mean_q,
+                     const float *mean_scale, int max_windows, const int32_t *seq_id,
+                     const int32_t *pos, const int32_t *slot, int T, int Hkv, uint8_t *symbols,
+                     float *dequant, void *cuda_stream);
+
+/* Comparison baseline (no counterpart in the paper's method: its reference point is bf16
+ * FlashAttention-2, Sec. 5.1): split-K decode attention over an un-quantised bf16 cache
+ * laid out [num_pages][Hkv][16][128].  Same page table, workspace and outputs as above. */
+int dq_bf16_decode_attention(const void *q_bf16, const void *k_bf16_pages, const void *v_bf16_pages,
+                             const int32_t *page_table, int max_pages, const int32_t *seq_lens,
+                             int B, int Hq, int Hkv, float sm_scale, void *out_bf16,
+                             void *workspace, size_t workspace_bytes, void *cuda_stream);
+
+const char *dq_strerror(int code);
+/* Text of the last CUDA error seen by this thread's calls ("" if none). */
+const char *dq_last_cuda_error(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* DQ_H_ */

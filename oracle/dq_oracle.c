@@ -565,7 +565,7 @@ void dqo_decode_tokens(const dqo_table *T, const uint8_t *cont, const int8_t *me
         int t = (int)(th / Hkv), h = (int)(th % Hkv);
         const int8_t *mq = NULL;
         float msc = 0.0f;
-        if (T->has_mean) {
+        if (T->has_mean && mean_q) {
             size_t mi = ((size_t)seq_id[t] * Wmax + pos[t] / DQO_WINDOW) * Hkv + h;
             mq = mean_q + mi * n; msc = mean_scale[mi];
         }

@@ -1,0 +1,185 @@
+"""Thin Python binding of the D-Quant B200 library (``libdquant.so``, C ABI in include/dq.h).
+
+Argument marshalling only: every step of the path runs in the library's CUDA kernels.
+PyTorch supplies device memory and the current stream.  There is no CPU fallback: if the
+shared library is missing or fails to load, every call raises.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_PKG, "libdquant.so")
+
+MAX_LEVELS = 16
+HEAD_DIM = 128
+PAGE_TOKENS = 16
+WINDOW_TOKENS = 128
+MEAN_COMPUTE = 0
+MEAN_REUSE = 1
+
+ERRORS = {0: "DQ_OK", -1: "DQ_ERR_ARG", -2: "DQ_ERR_INFEASIBLE", -3: "DQ_ERR_UNSUPPORTED",
+          -4: "DQ_ERR_WORKSPACE", -5: "DQ_ERR_CUDA"}
+
+EXPORTS = ["dq_build_tables", "dq_free_tables", "dq_tables_info", "dq_encode_tokens",
+           "dq_decode_workspace_bytes", "dq_decode_attention", "dq_decode_tokens",
+           "dq_bf16_decode_attention", "dq_strerror", "dq_last_cuda_error"]
+
+
+class DqError(RuntimeError):
+    def __init__(self, code, what):
+        self.code = code
+        super().__init__(f"{what}: {ERRORS.get(code, code)}")
+
+
+class TableOpts(C.Structure):
+    _fields_ = [("head_dim", C.c_int), ("alpha", C.c_double), ("has_mean", C.c_int), ("rotate", C.c_int)]
+
+
+class TableInfo(C.Structure):
+    _fields_ = [("levels", C.c_int), ("head_dim", C.c_int), ("rec_bytes", C.c_int),
+                ("container_bytes", C.c_int), ("budget_bits", C.c_int), ("mstar", C.c_int),
+                ("has_mean", C.c_int), ("rotate", C.c_int), ("alpha", C.c_double),
+                ("f", C.c_int32 * MAX_LEVELS), ("c", C.c_int32 * (MAX_LEVELS + 1)),
+                ("r", C.c_float * MAX_LEVELS), ("R", C.c_uint32 * MAX_LEVELS), ("lut", C.c_uint32 * 256)]
+
+
+_lib = None
+
+
+def lib():
+    """Load libdquant.so (built by ``_build.build()``); raises if it is missing."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise ImportError(f"{LIB_PATH} not found: build it with `python -m paper_2609_19880_b200._build` "
+                              "(there is no CPU fallback)")
+        L = C.CDLL(LIB_PATH)
+        vp, i32, f32, f64, sz = C.c_void_p, C.c_int, C.c_float, C.c_double, C.c_size_t
+        L.dq_build_tables.restype = i32
+        L.dq_build_tables.argtypes = [i32, f64, C.POINTER(TableOpts), C.POINTER(vp)]
+        L.dq_free_tables.restype = None
+        L.dq_free_tables.argtypes = [vp]
+        L.dq_tables_info.restype = i32
+        L.dq_tables_info.argtypes = [vp, C.POINTER(TableInfo)]
+        L.dq_encode_tokens.restype = i32
+        L.dq_encode_tokens.argtypes = [vp, vp, vp, vp, i32, i32, vp, vp, vp, vp, vp, vp, vp, i32, i32, vp, vp]
+        L.dq_decode_workspace_bytes.restype = sz
+        L.dq_decode_workspace_bytes.argtypes = [i32, i32, i32]
+        L.dq_decode_attention.restype = i32
+        L.dq_decode_attention.argtypes = [vp, vp, vp, vp, vp, vp, vp, i32, vp, i32, vp, i32, i32, i32, f32,
+                                          vp, vp, vp, sz, vp]
+        L.dq_decode_tokens.restype = i32
+        L.dq_decode_tokens.argtypes = [vp, vp, vp, vp, i32, vp, vp, vp, i32, i32, vp, vp, vp]
+        L.dq_bf16_decode_attention.restype = i32
+        L.dq_bf16_decode_attention.argtypes = [vp, vp, vp, vp, i32, vp, i32, i32, i32, f32, vp, vp, sz, vp]
+        L.dq_strerror.restype = C.c_char_p
+        L.dq_strerror.argtypes = [i32]
+        L.dq_last_cuda_error.restype = C.c_char_p
+        L.dq_last_cuda_error.argtypes = []
+        _lib = L
+    return _lib
+
+
+def _check(rc, what):
+    if rc != 0:
+        msg = what
+        if rc == -5:
+            msg += " [" + lib().dq_last_cuda_error().decode() + "]"
+        raise DqError(rc, msg)
+
+
+def _ptr(t):
+    return None if t is None else C.c_void_p(t.data_ptr())
+
+
+def _stream(stream=None):
+    import torch
+    s = stream if stream is not None else torch.cuda.current_stream()
+    return C.c_void_p(s.cuda_stream)
+
+
+class Tables:
+    """Owner of one ``dq_tables*`` (host memory inside the library)."""
+
+    def __init__(self, handle):
+        self._h = C.c_void_p(handle)
+
+    @property
+    def handle(self):
+        return self._h
+
+    def info(self) -> TableInfo:
+        out = TableInfo()
+        _check(lib().dq_tables_info(self._h, C.byref(out)), "dq_tables_info")
+        return out
+
+    def __del__(self):
+        try:
+            if self._h and _lib is not None:
+                _lib.dq_free_tables(self._h)
+                self._h = None
+        except Exception:
+            pass
+
+
+def dq_build_tables(levels: int, bits_per_elem: float, *, alpha: float = 1.4, has_mean: bool = False,
+                    rotate: bool = True, head_dim: int = HEAD_DIM) -> Tables:
+    opts = TableOpts(head_dim, float(alpha), int(has_mean), int(rotate))
+    h = C.c_void_p()
+    _check(lib().dq_build_tables(int(levels), float(bits_per_elem), C.byref(opts), C.byref(h)), "dq_build_tables")
+    return Tables(h.value)
+
+
+def dq_tables_info(t: Tables) -> TableInfo:
+    return t.info()
+
+
+def dq_encode_tokens(tk, tv, k_bf16, v_bf16, seq_id, pos, slot, k_cont, v_cont, k_mean_q=None,
+                     k_mean_scale=None, mean_mode: int = MEAN_COMPUTE, status=None, stream=None):
+    """K/V bf16 [T, Hkv, 128] -> containers (+ window means).  All tensors on the device."""
+    ref = k_bf16 if k_bf16 is not None else v_bf16
+    T, Hkv = int(ref.shape[0]), int(ref.shape[1])
+    max_windows = int(k_mean_q.shape[1]) if k_mean_q is not None else 0
+    rc = lib().dq_encode_tokens(tk.handle if tk else None, tv.handle if tv else None, _ptr(k_bf16), _ptr(v_bf16),
+                                T, Hkv, _ptr(seq_id), _ptr(pos), _ptr(slot), _ptr(k_cont), _ptr(v_cont),
+                                _ptr(k_mean_q), _ptr(k_mean_scale), max_windows, int(mean_mode), _ptr(status),
+                                _stream(stream))
+    _check(rc, "dq_encode_tokens")
+
+
+def dq_decode_workspace_bytes(B: int, Hq: int, max_pages: int) -> int:
+    return int(lib().dq_decode_workspace_bytes(int(B), int(Hq), int(max_pages)))
+
+
+def dq_decode_attention(tk, tv, q_bf16, k_cont, v_cont, k_mean_q, k_mean_scale, page_table, seq_lens,
+                        Hkv: int, sm_scale: float, out_bf16, workspace, out_f32=None, stream=None):
+    """q bf16 [B, Hq, 128], containers, seq_lens -> out bf16 [B, Hq, 128]."""
+    B, Hq = int(q_bf16.shape[0]), int(q_bf16.shape[1])
+    max_windows = int(k_mean_q.shape[1]) if k_mean_q is not None else 0
+    rc = lib().dq_decode_attention(tk.handle, tv.handle, _ptr(q_bf16), _ptr(k_cont), _ptr(v_cont), _ptr(k_mean_q),
+                                   _ptr(k_mean_scale), max_windows, _ptr(page_table), int(page_table.shape[1]),
+                                   _ptr(seq_lens), B, Hq, int(Hkv), float(sm_scale), _ptr(out_bf16),
+                                   _ptr(out_f32), _ptr(workspace), int(workspace.numel() * workspace.element_size()),
+                                   _stream(stream))
+    _check(rc, "dq_decode_attention")
+
+
+def dq_decode_tokens(t, cont, slot, Hkv: int, symbols=None, dequant=None, mean_q=None, mean_scale=None,
+                     seq_id=None, pos=None, stream=None):
+    max_windows = int(mean_q.shape[1]) if mean_q is not None else 0
+    rc = lib().dq_decode_tokens(t.handle, _ptr(cont), _ptr(mean_q), _ptr(mean_scale), max_windows, _ptr(seq_id),
+                                _ptr(pos), _ptr(slot), int(slot.shape[0]), int(Hkv), _ptr(symbols), _ptr(dequant),
+                                _stream(stream))
+    _check(rc, "dq_decode_tokens")
+
+
+def dq_bf16_decode_attention(q_bf16, k_pages, v_pages, page_table, seq_lens, Hkv: int, sm_scale: float,
+                             out_bf16, workspace, stream=None):
+    B, Hq = int(q_bf16.shape[0]), int(q_bf16.shape[1])
+    rc = lib().dq_bf16_decode_attention(_ptr(q_bf16), _ptr(k_pages), _ptr(v_pages), _ptr(page_table),
+                                        int(page_table.shape[1]), _ptr(seq_lens), B, Hq, int(Hkv), float(sm_scale),
+                                        _ptr(out_bf16), _ptr(workspace),
+                                        int(workspace.numel() * workspace.element_size()), _stream(stream))
+    _check(rc, "dq_bf16_decode_attention")

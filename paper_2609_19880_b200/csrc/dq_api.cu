@@ -1,0 +1,175 @@
+// C ABI of the library: argument validation and kernel launches (see include/dq.h).
+#include <cstdio>
+#include <cstring>
+#include <new>
+
+#include "dq_internal.h"
+
+namespace {
+
+thread_local char g_cuda_error[256] = "";
+
+int cuda_fail(cudaError_t e, const char* where) {
+    std::snprintf(g_cuda_error, sizeof g_cuda_error, "%s: %s", where, cudaGetErrorString(e));
+    return DQ_ERR_CUDA;
+}
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+}  // namespace
+
+extern "C" {
+
+int dq_build_tables(int levels, double bits_per_elem, const dq_table_opts* opts, dq_tables** out) {
+    if (!opts || !out) return DQ_ERR_ARG;
+    dq_tables* t = new (std::nothrow) dq_tables;
+    if (!t) return DQ_ERR_ARG;
+    const int rc = dq_host_build(levels, bits_per_elem, opts, t);
+    if (rc != DQ_OK) {
+        delete t;
+        return rc;
+    }
+    *out = t;
+    return DQ_OK;
+}
+
+void dq_free_tables(dq_tables* t) { delete t; }
+
+int dq_tables_info(const dq_tables* t, dq_table_info* out) {
+    if (!t || !out) return DQ_ERR_ARG;
+    *out = t->info;
+    return DQ_OK;
+}
+
+int dq_encode_tokens(const dq_tables* tk, const dq_tables* tv, const void* k_bf16, const void* v_bf16,
+                     int T, int Hkv, const int32_t* seq_id, const int32_t* pos, const int32_t* slot,
+                     uint8_t* k_cont, uint8_t* v_cont, int8_t* k_mean_q, float* k_mean_scale,
+                     int max_windows, int mean_mode, uint32_t* status, void* cuda_stream) {
+    if (T < 0 || Hkv <= 0 || (!tk && !tv)) return DQ_ERR_ARG;
+    if (!seq_id || !pos || !slot) return DQ_ERR_ARG;
+    if (tk && (!k_bf16 || !k_cont)) return DQ_ERR_ARG;
+    if (tv && (!v_bf16 || !v_cont)) return DQ_ERR_ARG;
+    if (mean_mode != DQ_MEAN_COMPUTE && mean_mode != DQ_MEAN_REUSE) return DQ_ERR_ARG;
+    const bool k_mean = tk && tk->info.has_mean;
+    if (k_mean && (!k_mean_q || !k_mean_scale || max_windows <= 0)) return DQ_ERR_ARG;
+    if (tv && tv->info.has_mean) return DQ_ERR_UNSUPPORTED;  // only keys carry window means
+    if ((k_bf16 && (reinterpret_cast<uintptr_t>(k_bf16) & 7u)) ||
+        (v_bf16 && (reinterpret_cast<uintptr_t>(v_bf16) & 7u)) ||
+        (k_mean && (reinterpret_cast<uintptr_t>(k_mean_q) & 3u)))
+        return DQ_ERR_ARG;
+    if (T == 0) return DQ_OK;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    cudaError_t e;
+    if (k_mean) {
+        e = dq_launch_means(tk->dev, k_bf16, T, Hkv, seq_id, pos, k_mean_q, k_mean_scale, max_windows,
+                            mean_mode, st);
+        if (e != cudaSuccess) return cuda_fail(e, "window means");
+    }
+    if (tk) {
+        e = dq_launch_encode(tk->dev, k_bf16, T, Hkv, seq_id, pos, slot, k_cont, k_mean_q, k_mean_scale,
+                             max_windows, status, st);
+        if (e != cudaSuccess) return cuda_fail(e, "encode K");
+    }
+    if (tv) {
+        e = dq_launch_encode(tv->dev, v_bf16, T, Hkv, seq_id, pos, slot, v_cont, nullptr, nullptr, 0,
+                             status, st);
+        if (e != cudaSuccess) return cuda_fail(e, "encode V");
+    }
+    return DQ_OK;
+}
+
+size_t dq_decode_workspace_bytes(int B, int Hq, int max_pages) {
+    if (B <= 0 || Hq <= 0 || max_pages <= 0) return 0;
+    return dq_attn_workspace_bytes(B, Hq, max_pages);
+}
+
+static int check_attn_common(const void* q, const int32_t* page_table, int max_pages,
+                             const int32_t* seq_lens, int B, int Hq, int Hkv, const void* out_a,
+                             const void* out_b, void* workspace, size_t workspace_bytes) {
+    if (!q || !page_table || !seq_lens || (!out_a && !out_b) || !workspace) return DQ_ERR_ARG;
+    if (B <= 0 || Hq <= 0 || Hkv <= 0 || max_pages <= 0) return DQ_ERR_ARG;
+    if (Hq % Hkv != 0) return DQ_ERR_ARG;
+    if (Hq / Hkv > DQ_MAX_GROUP || B > 4096) return DQ_ERR_UNSUPPORTED;
+    if (!aligned16(workspace) || (reinterpret_cast<uintptr_t>(q) & 7u)) return DQ_ERR_ARG;
+    if (workspace_bytes < dq_attn_workspace_bytes(B, Hq, max_pages)) return DQ_ERR_WORKSPACE;
+    return DQ_OK;
+}
+
+int dq_decode_attention(const dq_tables* tk, const dq_tables* tv, const void* q_bf16,
+                        const uint8_t* k_cont, const uint8_t* v_cont, const int8_t* k_mean_q,
+                        const float* k_mean_scale, int max_windows, const int32_t* page_table,
+                        int max_pages, const int32_t* seq_lens, int B, int Hq, int Hkv, float sm_scale,
+                        void* out_bf16, float* out_f32, void* workspace, size_t workspace_bytes,
+                        void* cuda_stream) {
+    if (!tk || !tv || !k_cont || !v_cont) return DQ_ERR_ARG;
+    int rc = check_attn_common(q_bf16, page_table, max_pages, seq_lens, B, Hq, Hkv, out_bf16, out_f32,
+                               workspace, workspace_bytes);
+    if (rc != DQ_OK) return rc;
+    if (tv->info.has_mean) return DQ_ERR_UNSUPPORTED;
+    if (tk->info.has_mean && (!k_mean_q || !k_mean_scale || max_windows <= 0)) return DQ_ERR_ARG;
+    if (tk->info.has_mean && (long long)max_windows * DQ_WINDOW_TOKENS < (long long)max_pages * DQ_PAGE_TOKENS)
+        return DQ_ERR_ARG;  // every addressable position needs a window slot
+    if (!aligned16(k_cont) || !aligned16(v_cont) || (tk->info.has_mean && !aligned16(k_mean_q))) return DQ_ERR_ARG;
+    if ((out_bf16 && (reinterpret_cast<uintptr_t>(out_bf16) & 7u)) || (out_f32 && !aligned16(out_f32)))
+        return DQ_ERR_ARG;
+    DqAttnArgs a;
+    a.q_bf16 = q_bf16; a.k_cont = k_cont; a.v_cont = v_cont;
+    a.mean_q = k_mean_q; a.mean_scale = k_mean_scale;
+    a.page_table = page_table; a.seq_lens = seq_lens;
+    a.out_bf16 = out_bf16; a.out_f32 = out_f32; a.workspace = workspace;
+    a.max_windows = max_windows; a.max_pages = max_pages;
+    a.B = B; a.Hq = Hq; a.Hkv = Hkv; a.sm_scale = sm_scale;
+    const cudaError_t e = dq_launch_attention(tk->dev, tv->dev, a, static_cast<cudaStream_t>(cuda_stream));
+    if (e != cudaSuccess) return cuda_fail(e, "decode attention");
+    return DQ_OK;
+}
+
+int dq_decode_tokens(const dq_tables* t, const uint8_t* cont, const int8_t* mean_q, const float* mean_scale,
+                     int max_windows, const int32_t* seq_id, const int32_t* pos, const int32_t* slot, int T,
+                     int Hkv, uint8_t* symbols, float* dequant, void* cuda_stream) {
+    if (!t || !cont || !slot || T < 0 || Hkv <= 0 || (!symbols && !dequant)) return DQ_ERR_ARG;
+    if (t->info.has_mean && mean_q && (!mean_scale || !seq_id || !pos || max_windows <= 0)) return DQ_ERR_ARG;
+    if (T == 0) return DQ_OK;
+    const cudaError_t e = dq_launch_decode_tokens(t->dev, cont, mean_q, mean_scale, max_windows, seq_id, pos,
+                                                  slot, T, Hkv, symbols, dequant,
+                                                  static_cast<cudaStream_t>(cuda_stream));
+    if (e != cudaSuccess) return cuda_fail(e, "decode tokens");
+    return DQ_OK;
+}
+
+int dq_bf16_decode_attention(const void* q_bf16, const void* k_bf16_pages, const void* v_bf16_pages,
+                             const int32_t* page_table, int max_pages, const int32_t* seq_lens, int B,
+                             int Hq, int Hkv, float sm_scale, void* out_bf16, void* workspace,
+                             size_t workspace_bytes, void* cuda_stream) {
+    if (!k_bf16_pages || !v_bf16_pages) return DQ_ERR_ARG;
+    int rc = check_attn_common(q_bf16, page_table, max_pages, seq_lens, B, Hq, Hkv, out_bf16, nullptr,
+                               workspace, workspace_bytes);
+    if (rc != DQ_OK) return rc;
+    if (!aligned16(k_bf16_pages) || !aligned16(v_bf16_pages) || (reinterpret_cast<uintptr_t>(out_bf16) & 7u))
+        return DQ_ERR_ARG;
+    DqAttnArgs a;
+    std::memset(&a, 0, sizeof a);
+    a.q_bf16 = q_bf16; a.page_table = page_table; a.seq_lens = seq_lens;
+    a.out_bf16 = out_bf16; a.workspace = workspace;
+    a.max_pages = max_pages; a.B = B; a.Hq = Hq; a.Hkv = Hkv; a.sm_scale = sm_scale;
+    const cudaError_t e = dq_launch_bf16_attention(a, k_bf16_pages, v_bf16_pages,
+                                                   static_cast<cudaStream_t>(cuda_stream));
+    if (e != cudaSuccess) return cuda_fail(e, "bf16 decode attention");
+    return DQ_OK;
+}
+
+const char* dq_strerror(int code) {
+    switch (code) {
+        case DQ_OK: return "ok";
+        case DQ_ERR_ARG: return "invalid argument";
+        case DQ_ERR_INFEASIBLE: return "levels do not fit the container budget";
+        case DQ_ERR_UNSUPPORTED: return "unsupported configuration";
+        case DQ_ERR_WORKSPACE: return "workspace too small";
+        case DQ_ERR_CUDA: return "CUDA error";
+        default: return "unknown error";
+    }
+}
+
+const char* dq_last_cuda_error(void) { return g_cuda_error; }
+
+}  // extern "C"

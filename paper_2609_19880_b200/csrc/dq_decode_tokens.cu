@@ -1,0 +1,59 @@
+// Check/debug decoder: Algorithm 2 on every record, one thread per stream, reading the
+// record straight from global memory.  Produces the symbols and the dequantised values
+// xhat = fma(m, s, o) (+ window mean for keys, Appendix A).  Not a performance path.
+#include <cuda_fp16.h>
+
+#include "dq_internal.h"
+
+namespace {
+
+__global__ void __launch_bounds__(128)
+dq_decode_tokens_kernel(const __grid_constant__ DqDevTable T, const uint8_t* __restrict__ cont,
+                        const int8_t* __restrict__ mean_q, const float* __restrict__ mean_scale,
+                        int Wmax, const int32_t* __restrict__ seq_id, const int32_t* __restrict__ pos,
+                        const int32_t* __restrict__ slot, int n_tok, int Hkv,
+                        uint8_t* __restrict__ symbols, float* __restrict__ dequant) {
+    const long long sid = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (sid >= (long long)n_tok * Hkv) return;
+    const int t = (int)(sid / Hkv), h = (int)(sid % Hkv);
+    const int sl = slot[t];
+    const uint8_t* rec = cont + (((size_t)(sl / DQ_PAGE_TOKENS) * Hkv + h) * DQ_PAGE_TOKENS +
+                                 (size_t)(sl % DQ_PAGE_TOKENS)) * T.rec;
+    const float s = __half2float(__ushort_as_half((unsigned short)(rec[0] | (rec[1] << 8))));
+    const float o = __half2float(__ushort_as_half((unsigned short)(rec[2] | (rec[3] << 8))));
+    uint32_t x = (uint32_t)rec[4] | ((uint32_t)rec[5] << 8) | ((uint32_t)rec[6] << 16) |
+                 ((uint32_t)rec[7] << 24);
+    int ptr = 8;
+    const int8_t* mq = nullptr;
+    float msc = 0.f;
+    if (T.has_mean && mean_q) {
+        const size_t mi = ((size_t)seq_id[t] * Wmax + pos[t] / DQ_WINDOW_TOKENS) * Hkv + h;
+        mq = mean_q + mi * DQ_HEAD_DIM;
+        msc = mean_scale[mi];
+    }
+    for (int j = 0; j < DQ_HEAD_DIM; ++j) {
+        const uint32_t e = T.lut[x & 255u];
+        x = ((e >> 8) & 255u) * (x >> 8) + (e & 255u);
+        if (x < (1u << 23) && ptr < T.rec) x = (x << 8) | rec[ptr++];  // at most one byte
+        const float lvl = __half2float(__ushort_as_half((unsigned short)(e >> 16)));
+        if (symbols) symbols[sid * DQ_HEAD_DIM + j] = (uint8_t)(int)lvl;
+        if (dequant) {
+            float v = __fmaf_rn(lvl, s, o);
+            if (mq) v = __fadd_rn(v, __fmul_rn(msc, (float)mq[j]));
+            dequant[sid * DQ_HEAD_DIM + j] = v;
+        }
+    }
+}
+
+}  // namespace
+
+cudaError_t dq_launch_decode_tokens(const DqDevTable& t, const uint8_t* cont, const int8_t* mean_q,
+                                    const float* mean_scale, int max_windows, const int32_t* seq_id,
+                                    const int32_t* pos, const int32_t* slot, int T, int Hkv,
+                                    uint8_t* symbols, float* dequant, cudaStream_t st) {
+    const long long n = (long long)T * Hkv;
+    if (n == 0) return cudaSuccess;
+    dq_decode_tokens_kernel<<<(unsigned)((n + 127) / 128), 128, 0, st>>>(
+        t, cont, mean_q, mean_scale, max_windows, seq_id, pos, slot, T, Hkv, symbols, dequant);
+    return cudaGetLastError();
+}

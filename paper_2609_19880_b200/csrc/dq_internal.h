@@ -1,0 +1,58 @@
+// Internal declarations shared by the library's translation units (not part of the ABI).
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "dq.h"
+
+// Table of one tensor kind as the kernels see it; passed by value as a kernel parameter
+// (constant bank), so building tables needs no device memory.
+struct DqDevTable {
+    int M, rec, mstar, budget_bits;
+    int has_mean, rotate, pad0, pad1;
+    uint32_t fc[DQ_MAX_LEVELS];  // f | c << 16           (encoder, Eq. rans Enc)
+    float r[DQ_MAX_LEVELS];      // ideal cost in bits     (Algorithm 1)
+    uint32_t R[DQ_MAX_LEVELS];   // ceil(r * 65536)
+    uint32_t lut[256];           // fp16(level) << 16 | f << 8 | (z - c)   (Algorithm 2)
+};
+
+struct dq_tables {
+    dq_table_info info;
+    DqDevTable dev;
+};
+
+// dq_tables.cu
+int dq_host_build(int levels, double bits_per_elem, const dq_table_opts* opts, dq_tables* out);
+
+// kernels' host launchers (each returns a cudaError_t from the launch)
+cudaError_t dq_launch_means(const DqDevTable& tk, const void* k_bf16, int T, int Hkv,
+                            const int32_t* seq_id, const int32_t* pos, int8_t* mean_q,
+                            float* mean_scale, int max_windows, int mode, cudaStream_t st);
+cudaError_t dq_launch_encode(const DqDevTable& t, const void* x_bf16, int T, int Hkv,
+                             const int32_t* seq_id, const int32_t* pos, const int32_t* slot,
+                             uint8_t* cont, const int8_t* mean_q, const float* mean_scale,
+                             int max_windows, uint32_t* status, cudaStream_t st);
+cudaError_t dq_launch_decode_tokens(const DqDevTable& t, const uint8_t* cont, const int8_t* mean_q,
+                                    const float* mean_scale, int max_windows, const int32_t* seq_id,
+                                    const int32_t* pos, const int32_t* slot, int T, int Hkv,
+                                    uint8_t* symbols, float* dequant, cudaStream_t st);
+
+struct DqAttnArgs {
+    const void* q_bf16;
+    const uint8_t* k_cont;
+    const uint8_t* v_cont;
+    const int8_t* mean_q;
+    const float* mean_scale;
+    const int32_t* page_table;
+    const int32_t* seq_lens;
+    void* out_bf16;
+    float* out_f32;
+    void* workspace;
+    int max_windows, max_pages, B, Hq, Hkv;
+    float sm_scale;
+};
+size_t dq_attn_workspace_bytes(int B, int Hq, int max_pages);
+cudaError_t dq_launch_attention(const DqDevTable& tk, const DqDevTable& tv, const DqAttnArgs& a,
+                                cudaStream_t st);
+cudaError_t dq_launch_bf16_attention(const DqAttnArgs& a, const void* k_pages, const void* v_pages,
+                                     cudaStream_t st);

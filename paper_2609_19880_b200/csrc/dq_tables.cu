@@ -1,0 +1,167 @@
+// Host-side construction of the calibration-free rANS tables (Sec. 3.1 "Entropy Coding",
+// Sec. 4.2 last paragraph, Sec. 4.4 "Distribution sharpening").  No device work.
+#include <cuda_fp16.h>
+
+#include <algorithm>
+#include <cmath>
+#include <cstring>
+#include <vector>
+
+#include "dq_internal.h"
+
+namespace {
+
+constexpr int kTotal = 256;  // 2^p, p = 8
+
+inline double normal_cdf(double x) { return 0.5 * std::erfc(-x * M_SQRT1_2); }
+
+// E[max of n iid standard normals] = integral of x n phi(x) Phi(x)^(n-1).  The integrand is
+// analytic and vanishes to all orders at +-9, so the trapezoid rule converges geometrically.
+double expected_maximum(int n) {
+    const int nodes = 1 << 17;
+    const double lo = -9.0, hi = 9.0, step = (hi - lo) / nodes;
+    const double inv_sqrt_2pi = 0.3989422804014326779;
+    double acc = 0.0;
+    for (int i = 1; i < nodes; ++i) {
+        const double x = lo + step * i;
+        acc += x * std::exp(-0.5 * x * x) * std::pow(normal_cdf(x), n - 1);
+    }
+    return acc * step * n * inv_sqrt_2pi;
+}
+
+struct Model {
+    std::vector<double> cell;  // analytic cell masses, normalised
+};
+
+Model cell_masses(int M, int n) {
+    const double span = expected_maximum(n);
+    const double width = 2.0 * span / (M - 1);
+    Model mod;
+    mod.cell.assign(M, 0.0);
+    for (int m = 0; 2 * m < M + 1 && m < M; ++m) {
+        const double centre = -span + width * m;
+        const double left = std::max(-span, centre - 0.5 * width);
+        const double right = std::min(span, centre + 0.5 * width);
+        const double mass = normal_cdf(right) - normal_cdf(left);
+        mod.cell[m] = mass;
+        mod.cell[M - 1 - m] = mass;  // the model is symmetric
+    }
+    double total = 0.0;
+    for (double v : mod.cell) total += v;
+    for (double& v : mod.cell) v /= total;
+    return mod;
+}
+
+// Integer frequencies summing to 256: floor with a floor of 1, then largest remainders up
+// (ties to the lowest index) or largest excesses down among f > 1 (ties to the highest index).
+void integer_frequencies(const Model& mod, double alpha, int32_t* f) {
+    const int M = (int)mod.cell.size();
+    std::vector<double> target(M);
+    double norm = 0.0;
+    for (int m = 0; m < M; ++m) norm += (target[m] = std::pow(mod.cell[m], alpha));
+    int sum = 0;
+    for (int m = 0; m < M; ++m) {
+        target[m] = target[m] / norm;
+        target[m] = kTotal * target[m];
+        f[m] = std::max(1, (int)std::floor(target[m]));
+        sum += f[m];
+    }
+    for (; sum < kTotal; ++sum) {
+        int pick = 0;
+        for (int m = 1; m < M; ++m)
+            if (target[m] - f[m] > target[pick] - f[pick]) pick = m;
+        ++f[pick];
+    }
+    for (; sum > kTotal; --sum) {
+        int pick = -1;
+        for (int m = 0; m < M; ++m)
+            if (f[m] > 1 && (pick < 0 || f[m] - target[m] >= f[pick] - target[pick])) pick = m;
+        --f[pick];
+    }
+}
+
+void finish(dq_table_info& t) {
+    t.c[0] = 0;
+    t.mstar = 0;
+    for (int m = 0; m < t.levels; ++m) {
+        t.c[m + 1] = t.c[m] + t.f[m];
+        const double bits = 8.0 - std::log2((double)t.f[m]);
+        t.r[m] = (float)bits;
+        t.R[m] = (uint32_t)std::ceil(bits * 65536.0);
+        if (t.f[m] > t.f[t.mstar]) t.mstar = m;
+    }
+    for (int m = 0; m < t.levels; ++m) {
+        const uint32_t level_bits = __half_as_ushort(__float2half((float)m));
+        for (int z = t.c[m]; z < t.c[m + 1]; ++z)
+            t.lut[z] = (level_bits << 16) | ((uint32_t)t.f[m] << 8) | (uint32_t)(z - t.c[m]);
+    }
+}
+
+bool all_central_fits(const dq_table_info& t) {
+    return (int64_t)t.head_dim * t.R[t.mstar] <= (int64_t)t.budget_bits * 65536;
+}
+
+double table_entropy(const dq_table_info& t) {
+    double h = 0.0;
+    for (int m = 0; m < t.levels; ++m) {
+        const double p = t.f[m] / (double)kTotal;
+        h -= p * std::log2(p);
+    }
+    return h;
+}
+
+}  // namespace
+
+int dq_host_build(int levels, double bits_per_elem, const dq_table_opts* opts, dq_tables* out) {
+    if (!opts || !out) return DQ_ERR_ARG;
+    if (opts->head_dim != DQ_HEAD_DIM) return DQ_ERR_UNSUPPORTED;
+    if (levels < 2 || !(bits_per_elem > 0.0) || !std::isfinite(bits_per_elem)) return DQ_ERR_ARG;
+    if (levels > DQ_MAX_LEVELS) return DQ_ERR_UNSUPPORTED;
+    const int n = DQ_HEAD_DIM;
+    const double rec_d = std::floor(bits_per_elem * n / 8.0 + 1e-9);
+    if (rec_d > DQ_MAX_REC_BYTES) return DQ_ERR_UNSUPPORTED;
+    const int rec = (int)rec_d;
+    if (rec < 9) return DQ_ERR_INFEASIBLE;  // header alone is 8 bytes
+
+    dq_table_info& t = out->info;
+    std::memset(out, 0, sizeof *out);
+    t.levels = levels;
+    t.head_dim = n;
+    t.rec_bytes = rec;
+    t.container_bytes = rec - 4;              // Eq. (budget): C bytes hold state + payload
+    t.budget_bits = 8 * t.container_bytes - 32;  // B = 8C - sigma, sigma = 32
+    t.has_mean = opts->has_mean ? 1 : 0;
+    t.rotate = opts->rotate ? 1 : 0;
+
+    const Model mod = cell_masses(levels, n);
+    bool ok = false;
+    if (opts->alpha >= 0.0) {
+        t.alpha = opts->alpha;
+        integer_frequencies(mod, t.alpha, t.f);
+        finish(t);
+        ok = all_central_fits(t);
+    } else {
+        for (int tenth = 14; tenth <= 320 && !ok; ++tenth) {
+            t.alpha = tenth / 10.0;
+            integer_frequencies(mod, t.alpha, t.f);
+            finish(t);
+            ok = all_central_fits(t) && table_entropy(t) <= (double)t.budget_bits / n;
+        }
+    }
+    if (!ok) return DQ_ERR_INFEASIBLE;
+
+    DqDevTable& d = out->dev;
+    d.M = levels;
+    d.rec = rec;
+    d.mstar = t.mstar;
+    d.budget_bits = t.budget_bits;
+    d.has_mean = t.has_mean;
+    d.rotate = t.rotate;
+    for (int m = 0; m < levels; ++m) {
+        d.fc[m] = (uint32_t)t.f[m] | ((uint32_t)t.c[m] << 16);
+        d.r[m] = t.r[m];
+        d.R[m] = t.R[m];
+    }
+    std::memcpy(d.lut, t.lut, sizeof d.lut);
+    return DQ_OK;
+}

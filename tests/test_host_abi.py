@@ -1,0 +1,113 @@
+"""CPU-side checks of the C-ABI library: it loads, exports every symbol the header declares,
+validates arguments before any launch, and its host-built tables equal the oracle's."""
+import ctypes as C
+import os
+import re
+
+import pytest
+
+import oracle
+import paper_2609_19880_b200 as dq
+from paper_2609_19880_b200 import _build, workloads
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def L():
+    _build.build()
+    return dq.lib()
+
+
+def test_header_symbols_are_exported(L):
+    hdr = open(os.path.join(ROOT, "include", "dq.h")).read()
+    hdr = re.sub(r"/\*.*?\*/", "", hdr, flags=re.S)
+    declared = set(re.findall(r"\b(dq_[a-z0-9_]+)\s*\(", hdr))
+    assert declared == set(dq.EXPORTS)
+    for name in declared:
+        assert hasattr(L, name), name
+
+
+CASES = [(5, 42, 1.4), (3, 29, 1.4), (16, 36, -1.0), (16, 75, 1.4), (9, 52, 1.4), (8, 56, 1.4),
+         (4, 37, 1.4), (3, 27, 1.4), (3, 20, 1.4), (3, 26, 1.4), (5, 39, 1.4), (2, 24, 0.0), (7, 40, 2.5)]
+
+
+@pytest.mark.parametrize("M,rec,alpha", CASES)
+def test_tables_equal_oracle(L, M, rec, alpha):
+    t = dq.dq_build_tables(M, rec * 8 / 128, alpha=alpha, has_mean=True, rotate=True)
+    i = t.info()
+    o = oracle.build_table(M, 128, rec, alpha)
+    assert (i.levels, i.rec_bytes, i.container_bytes, i.budget_bits, i.mstar) == (M, rec, o.C, o.B, o.mstar)
+    assert abs(i.alpha - o.alpha) < 1e-12
+    assert [i.f[m] for m in range(M)] == o.freqs() and [i.c[m] for m in range(M + 1)] == o.cum()
+    assert [i.r[m] for m in range(M)] == [o.r[m] for m in range(M)]
+    assert [i.R[m] for m in range(M)] == [o.R[m] for m in range(M)]
+    for z in range(256):
+        e = i.lut[z]
+        assert (e >> 8) & 255 == o.lut_f[z] and e & 255 == o.lut_d[z]
+        lvl = oracle.f16_bits_to_f32(e >> 16)
+        assert lvl == float(o.lut_m[z])
+
+
+def test_record_size_from_bits(L):
+    for bits, rec in [(2.25, 36), (2.625, 42), (1.8125, 29), (4.6875, 75), (2.26, 36), (3.0, 48)]:
+        assert dq.dq_build_tables(3, bits).info().rec_bytes == rec == oracle.rec_bytes(bits, 128)
+
+
+def test_build_errors(L):
+    with pytest.raises(dq.DqError) as e:
+        dq.dq_build_tables(16, 2.25, alpha=1.4)
+    assert e.value.code == -2
+    with pytest.raises(dq.DqError) as e:
+        dq.dq_build_tables(5, 2.625, head_dim=64)
+    assert e.value.code == -3
+    for lv, bits, code in [(1, 2.0, -1), (17, 4.0, -3), (5, -1.0, -1), (5, 20.0, -3), (3, 0.5, -2)]:
+        with pytest.raises(dq.DqError) as e:
+            dq.dq_build_tables(lv, bits)
+        assert e.value.code == code, (lv, bits)
+    h = C.c_void_p()
+    assert L.dq_build_tables(5, 2.625, None, C.byref(h)) == -1
+    assert L.dq_strerror(-2).decode().startswith("levels")
+
+
+def test_calls_validate_before_launch(L):
+    """No GPU here: every rejected call must return before touching CUDA."""
+    tk = dq.dq_build_tables(5, 2.625, has_mean=True)
+    tv = dq.dq_build_tables(3, 1.8125)
+    n = None
+    assert L.dq_encode_tokens(None, None, n, n, 4, 8, n, n, n, n, n, n, n, 0, 0, n, n) == -1
+    assert L.dq_encode_tokens(tk.handle, tv.handle, n, n, 4, 8, n, n, n, n, n, n, n, 0, 0, n, n) == -1
+    fake = C.c_void_p(0x1000)
+    assert L.dq_encode_tokens(tk.handle, None, fake, n, 4, 8, fake, fake, fake, fake, n, n, n, 4, 0, n, n) == -1
+    assert L.dq_encode_tokens(tk.handle, None, fake, n, 4, 8, fake, fake, fake, fake, n, fake, fake, 4, 7, n, n) == -1
+    assert L.dq_encode_tokens(tk.handle, None, fake, n, -1, 8, fake, fake, fake, fake, n, fake, fake, 4, 0, n, n) == -1
+    assert L.dq_encode_tokens(tk.handle, None, fake, n, 0, 8, fake, fake, fake, fake, n, fake, fake, 4, 0, n, n) == 0
+    ws = dq.dq_decode_workspace_bytes(2, 32, 8)
+    assert ws > 2 * 32 * 128 * 4 and dq.dq_decode_workspace_bytes(0, 32, 8) == 0
+    a = dict(tk=tk.handle, tv=tv.handle, q=fake, kc=fake, vc=fake, mq=fake, ms=fake, mw=1, pt=fake, mp=8,
+             sl=fake, B=2, Hq=32, Hkv=8, sm=C.c_float(0.1), ob=fake, of=n, ws=fake, wsb=ws, st=n)
+
+    def call(**kw):
+        d = dict(a); d.update(kw)
+        return L.dq_decode_attention(*[d[k] for k in ("tk", "tv", "q", "kc", "vc", "mq", "ms", "mw", "pt", "mp",
+                                                      "sl", "B", "Hq", "Hkv", "sm", "ob", "of", "ws", "wsb", "st")])
+
+    assert call(q=n) == -1 and call(tk=n) == -1 and call(ob=n) == -1 and call(ws=n) == -1
+    assert call(Hq=30) == -1 and call(Hq=128) == -3 and call(B=5000, wsb=1 << 40) == -3
+    assert call(wsb=ws - 1) == -4
+    assert call(mq=n) == -1 and call(mw=0) == -1       # key tables with a mean need the mean arrays
+    assert call(kc=C.c_void_p(0x1001)) == -1           # containers must be 16-byte aligned
+    assert L.dq_decode_tokens(tk.handle, n, n, n, 0, n, n, fake, 4, 8, fake, n, n) == -1
+    assert L.dq_bf16_decode_attention(fake, n, fake, fake, 8, fake, 2, 32, 8, C.c_float(0.1), fake, fake, ws, n) == -1
+
+
+def test_binding_fails_loudly_without_library(monkeypatch, tmp_path):
+    monkeypatch.setattr(dq, "_lib", None)
+    monkeypatch.setattr(dq, "LIB_PATH", str(tmp_path / "missing.so"))
+    with pytest.raises(ImportError):
+        dq.dq_build_tables(5, 2.625)
+
+
+def test_budget_table_matches_record_split():
+    for bits, (kr, vr, km, vm) in workloads.BUDGETS.items():
+        assert workloads.record_split(bits) == (kr, vr)
