@@ -1,0 +1,438 @@
+#!/usr/bin/env python
+"""Benchmark of the D-Quant hot path on B200: decode-attention KV tokens/s over the compressed
+cache (2.26 bits/element), with the encoder on the step's new tokens.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+                    [--config 2|3|4|5] [--budget 2.26]
+
+One *step* = one decode step of the whole hot path: encode one new token per sequence (K and
+V: Hadamard, mean removal, drift, rANS) into the cache, then decode-step attention over every
+cached token of every sequence.  KV tokens per step = sum of sequence lengths.  Prints ONE
+JSON line (rank 0).  With N > 1 (torchrun) every rank runs an independent replica on its own
+GPU (the path has no exchange step): weak scaling, max time over ranks.
+
+`--impl reference` times the CPU oracle (as it stands) on a bounded sample of the same
+workload, on the host cores, without touching the GPU.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import math
+import os
+import statistics
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "decode_attention_kv_tokens_per_s"
+UNIT = "KV tokens/s"
+L2_BYTES = 126 * 2 ** 20
+# Algorithmic integer work of Algorithm 2 per decoded symbol (lane operations): slot mask,
+# table address, table read, two field extracts, state shift, multiply-add, compare with L,
+# byte merge, pointer advance.
+ALU_OPS_PER_SYMBOL = 10.0
+SM_COUNT, LANES_PER_SM_CLK = 148, 128
+
+
+def _peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as fh:
+            d = json.load(fh)
+        return float(d["hbm_gbs"]), float(d.get("sm_max_mhz", 1965.0)), "measured"
+    return 6650.0, 1965.0, "fallback"
+
+
+class ClockSampler(threading.Thread):
+    """Polls SM clock, power and throttle reasons through NVML (read-only) while running."""
+
+    def __init__(self, index: int, period_s: float = 0.02):
+        super().__init__(daemon=True)
+        self.index, self.period, self.samples, self._stop_evt = index, period_s, [], threading.Event()
+        self.max_mhz = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+        except Exception:
+            self.nv = None
+
+    def run(self):
+        if self.nv is None:
+            return
+        nv = self.nv
+        while not self._stop_evt.is_set():
+            try:
+                mhz = nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM)
+                reasons = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h)
+                power = nv.nvmlDeviceGetPowerUsage(self.h) / 1000.0
+                self.samples.append((time.time(), mhz, reasons, power))
+            except Exception:
+                pass
+            time.sleep(self.period)
+
+    def stop(self):
+        self._stop_evt.set()
+        self.join(timeout=2)
+
+    def summary(self, t0=None, t1=None):
+        if self.nv is None or not self.samples:
+            return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": ["nvml unavailable"]}
+        nv = self.nv
+        sel = [s for s in self.samples if (t0 is None or s[0] >= t0) and (t1 is None or s[0] <= t1)] or self.samples
+        names = {
+            getattr(nv, "nvmlClocksThrottleReasonHwSlowdown", 0x8): "hw_slowdown",
+            getattr(nv, "nvmlClocksThrottleReasonHwThermalSlowdown", 0x40): "hw_thermal_slowdown",
+            getattr(nv, "nvmlClocksThrottleReasonSwThermalSlowdown", 0x20): "sw_thermal_slowdown",
+            getattr(nv, "nvmlClocksThrottleReasonSwPowerCap", 0x4): "sw_power_cap",
+        }
+        seen = set()
+        for _, _, r, _ in sel:
+            for bit, name in names.items():
+                if r & bit:
+                    seen.add(name)
+        return {"sm_mhz": statistics.median(s[1] for s in sel), "sm_max_mhz": self.max_mhz,
+                "reasons": sorted(seen), "samples": len(sel), "power_w_max": max(s[3] for s in sel)}
+
+
+# --------------------------------------------------------------------------- CPU oracle leg
+
+def oracle_step_runner(cfg_idx: int, budget: float):
+    """Builds the bounded oracle sample (sequence 0 of the workload, all KV heads) and returns
+    (step function, KV tokens per step, description).  GPU-free."""
+    import numpy as np
+    import oracle
+    from paper_2609_19880_b200 import workloads
+
+    cfg = workloads.make_config(cfg_idx, budget=budget)
+    cfg.batch, cfg.seq_lens = 1, [min(cfg.seq_lens[0], 8192)]
+    w = workloads.generate(cfg, device="cpu")
+    ok = oracle.build_table(cfg.k_levels, 128, cfg.k_rec, cfg.alpha, has_mean=True, rotate=True)
+    ov = oracle.build_table(cfg.v_levels, 128, cfg.v_rec, cfg.alpha, has_mean=False, rotate=True)
+    kb, vb, qb = workloads.bf16_bits(w.k), workloads.bf16_bits(w.v), workloads.bf16_bits(w.q)
+    seq_id, pos, slot = (t.numpy() for t in (w.seq_id, w.pos, w.slot))
+    mq = np.zeros((1, w.max_windows, cfg.hkv, 128), np.int8)
+    ms = np.zeros((1, w.max_windows, cfg.hkv), np.float32)
+    oracle.window_means(kb, seq_id, pos, mq, ms, 0)
+    kc = np.zeros((w.num_pages, cfg.hkv, 16, ok.rec), np.uint8)
+    vc = np.zeros((w.num_pages, cfg.hkv, 16, ov.rec), np.uint8)
+    oracle.encode_tokens(ok, kb, seq_id, pos, slot, kc, mq, ms)
+    oracle.encode_tokens(ov, vb, seq_id, pos, slot, vc)
+    last = slice(cfg.total_tokens - 1, cfg.total_tokens)
+    pt, sl = w.page_table.numpy(), w.seq_lens.numpy()
+    sm = 1.0 / math.sqrt(128.0)
+
+    def step():
+        oracle.window_means(kb[last], seq_id[last], pos[last], mq, ms, 1)
+        oracle.encode_tokens(ok, kb[last], seq_id[last], pos[last], slot[last], kc, mq, ms)
+        oracle.encode_tokens(ov, vb[last], seq_id[last], pos[last], slot[last], vc)
+        return oracle.attention(ok, ov, qb, kc, vc, mq, ms, pt, sl, cfg.hkv, sm)
+
+    desc = (f"sequence 0 of {cfg.name}: {cfg.seq_lens[0]} tokens x {cfg.hkv} KV heads x {cfg.hq} query heads, "
+            f"encode 1 token + fp64 attention per step")
+    return step, cfg.seq_lens[0], desc, oracle.num_threads()
+
+
+def time_oracle(cfg_idx, budget, budget_s=10.0, max_steps=1000, warmup=1):
+    step, toks, desc, cores = oracle_step_runner(cfg_idx, budget)
+    for _ in range(warmup):
+        step()
+    n, t0 = 0, time.perf_counter()
+    while True:
+        step()
+        n += 1
+        dt = time.perf_counter() - t0
+        if dt >= budget_s or n >= max_steps:
+            break
+    return {"value": toks * n / dt, "unit": UNIT, "cores": cores, "kind": "oracle",
+            "sample": f"{desc}; {n} steps in {dt:.1f} s"}
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    step, toks, desc, cores = oracle_step_runner(args.config, args.budget)
+    for _ in range(max(args.warmup, 1)):
+        step()
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        step()
+    dt = time.perf_counter() - t0
+    val = toks * args.steps / dt
+    line = {"impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * dt / args.steps,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": f"config {args.config} at {args.budget} bits/elem, bounded sample: {desc}"},
+            "cpu_baseline": {"value": val, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": desc},
+            "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+# --------------------------------------------------------------------------------- GPU leg
+
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+
+    import paper_2609_19880_b200 as dq
+    from paper_2609_19880_b200 import _build, workloads
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the library has no CPU path")
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    if not os.path.exists(dq.LIB_PATH):
+        _build.build()
+    dq.lib()
+    dev = torch.device("cuda", local)
+    hbm_peak, sm_max_mhz, peak_kind = _peaks()
+
+    cfg = workloads.make_config(args.config, budget=args.budget)
+    w = workloads.generate(cfg, device=dev)
+    B, Hq, Hkv = cfg.batch, cfg.hq, cfg.hkv
+    tk = dq.dq_build_tables(cfg.k_levels, cfg.bits_k, alpha=cfg.alpha, has_mean=True, rotate=True)
+    tv = dq.dq_build_tables(cfg.v_levels, cfg.bits_v, alpha=cfg.alpha, has_mean=False, rotate=True)
+    sm_scale = 1.0 / math.sqrt(128.0)
+
+    token_heads = cfg.total_tokens * Hkv
+    cache_bytes = token_heads * (cfg.k_rec + cfg.v_rec) + B * w.max_windows * Hkv * 132
+    copies = max(2, math.ceil(2.2 * L2_BYTES / cache_bytes)) if cache_bytes < 2 * L2_BYTES else 1
+
+    def new_cache():
+        return dict(
+            k=torch.zeros((w.num_pages, Hkv, 16, cfg.k_rec), dtype=torch.uint8, device=dev),
+            v=torch.zeros((w.num_pages, Hkv, 16, cfg.v_rec), dtype=torch.uint8, device=dev),
+            mq=torch.zeros((B, w.max_windows, Hkv, 128), dtype=torch.int8, device=dev),
+            ms=torch.zeros((B, w.max_windows, Hkv), dtype=torch.float32, device=dev))
+
+    # ---- prefill encode (timed once; also fills the cache the decode steps read)
+    caches = [new_cache()]
+    c0 = caches[0]
+    dq.dq_encode_tokens(tk, tv, w.k, w.v, w.seq_id, w.pos, w.slot, c0["k"], c0["v"], c0["mq"], c0["ms"])
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    dq.dq_encode_tokens(tk, tv, w.k, w.v, w.seq_id, w.pos, w.slot, c0["k"], c0["v"], c0["mq"], c0["ms"])
+    e1.record()
+    torch.cuda.synchronize()
+    enc_ms = e0.elapsed_time(e1)
+    for _ in range(copies - 1):
+        caches.append({k: v.clone() for k, v in c0.items()})
+
+    # ---- the step's inputs: q and one new token per sequence (the last position)
+    lens = torch.tensor(cfg.seq_lens, dtype=torch.int64)
+    last_idx = (torch.cumsum(lens, 0) - 1).to(dev)
+    new_k, new_v = w.k[last_idx].contiguous(), w.v[last_idx].contiguous()
+    new_seq, new_pos, new_slot = (t[last_idx].contiguous() for t in (w.seq_id, w.pos, w.slot))
+    out = torch.empty((B, Hq, 128), dtype=torch.bfloat16, device=dev)
+    ws = torch.empty(dq.dq_decode_workspace_bytes(B, Hq, w.page_table.shape[1]), dtype=torch.uint8, device=dev)
+    kv_tokens = cfg.total_tokens
+
+    def step(i, q=w.q, nk=new_k, nv=new_v):
+        c = caches[i % copies]
+        dq.dq_encode_tokens(tk, tv, nk, nv, new_seq, new_pos, new_slot, c["k"], c["v"], c["mq"], c["ms"],
+                            dq.MEAN_REUSE)
+        dq.dq_decode_attention(tk, tv, q, c["k"], c["v"], c["mq"], c["ms"], w.page_table, w.seq_lens, Hkv,
+                               sm_scale, out, ws)
+    launches_per_step = 6   # mean carry-forward, encode K, encode V, prepare, fused attention, combine
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    sampler = ClockSampler(local)
+    sampler.start()
+    for i in range(max(args.warmup, 3)):
+        step(i)
+    barrier()
+
+    # ---- timed region: exactly K steps, CUDA events on the launch stream
+    dq.dq_profile_enable(True)
+    t_wall0 = time.time()
+    e0.record()
+    for i in range(args.steps):
+        step(i)
+    e1.record()
+    barrier()
+    t_wall1 = time.time()
+    total_ms = e0.elapsed_time(e1)
+    kern_ms = dq.dq_profile_read(4096)
+    dq.dq_profile_enable(False)
+    if world > 1:
+        t = torch.tensor([total_ms], device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms = float(t.item())
+    ms_per_step = total_ms / args.steps
+    value = world * kv_tokens / (ms_per_step * 1e-3)
+
+    if args.profile_only:   # short run for an ncu capture: no soak, no e2e, no baselines
+        sampler.stop()
+        if rank == 0:
+            print(json.dumps({"profile_only": True, "ms_per_step": ms_per_step,
+                              "kernel_ms": statistics.mean(kern_ms) if kern_ms else None}), flush=True)
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    # keep the same load running briefly so the clock sampler sees it (not part of any number)
+    if t_wall1 - t_wall0 < 0.5:
+        t_end = time.time() + 0.6
+        i = 0
+        while time.time() < t_end:
+            for _ in range(50):
+                step(i); i += 1
+            torch.cuda.synchronize()
+        t_wall1 = time.time()
+    sampler.stop()
+    clocks = sampler.summary(t_wall0, t_wall1)
+
+    # ---- end to end: host buffers in, host buffer out, every step
+    hq = w.q.cpu().pin_memory()
+    hk, hv = new_k.cpu().pin_memory(), new_v.cpu().pin_memory()
+    hout = torch.empty((B, Hq, 128), dtype=torch.bfloat16).pin_memory()
+    dq_q, dk, dv = torch.empty_like(w.q), torch.empty_like(new_k), torch.empty_like(new_v)
+    h2d = hq.numel() * 2 + hk.numel() * 2 + hv.numel() * 2
+    d2h = hout.numel() * 2
+
+    def e2e_step(i):
+        dq_q.copy_(hq, non_blocking=True)
+        dk.copy_(hk, non_blocking=True)
+        dv.copy_(hv, non_blocking=True)
+        step(i, dq_q, dk, dv)
+        hout.copy_(out, non_blocking=True)
+        torch.cuda.synchronize()
+
+    for i in range(3):
+        e2e_step(i)
+    barrier()
+    t0 = time.perf_counter()
+    for i in range(args.steps):
+        e2e_step(i)
+    barrier()
+    e2e_s = time.perf_counter() - t0
+    if world > 1:
+        t = torch.tensor([e2e_s], device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_s = float(t.item())
+    e2e_value = world * kv_tokens * args.steps / e2e_s
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    # ---- roofline of the dominant kernel (fused decode attention)
+    k_ms = statistics.mean(kern_ms) if kern_ms else None
+    symbols = token_heads * 256.0
+    comp_bytes = token_heads * (cfg.k_rec + cfg.v_rec + 1.0)   # records + amortised INT8 mean byte
+    roofline = None
+    extra = {}
+    if k_ms:
+        alu_peak = SM_COUNT * LANES_PER_SM_CLK * sm_max_mhz * 1e6 / 1e9          # G lane-ops / s
+        alu_ach = symbols * ALU_OPS_PER_SYMBOL / (k_ms * 1e-3) / 1e9
+        gbs = comp_bytes / (k_ms * 1e-3) / 1e9
+        roofline = {"bound": "alu", "achieved": alu_ach, "peak": alu_peak, "unit": "Gop/s (int32 lane ops)",
+                    "frac": alu_ach / alu_peak, "traffic": args.traffic_bytes,
+                    "kernel": "dq_attention_kernel", "kernel_ms": k_ms, "launches_timed": len(kern_ms),
+                    "peak_source": f"148 SM x 128 lanes x {sm_max_mhz:.0f} MHz ({peak_kind} clocks)",
+                    "ops_per_symbol": ALU_OPS_PER_SYMBOL}
+        extra = {"hbm": {"bound": "hbm", "achieved": gbs, "peak": hbm_peak, "unit": "GB/s", "frac": gbs / hbm_peak,
+                         "frac_of_8TBps": gbs / 8000.0, "peak_source": peak_kind,
+                         "bytes_per_token_head": cfg.k_rec + cfg.v_rec + 1},
+                 "kernel_token_heads_per_s": token_heads / (k_ms * 1e-3),
+                 "kernel_symbols_per_s": symbols / (k_ms * 1e-3)}
+
+    # ---- bf16-cache baseline on the same GPU (context)
+    bf16 = None
+    try:
+        kp = torch.zeros((w.num_pages * 16, Hkv, 128), dtype=torch.bfloat16, device=dev)
+        vp = torch.zeros_like(kp)
+        kp[w.slot.long()] = w.k
+        vp[w.slot.long()] = w.v
+        kp = kp.view(w.num_pages, 16, Hkv, 128).transpose(1, 2).contiguous()
+        vp = vp.view(w.num_pages, 16, Hkv, 128).transpose(1, 2).contiguous()
+        bcopies = max(1, math.ceil(2.2 * L2_BYTES / (kp.numel() * 4)))
+        kps, vps = [kp] + [kp.clone() for _ in range(bcopies - 1)], [vp] + [vp.clone() for _ in range(bcopies - 1)]
+        for i in range(3):
+            dq.dq_bf16_decode_attention(w.q, kps[i % bcopies], vps[i % bcopies], w.page_table, w.seq_lens, Hkv,
+                                        sm_scale, out, ws)
+        torch.cuda.synchronize()
+        nb = 50
+        e0.record()
+        for i in range(nb):
+            dq.dq_bf16_decode_attention(w.q, kps[i % bcopies], vps[i % bcopies], w.page_table, w.seq_lens, Hkv,
+                                        sm_scale, out, ws)
+        e1.record()
+        torch.cuda.synchronize()
+        bms = e0.elapsed_time(e1) / nb
+        bf16 = {"ms_per_call": bms, "kv_tokens_per_s": kv_tokens / (bms * 1e-3),
+                "gb_per_s": token_heads * 512.0 / (bms * 1e-3) / 1e9, "bytes_per_token_head": 512}
+        del kps, vps, kp, vp
+    except Exception as ex:  # the baseline is context only
+        bf16 = {"error": str(ex)}
+
+    cpu = None
+    if world == 1 and not args.no_cpu_baseline:
+        cpu = time_oracle(args.config, args.budget)
+
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
+        "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "u32 rANS state / f16 mma, f32 accumulate", "data": "synthetic",
+        "config": {"workload": cfg.name, "batch": B, "q_heads": Hq, "kv_heads": Hkv, "head_dim": 128,
+                   "context": cfg.seq_lens if len(set(cfg.seq_lens)) > 1 and B <= 8 else
+                   {"min": min(cfg.seq_lens), "max": max(cfg.seq_lens), "sum": kv_tokens},
+                   "bits_per_elem": args.budget, "k_rec_bytes": cfg.k_rec, "v_rec_bytes": cfg.v_rec,
+                   "k_levels": cfg.k_levels, "v_levels": cfg.v_levels,
+                   "step": "encode 1 new token per sequence + decode attention over the whole cache",
+                   "l2": f"{copies} rotating copies of the cache ({copies * cache_bytes / 2**20:.0f} MiB > 126 MiB L2)",
+                   "parallelism": "replicas only" if world > 1 else "single GPU"},
+        "roofline": roofline, "cpu_baseline": cpu,
+        "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
+        "gpu_launches": launches_per_step * args.steps, "clocks": clocks,
+        "encoder": {"token_heads_per_s": 2 * token_heads / (enc_ms * 1e-3), "prefill_ms": enc_ms,
+                    "streams": 2 * token_heads},
+        "bf16_baseline": bf16,
+    }
+    line.update(extra)
+    print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--config", type=int, default=2, choices=[2, 3, 4, 5])
+    ap.add_argument("--budget", type=float, default=2.26)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--profile-only", action="store_true",
+                    help="warm-up and timed steps only (for profiler captures); prints a short line")
+    ap.add_argument("--traffic-bytes", type=float, default=None,
+                    help="DRAM bytes per launch of the fused kernel from an ncu capture (reported as-is)")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -77,7 +77,7 @@ typedef struct {
     int32_t c[DQ_MAX_LEVELS + 1];  /* cumulative frequencies          */
     float r[DQ_MAX_LEVELS];        /* -log2(f/256), bits (Algorithm 1) */
     uint32_t R[DQ_MAX_LEVELS];     /* ceil(r * 65536)                  */
-    uint32_t lut[256];             /* (fp16 bits of level) << 16 | f << 8 | (z - c) */
+    uint32_t lut[256];             /* f << 24 | (fp16 bits of level) << 8 | (z - c) */
 } dq_table_info;
 
 /* Probability model and rANS tables of one tensor kind (Sec. 3.1 "Entropy Coding",
@@ -151,6 +151,13 @@ int dq_bf16_decode_attention(const void *q_bf16, const void *k_bf16_pages, const
                              const int32_t *page_table, int max_pages, const int32_t *seq_lens,
                              int B, int Hq, int Hkv, float sm_scale, void *out_bf16,
                              void *workspace, size_t workspace_bytes, void *cuda_stream);
+
+/* Measurement aid (no counterpart in the paper): while enabled, every dq_decode_attention
+ * call records CUDA events on its stream around the fused kernel (up to 4096 calls).
+ * dq_profile_read waits for them, writes the kernel durations in milliseconds (host array,
+ * call order) and clears the record; returns how many it wrote.  Not thread-safe. */
+void dq_profile_enable(int on);
+int dq_profile_read(float *ms_out, int max_records);
 
 const char *dq_strerror(int code);
 /* Text of the last CUDA error seen by this thread's calls ("" if none). */

@@ -24,7 +24,8 @@ ERRORS = {0: "DQ_OK", -1: "DQ_ERR_ARG", -2: "DQ_ERR_INFEASIBLE", -3: "DQ_ERR_UNS
 
 EXPORTS = ["dq_build_tables", "dq_free_tables", "dq_tables_info", "dq_encode_tokens",
            "dq_decode_workspace_bytes", "dq_decode_attention", "dq_decode_tokens",
-           "dq_bf16_decode_attention", "dq_strerror", "dq_last_cuda_error"]
+           "dq_bf16_decode_attention", "dq_profile_enable", "dq_profile_read", "dq_strerror",
+           "dq_last_cuda_error"]
 
 
 class DqError(RuntimeError):
@@ -74,6 +75,10 @@ def lib():
         L.dq_decode_tokens.argtypes = [vp, vp, vp, vp, i32, vp, vp, vp, i32, i32, vp, vp, vp]
         L.dq_bf16_decode_attention.restype = i32
         L.dq_bf16_decode_attention.argtypes = [vp, vp, vp, vp, i32, vp, i32, i32, i32, f32, vp, vp, sz, vp]
+        L.dq_profile_enable.restype = None
+        L.dq_profile_enable.argtypes = [i32]
+        L.dq_profile_read.restype = i32
+        L.dq_profile_read.argtypes = [C.POINTER(C.c_float), i32]
         L.dq_strerror.restype = C.c_char_p
         L.dq_strerror.argtypes = [i32]
         L.dq_last_cuda_error.restype = C.c_char_p
@@ -183,3 +188,14 @@ def dq_bf16_decode_attention(q_bf16, k_pages, v_pages, page_table, seq_lens, Hkv
                                         _ptr(out_bf16), _ptr(workspace),
                                         int(workspace.numel() * workspace.element_size()), _stream(stream))
     _check(rc, "dq_bf16_decode_attention")
+
+
+def dq_profile_enable(on: bool):
+    lib().dq_profile_enable(int(bool(on)))
+
+
+def dq_profile_read(max_records: int = 4096):
+    """Durations (ms) of the fused attention kernel for the calls made since enabling."""
+    buf = (C.c_float * max_records)()
+    n = lib().dq_profile_read(buf, max_records)
+    return [float(buf[i]) for i in range(n)]

@@ -158,6 +158,13 @@ int dq_bf16_decode_attention(const void* q_bf16, const void* k_bf16_pages, const
     return DQ_OK;
 }
 
+void dq_profile_enable(int on) { dq_attn_profile_enable(on); }
+
+int dq_profile_read(float* ms_out, int max_records) {
+    if (!ms_out || max_records <= 0) return 0;
+    return dq_attn_profile_read(ms_out, max_records);
+}
+
 const char* dq_strerror(int code) {
     switch (code) {
         case DQ_OK: return "ok";

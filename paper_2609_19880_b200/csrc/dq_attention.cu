@@ -7,18 +7,22 @@
 //   dq_attention_kernel      persistent, one CTA per SM; CTAs pull work items
 //                            (sequence, KV head, block of NW*32 tokens) from an atomic
 //                            counter.  Each warp owns 32 tokens of the item: lane l runs the
-//                            rANS state machines of token l (K stream, then V stream) out of
-//                            shared memory, levels go to a small fp16 tile and from there
-//                            into mma.sync contractions against q' (K) and the softmax
-//                            weights (V).  s, o and the window mean are applied after the
-//                            contraction.  The next item's records are prefetched with
-//                            cp.async while the current one is decoded.
-//   dq_attn_combine_kernel   log-sum-exp merge of the per-block partials, inverse rotation
+//                            rANS state machine of token l out of shared memory, levels go to
+//                            a small fp16 tile and from there into mma.sync contractions
+//                            against q' (keys) and the softmax weights (values).  s, o and
+//                            the window mean are applied after the contraction.  The loop is
+//                            software-pipelined across items: while a warp decodes the K
+//                            streams of item n it also decodes the V streams of item n-1
+//                            (whose softmax weights are known), two independent dependency
+//                            chains per lane; records of item n+1 arrive by cp.async.
+//   dq_attn_combine_kernel   log-sum-exp merge of the per-item partials, inverse rotation
 //                            of the output when V was rotated, bf16 / f32 store.
 //
-// q' and the softmax weights enter the tensor cores as fp16 hi + lo pairs (rows g and g + 8
-// of the 16-row operand), so the contraction carries ~22 mantissa bits; levels 0..15 are
-// exact in fp16.
+// The integer ALU pipe (half rate) is what binds the decode, so the per-symbol step is
+// written to spread work over the pipes: table address and field extraction by dp4a (FMA
+// pipe), renormalisation byte merged by one byte-permute, selector bumped by a mad.
+// q' and the softmax weights enter the tensor cores as fp16 hi + lo pairs, so the
+// contractions carry ~22 mantissa bits; levels 0..15 are exact in fp16.
 #include <cuda_bf16.h>
 #include <cuda_fp16.h>
 
@@ -31,45 +35,47 @@ namespace {
 
 constexpr int kN = DQ_HEAD_DIM;
 constexpr int kChunk = 32;             // tokens per warp per item
-constexpr uint32_t kL = 1u << 23;
-constexpr int kTileStride = 48;        // bytes per token row of a [32 tok][16 ch] fp16 tile (+16 pad)
+constexpr int kTileStride = 48;        // bytes per token row of a [32 tok][16 ch] fp16 tile; the
+                                       // 16 pad bytes of the K tile rows hold (sK, oK, sV, oV)
 constexpr int kTileBytes = kChunk * kTileStride;
 constexpr int kQ16Stride = 272;        // bytes per row of the fp16 q' operand (128 halves + pad)
-constexpr int kPartial = 132;          // floats per partial record: 128 acc, m, l, 2 pad
-constexpr int kMergeStride = 136;      // floats per (slot, head) row of the merge buffer
+constexpr int kQ16Bytes = 16 * kQ16Stride;
+constexpr int kPartial = 132;          // floats per partial record: 128 acc, m, l, off, pad
+constexpr int kORow = 132;             // floats per head row of a warp's output slot
 constexpr int kMaxWarps = 16;
-constexpr int kMaxPerThread = DQ_MAX_GROUP * kN / 128;  // merge outputs per thread at 4 warps
+constexpr int kKTail = 32;             // bytes after a warp's K records: q'.mean of its window, per head
 
 struct Item {
     int b, h, blk, len, bg, valid, pad0, pad1;
 };
 
 struct Layout {
-    int stage_k, stage_v, stage_bytes;  // per warp per buffer
-    int off_lutk, off_lutv, off_prefix, off_qf32, off_q16, off_qsum, off_item, off_red, off_stage,
-        off_tiles, total;
-    int warp_tile_bytes;
+    int stage_k, stage_v;               // bytes of one warp's K (+ tail) / V record buffer
+    int off_lutk, off_lutv, off_prefix, off_q16, off_qsum, off_item, off_red, off_kst, off_vst, off_tiles,
+        off_obuf, total;
+    int warp_tile_bytes, warp_obuf_bytes;
 };
 
 __host__ __device__ inline int align16(int x) { return (x + 15) & ~15; }
 
-__host__ __device__ inline Layout make_layout(int nw, int rec_k, int rec_v, int B) {
+__host__ __device__ inline Layout make_layout(int nw, int rec_k, int rec_v, int B, int G) {
     Layout L;
-    L.stage_k = align16(kChunk * rec_k);
+    L.stage_k = align16(kChunk * rec_k) + kKTail;
     L.stage_v = align16(kChunk * rec_v);
-    L.stage_bytes = L.stage_k + L.stage_v + kN + 16;  // + INT8 mean row + its scale
-    L.warp_tile_bytes = 2 * kTileBytes + kChunk * 16;  // K tile, V tile, per-token (sK,oK,sV,oV)
+    L.warp_tile_bytes = 2 * kTileBytes;             // K tile (+ per-token metadata), V tile
+    L.warp_obuf_bytes = G * kORow * 4;              // this warp's O[g][channel], l, off
     int o = 0;
     L.off_lutk = o; o += 256 * 32 * 4;
     L.off_lutv = o; o += 256 * 32 * 4;
     L.off_prefix = o; o += align16((B + 1) * 4);
-    L.off_qf32 = o; o += 2 * DQ_MAX_GROUP * kN * 4;
-    L.off_q16 = o; o += 16 * kQ16Stride;
-    L.off_qsum = o; o += DQ_MAX_GROUP * 4;
-    L.off_item = o; o += 2 * (int)sizeof(Item);
-    L.off_red = o; o += 3 * kMaxWarps * DQ_MAX_GROUP * 4;
-    L.off_stage = o; o += 2 * nw * L.stage_bytes;
+    L.off_q16 = o; o += 2 * kQ16Bytes;
+    L.off_qsum = o; o += 2 * DQ_MAX_GROUP * 4;
+    L.off_item = o; o += 3 * (int)sizeof(Item);
+    L.off_red = o; o += (kMaxWarps + 1) * DQ_MAX_GROUP * 4;
+    L.off_kst = o; o += 2 * nw * L.stage_k;
+    L.off_vst = o; o += 2 * nw * L.stage_v;
     L.off_tiles = o; o += nw * L.warp_tile_bytes;
+    L.off_obuf = o; o += nw * L.warp_obuf_bytes;
     L.total = o + 256;  // slack: a malformed record may be over-read by up to 136 + 8 bytes
     return L;
 }
@@ -83,27 +89,71 @@ struct AttnParams {
     const int32_t* page_table;
     const int32_t* seq_lens;
     int* counter;
-    int* prefix;      // [B + 1] blocks before sequence b
-    float* qrot;      // [B][Hq][128]
-    float* partial;   // [blocks][Hq][kPartial]
+    int* prefix;        // [B + 1] blocks before sequence b
+    float* qrot;        // [B][Hq][128]              rotated q (bf16 baseline reads q itself)
+    uint16_t* q16;      // [B][Hkv][16][128] halves  fp16 hi (rows g) / lo (rows 8 + g) of q'
+    float* qsum;        // [B][Hq]                   sum_j q'_j
+    float* qmu;         // [B][Hq][windows]          sum_j q'_j mean_j of every window
+    float* partial;     // [blocks][Hq][kPartial]
     void* out_bf16;
     float* out_f32;
-    int max_windows, max_pages, B, Hq, Hkv, G, item_tokens, rotate_q, rotate_out;
-    float scale_log2;  // sm_scale * log2(e)
+    int max_windows, windows, max_pages, B, Hq, Hkv, G, item_tokens, rotate_q, rotate_out, has_mean;
+    float scale_log2;   // sm_scale * log2(e)
 };
 
 // ------------------------------------------------------------------ prepare
 
+// Warp roles: [0, B*Hq): rotate q, emit the fp16 hi/lo operand rows and the row sum;
+// [B*Hq, B*Hq*(1+windows)): q' . mean of one (head, window) (Eq. fold-key, third term);
+// block 0 additionally scans the blocks per sequence and resets the work counter.
 __global__ void __launch_bounds__(256)
 dq_attn_prepare_kernel(AttnParams p) {
     const int lane = threadIdx.x & 31;
-    const int wid = blockIdx.x * 8 + (threadIdx.x >> 5);
-    if (wid < p.B * p.Hq) {
-        const uint2 raw = *reinterpret_cast<const uint2*>(p.q + (size_t)wid * kN + 4 * lane);
+    const long long wid = (long long)blockIdx.x * 8 + (threadIdx.x >> 5);
+    const int heads = p.B * p.Hq;
+    if (wid < (long long)heads * (1 + (p.has_mean ? p.windows : 0))) {
+        const int head = (int)(wid % heads), win = (int)(wid / heads) - 1;
+        const uint2 raw = *reinterpret_cast<const uint2*>(p.q + (size_t)head * kN + 4 * lane);
         float v[4] = {bf16_bits_to_float(raw.x & 0xffffu), bf16_bits_to_float(raw.x >> 16),
                       bf16_bits_to_float(raw.y & 0xffffu), bf16_bits_to_float(raw.y >> 16)};
         if (p.rotate_q) warp_fwht128(v, lane);
-        *reinterpret_cast<float4*>(p.qrot + (size_t)wid * kN + 4 * lane) = make_float4(v[0], v[1], v[2], v[3]);
+        const int b = head / p.Hq, hq = head % p.Hq, h = hq / p.G, g = hq % p.G;
+        if (win < 0) {
+            *reinterpret_cast<float4*>(p.qrot + (size_t)head * kN + 4 * lane) = make_float4(v[0], v[1], v[2], v[3]);
+            uint16_t* rows = p.q16 + ((size_t)b * p.Hkv + h) * 16 * kN;
+            __half hi[4], lo[4];
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                hi[e] = __float2half_rn(v[e]);
+                lo[e] = __float2half_rn(v[e] - __half2float(hi[e]));
+            }
+            uint2 w;
+            w.x = (uint32_t)__half_as_ushort(hi[0]) | ((uint32_t)__half_as_ushort(hi[1]) << 16);
+            w.y = (uint32_t)__half_as_ushort(hi[2]) | ((uint32_t)__half_as_ushort(hi[3]) << 16);
+            *reinterpret_cast<uint2*>(rows + (size_t)g * kN + 4 * lane) = w;
+            w.x = (uint32_t)__half_as_ushort(lo[0]) | ((uint32_t)__half_as_ushort(lo[1]) << 16);
+            w.y = (uint32_t)__half_as_ushort(lo[2]) | ((uint32_t)__half_as_ushort(lo[3]) << 16);
+            *reinterpret_cast<uint2*>(rows + (size_t)(8 + g) * kN + 4 * lane) = w;
+            if (g == 0)  // unused operand rows of this KV head are zero
+                for (int r = p.G; r < 8; ++r) {
+                    *reinterpret_cast<uint2*>(rows + (size_t)r * kN + 4 * lane) = make_uint2(0u, 0u);
+                    *reinterpret_cast<uint2*>(rows + (size_t)(8 + r) * kN + 4 * lane) = make_uint2(0u, 0u);
+                }
+            float s = (v[0] + v[1]) + (v[2] + v[3]);
+#pragma unroll
+            for (int d = 16; d >= 1; d >>= 1) s += __shfl_xor_sync(kFullMask, s, d);
+            if (lane == 0) p.qsum[head] = s;
+        } else {
+            const size_t mi = ((size_t)b * p.max_windows + win) * p.Hkv + h;
+            const uint32_t q4 = *reinterpret_cast<const uint32_t*>(p.mean_q + mi * kN + 4 * lane);
+            const float msc = p.mean_scale[mi];
+            float s = 0.f;
+#pragma unroll
+            for (int e = 0; e < 4; ++e) s = fmaf(v[e], msc * (float)(int)(int8_t)((q4 >> (8 * e)) & 0xffu), s);
+#pragma unroll
+            for (int d = 16; d >= 1; d >>= 1) s += __shfl_xor_sync(kFullMask, s, d);
+            if (lane == 0) p.qmu[(size_t)head * p.windows + win] = s;
+        }
     }
     if (blockIdx.x == 0 && threadIdx.x < 32) {  // exclusive scan of blocks per sequence
         int carry = 0;
@@ -126,32 +176,106 @@ dq_attn_prepare_kernel(AttnParams p) {
 
 // --------------------------------------------------------------------- main
 
+__device__ __forceinline__ uint32_t dp4a_u32(uint32_t a, uint32_t b, uint32_t c) {
+    uint32_t d;
+    asm("dp4a.u32.u32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
+    return d;
+}
+
 // Decode 16 symbols of one stream (Algorithm 2) and pack their levels as 8 fp16x2 words.
-// x: rANS state; ptr: shared-memory byte address of the next renormalisation byte;
-// lut: shared address of this lane's column of the 32-way replicated table (entry z at
-// lut + z * 128).  Renormalisation bytes come from a 4-byte window refreshed every 4 symbols
-// (a symbol consumes at most one byte).
-__device__ __forceinline__ void decode16(uint32_t& x, uint32_t& ptr, uint32_t lut, uint32_t (&packed)[8]) {
+//   x    rANS state;  ptr  shared-memory byte address of the next renormalisation byte
+//   lut  shared address of this lane's column of the 32-way replicated table: entry z at
+//        lut + 128 z, entry = f << 24 | fp16(level) << 8 | (z - c)
+//   one  the value 1 in a register (keeps the selector bump a multiply-add)
+// Per symbol: z = x mod 256 addresses the table (dp4a: 128 * byte0(x) + lut); x = f * (x >> 8)
+// + (z - c) (f by dp4a, product by mad, addend by dp4a); if x < L one byte is appended with a
+// byte-permute from a 4-byte window that is reloaded every 4 symbols (a symbol takes at most
+// one byte because the state stays >= 2^15).
+__device__ __forceinline__ void decode16(uint32_t& x, uint32_t& ptr, uint32_t lut, uint32_t one,
+                                         uint32_t (&packed)[8]) {
 #pragma unroll
     for (int q4 = 0; q4 < 4; ++q4) {
-        const uint32_t win = lds32_unaligned(ptr);
+        const uint32_t base = ptr & ~3u;
+        const uint32_t win = __funnelshift_r(lds32(base), lds32(base + 4), ptr << 3);
         uint32_t sel = 0x2104u;
         uint32_t e[4];
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
-            e[i] = lds32(lut + ((x & 255u) << 7));
-            x = ((e[i] >> 8) & 255u) * (x >> 8) + (e[i] & 255u);
-            if (x < kL) { x = __byte_perm(x, win, sel); sel += 1u; }
+            e[i] = lds32(dp4a_u32(x, 0x80u, lut));
+            const uint32_t f = dp4a_u32(e[i], 0x01000000u, 0u);
+            const uint32_t t = f * (x >> 8);
+            x = dp4a_u32(e[i], 1u, t);
+            asm("{.reg .pred p; setp.lt.u32 p, %0, 0x800000; @p prmt.b32 %0, %0, %2, %1; "
+                "@p mad.lo.u32 %1, %3, %3, %1;}"
+                : "+r"(x), "+r"(sel) : "r"(win), "r"(one));
         }
         ptr += sel - 0x2104u;
-        packed[2 * q4] = __byte_perm(e[0], e[1], 0x7632u);
-        packed[2 * q4 + 1] = __byte_perm(e[2], e[3], 0x7632u);
+        packed[2 * q4] = __byte_perm(e[0], e[1], 0x6521u);
+        packed[2 * q4 + 1] = __byte_perm(e[2], e[3], 0x6521u);
     }
 }
 
 __device__ __forceinline__ uint32_t pack_half2(float a, float b) {
     const __half2 h = __floats2half2_rn(a, b);
     return *reinterpret_cast<const uint32_t*>(&h);
+}
+
+__device__ __forceinline__ void sts128(uint32_t addr, const uint32_t* v) {
+    asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};\n" ::"r"(addr), "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3])
+                 : "memory");
+}
+__device__ __forceinline__ void sts32f(uint32_t addr, float v) {
+    asm volatile("st.shared.f32 [%0], %1;\n" ::"r"(addr), "f"(v) : "memory");
+}
+
+// One pass over the 128 channels, 16 at a time.  With DO_K the K streams of the current item
+// are decoded and S[g][t] = sum_j q'_gj level_tj accumulated (Eq. fold-key, inner sum).  With
+// DO_V the V streams of the previous item are decoded and each finished 16-channel tile of
+// O[j][g] = sum_t (a_t s_t) level_tj (Eq. fold-value, first sum) goes to this warp's output
+// slot in shared memory.  Both decodes are interleaved in one instruction stream.
+template <bool DO_K, bool DO_V>
+__device__ __forceinline__ void fused_pass(uint32_t xk, uint32_t ptrk, uint32_t xv, uint32_t ptrv, uint32_t lutk,
+                                           uint32_t lutv, uint32_t one, uint32_t ktile, uint32_t vtile, uint32_t q16,
+                                           uint32_t obuf, int lane, int G, float (&sacc)[4][4],
+                                           const uint32_t (&pb_hi)[2][2], const uint32_t (&pb_lo)[2][2]) {
+    const uint32_t a_addr = q16 + ((lane & 7) + ((lane >> 3) & 1) * 8) * kQ16Stride + (lane >> 4) * 16;
+    const uint32_t bk_addr = ktile + ((lane & 7) + (lane >> 4) * 8) * kTileStride + ((lane >> 3) & 1) * 16;
+    const uint32_t av_addr = vtile + ((lane & 7) + (lane >> 4) * 8) * kTileStride + ((lane >> 3) & 1) * 16;
+    // output slot: thread holds channels (lane/4, lane/4 + 8) of heads (2 qd, 2 qd + 1)
+    const uint32_t o_addr = obuf + ((2 * (lane & 3)) * kORow + (lane >> 2)) * 4;
+#pragma unroll 1
+    for (int cg = 0; cg < 8; ++cg) {
+        uint32_t pk[8], pv[8];
+        if (DO_K) decode16(xk, ptrk, lutk, one, pk);
+        if (DO_V) decode16(xv, ptrv, lutv, one, pv);
+        if (DO_K) { sts128(ktile + lane * kTileStride, pk); sts128(ktile + lane * kTileStride + 16, pk + 4); }
+        if (DO_V) { sts128(vtile + lane * kTileStride, pv); sts128(vtile + lane * kTileStride + 16, pv + 4); }
+        __syncwarp();
+        if (DO_K) {
+            uint32_t a[4], b0[4], b1[4];
+            ldmatrix_x4(a, a_addr + cg * 32);
+            ldmatrix_x4(b0, bk_addr);
+            ldmatrix_x4(b1, bk_addr + 16 * kTileStride);
+            mma_f16_16816(sacc[0], a, b0[0], b0[1]);
+            mma_f16_16816(sacc[1], a, b0[2], b0[3]);
+            mma_f16_16816(sacc[2], a, b1[0], b1[1]);
+            mma_f16_16816(sacc[3], a, b1[2], b1[3]);
+        }
+        if (DO_V) {
+            uint32_t a0[4], a1[4];
+            float o[4] = {0.f, 0.f, 0.f, 0.f};
+            ldmatrix_x4_trans(a0, av_addr);                      // tokens 0..15, 16 channels
+            ldmatrix_x4_trans(a1, av_addr + 16 * kTileStride);   // tokens 16..31
+            mma_f16_16816(o, a0, pb_hi[0][0], pb_hi[0][1]);
+            mma_f16_16816(o, a1, pb_hi[1][0], pb_hi[1][1]);
+            mma_f16_16816(o, a0, pb_lo[0][0], pb_lo[0][1]);
+            mma_f16_16816(o, a1, pb_lo[1][0], pb_lo[1][1]);
+            const uint32_t oa = o_addr + cg * 64;
+            if (2 * (lane & 3) < G) { sts32f(oa, o[0]); sts32f(oa + 32, o[2]); }
+            if (2 * (lane & 3) + 1 < G) { sts32f(oa + kORow * 4, o[1]); sts32f(oa + kORow * 4 + 32, o[3]); }
+        }
+        __syncwarp();
+    }
 }
 
 __global__ void __launch_bounds__(kMaxWarps * 32, 1)
@@ -161,19 +285,17 @@ dq_attention_kernel(const __grid_constant__ DqDevTable TK, const __grid_constant
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int nthreads = blockDim.x, nw = nthreads >> 5;
     const int G = p.G;
-    const Layout L = make_layout(nw, TK.rec, TV.rec, p.B);
+    const Layout L = make_layout(nw, TK.rec, TV.rec, p.B, G);
     const uint32_t sbase = smem_addr(smem);
 
     uint32_t* lutk = reinterpret_cast<uint32_t*>(smem + L.off_lutk);
     uint32_t* lutv = reinterpret_cast<uint32_t*>(smem + L.off_lutv);
     int* prefix = reinterpret_cast<int*>(smem + L.off_prefix);
-    float* qf32 = reinterpret_cast<float*>(smem + L.off_qf32);
-    float* qsum = reinterpret_cast<float*>(smem + L.off_qsum);
+    float* qsum = reinterpret_cast<float*>(smem + L.off_qsum);      // [2][8]
     Item* items = reinterpret_cast<Item*>(smem + L.off_item);
-    float* red_m = reinterpret_cast<float*>(smem + L.off_red);
-    float* red_l = red_m + kMaxWarps * DQ_MAX_GROUP;
-    float* red_o = red_l + kMaxWarps * DQ_MAX_GROUP;
-    float* mbuf = reinterpret_cast<float*>(smem + L.off_tiles);  // aliases the tiles between items
+    float* red_m = reinterpret_cast<float*>(smem + L.off_red);      // [warp][head], then [head] maxima
+    float* red_M = red_m + kMaxWarps * DQ_MAX_GROUP;
+    float* obuf_all = reinterpret_cast<float*>(smem + L.off_obuf);  // [warp][head][kORow]
 
     for (int i = tid; i < 256 * 32; i += nthreads) {
         lutk[i] = TK.lut[i >> 5];
@@ -184,11 +306,12 @@ dq_attention_kernel(const __grid_constant__ DqDevTable TK, const __grid_constant
     const int total_items = prefix[p.B] * p.Hkv;
 
     const uint32_t my_lutk = sbase + L.off_lutk + lane * 4, my_lutv = sbase + L.off_lutv + lane * 4;
-    const uint32_t my_tiles = sbase + L.off_tiles + warp * L.warp_tile_bytes;
-    const uint32_t ktile = my_tiles, vtile = my_tiles + kTileBytes, scal = my_tiles + 2 * kTileBytes;
-    const int merge_slots = (nw * L.warp_tile_bytes) / (G * kMergeStride * 4);
+    const uint32_t ktile = sbase + L.off_tiles + warp * L.warp_tile_bytes, vtile = ktile + kTileBytes;
+    const uint32_t my_obuf = sbase + L.off_obuf + warp * L.warp_obuf_bytes;
+    const uint32_t one = (sbase >> 31) | 1u;
+    const int g_row = lane >> 2, qd = lane & 3;
 
-    auto fetch_item = [&](int buf) {  // thread 0 only
+    auto fetch_item = [&](int slot) {  // thread 0 only
         Item it;
         it.valid = 0; it.b = it.h = it.blk = it.len = it.bg = 0; it.pad0 = it.pad1 = 0;
         const int idx = atomicAdd(p.counter, 1);
@@ -205,278 +328,185 @@ dq_attention_kernel(const __grid_constant__ DqDevTable TK, const __grid_constant
             it.blk = it.bg - prefix[lo];
             it.len = min(p.seq_lens[lo], p.max_pages * DQ_PAGE_TOKENS);
         }
-        items[buf] = it;
+        items[slot] = it;
     };
 
-    auto issue_loads = [&](int buf) {
-        const Item it = items[buf];
-        if (it.valid) {
-            const uint32_t stage = sbase + L.off_stage + (buf * nw + warp) * L.stage_bytes;
-            const int tok0 = (it.blk * nw + warp) * kChunk;
-            if (tok0 < it.len) {
-                const int32_t* pt = p.page_table + (size_t)it.b * p.max_pages + (tok0 >> 4);
-                const int npg = (tok0 + 16 < it.len) ? 2 : 1;
-                for (int pg = 0; pg < npg; ++pg) {
-                    const size_t page = (size_t)pt[pg] * p.Hkv + it.h;
-                    const uint8_t* ks = p.k_cont + page * (size_t)(16 * TK.rec);
-                    const uint8_t* vs = p.v_cont + page * (size_t)(16 * TV.rec);
-                    for (int i = lane; i < TK.rec; i += 32) cp_async16(stage + pg * 16 * TK.rec + i * 16, ks + i * 16);
-                    for (int i = lane; i < TV.rec; i += 32)
-                        cp_async16(stage + L.stage_k + pg * 16 * TV.rec + i * 16, vs + i * 16);
+    // cp.async of the K records, q'.mean values and q' operand of item `nk`, V records of item `nv`
+    auto issue_loads = [&](int nk, int nv) {
+        if (nk >= 0) {
+            const Item it = items[nk % 3];
+            if (it.valid) {
+                const uint32_t kst = sbase + L.off_kst + ((nk & 1) * nw + warp) * L.stage_k;
+                const int tok0 = (it.blk * nw + warp) * kChunk;
+                if (tok0 < it.len) {
+                    const int32_t* pt = p.page_table + (size_t)it.b * p.max_pages + (tok0 >> 4);
+                    const int npg = (tok0 + 16 < it.len) ? 2 : 1;
+                    for (int pg = 0; pg < npg; ++pg) {
+                        const uint8_t* ks = p.k_cont + ((size_t)pt[pg] * p.Hkv + it.h) * (size_t)(16 * TK.rec);
+                        for (int i = lane; i < TK.rec; i += 32) cp_async16(kst + pg * 16 * TK.rec + i * 16, ks + i * 16);
+                    }
+                    if (p.has_mean && lane < G)
+                        cp_async4(kst + L.stage_k - kKTail + lane * 4,
+                                  p.qmu + ((size_t)it.b * p.Hq + (size_t)it.h * G + lane) * p.windows +
+                                      tok0 / DQ_WINDOW_TOKENS);
                 }
-                if (TK.has_mean) {
-                    const size_t mi = ((size_t)it.b * p.max_windows + tok0 / DQ_WINDOW_TOKENS) * p.Hkv + it.h;
-                    if (lane < 8) cp_async16(stage + L.stage_k + L.stage_v + lane * 16, p.mean_q + mi * kN + lane * 16);
-                    if (lane == 8) cp_async4(stage + L.stage_k + L.stage_v + kN, p.mean_scale + mi);
+                const uint16_t* qsrc = p.q16 + ((size_t)it.b * p.Hkv + it.h) * 16 * kN;
+                for (int i = tid; i < 16 * 16; i += nthreads)  // 16 rows x 16 chunks of 16 bytes
+                    cp_async16(sbase + L.off_q16 + (nk & 1) * kQ16Bytes + (i >> 4) * kQ16Stride + (i & 15) * 16,
+                               qsrc + i * 8);
+                if (tid < G)
+                    cp_async4(sbase + L.off_qsum + ((nk & 1) * DQ_MAX_GROUP + tid) * 4,
+                              p.qsum + (size_t)it.b * p.Hq + (size_t)it.h * G + tid);
+            }
+        }
+        if (nv >= 0) {
+            const Item it = items[nv % 3];
+            if (it.valid) {
+                const uint32_t vst = sbase + L.off_vst + ((nv & 1) * nw + warp) * L.stage_v;
+                const int tok0 = (it.blk * nw + warp) * kChunk;
+                if (tok0 < it.len) {
+                    const int32_t* pt = p.page_table + (size_t)it.b * p.max_pages + (tok0 >> 4);
+                    const int npg = (tok0 + 16 < it.len) ? 2 : 1;
+                    for (int pg = 0; pg < npg; ++pg) {
+                        const uint8_t* vs = p.v_cont + ((size_t)pt[pg] * p.Hkv + it.h) * (size_t)(16 * TV.rec);
+                        for (int i = lane; i < TV.rec; i += 32) cp_async16(vst + pg * 16 * TV.rec + i * 16, vs + i * 16);
+                    }
                 }
             }
-            for (int i = tid; i < G * 32; i += nthreads)  // q' rows of this KV head's group
-                cp_async16(sbase + L.off_qf32 + buf * (DQ_MAX_GROUP * kN * 4) + i * 16,
-                           p.qrot + ((size_t)it.b * p.Hq + (size_t)it.h * G) * kN + i * 4);
         }
         cp_async_commit();
     };
 
-    int buf = 0;
     if (tid == 0) fetch_item(0);
     __syncthreads();
-    issue_loads(0);
+    issue_loads(0, -1);
 
-    const int g_row = lane >> 2, qd = lane & 3;
+    // state carried from the item whose V streams are still to be decoded
+    bool have_prev = false;
+    Item prev = items[0];
+    uint32_t pb_hi[2][2] = {{0u, 0u}, {0u, 0u}}, pb_lo[2][2] = {{0u, 0u}, {0u, 0u}};
 
-    while (true) {
-        const Item it = items[buf];
-        if (!it.valid) break;
-        if (tid == 0) fetch_item(buf ^ 1);
+    for (int n = 0;; ++n) {
+        const Item cur = items[n % 3];
+        if (!cur.valid && !have_prev) break;
+        if (tid == 0) {
+            if (cur.valid) fetch_item((n + 1) % 3);
+            else items[(n + 1) % 3].valid = 0;
+        }
         __syncthreads();
-        issue_loads(buf ^ 1);
+        issue_loads(n + 1, cur.valid ? n : -1);
         cp_async_wait<1>();
         __syncthreads();
 
-        // fp16 hi/lo operand of q' (rows g: hi, rows 8 + g: lo) and row sums
-        {
-            const float* qf = qf32 + buf * (DQ_MAX_GROUP * kN);
-            for (int i = tid; i < 8 * kN; i += nthreads) {
-                const int g = i >> 7, ch = i & (kN - 1);
-                float v = (g < G) ? qf[g * kN + ch] : 0.f;
-                const __half hi = __float2half_rn(v);
-                const __half lo = __float2half_rn(v - __half2float(hi));
-                *reinterpret_cast<__half*>(smem + L.off_q16 + g * kQ16Stride + ch * 2) = hi;
-                *reinterpret_cast<__half*>(smem + L.off_q16 + (g + 8) * kQ16Stride + ch * 2) = lo;
-            }
-            for (int g = warp; g < DQ_MAX_GROUP; g += nw) {
-                float s = 0.f;
-                if (g < G) {
-                    const float4 v = *reinterpret_cast<const float4*>(qf + g * kN + 4 * lane);
-                    s = (v.x + v.y) + (v.z + v.w);
-                }
+        // ------------------------------------------ K streams of `cur`, V streams of `prev`
+        const int tok0 = (cur.blk * nw + warp) * kChunk;
+        const uint32_t kst = sbase + L.off_kst + ((n & 1) * nw + warp) * L.stage_k;
+        const uint32_t vst_prev = sbase + L.off_vst + (((n + 1) & 1) * nw + warp) * L.stage_v;
+        const uint32_t rk = kst + lane * TK.rec, rvp = vst_prev + lane * TV.rec;
+        const uint32_t q16 = sbase + L.off_q16 + (n & 1) * kQ16Bytes;
+        float sacc[4][4];
 #pragma unroll
-                for (int d = 16; d >= 1; d >>= 1) s += __shfl_xor_sync(kFullMask, s, d);
-                if (lane == 0) qsum[g] = s;
+        for (int i = 0; i < 4; ++i) { sacc[i][0] = sacc[i][1] = sacc[i][2] = sacc[i][3] = 0.f; }
+        {
+            const uint32_t xk = lds32_unaligned(rk + 4), xv = lds32_unaligned(rvp + 4);
+            if (cur.valid && have_prev)
+                fused_pass<true, true>(xk, rk + 8, xv, rvp + 8, my_lutk, my_lutv, one, ktile, vtile, q16, my_obuf, lane, G,
+                                       sacc, pb_hi, pb_lo);
+            else if (cur.valid)
+                fused_pass<true, false>(xk, rk + 8, xv, rvp + 8, my_lutk, my_lutv, one, ktile, vtile, q16, my_obuf, lane, G,
+                                        sacc, pb_hi, pb_lo);
+            else
+                fused_pass<false, true>(xk, rk + 8, xv, rvp + 8, my_lutk, my_lutv, one, ktile, vtile, q16, my_obuf, lane, G,
+                                        sacc, pb_hi, pb_lo);
+        }
+
+        // ------------------------------------------ finish `prev`: sum its warps' slots, write the partial
+        if (have_prev) {
+            __syncthreads();
+            for (int e = tid; e < G * 130; e += nthreads) {
+                const int g = e / 130, col = e - g * 130;
+                float s = 0.f;
+                for (int w = 0; w < nw; ++w) s += obuf_all[(w * G + g) * kORow + col];
+                float* dst = p.partial + ((size_t)prev.bg * p.Hq + (size_t)prev.h * G + g) * kPartial;
+                if (col < kN) dst[col] = s;
+                else dst[col + 1] = s;                       // l at 129, off at 130
+                if (col == 0) dst[kN] = red_M[g];
             }
         }
-        __syncthreads();
 
-        // ------------------------------------------------ this warp's 32 tokens
-        float oacc[16][4];
-#pragma unroll
-        for (int i = 0; i < 16; ++i) { oacc[i][0] = oacc[i][1] = oacc[i][2] = oacc[i][3] = 0.f; }
-        float m_run = -INFINITY, l_run = 0.f, off_run = 0.f;
-
-        const int tok0 = (it.blk * nw + warp) * kChunk;
-        if (tok0 < it.len) {
-            const uint32_t stage = sbase + L.off_stage + (buf * nw + warp) * L.stage_bytes;
-            const uint32_t rk = stage + lane * TK.rec, rv = stage + L.stage_k + lane * TV.rec;
-            const uint32_t hk = lds32_unaligned(rk), hv = lds32_unaligned(rv);
-            uint32_t xk = lds32_unaligned(rk + 4), xv = lds32_unaligned(rv + 4);
+        // ------------------------------------------ softmax weights of `cur` (base 2)
+        have_prev = cur.valid;
+        if (cur.valid) {
+            prev = cur;
+            cp_async_wait<0>();   // the V records of `cur` (header needed now) have landed
+            __syncwarp();
+            const uint32_t rv = sbase + L.off_vst + ((n & 1) * nw + warp) * L.stage_v + lane * TV.rec;
             {
+                const uint32_t hk = lds32_unaligned(rk), hv = lds32_unaligned(rv);
                 const float sK = __half2float(__ushort_as_half((unsigned short)(hk & 0xffffu)));
                 const float oK = __half2float(__ushort_as_half((unsigned short)(hk >> 16)));
                 const float sV = __half2float(__ushort_as_half((unsigned short)(hv & 0xffffu)));
                 const float oV = __half2float(__ushort_as_half((unsigned short)(hv >> 16)));
-                asm volatile("st.shared.v4.f32 [%0], {%1,%2,%3,%4};\n" ::"r"(scal + lane * 16), "f"(sK), "f"(oK),
-                             "f"(sV), "f"(oV) : "memory");
+                asm volatile("st.shared.v4.f32 [%0], {%1,%2,%3,%4};\n" ::"r"(ktile + lane * kTileStride + 32), "f"(sK),
+                             "f"(oK), "f"(sV), "f"(oV) : "memory");
             }
-            // q' . mean of this chunk's window, for the head row this thread owns
-            float qmu = 0.f;
-            if (TK.has_mean) {
-                const uint32_t mrow = stage + L.stage_k + L.stage_v;
-                const uint32_t q4 = lds32(mrow + lane * 4);
-                const float msc = __uint_as_float(lds32(mrow + kN));
-                float mu[4];
+            float qmu = 0.f, qs = 0.f;   // q' . window mean and sum of q', for the head row this thread owns
+            if (g_row < G) {
+                qs = qsum[(n & 1) * DQ_MAX_GROUP + g_row];
+                if (p.has_mean && tok0 < cur.len) qmu = __uint_as_float(lds32(kst + L.stage_k - kKTail + g_row * 4));
+            }
+            __syncwarp();
+            float lg[4][2], sv_t[4][2], ov_t[4][2];
+            float mx = -INFINITY;
 #pragma unroll
-                for (int e = 0; e < 4; ++e) mu[e] = msc * (float)(int)(int8_t)((q4 >> (8 * e)) & 0xffu);
-                const float* qf = qf32 + buf * (DQ_MAX_GROUP * kN);
-                for (int g = 0; g < G; ++g) {
-                    const float4 v = *reinterpret_cast<const float4*>(qf + g * kN + 4 * lane);
-                    float s = v.x * mu[0] + v.y * mu[1] + v.z * mu[2] + v.w * mu[3];
+            for (int i = 0; i < 4; ++i)
 #pragma unroll
-                    for (int d = 16; d >= 1; d >>= 1) s += __shfl_xor_sync(kFullMask, s, d);
-                    if (g == g_row) qmu = s;
+                for (int u = 0; u < 2; ++u) {
+                    const int tk = 8 * i + 2 * qd + u;
+                    float4 m4;
+                    asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4];\n"
+                                 : "=f"(m4.x), "=f"(m4.y), "=f"(m4.z), "=f"(m4.w) : "r"(ktile + tk * kTileStride + 32));
+                    const float S = sacc[i][u] + sacc[i][2 + u];
+                    const bool ok = tok0 + tk < cur.len;
+                    lg[i][u] = ok ? p.scale_log2 * fmaf(m4.x, S, fmaf(m4.y, qs, qmu)) : -INFINITY;
+                    sv_t[i][u] = ok ? m4.z : 0.f;
+                    ov_t[i][u] = ok ? m4.w : 0.f;
+                    mx = fmaxf(mx, lg[i][u]);
                 }
-            }
-            const float qs = (g_row < G) ? qsum[g_row] : 0.f;
-
-            // ---- keys: S[g][t] = sum_j q'_gj level_tj  (Eq. fold-key, inner sum)
-            float sacc[4][4];
-#pragma unroll
-            for (int i = 0; i < 4; ++i) { sacc[i][0] = sacc[i][1] = sacc[i][2] = sacc[i][3] = 0.f; }
-            {
-                uint32_t ptr = rk + 8;
-                const uint32_t a_addr = sbase + L.off_q16 + ((lane & 7) + ((lane >> 3) & 1) * 8) * kQ16Stride +
-                                        (lane >> 4) * 16;
-                const uint32_t b_addr = ktile + ((lane & 7) + (lane >> 4) * 8) * kTileStride + ((lane >> 3) & 1) * 16;
-#pragma unroll 1
-                for (int cg = 0; cg < 8; ++cg) {
-                    uint32_t pk[8];
-                    decode16(xk, ptr, my_lutk, pk);
-                    asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};\n" ::"r"(ktile + lane * kTileStride),
-                                 "r"(pk[0]), "r"(pk[1]), "r"(pk[2]), "r"(pk[3]) : "memory");
-                    asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};\n" ::"r"(ktile + lane * kTileStride + 16),
-                                 "r"(pk[4]), "r"(pk[5]), "r"(pk[6]), "r"(pk[7]) : "memory");
-                    __syncwarp();
-                    uint32_t a[4], b0[4], b1[4];
-                    ldmatrix_x4(a, a_addr + cg * 32);
-                    ldmatrix_x4(b0, b_addr);
-                    ldmatrix_x4(b1, b_addr + 16 * kTileStride);
-                    mma_f16_16816(sacc[0], a, b0[0], b0[1]);
-                    mma_f16_16816(sacc[1], a, b0[2], b0[3]);
-                    mma_f16_16816(sacc[2], a, b1[0], b1[1]);
-                    mma_f16_16816(sacc[3], a, b1[2], b1[3]);
-                    __syncwarp();
-                }
-            }
-
-            // ---- affine terms, softmax weights (base 2), fp16 hi/lo A operands for P.V
-            uint32_t pa[2][4];
-            {
-                float lg[4][2], sv_t[4][2], ov_t[4][2];
-                float mx = -INFINITY;
-#pragma unroll
-                for (int i = 0; i < 4; ++i)
-#pragma unroll
-                    for (int u = 0; u < 2; ++u) {
-                        const int tk = 8 * i + 2 * qd + u;
-                        float4 m4;
-                        asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4];\n"
-                                     : "=f"(m4.x), "=f"(m4.y), "=f"(m4.z), "=f"(m4.w) : "r"(scal + tk * 16));
-                        const float S = sacc[i][u] + sacc[i][2 + u];
-                        const bool ok = tok0 + tk < it.len;
-                        lg[i][u] = ok ? p.scale_log2 * fmaf(m4.x, S, fmaf(m4.y, qs, qmu)) : -INFINITY;
-                        sv_t[i][u] = ok ? m4.z : 0.f;
-                        ov_t[i][u] = ok ? m4.w : 0.f;
-                        mx = fmaxf(mx, lg[i][u]);
-                    }
-                mx = fmaxf(mx, __shfl_xor_sync(kFullMask, mx, 1));
-                mx = fmaxf(mx, __shfl_xor_sync(kFullMask, mx, 2));
-                m_run = mx;
-                const float m_use = (mx == -INFINITY) ? 0.f : mx;
-#pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    float hi[2], lo[2];
-#pragma unroll
-                    for (int u = 0; u < 2; ++u) {
-                        const float pr = exp2f(lg[i][u] - m_use);
-                        l_run += pr;
-                        off_run = fmaf(pr, ov_t[i][u], off_run);
-                        const float ps = pr * sv_t[i][u];
-                        hi[u] = __half2float(__float2half_rn(ps));
-                        lo[u] = ps - hi[u];
-                    }
-                    pa[i >> 1][(i & 1) * 2 + 0] = pack_half2(hi[0], hi[1]);
-                    pa[i >> 1][(i & 1) * 2 + 1] = pack_half2(lo[0], lo[1]);
-                }
-            }
-
-            // ---- values: O[g][j] += sum_t (a_t s_t) level_tj  (Eq. fold-value, first sum)
-            {
-                uint32_t ptr = rv + 8;
-                const uint32_t b_addr = vtile + ((lane & 7) + ((lane >> 3) & 1) * 8) * kTileStride + (lane >> 4) * 16;
-#pragma unroll
-                for (int cg = 0; cg < 8; ++cg) {
-                    uint32_t pk[8];
-                    decode16(xv, ptr, my_lutv, pk);
-                    asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};\n" ::"r"(vtile + lane * kTileStride),
-                                 "r"(pk[0]), "r"(pk[1]), "r"(pk[2]), "r"(pk[3]) : "memory");
-                    asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};\n" ::"r"(vtile + lane * kTileStride + 16),
-                                 "r"(pk[4]), "r"(pk[5]), "r"(pk[6]), "r"(pk[7]) : "memory");
-                    __syncwarp();
-                    uint32_t b0[4], b1[4];
-                    ldmatrix_x4_trans(b0, b_addr);                      // tokens 0..15
-                    ldmatrix_x4_trans(b1, b_addr + 16 * kTileStride);   // tokens 16..31
-                    mma_f16_16816(oacc[2 * cg], pa[0], b0[0], b0[1]);
-                    mma_f16_16816(oacc[2 * cg + 1], pa[0], b0[2], b0[3]);
-                    mma_f16_16816(oacc[2 * cg], pa[1], b1[0], b1[1]);
-                    mma_f16_16816(oacc[2 * cg + 1], pa[1], b1[2], b1[3]);
-                    __syncwarp();
-                }
-            }
-        }
-
-        // ------------------------------------------------ merge the warps of this item
-        l_run += __shfl_xor_sync(kFullMask, l_run, 1);
-        l_run += __shfl_xor_sync(kFullMask, l_run, 2);
-        off_run += __shfl_xor_sync(kFullMask, off_run, 1);
-        off_run += __shfl_xor_sync(kFullMask, off_run, 2);
-        if (qd == 0) {
-            red_m[warp * DQ_MAX_GROUP + g_row] = m_run;
-            red_l[warp * DQ_MAX_GROUP + g_row] = l_run;
-            red_o[warp * DQ_MAX_GROUP + g_row] = off_run;
-        }
-        __syncthreads();  // also: every warp is done with its tiles -> merge buffer may alias them
-        float m_all = -INFINITY;
-        for (int w = 0; w < nw; ++w) m_all = fmaxf(m_all, red_m[w * DQ_MAX_GROUP + g_row]);
-        const float m_base = (m_all == -INFINITY) ? 0.f : m_all;
-        const float my_scale = exp2f(m_run - m_base);
-
-        // output slot of this thread: (head og, channel oc) and (og + G/.., ...) handled below
-        float tot[kMaxPerThread];
-#pragma unroll
-        for (int r = 0; r < kMaxPerThread; ++r) tot[r] = 0.f;
-        for (int w0 = 0; w0 < nw; w0 += merge_slots) {
-            if (warp >= w0 && warp < w0 + merge_slots && g_row < G) {
-                float* dst = mbuf + ((warp - w0) * G + g_row) * kMergeStride + 2 * qd;
-#pragma unroll
-                for (int nt = 0; nt < 16; ++nt) {
-                    const float2 v = make_float2((oacc[nt][0] + oacc[nt][2]) * my_scale,
-                                                 (oacc[nt][1] + oacc[nt][3]) * my_scale);
-                    *reinterpret_cast<float2*>(dst + 8 * nt) = v;
-                }
-            }
+            mx = fmaxf(mx, __shfl_xor_sync(kFullMask, mx, 1));
+            mx = fmaxf(mx, __shfl_xor_sync(kFullMask, mx, 2));
+            // item-wide maximum per head, so that every warp's weights share one scale
+            if (qd == 0) red_m[warp * DQ_MAX_GROUP + g_row] = mx;
             __syncthreads();
-            const int cnt = min(merge_slots, nw - w0);
-#pragma unroll
-            for (int r = 0; r < kMaxPerThread; ++r) {
-                const int e = tid + r * nthreads;
-                if (e < G * kN) {
-                    const int g = e >> 7, ch = e & (kN - 1);
-                    float s = 0.f;
-                    for (int w = 0; w < cnt; ++w) s += mbuf[(w * G + g) * kMergeStride + ch];
-                    tot[r] += s;
-                }
-            }
-            __syncthreads();
-        }
-#pragma unroll
-        for (int r = 0; r < kMaxPerThread; ++r) {
-            const int e = tid + r * nthreads;
-            if (e >= G * kN) break;
-            const int g = e >> 7, ch = e & (kN - 1);
-            float mg = -INFINITY;
-            for (int w = 0; w < nw; ++w) mg = fmaxf(mg, red_m[w * DQ_MAX_GROUP + g]);
-            const float mb = (mg == -INFINITY) ? 0.f : mg;
+            float m_item = -INFINITY;
+            for (int w = 0; w < nw; ++w) m_item = fmaxf(m_item, red_m[w * DQ_MAX_GROUP + g_row]);
+            if (warp == 0 && qd == 0) red_M[g_row] = m_item;
+            const float m_use = (m_item == -INFINITY) ? 0.f : m_item;
             float lsum = 0.f, osum = 0.f;
-            for (int w = 0; w < nw; ++w) {
-                const float sc = exp2f(red_m[w * DQ_MAX_GROUP + g] - mb);
-                lsum = fmaf(red_l[w * DQ_MAX_GROUP + g], sc, lsum);
-                osum = fmaf(red_o[w * DQ_MAX_GROUP + g], sc, osum);
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                float hi[2], lo[2];
+#pragma unroll
+                for (int u = 0; u < 2; ++u) {
+                    const float pr = exp2f(lg[i][u] - m_use);
+                    lsum += pr;
+                    osum = fmaf(pr, ov_t[i][u], osum);
+                    const float ps = pr * sv_t[i][u];
+                    hi[u] = __half2float(__float2half_rn(ps));
+                    lo[u] = ps - hi[u];
+                }
+                pb_hi[i >> 1][i & 1] = pack_half2(hi[0], hi[1]);
+                pb_lo[i >> 1][i & 1] = pack_half2(lo[0], lo[1]);
             }
-            float* dst = p.partial + ((size_t)it.bg * p.Hq + (size_t)it.h * G + g) * kPartial;
-            dst[ch] = tot[r] + osum;               // Eq. fold-value: + sum_t a_t o_t
-            if (ch == 0) { dst[kN] = mg; dst[kN + 1] = lsum; }
+            lsum += __shfl_xor_sync(kFullMask, lsum, 1);
+            lsum += __shfl_xor_sync(kFullMask, lsum, 2);
+            osum += __shfl_xor_sync(kFullMask, osum, 1);
+            osum += __shfl_xor_sync(kFullMask, osum, 2);
+            if (qd == 0 && g_row < G) {   // l and off ride along in this warp's output slot
+                sts32f(my_obuf + (g_row * kORow + kN) * 4, lsum);
+                sts32f(my_obuf + (g_row * kORow + kN + 1) * 4, osum);
+            }
         }
-        __syncthreads();
-        buf ^= 1;
     }
     cp_async_wait<0>();
 }
@@ -492,7 +522,7 @@ dq_attn_combine_kernel(AttnParams p) {
     const int bg0 = p.prefix[b], nb = p.prefix[b + 1] - bg0;
     float mx = -INFINITY;
     for (int i = 0; i < nb; ++i) mx = fmaxf(mx, p.partial[((size_t)(bg0 + i) * p.Hq + hq) * kPartial + kN]);
-    float acc[4] = {0.f, 0.f, 0.f, 0.f}, lsum = 0.f;
+    float acc[4] = {0.f, 0.f, 0.f, 0.f}, lsum = 0.f, osum = 0.f;
     if (mx != -INFINITY) {
         for (int i = 0; i < nb; ++i) {
             const float* src = p.partial + ((size_t)(bg0 + i) * p.Hq + hq) * kPartial;
@@ -501,10 +531,11 @@ dq_attn_combine_kernel(AttnParams p) {
             acc[0] = fmaf(v.x, sc, acc[0]); acc[1] = fmaf(v.y, sc, acc[1]);
             acc[2] = fmaf(v.z, sc, acc[2]); acc[3] = fmaf(v.w, sc, acc[3]);
             lsum = fmaf(src[kN + 1], sc, lsum);
+            osum = fmaf(src[kN + 2], sc, osum);    // Eq. fold-value: + sum_t a_t o_t
         }
         const float inv = 1.0f / lsum;
 #pragma unroll
-        for (int e = 0; e < 4; ++e) acc[e] *= inv;
+        for (int e = 0; e < 4; ++e) acc[e] = (acc[e] + osum) * inv;
         if (p.rotate_out) warp_fwht128(acc, lane);
     }
     if (p.out_f32)
@@ -524,7 +555,7 @@ constexpr int kBfWarps = 4;
 constexpr int kBfRowStride = 272;                       // 128 bf16 + 16 bytes pad
 constexpr int kBfTileBytes = kChunk * kBfRowStride;     // one warp's K (or V) tile
 constexpr int kBfSmem = 16 * kBfRowStride + kBfWarps * 2 * kBfTileBytes + 3 * kBfWarps * 8 * 4 +
-                        kBfWarps * 8 * kMergeStride * 4;
+                        kBfWarps * 8 * kORow * 4;
 
 __device__ __forceinline__ void mma_bf16_16816(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
     asm volatile(
@@ -646,7 +677,7 @@ dq_bf16_attention_kernel(const AttnParams p, const uint16_t* __restrict__ kp, co
     for (int w = 0; w < kBfWarps; ++w) m_all = fmaxf(m_all, red_m[w * 8 + g_row]);
     const float my_scale = exp2f(m_run - ((m_all == -INFINITY) ? 0.f : m_all));
     if (g_row < G) {
-        float* dst = mbuf + (warp * G + g_row) * kMergeStride + 2 * qd;
+        float* dst = mbuf + (warp * G + g_row) * kORow + 2 * qd;
 #pragma unroll
         for (int nt = 0; nt < 16; ++nt)
             *reinterpret_cast<float2*>(dst + 8 * nt) = make_float2(oacc[nt][0] * my_scale, oacc[nt][1] * my_scale);
@@ -658,27 +689,35 @@ dq_bf16_attention_kernel(const AttnParams p, const uint16_t* __restrict__ kp, co
         for (int w = 0; w < kBfWarps; ++w) mg = fmaxf(mg, red_m[w * 8 + g]);
         const float mb = (mg == -INFINITY) ? 0.f : mg;
         for (int w = 0; w < kBfWarps; ++w) {
-            s += mbuf[(w * G + g) * kMergeStride + ch];
+            s += mbuf[(w * G + g) * kORow + ch];
             lsum = fmaf(red_l[w * 8 + g], exp2f(red_m[w * 8 + g] - mb), lsum);
         }
         float* dst = p.partial + ((size_t)(bg0 + blk) * p.Hq + (size_t)h * G + g) * kPartial;
         dst[ch] = s;
-        if (ch == 0) { dst[kN] = mg; dst[kN + 1] = lsum; }
+        if (ch == 0) { dst[kN] = mg; dst[kN + 1] = lsum; dst[kN + 2] = 0.f; }
     }
 }
 
 constexpr int kMinItemTokens = 4 * kChunk;  // smallest CTA the launcher may pick (4 warps)
 
 struct WsLayout {
-    size_t off_counter, off_prefix, off_qrot, off_partial, total;
+    size_t off_counter, off_prefix, off_qrot, off_q16, off_qsum, off_qmu, off_partial, total;
 };
+
+inline int windows_for(int max_pages) {
+    return (max_pages * DQ_PAGE_TOKENS + DQ_WINDOW_TOKENS - 1) / DQ_WINDOW_TOKENS;
+}
 
 WsLayout ws_layout(int B, int Hq, int max_pages) {
     WsLayout w;
     size_t o = 0;
+    auto up = [](size_t x) { return (x + 15) & ~(size_t)15; };
     w.off_counter = o; o += 16;
-    w.off_prefix = o; o += ((size_t)(B + 1) * 4 + 15) & ~(size_t)15;
+    w.off_prefix = o; o += up((size_t)(B + 1) * 4);
     w.off_qrot = o; o += (size_t)B * Hq * kN * 4;
+    w.off_q16 = o; o += (size_t)B * Hq * 16 * kN * 2;   // Hkv <= Hq rows blocks
+    w.off_qsum = o; o += up((size_t)B * Hq * 4);
+    w.off_qmu = o; o += up((size_t)B * Hq * windows_for(max_pages) * 4);
     const size_t blocks = (size_t)B * (((size_t)max_pages * DQ_PAGE_TOKENS + kMinItemTokens - 1) / kMinItemTokens);
     w.off_partial = o; o += blocks * Hq * kPartial * 4;
     w.total = o;
@@ -688,6 +727,33 @@ WsLayout ws_layout(int B, int Hq, int max_pages) {
 }  // namespace
 
 size_t dq_attn_workspace_bytes(int B, int Hq, int max_pages) { return ws_layout(B, Hq, max_pages).total; }
+
+// Optional timing of the main kernel: CUDA events recorded on the launch stream around
+// dq_attention_kernel, kept in a ring the caller drains with dq_profile_read().
+namespace {
+constexpr int kProfRing = 4096;
+bool g_prof_on = false;
+int g_prof_count = 0;
+cudaEvent_t g_prof_ev[kProfRing][2];
+bool g_prof_made[kProfRing];
+}  // namespace
+
+void dq_attn_profile_enable(int on) {
+    g_prof_on = on != 0;
+    g_prof_count = 0;
+}
+
+int dq_attn_profile_read(float* ms, int max_records) {
+    int n = 0;
+    for (int i = 0; i < g_prof_count && n < max_records; ++i) {
+        if (cudaEventSynchronize(g_prof_ev[i][1]) != cudaSuccess) break;
+        float t = 0.f;
+        if (cudaEventElapsedTime(&t, g_prof_ev[i][0], g_prof_ev[i][1]) != cudaSuccess) break;
+        ms[n++] = t;
+    }
+    g_prof_count = 0;
+    return n;
+}
 
 cudaError_t dq_launch_attention(const DqDevTable& tk, const DqDevTable& tv, const DqAttnArgs& a,
                                 cudaStream_t st) {
@@ -702,10 +768,11 @@ cudaError_t dq_launch_attention(const DqDevTable& tk, const DqDevTable& tv, cons
         if (e != cudaSuccess) return e;
     }
     int nw = kMaxWarps;
-    Layout L = make_layout(nw, tk.rec, tv.rec, a.B);
+    const int G = a.Hq / a.Hkv;
+    Layout L = make_layout(nw, tk.rec, tv.rec, a.B, G);
     while (L.total > smem_max && nw > 4) {
-        nw -= 4;
-        L = make_layout(nw, tk.rec, tv.rec, a.B);
+        nw -= 2;
+        L = make_layout(nw, tk.rec, tv.rec, a.B, G);
     }
     if (L.total > smem_max) return cudaErrorInvalidConfiguration;
 
@@ -719,23 +786,37 @@ cudaError_t dq_launch_attention(const DqDevTable& tk, const DqDevTable& tv, cons
     p.counter = reinterpret_cast<int*>(ws + w.off_counter);
     p.prefix = reinterpret_cast<int*>(ws + w.off_prefix);
     p.qrot = reinterpret_cast<float*>(ws + w.off_qrot);
+    p.q16 = reinterpret_cast<uint16_t*>(ws + w.off_q16);
+    p.qsum = reinterpret_cast<float*>(ws + w.off_qsum);
+    p.qmu = reinterpret_cast<float*>(ws + w.off_qmu);
     p.partial = reinterpret_cast<float*>(ws + w.off_partial);
     p.out_bf16 = a.out_bf16; p.out_f32 = a.out_f32;
-    p.max_windows = a.max_windows; p.max_pages = a.max_pages;
-    p.B = a.B; p.Hq = a.Hq; p.Hkv = a.Hkv; p.G = a.Hq / a.Hkv;
+    p.max_windows = a.max_windows; p.windows = windows_for(a.max_pages); p.max_pages = a.max_pages;
+    p.B = a.B; p.Hq = a.Hq; p.Hkv = a.Hkv; p.G = G;
     p.item_tokens = nw * kChunk;
-    p.rotate_q = tk.rotate; p.rotate_out = tv.rotate;
+    p.rotate_q = tk.rotate; p.rotate_out = tv.rotate; p.has_mean = tk.has_mean;
     p.scale_log2 = a.sm_scale * 1.4426950408889634f;
 
     const int heads = a.B * a.Hq;
-    dq_attn_prepare_kernel<<<(heads + 7) / 8, 256, 0, st>>>(p);
+    const long long prep_warps = (long long)heads * (1 + (p.has_mean ? p.windows : 0));
+    dq_attn_prepare_kernel<<<(unsigned)((prep_warps + 7) / 8), 256, 0, st>>>(p);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
     e = cudaFuncSetAttribute(dq_attention_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, L.total);
     if (e != cudaSuccess) return e;
+    const bool prof = g_prof_on && g_prof_count < kProfRing;
+    if (prof) {
+        if (!g_prof_made[g_prof_count]) {
+            if ((e = cudaEventCreate(&g_prof_ev[g_prof_count][0])) != cudaSuccess) return e;
+            if ((e = cudaEventCreate(&g_prof_ev[g_prof_count][1])) != cudaSuccess) return e;
+            g_prof_made[g_prof_count] = true;
+        }
+        cudaEventRecord(g_prof_ev[g_prof_count][0], st);
+    }
     dq_attention_kernel<<<sm_count, nw * 32, L.total, st>>>(tk, tv, p);
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;
+    if (prof) cudaEventRecord(g_prof_ev[g_prof_count++][1], st);
     dq_attn_combine_kernel<<<(heads + 7) / 8, 256, 0, st>>>(p);
     return cudaGetLastError();
 }
@@ -751,9 +832,12 @@ cudaError_t dq_launch_bf16_attention(const DqAttnArgs& a, const void* k_pages, c
     p.counter = reinterpret_cast<int*>(ws + w.off_counter);
     p.prefix = reinterpret_cast<int*>(ws + w.off_prefix);
     p.qrot = reinterpret_cast<float*>(ws + w.off_qrot);
+    p.q16 = reinterpret_cast<uint16_t*>(ws + w.off_q16);
+    p.qsum = reinterpret_cast<float*>(ws + w.off_qsum);
+    p.qmu = reinterpret_cast<float*>(ws + w.off_qmu);
     p.partial = reinterpret_cast<float*>(ws + w.off_partial);
     p.out_bf16 = a.out_bf16; p.out_f32 = nullptr;
-    p.max_windows = 0; p.max_pages = a.max_pages;
+    p.max_windows = 0; p.windows = 0; p.has_mean = 0; p.max_pages = a.max_pages;
     p.B = a.B; p.Hq = a.Hq; p.Hkv = a.Hkv; p.G = a.Hq / a.Hkv;
     p.item_tokens = kBfWarps * kChunk;
     p.rotate_q = 0; p.rotate_out = 0;

@@ -33,9 +33,9 @@ dq_decode_tokens_kernel(const __grid_constant__ DqDevTable T, const uint8_t* __r
     }
     for (int j = 0; j < DQ_HEAD_DIM; ++j) {
         const uint32_t e = T.lut[x & 255u];
-        x = ((e >> 8) & 255u) * (x >> 8) + (e & 255u);
+        x = (e >> 24) * (x >> 8) + (e & 255u);
         if (x < (1u << 23) && ptr < T.rec) x = (x << 8) | rec[ptr++];  // at most one byte
-        const float lvl = __half2float(__ushort_as_half((unsigned short)(e >> 16)));
+        const float lvl = __half2float(__ushort_as_half((unsigned short)((e >> 8) & 0xffffu)));
         if (symbols) symbols[sid * DQ_HEAD_DIM + j] = (uint8_t)(int)lvl;
         if (dequant) {
             float v = __fmaf_rn(lvl, s, o);

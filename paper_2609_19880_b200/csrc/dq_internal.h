@@ -13,7 +13,7 @@ struct DqDevTable {
     uint32_t fc[DQ_MAX_LEVELS];  // f | c << 16           (encoder, Eq. rans Enc)
     float r[DQ_MAX_LEVELS];      // ideal cost in bits     (Algorithm 1)
     uint32_t R[DQ_MAX_LEVELS];   // ceil(r * 65536)
-    uint32_t lut[256];           // fp16(level) << 16 | f << 8 | (z - c)   (Algorithm 2)
+    uint32_t lut[256];           // f << 24 | fp16(level) << 8 | (z - c)   (Algorithm 2)
 };
 
 struct dq_tables {
@@ -54,5 +54,7 @@ struct DqAttnArgs {
 size_t dq_attn_workspace_bytes(int B, int Hq, int max_pages);
 cudaError_t dq_launch_attention(const DqDevTable& tk, const DqDevTable& tv, const DqAttnArgs& a,
                                 cudaStream_t st);
+void dq_attn_profile_enable(int on);
+int dq_attn_profile_read(float* ms, int max_records);
 cudaError_t dq_launch_bf16_attention(const DqAttnArgs& a, const void* k_pages, const void* v_pages,
                                      cudaStream_t st);

@@ -93,7 +93,7 @@ void finish(dq_table_info& t) {
     for (int m = 0; m < t.levels; ++m) {
         const uint32_t level_bits = __half_as_ushort(__float2half((float)m));
         for (int z = t.c[m]; z < t.c[m + 1]; ++z)
-            t.lut[z] = (level_bits << 16) | ((uint32_t)t.f[m] << 8) | (uint32_t)(z - t.c[m]);
+            t.lut[z] = ((uint32_t)t.f[m] << 24) | (level_bits << 8) | (uint32_t)(z - t.c[m]);
     }
 }
 

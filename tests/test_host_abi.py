@@ -44,8 +44,8 @@ def test_tables_equal_oracle(L, M, rec, alpha):
     assert [i.R[m] for m in range(M)] == [o.R[m] for m in range(M)]
     for z in range(256):
         e = i.lut[z]
-        assert (e >> 8) & 255 == o.lut_f[z] and e & 255 == o.lut_d[z]
-        lvl = oracle.f16_bits_to_f32(e >> 16)
+        assert e >> 24 == o.lut_f[z] and e & 255 == o.lut_d[z]
+        lvl = oracle.f16_bits_to_f32((e >> 8) & 0xFFFF)
         assert lvl == float(o.lut_m[z])
 
 
