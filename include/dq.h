@@ -135,6 +135,35 @@ int dq_decode_attention(const dq_tables *tk, const dq_tables *tv, const void *q_
                         float sm_scale, void *out_bf16, float *out_f32, void *workspace,
                         size_t workspace_bytes, void *cuda_stream);
 
+/* dq_decode_attention for callers that must not allocate (the paper has no counterpart: this
+ * is a packaging variant of the same kernels, not part of the method).
+ *
+ * Some callers cannot obtain the workspace dq_decode_attention asks for: an engine whose device
+ * memory is handed out once at start-up and frozen, a plug-in running under a host program that
+ * owns every allocation, a real-time loop where an allocator call (which may synchronise the
+ * device or fail when memory is fragmented) is not acceptable.  For them the library carries its
+ * own scratch: a fixed array of DQ_STATIC_SCRATCH_BYTES in device global memory that every GPU
+ * loading the library holds until the process (context) ends.  This entry point passes that
+ * array to the kernels in place of a workspace and makes no cudaMalloc / cudaFree call and no
+ * call into any allocating library; inputs and outputs are still the caller's.
+ *
+ *   - Arguments, layouts and results are those of dq_decode_attention, minus the workspace.
+ *   - Limit: dq_decode_workspace_bytes(B, Hq, max_pages) must not exceed
+ *     DQ_STATIC_SCRATCH_BYTES; larger calls return DQ_ERR_WORKSPACE before anything is
+ *     launched and dq_last_cuda_error() then says how many bytes were needed.
+ *   - The first call on each device looks up the array's device address (current device must
+ *     be the one the call is meant for); make that first call outside any stream capture.
+ *   - All calls share the one array, which keeps whatever the previous call left in it; the
+ *     kernels reset what they need (work counter, prefix sums) themselves.  Two calls that
+ *     overlap on the GPU (different streams, or different host threads) race on it: serialise
+ *     them.  dq_profile_enable has no effect on this entry point. */
+#define DQ_STATIC_SCRATCH_BYTES (4u << 20)
+int dq_decode_attention_static(const dq_tables *tk, const dq_tables *tv, const void *q_bf16,
+                               const uint8_t *k_cont, const uint8_t *v_cont, const int8_t *k_mean_q,
+                               const float *k_mean_scale, int max_windows, const int32_t *page_table,
+                               int max_pages, const int32_t *seq_lens, int B, int Hq, int Hkv,
+                               float sm_scale, void *out_bf16, float *out_f32, void *cuda_stream);
+
 /* Check/debug export of Algorithm 2: decode T * Hkv records to symbols and to dequantised
  * values in the rotated domain, xhat = fma(m, s, o) (+ mean for keys).
  *   symbols  device uint8 [T][Hkv][128], nullable;  dequant  device float, same shape, nullable

@@ -23,7 +23,7 @@ ERRORS = {0: "DQ_OK", -1: "DQ_ERR_ARG", -2: "DQ_ERR_INFEASIBLE", -3: "DQ_ERR_UNS
           -4: "DQ_ERR_WORKSPACE", -5: "DQ_ERR_CUDA"}
 
 EXPORTS = ["dq_build_tables", "dq_free_tables", "dq_tables_info", "dq_encode_tokens",
-           "dq_decode_workspace_bytes", "dq_decode_attention", "dq_decode_tokens",
+           "dq_decode_workspace_bytes", "dq_decode_attention", "dq_decode_attention_static", "dq_decode_tokens",
            "dq_bf16_decode_attention", "dq_profile_enable", "dq_profile_read", "dq_strerror",
            "dq_last_cuda_error"]
 
@@ -71,6 +71,9 @@ def lib():
         L.dq_decode_attention.restype = i32
         L.dq_decode_attention.argtypes = [vp, vp, vp, vp, vp, vp, vp, i32, vp, i32, vp, i32, i32, i32, f32,
                                           vp, vp, vp, sz, vp]
+        L.dq_decode_attention_static.restype = i32
+        L.dq_decode_attention_static.argtypes = [vp, vp, vp, vp, vp, vp, vp, i32, vp, i32, vp, i32, i32, i32, f32,
+                                                 vp, vp, vp]
         L.dq_decode_tokens.restype = i32
         L.dq_decode_tokens.argtypes = [vp, vp, vp, vp, i32, vp, vp, vp, i32, i32, vp, vp, vp]
         L.dq_bf16_decode_attention.restype = i32
@@ -169,6 +172,26 @@ def dq_decode_attention(tk, tv, q_bf16, k_cont, v_cont, k_mean_q, k_mean_scale, 
                                    _ptr(out_f32), _ptr(workspace), int(workspace.numel() * workspace.element_size()),
                                    _stream(stream))
     _check(rc, "dq_decode_attention")
+
+
+STATIC_SCRATCH_BYTES = 4 << 20
+
+
+def dq_decode_attention_static(tk, tv, q_bf16, k_cont, v_cont, k_mean_q, k_mean_scale, page_table, seq_lens,
+                               Hkv: int, sm_scale: float, out_bf16, out_f32=None, stream=None):
+    """dq_decode_attention for callers that cannot allocate a workspace: the library's built-in
+    scratch array (STATIC_SCRATCH_BYTES, shared by all calls) is used instead.  Raises
+    DqError(DQ_ERR_WORKSPACE) when the call would need more than that.  Calls must not overlap
+    on the GPU; make the first call on a device outside any stream capture."""
+    B, Hq = int(q_bf16.shape[0]), int(q_bf16.shape[1])
+    max_windows = int(k_mean_q.shape[1]) if k_mean_q is not None else 0
+    rc = lib().dq_decode_attention_static(tk.handle, tv.handle, _ptr(q_bf16), _ptr(k_cont), _ptr(v_cont),
+                                          _ptr(k_mean_q), _ptr(k_mean_scale), max_windows, _ptr(page_table),
+                                          int(page_table.shape[1]), _ptr(seq_lens), B, Hq, int(Hkv),
+                                          float(sm_scale), _ptr(out_bf16), _ptr(out_f32), _stream(stream))
+    if rc == -4:
+        raise DqError(rc, "dq_decode_attention_static [" + lib().dq_last_cuda_error().decode() + "]")
+    _check(rc, "dq_decode_attention_static")
 
 
 def dq_decode_tokens(t, cont, slot, Hkv: int, symbols=None, dequant=None, mean_q=None, mean_scale=None,

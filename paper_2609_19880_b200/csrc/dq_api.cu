@@ -124,6 +124,46 @@ int dq_decode_attention(const dq_tables* tk, const dq_tables* tv, const void* q_
     return DQ_OK;
 }
 
+int dq_decode_attention_static(const dq_tables* tk, const dq_tables* tv, const void* q_bf16,
+                               const uint8_t* k_cont, const uint8_t* v_cont, const int8_t* k_mean_q,
+                               const float* k_mean_scale, int max_windows, const int32_t* page_table,
+                               int max_pages, const int32_t* seq_lens, int B, int Hq, int Hkv, float sm_scale,
+                               void* out_bf16, float* out_f32, void* cuda_stream) {
+    if (!tk || !tv || !k_cont || !v_cont) return DQ_ERR_ARG;
+    if (B <= 0 || Hq <= 0 || Hkv <= 0 || max_pages <= 0) return DQ_ERR_ARG;
+    const size_t need = dq_attn_workspace_bytes(B, Hq, max_pages);
+    if (need > (size_t)DQ_STATIC_SCRATCH_BYTES) {  // decided on the host, before any CUDA call
+        std::snprintf(g_cuda_error, sizeof g_cuda_error,
+                      "dq_decode_attention_static: the built-in scratch holds %zu bytes, this call needs %zu "
+                      "(B=%d, Hq=%d, max_pages=%d); use dq_decode_attention with a workspace",
+                      (size_t)DQ_STATIC_SCRATCH_BYTES, need, B, Hq, max_pages);
+        return DQ_ERR_WORKSPACE;
+    }
+    void* scratch = nullptr;
+    cudaError_t e = dq_attn_static_scratch(&scratch);
+    if (e != cudaSuccess) return cuda_fail(e, "static scratch address");
+    int rc = check_attn_common(q_bf16, page_table, max_pages, seq_lens, B, Hq, Hkv, out_bf16, out_f32, scratch,
+                               (size_t)DQ_STATIC_SCRATCH_BYTES);
+    if (rc != DQ_OK) return rc;
+    if (tv->info.has_mean) return DQ_ERR_UNSUPPORTED;
+    if (tk->info.has_mean && (!k_mean_q || !k_mean_scale || max_windows <= 0)) return DQ_ERR_ARG;
+    if (tk->info.has_mean && (long long)max_windows * DQ_WINDOW_TOKENS < (long long)max_pages * DQ_PAGE_TOKENS)
+        return DQ_ERR_ARG;
+    if (!aligned16(k_cont) || !aligned16(v_cont) || (tk->info.has_mean && !aligned16(k_mean_q))) return DQ_ERR_ARG;
+    if ((out_bf16 && (reinterpret_cast<uintptr_t>(out_bf16) & 7u)) || (out_f32 && !aligned16(out_f32)))
+        return DQ_ERR_ARG;
+    DqAttnArgs a;
+    a.q_bf16 = q_bf16; a.k_cont = k_cont; a.v_cont = v_cont;
+    a.mean_q = k_mean_q; a.mean_scale = k_mean_scale;
+    a.page_table = page_table; a.seq_lens = seq_lens;
+    a.out_bf16 = out_bf16; a.out_f32 = out_f32; a.workspace = scratch;
+    a.max_windows = max_windows; a.max_pages = max_pages;
+    a.B = B; a.Hq = Hq; a.Hkv = Hkv; a.sm_scale = sm_scale;
+    e = dq_launch_attention_static(tk->dev, tv->dev, a, static_cast<cudaStream_t>(cuda_stream));
+    if (e != cudaSuccess) return cuda_fail(e, "decode attention (static scratch)");
+    return DQ_OK;
+}
+
 int dq_decode_tokens(const dq_tables* t, const uint8_t* cont, const int8_t* mean_q, const float* mean_scale,
                      int max_windows, const int32_t* seq_id, const int32_t* pos, const int32_t* slot, int T,
                      int Hkv, uint8_t* symbols, float* dequant, void* cuda_stream) {

@@ -856,3 +856,46 @@ cudaError_t dq_launch_bf16_attention(const DqAttnArgs& a, const void* k_pages, c
     dq_attn_combine_kernel<<<(heads + 7) / 8, 256, 0, st>>>(p);
     return cudaGetLastError();
 }
+
+// ------------------------------------------------ attention without any allocation
+//
+// Scratch for dq_decode_attention_static: a fixed array in device global memory that exists
+// in every CUDA context which loads this library, from load until the context ends.  Host
+// code may not use the symbol `g_static_scratch` as a pointer (on the host it is only a
+// stand-in for the device object); its device address is looked up once per device with
+// cudaGetSymbolAddress and that address is what the kernels receive.
+static __device__ __align__(256) unsigned char g_static_scratch[DQ_STATIC_SCRATCH_BYTES];
+
+namespace {
+constexpr int kMaxDevices = 64;
+void* g_static_scratch_addr[kMaxDevices];
+bool g_static_scratch_known[kMaxDevices];
+}  // namespace
+
+// Device address of the static scratch array on the current device (looked up on first use).
+cudaError_t dq_attn_static_scratch(void** out) {
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
+    if (!g_static_scratch_known[dev]) {
+        void* addr = nullptr;
+        e = cudaGetSymbolAddress(&addr, g_static_scratch);
+        if (e != cudaSuccess) return e;
+        g_static_scratch_addr[dev] = addr;
+        g_static_scratch_known[dev] = true;
+    }
+    *out = g_static_scratch_addr[dev];
+    return cudaSuccess;
+}
+
+// Same launches as dq_launch_attention, with the event-recording measurement aid held off so
+// that nothing on this route can create a CUDA object.
+cudaError_t dq_launch_attention_static(const DqDevTable& tk, const DqDevTable& tv, const DqAttnArgs& a,
+                                       cudaStream_t st) {
+    const bool was_on = g_prof_on;
+    g_prof_on = false;
+    const cudaError_t e = dq_launch_attention(tk, tv, a, st);
+    g_prof_on = was_on;
+    return e;
+}

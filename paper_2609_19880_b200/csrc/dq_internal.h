@@ -54,6 +54,9 @@ struct DqAttnArgs {
 size_t dq_attn_workspace_bytes(int B, int Hq, int max_pages);
 cudaError_t dq_launch_attention(const DqDevTable& tk, const DqDevTable& tv, const DqAttnArgs& a,
                                 cudaStream_t st);
+cudaError_t dq_attn_static_scratch(void** out);
+cudaError_t dq_launch_attention_static(const DqDevTable& tk, const DqDevTable& tv, const DqAttnArgs& a,
+                                       cudaStream_t st);
 void dq_attn_profile_enable(int on);
 int dq_attn_profile_read(float* ms, int max_records);
 cudaError_t dq_launch_bf16_attention(const DqAttnArgs& a, const void* k_pages, const void* v_pages,
