@@ -247,7 +247,7 @@ def run_ours(args):
                             dq.MEAN_REUSE)
         dq.dq_decode_attention(tk, tv, q, c["k"], c["v"], c["mq"], c["ms"], w.page_table, w.seq_lens, Hkv,
                                sm_scale, out, ws)
-    launches_per_step = 6   # mean carry-forward, encode K, encode V, prepare, fused attention, combine
+    launches_per_step = 4   # encode (K and V), prepare, fused attention, combine
 
     def barrier():
         if world > 1:

@@ -60,21 +60,20 @@ int dq_encode_tokens(const dq_tables* tk, const dq_tables* tv, const void* k_bf1
     if (T == 0) return DQ_OK;
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     cudaError_t e;
-    if (k_mean) {
+    if (k_mean && mean_mode == DQ_MEAN_COMPUTE) {
         e = dq_launch_means(tk->dev, k_bf16, T, Hkv, seq_id, pos, k_mean_q, k_mean_scale, max_windows,
                             mean_mode, st);
         if (e != cudaSuccess) return cuda_fail(e, "window means");
     }
-    if (tk) {
-        e = dq_launch_encode(tk->dev, k_bf16, T, Hkv, seq_id, pos, slot, k_cont, k_mean_q, k_mean_scale,
-                             max_windows, status, st);
-        if (e != cudaSuccess) return cuda_fail(e, "encode K");
-    }
-    if (tv) {
-        e = dq_launch_encode(tv->dev, v_bf16, T, Hkv, seq_id, pos, slot, v_cont, nullptr, nullptr, 0,
-                             status, st);
-        if (e != cudaSuccess) return cuda_fail(e, "encode V");
-    }
+    // keys and values go through one launch; in DQ_MEAN_REUSE mode the encoder warp of a
+    // window's first token carries the previous mean forward itself
+    DqEncodeArgs a;
+    a.k_bf16 = k_bf16; a.v_bf16 = v_bf16; a.seq_id = seq_id; a.pos = pos; a.slot = slot;
+    a.k_cont = k_cont; a.v_cont = v_cont; a.mean_q = k_mean_q; a.mean_scale = k_mean_scale;
+    a.status = status; a.T = T; a.Hkv = Hkv; a.max_windows = max_windows; a.mean_mode = mean_mode;
+    a.do_k = tk ? 1 : 0; a.do_v = tv ? 1 : 0;
+    e = dq_launch_encode(tk ? tk->dev : tv->dev, tv ? tv->dev : tk->dev, a, st);
+    if (e != cudaSuccess) return cuda_fail(e, "encode");
     return DQ_OK;
 }
 

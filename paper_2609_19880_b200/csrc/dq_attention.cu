@@ -104,14 +104,16 @@ struct AttnParams {
 // ------------------------------------------------------------------ prepare
 
 // Warp roles: [0, B*Hq): rotate q, emit the fp16 hi/lo operand rows and the row sum;
-// [B*Hq, B*Hq*(1+windows)): q' . mean of one (head, window) (Eq. fold-key, third term);
-// block 0 additionally scans the blocks per sequence and resets the work counter.
+// then B*Hq warps per group of 8 windows: q' . mean of each (head, window) (Eq. fold-key, third
+// term); block 0 additionally scans the blocks per sequence and resets the work counter.
+constexpr int kPrepWindows = 8;
 __global__ void __launch_bounds__(256)
 dq_attn_prepare_kernel(AttnParams p) {
     const int lane = threadIdx.x & 31;
     const long long wid = (long long)blockIdx.x * 8 + (threadIdx.x >> 5);
     const int heads = p.B * p.Hq;
-    if (wid < (long long)heads * (1 + (p.has_mean ? p.windows : 0))) {
+    const int wgroups = p.has_mean ? (p.windows + kPrepWindows - 1) / kPrepWindows : 0;
+    if (wid < (long long)heads * (1 + wgroups)) {
         const int head = (int)(wid % heads), win = (int)(wid / heads) - 1;
         const uint2 raw = *reinterpret_cast<const uint2*>(p.q + (size_t)head * kN + 4 * lane);
         float v[4] = {bf16_bits_to_float(raw.x & 0xffffu), bf16_bits_to_float(raw.x >> 16),
@@ -144,15 +146,28 @@ dq_attn_prepare_kernel(AttnParams p) {
             for (int d = 16; d >= 1; d >>= 1) s += __shfl_xor_sync(kFullMask, s, d);
             if (lane == 0) p.qsum[head] = s;
         } else {
-            const size_t mi = ((size_t)b * p.max_windows + win) * p.Hkv + h;
-            const uint32_t q4 = *reinterpret_cast<const uint32_t*>(p.mean_q + mi * kN + 4 * lane);
-            const float msc = p.mean_scale[mi];
-            float s = 0.f;
+            uint32_t q4[kPrepWindows];
+            float msc[kPrepWindows], s[kPrepWindows];
 #pragma unroll
-            for (int e = 0; e < 4; ++e) s = fmaf(v[e], msc * (float)(int)(int8_t)((q4 >> (8 * e)) & 0xffu), s);
+            for (int u = 0; u < kPrepWindows; ++u) {   // all loads first
+                const int w = min(win * kPrepWindows + u, p.windows - 1);
+                const size_t mi = ((size_t)b * p.max_windows + w) * p.Hkv + h;
+                q4[u] = *reinterpret_cast<const uint32_t*>(p.mean_q + mi * kN + 4 * lane);
+                msc[u] = p.mean_scale[mi];
+            }
 #pragma unroll
-            for (int d = 16; d >= 1; d >>= 1) s += __shfl_xor_sync(kFullMask, s, d);
-            if (lane == 0) p.qmu[(size_t)head * p.windows + win] = s;
+            for (int u = 0; u < kPrepWindows; ++u) {
+                s[u] = 0.f;
+#pragma unroll
+                for (int e = 0; e < 4; ++e) s[u] = fmaf(v[e], msc[u] * (float)(int)(int8_t)((q4[u] >> (8 * e)) & 0xffu), s[u]);
+            }
+#pragma unroll
+            for (int d = 16; d >= 1; d >>= 1)
+#pragma unroll
+                for (int u = 0; u < kPrepWindows; ++u) s[u] += __shfl_xor_sync(kFullMask, s[u], d);
+#pragma unroll
+            for (int u = 0; u < kPrepWindows; ++u)
+                if (lane == u && win * kPrepWindows + u < p.windows) p.qmu[(size_t)head * p.windows + win * kPrepWindows + u] = s[u];
         }
     }
     if (blockIdx.x == 0 && threadIdx.x < 32) {  // exclusive scan of blocks per sequence
@@ -520,18 +535,31 @@ dq_attn_combine_kernel(AttnParams p) {
     if (wid >= p.B * p.Hq) return;
     const int b = wid / p.Hq, hq = wid % p.Hq;
     const int bg0 = p.prefix[b], nb = p.prefix[b + 1] - bg0;
+    const float* base = p.partial + ((size_t)bg0 * p.Hq + hq) * kPartial;
+    const size_t stride = (size_t)p.Hq * kPartial;
     float mx = -INFINITY;
-    for (int i = 0; i < nb; ++i) mx = fmaxf(mx, p.partial[((size_t)(bg0 + i) * p.Hq + hq) * kPartial + kN]);
+    for (int i = lane; i < nb; i += 32) mx = fmaxf(mx, base[i * stride + kN]);
+#pragma unroll
+    for (int d = 16; d >= 1; d >>= 1) mx = fmaxf(mx, __shfl_xor_sync(kFullMask, mx, d));
     float acc[4] = {0.f, 0.f, 0.f, 0.f}, lsum = 0.f, osum = 0.f;
     if (mx != -INFINITY) {
-        for (int i = 0; i < nb; ++i) {
-            const float* src = p.partial + ((size_t)(bg0 + i) * p.Hq + hq) * kPartial;
-            const float sc = exp2f(src[kN] - mx);
-            const float4 v = *reinterpret_cast<const float4*>(src + 4 * lane);
-            acc[0] = fmaf(v.x, sc, acc[0]); acc[1] = fmaf(v.y, sc, acc[1]);
-            acc[2] = fmaf(v.z, sc, acc[2]); acc[3] = fmaf(v.w, sc, acc[3]);
-            lsum = fmaf(src[kN + 1], sc, lsum);
-            osum = fmaf(src[kN + 2], sc, osum);    // Eq. fold-value: + sum_t a_t o_t
+        for (int i0 = 0; i0 < nb; i0 += 4) {   // four partials in flight
+            float4 v[4];
+            float m[4], l[4], o[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const float* src = base + (size_t)min(i0 + u, nb - 1) * stride;
+                v[u] = *reinterpret_cast<const float4*>(src + 4 * lane);
+                m[u] = src[kN]; l[u] = src[kN + 1]; o[u] = src[kN + 2];
+            }
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const float sc = (i0 + u < nb) ? exp2f(m[u] - mx) : 0.f;
+                acc[0] = fmaf(v[u].x, sc, acc[0]); acc[1] = fmaf(v[u].y, sc, acc[1]);
+                acc[2] = fmaf(v[u].z, sc, acc[2]); acc[3] = fmaf(v[u].w, sc, acc[3]);
+                lsum = fmaf(l[u], sc, lsum);
+                osum = fmaf(o[u], sc, osum);    // Eq. fold-value: + sum_t a_t o_t
+            }
         }
         const float inv = 1.0f / lsum;
 #pragma unroll
@@ -798,7 +826,7 @@ cudaError_t dq_launch_attention(const DqDevTable& tk, const DqDevTable& tv, cons
     p.scale_log2 = a.sm_scale * 1.4426950408889634f;
 
     const int heads = a.B * a.Hq;
-    const long long prep_warps = (long long)heads * (1 + (p.has_mean ? p.windows : 0));
+    const long long prep_warps = (long long)heads * (1 + (p.has_mean ? (p.windows + kPrepWindows - 1) / kPrepWindows : 0));
     dq_attn_prepare_kernel<<<(unsigned)((prep_warps + 7) / 8), 256, 0, st>>>(p);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;

@@ -63,39 +63,23 @@ dq_means_compute_kernel(const uint16_t* __restrict__ k, int T, int Hkv, int rota
     if (lane == 0) mean_scale[mi] = sc;
 }
 
-// DQ_MEAN_REUSE.  A token at the first position of a window copies the previous window's
-// mean into its own (window 0: zeros).  One warp per (token, KV head).
-__global__ void __launch_bounds__(256)
-dq_means_reuse_kernel(int T, int Hkv, const int32_t* __restrict__ seq_id,
-                      const int32_t* __restrict__ pos, int8_t* __restrict__ mean_q,
-                      float* __restrict__ mean_scale, int Wmax) {
-    const int lane = threadIdx.x & 31;
-    const long long wid = (long long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
-    if (wid >= (long long)T * Hkv) return;
-    const int t = (int)(wid / Hkv), h = (int)(wid % Hkv);
-    const int p = pos[t];
-    if (p % DQ_WINDOW_TOKENS) return;
-    const int w = p / DQ_WINDOW_TOKENS;
-    const size_t dst = ((size_t)seq_id[t] * Wmax + w) * Hkv + h;
-    uint32_t q = 0;
-    float sc = 0.f;
-    if (w > 0) {
-        const size_t src = ((size_t)seq_id[t] * Wmax + (w - 1)) * Hkv + h;
-        q = *reinterpret_cast<const uint32_t*>(mean_q + src * kN + 4 * lane);
-        sc = mean_scale[src];
-    }
-    *reinterpret_cast<uint32_t*>(mean_q + dst * kN + 4 * lane) = q;
-    if (lane == 0) mean_scale[dst] = sc;
-}
-
 // ------------------------------------------------------------------------ drift
+
+// Per-CTA copy of the table fields the encoder touches (a CTA encodes one tensor kind).
+struct EncTable {
+    float r[DQ_MAX_LEVELS];
+    uint32_t R[DQ_MAX_LEVELS];
+    uint32_t rcp[DQ_MAX_LEVELS];
+    uint32_t aux[DQ_MAX_LEVELS];
+    int M, rec, mstar, budget_bits, has_mean, rotate;
+};
 
 // Function Drift of Algorithm 1 on a stream held 4 values per lane.  The bisection of
 // log2(lambda) over T = 12 steps is carried out as the geometric mean of the bracket
 // [hi * 2^-40, hi], hi = 8 (max D - min D); the code length is an integer sum of
 // ceil(65536 r_m), so the feasibility test does not depend on summation order.
 // Returns the length of the final assignment (the argmin at the bracket's upper end).
-__device__ __forceinline__ uint32_t drift(const DqDevTable& T, const float (&z)[4], float s, float o,
+__device__ __forceinline__ uint32_t drift(const EncTable& T, const float (&z)[4], float s, float o,
                                           uint32_t (&sym)[4]) {
     const int M = T.M;
     float maxD = -INFINITY, minD = INFINITY;
@@ -145,18 +129,34 @@ __device__ __forceinline__ uint32_t drift(const DqDevTable& T, const float (&z)[
 
 constexpr int kEncWarps = 8;
 
-// One warp per stream (token, KV head).  Lane l owns elements 4l .. 4l+3.
+// One warp per stream (token, KV head); lane l owns elements 4l .. 4l+3.  blockIdx.y selects
+// the tensor kind when keys and values are encoded by one launch.
 __global__ void __launch_bounds__(kEncWarps * 32)
-dq_encode_kernel(const __grid_constant__ DqDevTable T, const uint16_t* __restrict__ x, int n_tok,
-                 int Hkv, const int32_t* __restrict__ seq_id, const int32_t* __restrict__ pos,
-                 const int32_t* __restrict__ slot, uint8_t* __restrict__ cont,
-                 const int8_t* __restrict__ mean_q, const float* __restrict__ mean_scale, int Wmax,
-                 uint32_t* __restrict__ status) {
+dq_encode_kernel(const __grid_constant__ DqDevTable TK, const __grid_constant__ DqDevTable TV,
+                 const DqEncodeArgs a) {
+    __shared__ EncTable T;
     __shared__ uint8_t s_bytes[kEncWarps][DQ_MAX_REC_BYTES];
+    __shared__ __align__(4) uint8_t s_sym[kEncWarps][kN];
+    const bool is_v = a.do_k ? (blockIdx.y == 1) : true;
+    if (threadIdx.x < DQ_MAX_LEVELS) {
+        const int i = threadIdx.x;
+        T.r[i] = is_v ? TV.r[i] : TK.r[i];
+        T.R[i] = is_v ? TV.R[i] : TK.R[i];
+        T.rcp[i] = is_v ? TV.enc_rcp[i] : TK.enc_rcp[i];
+        T.aux[i] = is_v ? TV.enc_aux[i] : TK.enc_aux[i];
+    }
+    if (threadIdx.x == 0) {
+        T.M = is_v ? TV.M : TK.M; T.rec = is_v ? TV.rec : TK.rec; T.mstar = is_v ? TV.mstar : TK.mstar;
+        T.budget_bits = is_v ? TV.budget_bits : TK.budget_bits;
+        T.has_mean = is_v ? TV.has_mean : TK.has_mean; T.rotate = is_v ? TV.rotate : TK.rotate;
+    }
+    __syncthreads();
     const int lane = threadIdx.x & 31, wib = threadIdx.x >> 5;
     const long long wid = (long long)blockIdx.x * kEncWarps + wib;
-    if (wid >= (long long)n_tok * Hkv) return;
-    const int t = (int)(wid / Hkv), h = (int)(wid % Hkv);
+    if (wid >= (long long)a.T * a.Hkv) return;
+    const int t = (int)(wid / a.Hkv), h = (int)(wid % a.Hkv), Hkv = a.Hkv;
+    const uint16_t* x = static_cast<const uint16_t*>(is_v ? a.v_bf16 : a.k_bf16);
+    uint8_t* cont = is_v ? a.v_cont : a.k_cont;
 
     float z[4];
     {
@@ -166,9 +166,25 @@ dq_encode_kernel(const __grid_constant__ DqDevTable T, const uint16_t* __restric
     }
     if (T.rotate) warp_fwht128(z, lane);
     if (T.has_mean) {  // remove the (dequantised) windowed channel mean, Sec. 4.2
-        const size_t mi = ((size_t)seq_id[t] * Wmax + pos[t] / DQ_WINDOW_TOKENS) * Hkv + h;
-        const float sc = mean_scale[mi];
-        const uint32_t q4 = *reinterpret_cast<const uint32_t*>(mean_q + mi * kN + 4 * lane);
+        const int ps = a.pos[t], w = ps / DQ_WINDOW_TOKENS;
+        const size_t mi = ((size_t)a.seq_id[t] * a.max_windows + w) * Hkv + h;
+        uint32_t q4;
+        float sc;
+        if (a.mean_mode == DQ_MEAN_REUSE && ps % DQ_WINDOW_TOKENS == 0) {
+            // first position of a window: carry the previous window's mean forward (window 0: zero).
+            // Rows are per head, so this warp is the only writer and reader of the row in this call.
+            q4 = 0u; sc = 0.f;
+            if (w > 0) {
+                const size_t src = mi - (size_t)Hkv;
+                q4 = *reinterpret_cast<const uint32_t*>(a.mean_q + src * kN + 4 * lane);
+                sc = a.mean_scale[src];
+            }
+            *reinterpret_cast<uint32_t*>(a.mean_q + mi * kN + 4 * lane) = q4;
+            if (lane == 0) a.mean_scale[mi] = sc;
+        } else {
+            sc = a.mean_scale[mi];
+            q4 = *reinterpret_cast<const uint32_t*>(a.mean_q + mi * kN + 4 * lane);
+        }
 #pragma unroll
         for (int e = 0; e < 4; ++e) {
             const float q = (float)(int)(int8_t)((q4 >> (8 * e)) & 0xffu);
@@ -192,26 +208,26 @@ dq_encode_kernel(const __grid_constant__ DqDevTable T, const uint16_t* __restric
         const float s = __fdiv_rn(__fsub_rn(mx, mn), (float)(T.M - 1));
         drift(T, z, s, o, sym);
         // Refit: least squares of z on the symbols; binary64 sums in a fixed order
-        double a = (double)z[0], b = __dmul_rn((double)sym[0], (double)z[0]);
+        double sa = (double)z[0], sb = __dmul_rn((double)sym[0], (double)z[0]);
         int sm = (int)sym[0], smm = (int)(sym[0] * sym[0]);
 #pragma unroll
         for (int e = 1; e < 4; ++e) {
-            a = __dadd_rn(a, (double)z[e]);
-            b = __dadd_rn(b, __dmul_rn((double)sym[e], (double)z[e]));
+            sa = __dadd_rn(sa, (double)z[e]);
+            sb = __dadd_rn(sb, __dmul_rn((double)sym[e], (double)z[e]));
             sm += (int)sym[e];
             smm += (int)(sym[e] * sym[e]);
         }
 #pragma unroll
         for (int d = 16; d >= 1; d >>= 1) {
-            a = __dadd_rn(a, __shfl_xor_sync(kFull, a, d));
-            b = __dadd_rn(b, __shfl_xor_sync(kFull, b, d));
+            sa = __dadd_rn(sa, __shfl_xor_sync(kFull, sa, d));
+            sb = __dadd_rn(sb, __shfl_xor_sync(kFull, sb, d));
         }
         const long long Sm = __reduce_add_sync(kFull, sm), Smm = __reduce_add_sync(kFull, smm);
         const long long den = (long long)kN * Smm - Sm * Sm;
         double sd = (double)s, od = (double)o;
         if (den != 0) {
-            sd = __ddiv_rn(__dsub_rn(__dmul_rn((double)kN, b), __dmul_rn((double)Sm, a)), (double)den);
-            od = __ddiv_rn(__dsub_rn(a, __dmul_rn(sd, (double)Sm)), (double)kN);
+            sd = __ddiv_rn(__dsub_rn(__dmul_rn((double)kN, sb), __dmul_rn((double)Sm, sa)), (double)den);
+            od = __ddiv_rn(__dsub_rn(sa, __dmul_rn(sd, (double)Sm)), (double)kN);
         }
         s16 = __double2half(sd);                                    // fp16 metadata
         o16 = __double2half(od);
@@ -240,26 +256,27 @@ dq_encode_kernel(const __grid_constant__ DqDevTable T, const uint16_t* __restric
     }
 
     // rANS, Eq. (rans) Enc on symbols 127 .. 0 so that decoding runs forward.  Every lane
-    // carries the same state; lane 0 records the emitted bytes.
-    const uint32_t sym4 = sym[0] | (sym[1] << 8) | (sym[2] << 16) | (sym[3] << 24);
+    // carries the same state (the symbols come from shared memory); lane 0 records the bytes.
+    *reinterpret_cast<uint32_t*>(&s_sym[wib][4 * lane]) = sym[0] | (sym[1] << 8) | (sym[2] << 16) | (sym[3] << 24);
+    __syncwarp();
     uint32_t xs = kL;
     int k = 0;
     uint8_t* bytes = s_bytes[wib];
+#pragma unroll 4
     for (int j = kN - 1; j >= 0; --j) {
-        const uint32_t word = __shfl_sync(kFull, sym4, j >> 2);
-        const uint32_t m = (word >> (8 * (j & 3))) & 0xffu;
-        const uint32_t fc = T.fc[m];
-        const uint32_t f = fc & 0xffffu, c = fc >> 16;
-        if (xs >= (f << 23)) {  // at most once: xs < 2^31 <= 2^8 * (f << 23)
+        const uint32_t m = s_sym[wib][j];
+        const uint32_t aux = T.aux[m], rcp = T.rcp[m];
+        const uint32_t cmpl = (aux >> 10) & 511u;                  // 2^p - f
+        if (xs >= ((256u - cmpl) << 23)) {  // at most once: xs < 2^31 <= 2^8 * (f << 23)
             if (lane == 0) bytes[k] = (uint8_t)(xs & 0xffu);
             ++k;
             xs >>= 8;
         }
-        xs = (xs / f) * 256u + (xs % f) + c;
+        xs = xs + (aux & 1023u) + (__umulhi(xs, rcp) >> (aux >> 19)) * cmpl;
     }
     __syncwarp();
     const uint32_t hdr0 = (uint32_t)__half_as_ushort(s16) | ((uint32_t)__half_as_ushort(o16) << 16);
-    const int sl = slot[t];
+    const int sl = a.slot[t];
     uint8_t* rec = cont + (((size_t)(sl / DQ_PAGE_TOKENS) * Hkv + h) * DQ_PAGE_TOKENS +
                            (size_t)(sl % DQ_PAGE_TOKENS)) * T.rec;
     const int used = min(8 + k, T.rec);  // the budget test keeps 8 + k <= rec
@@ -270,11 +287,11 @@ dq_encode_kernel(const __grid_constant__ DqDevTable T, const uint16_t* __restric
         else if (i < used) v = bytes[k - 1 - (i - 8)];
         rec[i] = v;
     }
-    if (status && lane == 0) {
-        if (st_fallback) atomicAdd(status + 0, 1u);
-        if (degenerate) atomicAdd(status + 1, 1u);
-        if (st_refit) atomicAdd(status + 2, 1u);
-        atomicMax(status + 3, (uint32_t)(8 + k));
+    if (a.status && lane == 0) {
+        if (st_fallback) atomicAdd(a.status + 0, 1u);
+        if (degenerate) atomicAdd(a.status + 1, 1u);
+        if (st_refit) atomicAdd(a.status + 2, 1u);
+        atomicMax(a.status + 3, (uint32_t)(8 + k));
     }
 }
 
@@ -286,24 +303,16 @@ cudaError_t dq_launch_means(const DqDevTable& tk, const void* k_bf16, int T, int
     const long long warps = (long long)T * Hkv;
     if (warps == 0) return cudaSuccess;
     const unsigned blocks = (unsigned)((warps + 7) / 8);
-    if (mode == DQ_MEAN_COMPUTE)
-        dq_means_compute_kernel<<<blocks, 256, 0, st>>>((const uint16_t*)k_bf16, T, Hkv, tk.rotate,
-                                                        seq_id, pos, mean_q, mean_scale, max_windows);
-    else
-        dq_means_reuse_kernel<<<blocks, 256, 0, st>>>(T, Hkv, seq_id, pos, mean_q, mean_scale,
-                                                      max_windows);
+    if (mode != DQ_MEAN_COMPUTE) return cudaSuccess;  // carry-forward is done by the encoder warps
+    dq_means_compute_kernel<<<blocks, 256, 0, st>>>((const uint16_t*)k_bf16, T, Hkv, tk.rotate, seq_id, pos,
+                                                    mean_q, mean_scale, max_windows);
     return cudaGetLastError();
 }
 
-cudaError_t dq_launch_encode(const DqDevTable& t, const void* x_bf16, int T, int Hkv,
-                             const int32_t* seq_id, const int32_t* pos, const int32_t* slot,
-                             uint8_t* cont, const int8_t* mean_q, const float* mean_scale,
-                             int max_windows, uint32_t* status, cudaStream_t st) {
-    const long long warps = (long long)T * Hkv;
-    if (warps == 0) return cudaSuccess;
+cudaError_t dq_launch_encode(const DqDevTable& tk, const DqDevTable& tv, const DqEncodeArgs& a, cudaStream_t st) {
+    const long long warps = (long long)a.T * a.Hkv;
+    if (warps == 0 || (!a.do_k && !a.do_v)) return cudaSuccess;
     const unsigned blocks = (unsigned)((warps + kEncWarps - 1) / kEncWarps);
-    dq_encode_kernel<<<blocks, kEncWarps * 32, 0, st>>>(t, (const uint16_t*)x_bf16, T, Hkv, seq_id,
-                                                        pos, slot, cont, mean_q, mean_scale,
-                                                        max_windows, status);
+    dq_encode_kernel<<<dim3(blocks, (a.do_k && a.do_v) ? 2 : 1), kEncWarps * 32, 0, st>>>(tk, tv, a);
     return cudaGetLastError();
 }

@@ -10,7 +10,8 @@
 struct DqDevTable {
     int M, rec, mstar, budget_bits;
     int has_mean, rotate, pad0, pad1;
-    uint32_t fc[DQ_MAX_LEVELS];  // f | c << 16           (encoder, Eq. rans Enc)
+    uint32_t enc_rcp[DQ_MAX_LEVELS];  // encoder, Eq. rans Enc by reciprocal: floor(x / f) = umulhi(x, rcp) >> rsh
+    uint32_t enc_aux[DQ_MAX_LEVELS];  // bias | (256 - f) << 10 | rsh << 19, bias = c (+ 255 when f = 1)
     float r[DQ_MAX_LEVELS];      // ideal cost in bits     (Algorithm 1)
     uint32_t R[DQ_MAX_LEVELS];   // ceil(r * 65536)
     uint32_t lut[256];           // f << 24 | fp16(level) << 8 | (z - c)   (Algorithm 2)
@@ -28,10 +29,20 @@ int dq_host_build(int levels, double bits_per_elem, const dq_table_opts* opts, d
 cudaError_t dq_launch_means(const DqDevTable& tk, const void* k_bf16, int T, int Hkv,
                             const int32_t* seq_id, const int32_t* pos, int8_t* mean_q,
                             float* mean_scale, int max_windows, int mode, cudaStream_t st);
-cudaError_t dq_launch_encode(const DqDevTable& t, const void* x_bf16, int T, int Hkv,
-                             const int32_t* seq_id, const int32_t* pos, const int32_t* slot,
-                             uint8_t* cont, const int8_t* mean_q, const float* mean_scale,
-                             int max_windows, uint32_t* status, cudaStream_t st);
+struct DqEncodeArgs {
+    const void* k_bf16;
+    const void* v_bf16;
+    const int32_t* seq_id;
+    const int32_t* pos;
+    const int32_t* slot;
+    uint8_t* k_cont;
+    uint8_t* v_cont;
+    int8_t* mean_q;
+    float* mean_scale;
+    uint32_t* status;
+    int T, Hkv, max_windows, mean_mode, do_k, do_v;
+};
+cudaError_t dq_launch_encode(const DqDevTable& tk, const DqDevTable& tv, const DqEncodeArgs& a, cudaStream_t st);
 cudaError_t dq_launch_decode_tokens(const DqDevTable& t, const uint8_t* cont, const int8_t* mean_q,
                                     const float* mean_scale, int max_windows, const int32_t* seq_id,
                                     const int32_t* pos, const int32_t* slot, int T, int Hkv,

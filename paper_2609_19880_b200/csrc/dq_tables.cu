@@ -158,7 +158,20 @@ int dq_host_build(int levels, double bits_per_elem, const dq_table_opts* opts, d
     d.has_mean = t.has_mean;
     d.rotate = t.rotate;
     for (int m = 0; m < levels; ++m) {
-        d.fc[m] = (uint32_t)t.f[m] | ((uint32_t)t.c[m] << 16);
+        // Enc(x, m) = floor(x / f) 2^p + x mod f + c = x + c + floor(x / f) (2^p - f); the quotient of a
+        // 31-bit x by f comes from one high multiply with rcp = ceil(2^(31 + s) / f), s = ceil(log2 f),
+        // followed by a shift of s - 1.  f = 1: rcp = 2^32 - 1 gives x - 1 and the bias absorbs it.
+        const uint32_t f = (uint32_t)t.f[m];
+        uint32_t rcp = 0xffffffffu, rsh = 0, bias = (uint32_t)t.c[m] + 255u;
+        if (f > 1) {
+            uint32_t s = 0;
+            while ((1u << s) < f) ++s;
+            rcp = (uint32_t)((((uint64_t)1 << (s + 31)) + f - 1) / f);
+            rsh = s - 1;
+            bias = (uint32_t)t.c[m];
+        }
+        d.enc_rcp[m] = rcp;
+        d.enc_aux[m] = bias | ((256u - f) << 10) | (rsh << 19);
         d.r[m] = t.r[m];
         d.R[m] = t.R[m];
     }

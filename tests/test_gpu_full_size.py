@@ -1,0 +1,208 @@
+"""Full-size GPU parity: the benchmark configurations at their real sizes, in the launch
+configuration bench.py times.  The oracle cannot redo millions of streams in seconds, so it
+is run on seeded samples: whole windows of tokens for the encoder (containers and means bit
+for bit), sampled tokens for the decoder, sampled (sequence, query head) rows for attention
+(each row needs every token of that sequence and KV head), plus properties that hold at any
+size."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_2609_19880_b200 as dq
+from paper_2609_19880_b200 import _build, workloads
+
+import gpu_common as gc
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _lib():
+    _build.build()
+    dq.lib()
+
+
+def _np(t):
+    return t.cpu().numpy()
+
+
+def _rec_view(cont):
+    """[pages, Hkv, 16, rec] -> [slot, Hkv, rec] view on the host."""
+    p, h, s, r = cont.shape
+    return cont.transpose(0, 2, 1, 3).reshape(p * s, h, r)
+
+
+def _host(cache):
+    return dict(kc=_np(cache.k_cont), vc=_np(cache.v_cont), mq=_np(cache.mean_q), ms=_np(cache.mean_scale))
+
+
+def _check_encoder_sample(w, ok, ov, host, rng, n_windows=6):
+    """Oracle re-encodes a few whole (sequence, window) runs (into compact containers of its
+    own) and compares their records and window means with what the GPU wrote."""
+    cfg = w.cfg
+    seq_id, pos, slot = _np(w.seq_id), _np(w.pos), _np(w.slot)
+    starts = np.concatenate([[0], np.cumsum(cfg.seq_lens)[:-1]])
+    picked = set()
+    for _ in range(n_windows):
+        b = int(rng.integers(0, cfg.batch))
+        nwin = (cfg.seq_lens[b] + 127) // 128
+        picked.add((b, int(rng.choice([0, nwin - 1, int(rng.integers(0, nwin))]))))
+    for (b, win) in sorted(picked):
+        lo = int(starts[b]) + win * 128
+        hi = int(starts[b]) + min(cfg.seq_lens[b], (win + 1) * 128)
+        assert (seq_id[lo:hi] == b).all() and (pos[lo:hi] // 128 == win).all()
+        kb, vb = workloads.bf16_bits(w.k[lo:hi]), workloads.bf16_bits(w.v[lo:hi])
+        n = hi - lo
+        compact = np.arange(n, dtype=np.int32)
+        mq = np.zeros((cfg.batch, w.max_windows, cfg.hkv, 128), np.int8)
+        ms = np.zeros((cfg.batch, w.max_windows, cfg.hkv), np.float32)
+        oracle.window_means(kb, seq_id[lo:hi], pos[lo:hi], mq, ms, 0)
+        kc = np.zeros(((n + 15) // 16, cfg.hkv, 16, ok.rec), np.uint8)
+        vc = np.zeros(((n + 15) // 16, cfg.hkv, 16, ov.rec), np.uint8)
+        oracle.encode_tokens(ok, kb, seq_id[lo:hi], pos[lo:hi], compact, kc, mq, ms)
+        oracle.encode_tokens(ov, vb, seq_id[lo:hi], pos[lo:hi], compact, vc)
+        sl = slot[lo:hi]
+        assert np.array_equal(mq[b, win], host["mq"][b, win]) and np.array_equal(ms[b, win], host["ms"][b, win])
+        assert np.array_equal(kc[compact // 16, :, compact % 16], host["kc"][sl // 16, :, sl % 16]), (b, win)
+        assert np.array_equal(vc[compact // 16, :, compact % 16], host["vc"][sl // 16, :, sl % 16]), (b, win)
+
+
+def _check_decoder_sample(w, tk, tv, ok, ov, cache, host, rng, n_tokens=256):
+    cfg = w.cfg
+    idx = np.sort(rng.choice(cfg.total_tokens, size=min(n_tokens, cfg.total_tokens), replace=False))
+    sel = torch.from_numpy(idx).to(w.k.device)
+    seq_id, pos, slot = w.seq_id[sel].contiguous(), w.pos[sel].contiguous(), w.slot[sel].contiguous()
+    kc, vc, mq, ms = host["kc"], host["vc"], host["mq"], host["ms"]
+    for (t_lib, t_or, cont_d, cont_h, m_q, m_s, mqd, msd) in (
+            (tk, ok, cache.k_cont, kc, mq, ms, cache.mean_q, cache.mean_scale),
+            (tv, ov, cache.v_cont, vc, None, None, None, None)):
+        sym_ref, deq_ref = oracle.decode_tokens(t_or, cont_h, _np(seq_id), _np(pos), _np(slot), cfg.hkv, m_q, m_s)
+        sym = torch.zeros(sym_ref.shape, dtype=torch.uint8, device="cuda")
+        deq = torch.zeros(deq_ref.shape, dtype=torch.float32, device="cuda")
+        dq.dq_decode_tokens(t_lib, cont_d, slot, cfg.hkv, sym, deq, mqd, msd, seq_id, pos)
+        torch.cuda.synchronize()
+        assert np.array_equal(_np(sym), sym_ref)
+        assert np.array_equal(_np(deq).view(np.uint32), deq_ref.view(np.uint32))
+
+
+def _check_attention_sample(w, tk, tv, ok, ov, cache, host, rng, rows=3, seq_lens=None):
+    cfg = w.cfg
+    out, out32 = gc.gpu_attention(w, tk, tv, cache, seq_lens=seq_lens)
+    assert torch.isfinite(out32).all()
+    lens = _np(w.seq_lens if seq_lens is None else seq_lens)
+    kc, vc, mq, ms = host["kc"], host["vc"], host["mq"], host["ms"]
+    qb, pt = workloads.bf16_bits(w.q), _np(w.page_table)
+    ref = np.full((cfg.batch, cfg.hq, 128), np.nan)
+    picked = []
+    order = np.argsort(lens)
+    cand_b = [int(order[0]), int(order[-1])] + [int(rng.integers(0, cfg.batch)) for _ in range(rows)]
+    for b in cand_b[:rows]:
+        hq = int(rng.integers(0, cfg.hq))
+        r = oracle.attention(ok, ov, qb, kc, vc, mq, ms, pt, lens, cfg.hkv, gc.SM_SCALE, only=(b, hq))
+        ref[b, hq] = r[b, hq]
+        picked.append((b, hq))
+    worst = gc.check_attention(out, out32, ref, rows=picked)
+    assert worst < 5e-4
+    return out32
+
+
+def _run_config(cfg, seed):
+    rng = np.random.default_rng(seed)
+    w = workloads.generate(cfg, device="cuda")
+    tk, tv, ok, ov = gc.tables(cfg)
+    cache = gc.GpuCache(w, ok.rec, ov.rec)
+    gc.gpu_encode(w, tk, tv, cache)
+    torch.cuda.synchronize()
+    st = _np(cache.status)
+    assert st[0] == 0 and st[3] <= max(ok.rec, ov.rec)     # every stream fits; no all-central fallback
+    host = _host(cache)
+    _check_encoder_sample(w, ok, ov, host, rng)
+    _check_decoder_sample(w, tk, tv, ok, ov, cache, host, rng)
+    _check_attention_sample(w, tk, tv, ok, ov, cache, host, rng)
+    return w, tk, tv, ok, ov, cache
+
+
+def test_config2_llama3_8b_full():
+    cfg = workloads.make_config(2)
+    assert cfg.total_tokens * cfg.hkv == 524288
+    _run_config(cfg, 2)
+
+
+@pytest.mark.parametrize("budget", [1.5, 2.0, 2.26, 3.0, 4.0])
+def test_config3_long_context_budget_sweep_full(budget):
+    cfg = workloads.make_config(3, budget=budget)
+    assert cfg.seq_lens == [131072] and cfg.hq // cfg.hkv == 8
+    _run_config(cfg, 30 + int(budget * 10))
+
+
+def test_config4_ragged_paged_full():
+    cfg = workloads.make_config(4)
+    assert cfg.batch == 128 and cfg.shuffle_pages
+    w, tk, tv, ok, ov, cache = _run_config(cfg, 4)
+    pt = _np(w.page_table)
+    assert not np.array_equal(pt[0, :8], np.sort(pt[0, :8]))     # pages really are shuffled
+
+
+def test_config5_encode_decode_loop_full():
+    """Prefill-encode 4 x 32768 tokens, then 256 decode steps, each appending one freshly
+    encoded token per sequence (means carried forward) before attention."""
+    cfg = workloads.make_config(5)
+    steps = cfg.decode_steps
+    assert steps == 256 and cfg.hq // cfg.hkv == 7
+    rng = np.random.default_rng(5)
+    w = workloads.generate(cfg, device="cuda", extra_tokens_per_seq=steps)
+    tk, tv, ok, ov = gc.tables(cfg)
+    cache = gc.GpuCache(w, ok.rec, ov.rec)
+    gc.gpu_encode(w, tk, tv, cache)
+    torch.cuda.synchronize()
+    _check_encoder_sample(w, ok, ov, _host(cache), rng, n_windows=4)
+
+    # oracle mirror of the append loop for one sequence: its last prefill window, then every step
+    b0 = int(rng.integers(0, cfg.batch))
+    L0 = cfg.seq_lens[b0]
+    start = int(np.cumsum([0] + cfg.seq_lens)[b0])
+    last_win = torch.arange(start + L0 - 128, start + L0, device="cuda")
+    _, _, mq_o, ms_o, _, _ = gc.oracle_encode(w, ok, ov, sel=last_win)
+    kc_o = np.zeros((w.num_pages, cfg.hkv, 16, ok.rec), np.uint8)
+    vc_o = np.zeros((w.num_pages, cfg.hkv, 16, ov.rec), np.uint8)
+
+    gen = torch.Generator(device="cuda").manual_seed(55)
+    lens = torch.tensor(cfg.seq_lens)
+    seq = torch.arange(cfg.batch, dtype=torch.int32)
+    pt_cpu = w.page_table.cpu()
+    out = torch.empty((cfg.batch, cfg.hq, 128), dtype=torch.bfloat16, device="cuda")
+    out32 = torch.empty((cfg.batch, cfg.hq, 128), dtype=torch.float32, device="cuda")
+    ws = torch.empty(dq.dq_decode_workspace_bytes(cfg.batch, cfg.hq, w.page_table.shape[1]), dtype=torch.uint8,
+                     device="cuda")
+    new_slots = []
+    for s in range(steps):
+        k1, v1 = workloads.make_kv(cfg, cfg.batch, gen, torch.device("cuda"), w.k_offsets, w.k_gain)
+        pos = (lens + s).to(torch.int32)
+        slot = (pt_cpu[seq.long(), (pos // 16).long()] * 16 + pos % 16).to(torch.int32)
+        dq.dq_encode_tokens(tk, tv, k1, v1, seq.cuda(), pos.cuda(), slot.cuda(), cache.k_cont, cache.v_cont,
+                            cache.mean_q, cache.mean_scale, dq.MEAN_REUSE, cache.status)
+        cur = (lens + s + 1).to(torch.int32).cuda()
+        dq.dq_decode_attention(tk, tv, w.q, cache.k_cont, cache.v_cont, cache.mean_q, cache.mean_scale,
+                               w.page_table, cur, cfg.hkv, gc.SM_SCALE, out, ws, out32)
+        kb, vb = workloads.bf16_bits(k1[b0:b0 + 1]), workloads.bf16_bits(v1[b0:b0 + 1])
+        sid, ps, sl = np.array([b0], np.int32), pos[b0:b0 + 1].numpy(), slot[b0:b0 + 1].numpy()
+        oracle.window_means(kb, sid, ps, mq_o, ms_o, 1)
+        oracle.encode_tokens(ok, kb, sid, ps, sl, kc_o, mq_o, ms_o)
+        oracle.encode_tokens(ov, vb, sid, ps, sl, vc_o)
+        new_slots.append(int(sl[0]))
+    torch.cuda.synchronize()
+    assert int(_np(cache.status)[0]) == 0
+    new_slots = np.array(new_slots)
+    kc, vc = _np(cache.k_cont), _np(cache.v_cont)
+    assert np.array_equal(_rec_view(kc)[new_slots], _rec_view(kc_o)[new_slots])
+    assert np.array_equal(_rec_view(vc)[new_slots], _rec_view(vc_o)[new_slots])
+    wins = slice(L0 // 128 - 1, (L0 + steps - 1) // 128 + 1)
+    assert np.array_equal(_np(cache.mean_q)[b0, wins], mq_o[b0, wins])
+    assert np.array_equal(_np(cache.mean_scale)[b0, wins], ms_o[b0, wins])
+    # attention of the last step against the oracle over the grown cache
+    final = (lens + steps).to(torch.int32).cuda()
+    _check_attention_sample(w, tk, tv, ok, ov, cache, _host(cache), rng, rows=3, seq_lens=final)
+    ref_rows = oracle.attention(ok, ov, workloads.bf16_bits(w.q), kc, vc, _np(cache.mean_q), _np(cache.mean_scale),
+                                _np(w.page_table), _np(final), cfg.hkv, gc.SM_SCALE, only=(b0, 3))
+    gc.check_attention(out, out32, ref_rows, rows=[(b0, 3)])     # the loop's own last output
