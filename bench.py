@@ -179,6 +179,22 @@ def run_reference(args):
 
 # --------------------------------------------------------------------------------- GPU leg
 
+def max_over_ranks(value: float, world: int, device="cpu") -> float:
+    """Slowest rank's figure (every rank gets it).  Replicas share nothing else."""
+    if world <= 1:
+        return float(value)
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([value], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def job_throughput(units_per_rank_per_step: float, seconds_per_step: float, world: int) -> float:
+    """Whole-job rate of `world` independent replicas timed by the slowest one (weak scaling)."""
+    return world * units_per_rank_per_step / seconds_per_step
+
+
 def run_ours(args):
     import torch
     import torch.distributed as dist
@@ -272,12 +288,9 @@ def run_ours(args):
     total_ms = e0.elapsed_time(e1)
     kern_ms = dq.dq_profile_read(4096)
     dq.dq_profile_enable(False)
-    if world > 1:
-        t = torch.tensor([total_ms], device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms = float(t.item())
+    total_ms = max_over_ranks(total_ms, world, dev)
     ms_per_step = total_ms / args.steps
-    value = world * kv_tokens / (ms_per_step * 1e-3)
+    value = job_throughput(kv_tokens, ms_per_step * 1e-3, world)
 
     if args.profile_only:   # short run for an ncu capture: no soak, no e2e, no baselines
         sampler.stop()
@@ -324,11 +337,8 @@ def run_ours(args):
         e2e_step(i)
     barrier()
     e2e_s = time.perf_counter() - t0
-    if world > 1:
-        t = torch.tensor([e2e_s], device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_s = float(t.item())
-    e2e_value = world * kv_tokens * args.steps / e2e_s
+    e2e_s = max_over_ranks(e2e_s, world, dev)
+    e2e_value = job_throughput(kv_tokens, e2e_s / args.steps, world)
 
     if rank != 0:
         if world > 1:
@@ -341,6 +351,10 @@ def run_ours(args):
     comp_bytes = token_heads * (cfg.k_rec + cfg.v_rec + 1.0)   # records + amortised INT8 mean byte
     roofline = None
     extra = {}
+    if args.traffic_bytes is None:
+        # ncu, config 2: dram__bytes_read + write = 37.62 MB for 524288 token-heads at 42 + 29 byte records;
+        # the kernel reads every record once, so traffic grows with the records' bytes
+        args.traffic_bytes = 37.62e6 * (token_heads * (cfg.k_rec + cfg.v_rec + 1.0)) / (524288 * 72.0)
     if k_ms:
         alu_peak = SM_COUNT * LANES_PER_SM_CLK * sm_max_mhz * 1e6 / 1e9          # G lane-ops / s
         alu_ach = symbols * ALU_OPS_PER_SYMBOL / (k_ms * 1e-3) / 1e9
@@ -426,7 +440,8 @@ def main():
     ap.add_argument("--profile-only", action="store_true",
                     help="warm-up and timed steps only (for profiler captures); prints a short line")
     ap.add_argument("--traffic-bytes", type=float, default=None,
-                    help="DRAM bytes per launch of the fused kernel from an ncu capture (reported as-is)")
+                    help="DRAM bytes per launch of the fused kernel from an ncu capture; default: the captured "
+                         "figure of profiles/dq_attention_kernel_config2_ncu.md scaled by the token-heads processed")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)

@@ -4,9 +4,8 @@
 // Launch sequence per call (one stream):
 //   dq_attn_prepare_kernel   rotate q (q' = H q / sqrt(128)), per-sequence block prefix
 //                            sums, reset of the work counter
-//   dq_attention_kernel      persistent, one CTA per SM; CTAs pull work items
-//                            (sequence, KV head, block of NW*32 tokens) from an atomic
-//                            counter.  Each warp owns 32 tokens of the item: lane l runs the
+//   dq_attention_kernel      persistent, one CTA per SM; work items (sequence, KV head,
+//                            block of NW*32 tokens) are dealt round-robin to the CTAs.  Each warp owns 32 tokens of the item: lane l runs the
 //                            rANS state machine of token l out of shared memory, levels go to
 //                            a small fp16 tile and from there into mma.sync contractions
 //                            against q' (keys) and the softmax weights (values).  s, o and
@@ -51,7 +50,7 @@ struct Item {
 
 struct Layout {
     int stage_k, stage_v;               // bytes of one warp's K (+ tail) / V record buffer
-    int off_lutk, off_lutv, off_prefix, off_q16, off_qsum, off_item, off_red, off_kst, off_vst, off_tiles,
+    int off_lutk, off_lutv, off_prefix, off_q16, off_qsum, off_red, off_pages, off_kst, off_vst, off_tiles,
         off_obuf, total;
     int warp_tile_bytes, warp_obuf_bytes;
 };
@@ -67,11 +66,11 @@ __host__ __device__ inline Layout make_layout(int nw, int rec_k, int rec_v, int 
     int o = 0;
     L.off_lutk = o; o += 256 * 32 * 4;
     L.off_lutv = o; o += 256 * 32 * 4;
-    L.off_prefix = o; o += align16((B + 1) * 4);
+    L.off_prefix = o; o += align16((2 * B + 1) * 4);   // block prefix sums, sequence lengths
     L.off_q16 = o; o += 2 * kQ16Bytes;
     L.off_qsum = o; o += 2 * DQ_MAX_GROUP * 4;
-    L.off_item = o; o += 3 * (int)sizeof(Item);
-    L.off_red = o; o += (kMaxWarps + 1) * DQ_MAX_GROUP * 4;
+    L.off_red = o; o += (kMaxWarps + 2) * DQ_MAX_GROUP * 4;
+    L.off_pages = o; o += kMaxWarps * 3 * 2 * 4 + 16;   // per warp: page ids of 3 items in flight; prev row
     L.off_kst = o; o += 2 * nw * L.stage_k;
     L.off_vst = o; o += 2 * nw * L.stage_v;
     L.off_tiles = o; o += nw * L.warp_tile_bytes;
@@ -305,18 +304,21 @@ dq_attention_kernel(const __grid_constant__ DqDevTable TK, const __grid_constant
 
     uint32_t* lutk = reinterpret_cast<uint32_t*>(smem + L.off_lutk);
     uint32_t* lutv = reinterpret_cast<uint32_t*>(smem + L.off_lutv);
-    int* prefix = reinterpret_cast<int*>(smem + L.off_prefix);
+    int* prefix = reinterpret_cast<int*>(smem + L.off_prefix);      // [B + 1] blocks before sequence b
+    int* s_len = prefix + (p.B + 1);                                // [B] clamped sequence lengths
     float* qsum = reinterpret_cast<float*>(smem + L.off_qsum);      // [2][8]
-    Item* items = reinterpret_cast<Item*>(smem + L.off_item);
-    float* red_m = reinterpret_cast<float*>(smem + L.off_red);      // [warp][head], then [head] maxima
-    float* red_M = red_m + kMaxWarps * DQ_MAX_GROUP;
+    float* red_m = reinterpret_cast<float*>(smem + L.off_red);      // [warp][head] chunk maxima
+    float* red_M = red_m + kMaxWarps * DQ_MAX_GROUP;                // [2][head] item maxima
     float* obuf_all = reinterpret_cast<float*>(smem + L.off_obuf);  // [warp][head][kORow]
 
     for (int i = tid; i < 256 * 32; i += nthreads) {
         lutk[i] = TK.lut[i >> 5];
         lutv[i] = TV.lut[i >> 5];
     }
-    for (int i = tid; i <= p.B; i += nthreads) prefix[i] = p.prefix[i];
+    for (int i = tid; i <= p.B; i += nthreads) {
+        prefix[i] = p.prefix[i];
+        if (i < p.B) s_len[i] = min(p.seq_lens[i], p.max_pages * DQ_PAGE_TOKENS);
+    }
     __syncthreads();
     const int total_items = prefix[p.B] * p.Hkv;
 
@@ -326,92 +328,102 @@ dq_attention_kernel(const __grid_constant__ DqDevTable TK, const __grid_constant
     const uint32_t one = (sbase >> 31) | 1u;
     const int g_row = lane >> 2, qd = lane & 3;
 
-    auto fetch_item = [&](int slot) {  // thread 0 only
+    // Items are dealt round-robin to the CTAs; every thread derives the descriptor itself from
+    // the tables in shared memory, so no broadcast or global atomic sits on the critical path.
+    // (Item indices of one CTA grow with n, so the sequence is found by walking forward from `hint`,
+    // the sequence of an earlier item.)
+    auto item_of = [&](int n, int hint) {
         Item it;
-        it.valid = 0; it.b = it.h = it.blk = it.len = it.bg = 0; it.pad0 = it.pad1 = 0;
-        const int idx = atomicAdd(p.counter, 1);
-        if (idx < total_items) {
+        it.valid = 0; it.b = hint; it.h = it.blk = it.len = it.bg = 0; it.pad0 = it.pad1 = 0;
+        const unsigned idx = blockIdx.x + (unsigned)n * gridDim.x;   // < 2^31: total_items is an int
+        if (idx < (unsigned)total_items) {
             it.valid = 1;
-            it.h = idx % p.Hkv;
-            it.bg = idx / p.Hkv;
-            int lo = 0, hi = p.B;
-            while (hi - lo > 1) {
-                const int mid = (lo + hi) >> 1;
-                if (prefix[mid] <= it.bg) lo = mid; else hi = mid;
-            }
-            it.b = lo;
-            it.blk = it.bg - prefix[lo];
-            it.len = min(p.seq_lens[lo], p.max_pages * DQ_PAGE_TOKENS);
+            it.bg = (int)(idx / (unsigned)p.Hkv);
+            it.h = (int)(idx - (unsigned)it.bg * (unsigned)p.Hkv);
+            int b = hint;
+            while (prefix[b + 1] <= it.bg) ++b;   // prefix[B] > bg because idx < total_items
+            it.b = b;
+            it.blk = it.bg - prefix[b];
+            it.len = s_len[b];
         }
-        items[slot] = it;
+        return it;
+    };
+    // The physical page ids of this warp's 32 tokens are fetched two items ahead by cp.async into
+    // a small ring in shared memory (slot n % 3), so neither their latency nor registers are spent.
+    int* my_pages = reinterpret_cast<int*>(smem + L.off_pages) + warp * 6;
+    long long* s_prev_row = reinterpret_cast<long long*>(smem + L.off_pages + kMaxWarps * 24);
+    auto fetch_pages = [&](int n, const Item& it) {
+        const int tok0 = (it.blk * nw + warp) * kChunk;
+        if (it.valid && tok0 < it.len && lane < 2 && tok0 + 16 * lane < it.len)
+            cp_async4(smem_addr(my_pages + (n % 3) * 2 + lane),
+                      p.page_table + (size_t)it.b * p.max_pages + (tok0 >> 4) + lane);
+    };
+    // cp.async of the K records, q'.mean values and q' operand of item n_k, V records of item n_v
+    auto issue_loads = [&](int nk, const Item& ik, int nv, const Item& iv) {
+        if (ik.valid) {
+            const uint32_t kst = sbase + L.off_kst + ((nk & 1) * nw + warp) * L.stage_k;
+            const int tok0 = (ik.blk * nw + warp) * kChunk;
+            if (tok0 < ik.len) {
+                const int npg = (tok0 + 16 < ik.len) ? 2 : 1;
+                for (int pg = 0; pg < npg; ++pg) {
+                    const uint8_t* ks = p.k_cont + ((size_t)my_pages[(nk % 3) * 2 + pg] * p.Hkv + ik.h) * (size_t)(16 * TK.rec);
+                    for (int i = lane; i < TK.rec; i += 32) cp_async16(kst + pg * 16 * TK.rec + i * 16, ks + i * 16);
+                }
+                if (p.has_mean && lane < G)
+                    cp_async4(kst + L.stage_k - kKTail + lane * 4,
+                              p.qmu + ((size_t)ik.b * p.Hq + (size_t)ik.h * G + lane) * p.windows + tok0 / DQ_WINDOW_TOKENS);
+            }
+            const uint16_t* qsrc = p.q16 + ((size_t)ik.b * p.Hkv + ik.h) * 16 * kN;
+            for (int i = tid; i < 16 * 16; i += nthreads)  // 16 rows x 16 chunks of 16 bytes
+                cp_async16(sbase + L.off_q16 + (nk & 1) * kQ16Bytes + (i >> 4) * kQ16Stride + (i & 15) * 16, qsrc + i * 8);
+            if (tid < G)
+                cp_async4(sbase + L.off_qsum + ((nk & 1) * DQ_MAX_GROUP + tid) * 4,
+                          p.qsum + (size_t)ik.b * p.Hq + (size_t)ik.h * G + tid);
+        }
+        if (iv.valid) {
+            const uint32_t vst = sbase + L.off_vst + ((nv & 1) * nw + warp) * L.stage_v;
+            const int tok0 = (iv.blk * nw + warp) * kChunk;
+            if (tok0 < iv.len) {
+                const int npg = (tok0 + 16 < iv.len) ? 2 : 1;
+                for (int pg = 0; pg < npg; ++pg) {
+                    const uint8_t* vs = p.v_cont + ((size_t)my_pages[(nv % 3) * 2 + pg] * p.Hkv + iv.h) * (size_t)(16 * TV.rec);
+                    for (int i = lane; i < TV.rec; i += 32) cp_async16(vst + pg * 16 * TV.rec + i * 16, vs + i * 16);
+                }
+            }
+        }
     };
 
-    // cp.async of the K records, q'.mean values and q' operand of item `nk`, V records of item `nv`
-    auto issue_loads = [&](int nk, int nv) {
-        if (nk >= 0) {
-            const Item it = items[nk % 3];
-            if (it.valid) {
-                const uint32_t kst = sbase + L.off_kst + ((nk & 1) * nw + warp) * L.stage_k;
-                const int tok0 = (it.blk * nw + warp) * kChunk;
-                if (tok0 < it.len) {
-                    const int32_t* pt = p.page_table + (size_t)it.b * p.max_pages + (tok0 >> 4);
-                    const int npg = (tok0 + 16 < it.len) ? 2 : 1;
-                    for (int pg = 0; pg < npg; ++pg) {
-                        const uint8_t* ks = p.k_cont + ((size_t)pt[pg] * p.Hkv + it.h) * (size_t)(16 * TK.rec);
-                        for (int i = lane; i < TK.rec; i += 32) cp_async16(kst + pg * 16 * TK.rec + i * 16, ks + i * 16);
-                    }
-                    if (p.has_mean && lane < G)
-                        cp_async4(kst + L.stage_k - kKTail + lane * 4,
-                                  p.qmu + ((size_t)it.b * p.Hq + (size_t)it.h * G + lane) * p.windows +
-                                      tok0 / DQ_WINDOW_TOKENS);
-                }
-                const uint16_t* qsrc = p.q16 + ((size_t)it.b * p.Hkv + it.h) * 16 * kN;
-                for (int i = tid; i < 16 * 16; i += nthreads)  // 16 rows x 16 chunks of 16 bytes
-                    cp_async16(sbase + L.off_q16 + (nk & 1) * kQ16Bytes + (i >> 4) * kQ16Stride + (i & 15) * 16,
-                               qsrc + i * 8);
-                if (tid < G)
-                    cp_async4(sbase + L.off_qsum + ((nk & 1) * DQ_MAX_GROUP + tid) * 4,
-                              p.qsum + (size_t)it.b * p.Hq + (size_t)it.h * G + tid);
-            }
-        }
-        if (nv >= 0) {
-            const Item it = items[nv % 3];
-            if (it.valid) {
-                const uint32_t vst = sbase + L.off_vst + ((nv & 1) * nw + warp) * L.stage_v;
-                const int tok0 = (it.blk * nw + warp) * kChunk;
-                if (tok0 < it.len) {
-                    const int32_t* pt = p.page_table + (size_t)it.b * p.max_pages + (tok0 >> 4);
-                    const int npg = (tok0 + 16 < it.len) ? 2 : 1;
-                    for (int pg = 0; pg < npg; ++pg) {
-                        const uint8_t* vs = p.v_cont + ((size_t)pt[pg] * p.Hkv + it.h) * (size_t)(16 * TV.rec);
-                        for (int i = lane; i < TV.rec; i += 32) cp_async16(vst + pg * 16 * TV.rec + i * 16, vs + i * 16);
-                    }
-                }
-            }
-        }
+    // prologue: page ids of items 0 and 1, then the K records of item 0
+    int hint = 0;   // sequence of the current item: search start for later items
+    {
+        const Item i0 = item_of(0, 0);
+        fetch_pages(0, i0);
+        fetch_pages(1, item_of(1, i0.b));
         cp_async_commit();
-    };
-
-    if (tid == 0) fetch_item(0);
-    __syncthreads();
-    issue_loads(0, -1);
+        cp_async_wait<0>();
+        __syncwarp();
+        Item none = i0; none.valid = 0;
+        issue_loads(0, i0, 0, none);
+        cp_async_commit();
+        hint = i0.b;
+    }
 
     // state carried from the item whose V streams are still to be decoded
     bool have_prev = false;
-    Item prev = items[0];
     uint32_t pb_hi[2][2] = {{0u, 0u}, {0u, 0u}}, pb_lo[2][2] = {{0u, 0u}, {0u, 0u}};
 
     for (int n = 0;; ++n) {
-        const Item cur = items[n % 3];
+        Item cur = item_of(n, hint);
         if (!cur.valid && !have_prev) break;
-        if (tid == 0) {
-            if (cur.valid) fetch_item((n + 1) % 3);
-            else items[(n + 1) % 3].valid = 0;
+        hint = cur.b;
+        {   // records of item n + 1 (its page ids arrived last iteration), page ids of item n + 2
+            const Item nxt = item_of(n + 1, cur.b);
+            issue_loads(n + 1, nxt, n, cur);
+            fetch_pages(n + 2, item_of(n + 2, nxt.b));
+            cp_async_commit();
         }
-        __syncthreads();
-        issue_loads(n + 1, cur.valid ? n : -1);
         cp_async_wait<1>();
-        __syncthreads();
+        __syncthreads();   // q' operand of `cur` visible; last iteration's merge reads are done
 
         // ------------------------------------------ K streams of `cur`, V streams of `prev`
         const int tok0 = (cur.blk * nw + warp) * kChunk;
@@ -435,24 +447,9 @@ dq_attention_kernel(const __grid_constant__ DqDevTable TK, const __grid_constant
                                         sacc, pb_hi, pb_lo);
         }
 
-        // ------------------------------------------ finish `prev`: sum its warps' slots, write the partial
-        if (have_prev) {
-            __syncthreads();
-            for (int e = tid; e < G * 130; e += nthreads) {
-                const int g = e / 130, col = e - g * 130;
-                float s = 0.f;
-                for (int w = 0; w < nw; ++w) s += obuf_all[(w * G + g) * kORow + col];
-                float* dst = p.partial + ((size_t)prev.bg * p.Hq + (size_t)prev.h * G + g) * kPartial;
-                if (col < kN) dst[col] = s;
-                else dst[col + 1] = s;                       // l at 129, off at 130
-                if (col == 0) dst[kN] = red_M[g];
-            }
-        }
-
-        // ------------------------------------------ softmax weights of `cur` (base 2)
-        have_prev = cur.valid;
+        // ------------------------------------------ logits of `cur` and this warp's maximum (base 2)
+        float lg[4][2], sv_t[4][2], ov_t[4][2];
         if (cur.valid) {
-            prev = cur;
             cp_async_wait<0>();   // the V records of `cur` (header needed now) have landed
             __syncwarp();
             const uint32_t rv = sbase + L.off_vst + ((n & 1) * nw + warp) * L.stage_v + lane * TV.rec;
@@ -471,7 +468,6 @@ dq_attention_kernel(const __grid_constant__ DqDevTable TK, const __grid_constant
                 if (p.has_mean && tok0 < cur.len) qmu = __uint_as_float(lds32(kst + L.stage_k - kKTail + g_row * 4));
             }
             __syncwarp();
-            float lg[4][2], sv_t[4][2], ov_t[4][2];
             float mx = -INFINITY;
 #pragma unroll
             for (int i = 0; i < 4; ++i)
@@ -490,12 +486,31 @@ dq_attention_kernel(const __grid_constant__ DqDevTable TK, const __grid_constant
                 }
             mx = fmaxf(mx, __shfl_xor_sync(kFullMask, mx, 1));
             mx = fmaxf(mx, __shfl_xor_sync(kFullMask, mx, 2));
-            // item-wide maximum per head, so that every warp's weights share one scale
             if (qd == 0) red_m[warp * DQ_MAX_GROUP + g_row] = mx;
-            __syncthreads();
+        }
+        __syncthreads();   // output slots of `prev` complete; chunk maxima of `cur` published
+
+        // ------------------------------------------ finish `prev`: sum its warps' slots, write the partial
+        if (have_prev) {
+            const int lcol = kN + 2 * ((n + 1) & 1);   // l, off columns written when `prev` was `cur`
+            for (int e = tid; e < G * 130; e += nthreads) {
+                const int g = e / 130, col = e - g * 130;
+                const int src = col < kN ? col : lcol + (col - kN);
+                float s = 0.f;
+                for (int w = 0; w < nw; ++w) s += obuf_all[(w * G + g) * kORow + src];
+                float* dst = p.partial + ((size_t)s_prev_row[(n + 1) & 1] + g) * kPartial;
+                if (col < kN) dst[col] = s;
+                else dst[col + 1] = s;                       // l at 129, off at 130
+                if (col == 0) dst[kN] = red_M[((n + 1) & 1) * DQ_MAX_GROUP + g];
+            }
+        }
+
+        // ------------------------------------------ softmax weights of `cur`, scaled by the item maximum
+        have_prev = cur.valid;
+        if (cur.valid) {
             float m_item = -INFINITY;
             for (int w = 0; w < nw; ++w) m_item = fmaxf(m_item, red_m[w * DQ_MAX_GROUP + g_row]);
-            if (warp == 0 && qd == 0) red_M[g_row] = m_item;
+            if (warp == 0 && qd == 0) red_M[(n & 1) * DQ_MAX_GROUP + g_row] = m_item;
             const float m_use = (m_item == -INFINITY) ? 0.f : m_item;
             float lsum = 0.f, osum = 0.f;
 #pragma unroll
@@ -517,11 +532,12 @@ dq_attention_kernel(const __grid_constant__ DqDevTable TK, const __grid_constant
             lsum += __shfl_xor_sync(kFullMask, lsum, 2);
             osum += __shfl_xor_sync(kFullMask, osum, 1);
             osum += __shfl_xor_sync(kFullMask, osum, 2);
-            if (qd == 0 && g_row < G) {   // l and off ride along in this warp's output slot
-                sts32f(my_obuf + (g_row * kORow + kN) * 4, lsum);
-                sts32f(my_obuf + (g_row * kORow + kN + 1) * 4, osum);
+            if (qd == 0 && g_row < G) {   // l and off ride along in this warp's output slot (columns by parity)
+                sts32f(my_obuf + (g_row * kORow + kN + 2 * (n & 1)) * 4, lsum);
+                sts32f(my_obuf + (g_row * kORow + kN + 2 * (n & 1) + 1) * 4, osum);
             }
         }
+        if (tid == 0) s_prev_row[n & 1] = (long long)cur.bg * p.Hq + (long long)cur.h * G;   // read after two barriers
     }
     cp_async_wait<0>();
 }
