@@ -181,8 +181,9 @@ int dq_bf16_decode_attention(const void *q_bf16, const void *k_bf16_pages, const
                              int B, int Hq, int Hkv, float sm_scale, void *out_bf16,
                              void *workspace, size_t workspace_bytes, void *cuda_stream);
 
-/* Measurement aid (no counterpart in the paper): while enabled, every dq_decode_attention
- * call records CUDA events on its stream around the fused kernel (up to 4096 calls).
+/* Measurement aid (no counterpart in the paper): while enabled (on > 0), every on-th
+ * dq_decode_attention call records CUDA events on its stream around the fused kernel (up to
+ * 4096 records; the events keep that call's kernels from overlapping their neighbours).
  * dq_profile_read waits for them, writes the kernel durations in milliseconds (host array,
  * call order) and clears the record; returns how many it wrote.  Not thread-safe. */
 void dq_profile_enable(int on);

@@ -213,8 +213,9 @@ def dq_bf16_decode_attention(q_bf16, k_pages, v_pages, page_table, seq_lens, Hkv
     _check(rc, "dq_bf16_decode_attention")
 
 
-def dq_profile_enable(on: bool):
-    lib().dq_profile_enable(int(bool(on)))
+def dq_profile_enable(on):
+    """0 / False: off; k > 0: time the fused kernel of every k-th dq_decode_attention call."""
+    lib().dq_profile_enable(int(on))
 
 
 def dq_profile_read(max_records: int = 4096):

@@ -108,6 +108,8 @@ struct AttnParams {
 constexpr int kPrepWindows = 8;
 __global__ void __launch_bounds__(256)
 dq_attn_prepare_kernel(AttnParams p) {
+    pdl_launch_dependents();
+    pdl_wait_prior_grid();   // q, the window means and seq_lens may come from the previous kernel
     const int lane = threadIdx.x & 31;
     const long long wid = (long long)blockIdx.x * 8 + (threadIdx.x >> 5);
     const int heads = p.B * p.Hq;
@@ -311,10 +313,12 @@ dq_attention_kernel(const __grid_constant__ DqDevTable TK, const __grid_constant
     float* red_M = red_m + kMaxWarps * DQ_MAX_GROUP;                // [2][head] item maxima
     float* obuf_all = reinterpret_cast<float*>(smem + L.off_obuf);  // [warp][head][kORow]
 
-    for (int i = tid; i < 256 * 32; i += nthreads) {
+    pdl_launch_dependents();
+    for (int i = tid; i < 256 * 32; i += nthreads) {   // tables come from the kernel parameters
         lutk[i] = TK.lut[i >> 5];
         lutv[i] = TV.lut[i >> 5];
     }
+    pdl_wait_prior_grid();   // everything below reads what the prepare kernel wrote
     for (int i = tid; i <= p.B; i += nthreads) {
         prefix[i] = p.prefix[i];
         if (i < p.B) s_len[i] = min(p.seq_lens[i], p.max_pages * DQ_PAGE_TOKENS);
@@ -544,38 +548,66 @@ dq_attention_kernel(const __grid_constant__ DqDevTable TK, const __grid_constant
 
 // ------------------------------------------------------------------ combine
 
+// One CTA of 8 warps per (sequence, query head): warp w merges partials w*4 .. w*4+3, w*4+32 ...
+// with a running maximum, the warps are merged through shared memory, warp 0 normalises,
+// applies the inverse rotation and stores.
 __global__ void __launch_bounds__(256)
 dq_attn_combine_kernel(AttnParams p) {
-    const int lane = threadIdx.x & 31;
-    const int wid = blockIdx.x * 8 + (threadIdx.x >> 5);
-    if (wid >= p.B * p.Hq) return;
+    pdl_launch_dependents();
+    pdl_wait_prior_grid();
+    __shared__ float s_acc[8][kN];
+    __shared__ float s_mlo[8][4];
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+    const int wid = blockIdx.x;
     const int b = wid / p.Hq, hq = wid % p.Hq;
     const int bg0 = p.prefix[b], nb = p.prefix[b + 1] - bg0;
     const float* base = p.partial + ((size_t)bg0 * p.Hq + hq) * kPartial;
     const size_t stride = (size_t)p.Hq * kPartial;
+    float acc[4] = {0.f, 0.f, 0.f, 0.f}, lsum = 0.f, osum = 0.f, m_run = -INFINITY;
+    for (int i0 = 4 * w; i0 < nb; i0 += 32) {   // four partials in flight per warp
+        float4 v[4];
+        float m[4], l[4], o[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const float* src = base + (size_t)min(i0 + u, nb - 1) * stride;
+            v[u] = *reinterpret_cast<const float4*>(src + 4 * lane);
+            m[u] = (i0 + u < nb) ? src[kN] : -INFINITY;
+            l[u] = src[kN + 1]; o[u] = src[kN + 2];
+        }
+        const float m_new = fmaxf(fmaxf(fmaxf(m[0], m[1]), fmaxf(m[2], m[3])), m_run);
+        if (m_new == -INFINITY) continue;
+        const float keep = exp2f(m_run - m_new);
+#pragma unroll
+        for (int e = 0; e < 4; ++e) acc[e] *= keep;
+        lsum *= keep; osum *= keep;
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const float sc = exp2f(m[u] - m_new);   // 0 for the padding entries
+            acc[0] = fmaf(v[u].x, sc, acc[0]); acc[1] = fmaf(v[u].y, sc, acc[1]);
+            acc[2] = fmaf(v[u].z, sc, acc[2]); acc[3] = fmaf(v[u].w, sc, acc[3]);
+            lsum = fmaf(l[u], sc, lsum);
+            osum = fmaf(o[u], sc, osum);            // Eq. fold-value: + sum_t a_t o_t
+        }
+        m_run = m_new;
+    }
+    *reinterpret_cast<float4*>(&s_acc[w][4 * lane]) = make_float4(acc[0], acc[1], acc[2], acc[3]);
+    if (lane == 0) { s_mlo[w][0] = m_run; s_mlo[w][1] = lsum; s_mlo[w][2] = osum; }
+    __syncthreads();
+    if (w != 0) return;
     float mx = -INFINITY;
-    for (int i = lane; i < nb; i += 32) mx = fmaxf(mx, base[i * stride + kN]);
 #pragma unroll
-    for (int d = 16; d >= 1; d >>= 1) mx = fmaxf(mx, __shfl_xor_sync(kFullMask, mx, d));
-    float acc[4] = {0.f, 0.f, 0.f, 0.f}, lsum = 0.f, osum = 0.f;
+    for (int i = 0; i < 8; ++i) mx = fmaxf(mx, s_mlo[i][0]);
+    acc[0] = acc[1] = acc[2] = acc[3] = 0.f;
+    lsum = osum = 0.f;
     if (mx != -INFINITY) {
-        for (int i0 = 0; i0 < nb; i0 += 4) {   // four partials in flight
-            float4 v[4];
-            float m[4], l[4], o[4];
 #pragma unroll
-            for (int u = 0; u < 4; ++u) {
-                const float* src = base + (size_t)min(i0 + u, nb - 1) * stride;
-                v[u] = *reinterpret_cast<const float4*>(src + 4 * lane);
-                m[u] = src[kN]; l[u] = src[kN + 1]; o[u] = src[kN + 2];
-            }
-#pragma unroll
-            for (int u = 0; u < 4; ++u) {
-                const float sc = (i0 + u < nb) ? exp2f(m[u] - mx) : 0.f;
-                acc[0] = fmaf(v[u].x, sc, acc[0]); acc[1] = fmaf(v[u].y, sc, acc[1]);
-                acc[2] = fmaf(v[u].z, sc, acc[2]); acc[3] = fmaf(v[u].w, sc, acc[3]);
-                lsum = fmaf(l[u], sc, lsum);
-                osum = fmaf(o[u], sc, osum);    // Eq. fold-value: + sum_t a_t o_t
-            }
+        for (int i = 0; i < 8; ++i) {
+            const float sc = exp2f(s_mlo[i][0] - mx);
+            const float4 v = *reinterpret_cast<const float4*>(&s_acc[i][4 * lane]);
+            acc[0] = fmaf(v.x, sc, acc[0]); acc[1] = fmaf(v.y, sc, acc[1]);
+            acc[2] = fmaf(v.z, sc, acc[2]); acc[3] = fmaf(v.w, sc, acc[3]);
+            lsum = fmaf(s_mlo[i][1], sc, lsum);
+            osum = fmaf(s_mlo[i][2], sc, osum);
         }
         const float inv = 1.0f / lsum;
 #pragma unroll
@@ -586,10 +618,10 @@ dq_attn_combine_kernel(AttnParams p) {
         *reinterpret_cast<float4*>(p.out_f32 + (size_t)wid * kN + 4 * lane) = make_float4(acc[0], acc[1], acc[2], acc[3]);
     if (p.out_bf16) {
         const __nv_bfloat162 lo = __floats2bfloat162_rn(acc[0], acc[1]), hi = __floats2bfloat162_rn(acc[2], acc[3]);
-        uint2 w;
-        w.x = *reinterpret_cast<const uint32_t*>(&lo);
-        w.y = *reinterpret_cast<const uint32_t*>(&hi);
-        *reinterpret_cast<uint2*>(reinterpret_cast<uint16_t*>(p.out_bf16) + (size_t)wid * kN + 4 * lane) = w;
+        uint2 wv;
+        wv.x = *reinterpret_cast<const uint32_t*>(&lo);
+        wv.y = *reinterpret_cast<const uint32_t*>(&hi);
+        *reinterpret_cast<uint2*>(reinterpret_cast<uint16_t*>(p.out_bf16) + (size_t)wid * kN + 4 * lane) = wv;
     }
 }
 
@@ -614,6 +646,8 @@ __device__ __forceinline__ void mma_bf16_16816(float (&d)[4], const uint32_t (&a
 __global__ void __launch_bounds__(kBfWarps * 32)
 dq_bf16_attention_kernel(const AttnParams p, const uint16_t* __restrict__ kp, const uint16_t* __restrict__ vp) {
     extern __shared__ __align__(128) uint8_t smem[];
+    pdl_launch_dependents();
+    pdl_wait_prior_grid();
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int b = blockIdx.z, h = blockIdx.y, blk = blockIdx.x, G = p.G;
     const int bg0 = p.prefix[b];
@@ -777,13 +811,16 @@ size_t dq_attn_workspace_bytes(int B, int Hq, int max_pages) { return ws_layout(
 namespace {
 constexpr int kProfRing = 4096;
 bool g_prof_on = false;
+int g_prof_period = 1, g_prof_calls = 0;
 int g_prof_count = 0;
 cudaEvent_t g_prof_ev[kProfRing][2];
 bool g_prof_made[kProfRing];
 }  // namespace
 
 void dq_attn_profile_enable(int on) {
-    g_prof_on = on != 0;
+    g_prof_on = on > 0;
+    g_prof_period = on > 0 ? on : 1;   // record every on-th call
+    g_prof_calls = 0;
     g_prof_count = 0;
 }
 
@@ -843,12 +880,11 @@ cudaError_t dq_launch_attention(const DqDevTable& tk, const DqDevTable& tv, cons
 
     const int heads = a.B * a.Hq;
     const long long prep_warps = (long long)heads * (1 + (p.has_mean ? (p.windows + kPrepWindows - 1) / kPrepWindows : 0));
-    dq_attn_prepare_kernel<<<(unsigned)((prep_warps + 7) / 8), 256, 0, st>>>(p);
-    cudaError_t e = cudaGetLastError();
+    cudaError_t e = dq_launch_pdl(dq_attn_prepare_kernel, dim3((unsigned)((prep_warps + 7) / 8)), dim3(256), 0, st, p);
     if (e != cudaSuccess) return e;
     e = cudaFuncSetAttribute(dq_attention_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, L.total);
     if (e != cudaSuccess) return e;
-    const bool prof = g_prof_on && g_prof_count < kProfRing;
+    const bool prof = g_prof_on && g_prof_count < kProfRing && (g_prof_calls++ % g_prof_period) == 0;
     if (prof) {
         if (!g_prof_made[g_prof_count]) {
             if ((e = cudaEventCreate(&g_prof_ev[g_prof_count][0])) != cudaSuccess) return e;
@@ -857,12 +893,10 @@ cudaError_t dq_launch_attention(const DqDevTable& tk, const DqDevTable& tv, cons
         }
         cudaEventRecord(g_prof_ev[g_prof_count][0], st);
     }
-    dq_attention_kernel<<<sm_count, nw * 32, L.total, st>>>(tk, tv, p);
-    e = cudaGetLastError();
+    e = dq_launch_pdl(dq_attention_kernel, dim3(sm_count), dim3(nw * 32), (size_t)L.total, st, tk, tv, p);
     if (e != cudaSuccess) return e;
     if (prof) cudaEventRecord(g_prof_ev[g_prof_count++][1], st);
-    dq_attn_combine_kernel<<<(heads + 7) / 8, 256, 0, st>>>(p);
-    return cudaGetLastError();
+    return dq_launch_pdl(dq_attn_combine_kernel, dim3(heads), dim3(256), 0, st, p);
 }
 
 cudaError_t dq_launch_bf16_attention(const DqAttnArgs& a, const void* k_pages, const void* v_pages,
@@ -897,8 +931,7 @@ cudaError_t dq_launch_bf16_attention(const DqAttnArgs& a, const void* k_pages, c
         p, static_cast<const uint16_t*>(k_pages), static_cast<const uint16_t*>(v_pages));
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;
-    dq_attn_combine_kernel<<<(heads + 7) / 8, 256, 0, st>>>(p);
-    return cudaGetLastError();
+    return dq_launch_pdl(dq_attn_combine_kernel, dim3(heads), dim3(256), 0, st, p);
 }
 
 // ------------------------------------------------ attention without any allocation

@@ -69,8 +69,11 @@ dq_means_compute_kernel(const uint16_t* __restrict__ k, int T, int Hkv, int rota
 struct EncTable {
     float r[DQ_MAX_LEVELS];
     uint32_t R[DQ_MAX_LEVELS];
-    uint32_t rcp[DQ_MAX_LEVELS];
-    uint32_t aux[DQ_MAX_LEVELS];
+    uint32_t rcp[DQ_MAX_LEVELS];   // Eq. rans Enc by reciprocal: floor(x / f) = umulhi(x, rcp) >> rsh
+    uint32_t rsh[DQ_MAX_LEVELS];
+    uint32_t bias[DQ_MAX_LEVELS];  // c (+ 255 when f = 1)
+    uint32_t cmpl[DQ_MAX_LEVELS];  // 2^p - f
+    uint32_t thr[DQ_MAX_LEVELS];   // f << 23: renormalise while the state is not below it
     int M, rec, mstar, budget_bits, has_mean, rotate;
 };
 
@@ -79,20 +82,32 @@ struct EncTable {
 // [hi * 2^-40, hi], hi = 8 (max D - min D); the code length is an integer sum of
 // ceil(65536 r_m), so the feasibility test does not depend on summation order.
 // Returns the length of the final assignment (the argmin at the bracket's upper end).
-__device__ __forceinline__ uint32_t drift(const EncTable& T, const float (&z)[4], float s, float o,
-                                          uint32_t (&sym)[4]) {
-    const int M = T.M;
-    float maxD = -INFINITY, minD = INFINITY;
-    for (int m = 0; m < M; ++m) {
-        const float tm = __fmaf_rn((float)m, s, o);
+// M is a template parameter so that the M candidate costs of a value are independent
+// instructions and the table sits in registers; the minimum keeps the lowest index among equal
+// costs, exactly as an ascending scan with a strict comparison does.
+template <int M>
+__device__ __noinline__ uint32_t drift_m(const EncTable& T, float z0, float z1, float z2, float z3, float s, float o,
+                                         uint32_t& sym_packed) {
+    const float z[4] = {z0, z1, z2, z3};
+    float tm[M], rm[M];
+    uint32_t Rm[M];
 #pragma unroll
-        for (int e = 0; e < 4; ++e) {
-            const float d = __fsub_rn(z[e], tm);
-            const float D = __fmul_rn(d, d);
-            maxD = fmaxf(maxD, D);
-            minD = fminf(minD, D);
-        }
+    for (int m = 0; m < M; ++m) {
+        tm[m] = __fmaf_rn((float)m, s, o);
+        rm[m] = T.r[m];
+        Rm[m] = T.R[m];
     }
+    float D[4][M];
+    float maxD = -INFINITY, minD = INFINITY;
+#pragma unroll
+    for (int e = 0; e < 4; ++e)
+#pragma unroll
+        for (int m = 0; m < M; ++m) {
+            const float d = __fsub_rn(z[e], tm[m]);
+            D[e][m] = __fmul_rn(d, d);
+            maxD = fmaxf(maxD, D[e][m]);
+            minD = fminf(minD, D[e][m]);
+        }
 #pragma unroll
     for (int d = 16; d >= 1; d >>= 1) {
         maxD = fmaxf(maxD, __shfl_xor_sync(kFull, maxD, d));
@@ -101,27 +116,51 @@ __device__ __forceinline__ uint32_t drift(const EncTable& T, const float (&z)[4]
     const uint32_t budget = (uint32_t)T.budget_bits << 16;
     float lam_hi = __fmul_rn(8.0f, __fsub_rn(maxD, minD));
     float lam_lo = __fmul_rn(lam_hi, 0x1p-40f);
-    uint32_t len = 0;
+    uint32_t len = 0, sym[4] = {0u, 0u, 0u, 0u};
+#pragma unroll 1
     for (int it = 0; it <= 12; ++it) {
         const float lam = (it < 12) ? __fsqrt_rn(__fmul_rn(lam_lo, lam_hi)) : lam_hi;
-        float best[4];
-        uint32_t cost_fx[4];
-        for (int m = 0; m < M; ++m) {
-            const float tm = __fmaf_rn((float)m, s, o);
-            const float rm = T.r[m];
-            const uint32_t Rm = T.R[m];
+        uint32_t cost_sum = 0;
 #pragma unroll
-            for (int e = 0; e < 4; ++e) {
-                const float d = __fsub_rn(z[e], tm);
-                const float c = __fmaf_rn(lam, rm, __fmul_rn(d, d));
-                if (m == 0 || c < best[e]) { best[e] = c; sym[e] = (uint32_t)m; cost_fx[e] = Rm; }
-            }
+        for (int e = 0; e < 4; ++e) {
+            float c[M];
+            uint32_t idx[M];
+#pragma unroll
+            for (int m = 0; m < M; ++m) { c[m] = __fmaf_rn(lam, rm[m], D[e][m]); idx[m] = (uint32_t)m; }
+            // pairwise minimum, the left (lower index) operand wins ties
+#pragma unroll
+            for (int w = 1; w < M; w <<= 1)
+#pragma unroll
+                for (int m = 0; m + w < M; m += 2 * w)
+                    if (c[m + w] < c[m]) { c[m] = c[m + w]; idx[m] = idx[m + w]; }
+            sym[e] = idx[0];
+            uint32_t Rsel = Rm[0];
+#pragma unroll
+            for (int m = 1; m < M; ++m) Rsel = (idx[0] == (uint32_t)m) ? Rm[m] : Rsel;
+            cost_sum += Rsel;
         }
-        len = __reduce_add_sync(kFull, cost_fx[0] + cost_fx[1] + cost_fx[2] + cost_fx[3]);
+        len = __reduce_add_sync(kFull, cost_sum);
         if (it < 12) {
             if (len <= budget) lam_hi = lam; else lam_lo = lam;
         }
     }
+    sym_packed = sym[0] | (sym[1] << 8) | (sym[2] << 16) | (sym[3] << 24);
+    return len;
+}
+
+__device__ __forceinline__ uint32_t drift(const EncTable& T, const float (&z)[4], float s, float o,
+                                          uint32_t (&sym)[4]) {
+    uint32_t packed = 0, len = 0;
+    switch (T.M) {   // uniform across the CTA
+#define DQ_DRIFT_CASE(M_) case M_: len = drift_m<M_>(T, z[0], z[1], z[2], z[3], s, o, packed); break;
+        DQ_DRIFT_CASE(2) DQ_DRIFT_CASE(3) DQ_DRIFT_CASE(4) DQ_DRIFT_CASE(5) DQ_DRIFT_CASE(6) DQ_DRIFT_CASE(7)
+        DQ_DRIFT_CASE(8) DQ_DRIFT_CASE(9) DQ_DRIFT_CASE(10) DQ_DRIFT_CASE(11) DQ_DRIFT_CASE(12) DQ_DRIFT_CASE(13)
+        DQ_DRIFT_CASE(14) DQ_DRIFT_CASE(15) DQ_DRIFT_CASE(16)
+#undef DQ_DRIFT_CASE
+        default: break;
+    }
+#pragma unroll
+    for (int e = 0; e < 4; ++e) sym[e] = (packed >> (8 * e)) & 0xffu;
     return len;
 }
 
@@ -137,13 +176,18 @@ dq_encode_kernel(const __grid_constant__ DqDevTable TK, const __grid_constant__ 
     __shared__ EncTable T;
     __shared__ uint8_t s_bytes[kEncWarps][DQ_MAX_REC_BYTES];
     __shared__ __align__(4) uint8_t s_sym[kEncWarps][kN];
+    dqdev::pdl_launch_dependents();
     const bool is_v = a.do_k ? (blockIdx.y == 1) : true;
     if (threadIdx.x < DQ_MAX_LEVELS) {
         const int i = threadIdx.x;
         T.r[i] = is_v ? TV.r[i] : TK.r[i];
         T.R[i] = is_v ? TV.R[i] : TK.R[i];
         T.rcp[i] = is_v ? TV.enc_rcp[i] : TK.enc_rcp[i];
-        T.aux[i] = is_v ? TV.enc_aux[i] : TK.enc_aux[i];
+        const uint32_t aux = is_v ? TV.enc_aux[i] : TK.enc_aux[i];
+        T.bias[i] = aux & 1023u;
+        T.cmpl[i] = (aux >> 10) & 511u;
+        T.rsh[i] = aux >> 19;
+        T.thr[i] = (256u - ((aux >> 10) & 511u)) << 23;
     }
     if (threadIdx.x == 0) {
         T.M = is_v ? TV.M : TK.M; T.rec = is_v ? TV.rec : TK.rec; T.mstar = is_v ? TV.mstar : TK.mstar;
@@ -151,6 +195,7 @@ dq_encode_kernel(const __grid_constant__ DqDevTable TK, const __grid_constant__ 
         T.has_mean = is_v ? TV.has_mean : TK.has_mean; T.rotate = is_v ? TV.rotate : TK.rotate;
     }
     __syncthreads();
+    dqdev::pdl_wait_prior_grid();   // inputs and the cache may be written / read by the previous kernel
     const int lane = threadIdx.x & 31, wib = threadIdx.x >> 5;
     const long long wid = (long long)blockIdx.x * kEncWarps + wib;
     if (wid >= (long long)a.T * a.Hkv) return;
@@ -261,20 +306,22 @@ dq_encode_kernel(const __grid_constant__ DqDevTable TK, const __grid_constant__ 
     __syncwarp();
     uint32_t xs = kL;
     int k = 0;
-    uint8_t* bytes = s_bytes[wib];
-#pragma unroll 4
+    // emitted bytes go to shared memory through stores the compiler does not treat as aliasing
+    // the symbol / table loads, so those loads are issued ahead of the serial state chain
+    const uint32_t bytes_addr = dqdev::smem_addr(s_bytes[wib]);
+#pragma unroll 8
     for (int j = kN - 1; j >= 0; --j) {
         const uint32_t m = s_sym[wib][j];
-        const uint32_t aux = T.aux[m], rcp = T.rcp[m];
-        const uint32_t cmpl = (aux >> 10) & 511u;                  // 2^p - f
-        if (xs >= ((256u - cmpl) << 23)) {  // at most once: xs < 2^31 <= 2^8 * (f << 23)
-            if (lane == 0) bytes[k] = (uint8_t)(xs & 0xffu);
+        const uint32_t rcp = T.rcp[m], rsh = T.rsh[m], bias = T.bias[m], cmpl = T.cmpl[m], thr = T.thr[m];
+        if (xs >= thr) {  // at most once: xs < 2^31 <= 2^8 * (f << 23)
+            if (lane == 0) asm volatile("st.shared.u8 [%0], %1;" ::"r"(bytes_addr + k), "r"(xs & 0xffu));
             ++k;
             xs >>= 8;
         }
-        xs = xs + (aux & 1023u) + (__umulhi(xs, rcp) >> (aux >> 19)) * cmpl;
+        xs = (__umulhi(xs, rcp) >> rsh) * cmpl + (xs + bias);
     }
     __syncwarp();
+    asm volatile("" ::: "memory");
     const uint32_t hdr0 = (uint32_t)__half_as_ushort(s16) | ((uint32_t)__half_as_ushort(o16) << 16);
     const int sl = a.slot[t];
     uint8_t* rec = cont + (((size_t)(sl / DQ_PAGE_TOKENS) * Hkv + h) * DQ_PAGE_TOKENS +
@@ -284,7 +331,7 @@ dq_encode_kernel(const __grid_constant__ DqDevTable TK, const __grid_constant__ 
         uint8_t v = 0;
         if (i < 4) v = (uint8_t)(hdr0 >> (8 * i));
         else if (i < 8) v = (uint8_t)(xs >> (8 * (i - 4)));
-        else if (i < used) v = bytes[k - 1 - (i - 8)];
+        else if (i < used) v = s_bytes[wib][k - 1 - (i - 8)];
         rec[i] = v;
     }
     if (a.status && lane == 0) {
@@ -313,6 +360,5 @@ cudaError_t dq_launch_encode(const DqDevTable& tk, const DqDevTable& tv, const D
     const long long warps = (long long)a.T * a.Hkv;
     if (warps == 0 || (!a.do_k && !a.do_v)) return cudaSuccess;
     const unsigned blocks = (unsigned)((warps + kEncWarps - 1) / kEncWarps);
-    dq_encode_kernel<<<dim3(blocks, (a.do_k && a.do_v) ? 2 : 1), kEncWarps * 32, 0, st>>>(tk, tv, a);
-    return cudaGetLastError();
+    return dq_launch_pdl(dq_encode_kernel, dim3(blocks, (a.do_k && a.do_v) ? 2 : 1), dim3(kEncWarps * 32), 0, st, tk, tv, a);
 }
