@@ -98,6 +98,7 @@ struct AttnParams {
     float* out_f32;
     int max_windows, windows, max_pages, B, Hq, Hkv, G, item_tokens, rotate_q, rotate_out, has_mean;
     float scale_log2;   // sm_scale * log2(e)
+    unsigned hkv_magic; // ceil(2^32 / Hkv), 0 when Hkv = 1
 };
 
 // ------------------------------------------------------------------ prepare
@@ -342,7 +343,8 @@ dq_attention_kernel(const __grid_constant__ DqDevTable TK, const __grid_constant
         const unsigned idx = blockIdx.x + (unsigned)n * gridDim.x;   // < 2^31: total_items is an int
         if (idx < (unsigned)total_items) {
             it.valid = 1;
-            it.bg = (int)(idx / (unsigned)p.Hkv);
+            // idx / Hkv by a high multiply: exact for idx < 2^32 / Hkv (hkv_magic = ceil(2^32 / Hkv); 0: Hkv = 1)
+            it.bg = p.hkv_magic ? (int)__umulhi(idx, p.hkv_magic) : (int)idx;
             it.h = (int)(idx - (unsigned)it.bg * (unsigned)p.Hkv);
             int b = hint;
             while (prefix[b + 1] <= it.bg) ++b;   // prefix[B] > bg because idx < total_items
@@ -877,6 +879,7 @@ cudaError_t dq_launch_attention(const DqDevTable& tk, const DqDevTable& tv, cons
     p.item_tokens = nw * kChunk;
     p.rotate_q = tk.rotate; p.rotate_out = tv.rotate; p.has_mean = tk.has_mean;
     p.scale_log2 = a.sm_scale * 1.4426950408889634f;
+    p.hkv_magic = a.Hkv > 1 ? (unsigned)((0x100000000ull + a.Hkv - 1) / a.Hkv) : 0u;
 
     const int heads = a.B * a.Hq;
     const long long prep_warps = (long long)heads * (1 + (p.has_mean ? (p.windows + kPrepWindows - 1) / kPrepWindows : 0));
@@ -920,6 +923,7 @@ cudaError_t dq_launch_bf16_attention(const DqAttnArgs& a, const void* k_pages, c
     p.item_tokens = kBfWarps * kChunk;
     p.rotate_q = 0; p.rotate_out = 0;
     p.scale_log2 = a.sm_scale * 1.4426950408889634f;
+    p.hkv_magic = 0;
     const int heads = a.B * a.Hq;
     dq_attn_prepare_kernel<<<(heads + 7) / 8, 256, 0, st>>>(p);
     cudaError_t e = cudaGetLastError();
