@@ -216,17 +216,25 @@ def decode_tokens(T: Table, cont: np.ndarray, seq_id, pos, slot, Hkv: int, mean_
 
 
 def attention(TK: Table, TV: Table, q_bf16: np.ndarray, k_cont, v_cont, mean_q, mean_scale,
-              page_table: np.ndarray, seq_lens, Hkv: int, sm_scale: float, only=None):
+              page_table: np.ndarray, seq_lens, Hkv: int, sm_scale: float, only=None,
+              resid_k=None, resid_v=None, resid_lens=None):
     """fp64 decode-step attention over the containers.  q_bf16: uint16 [B, Hq, n].
-    only=(b, hq) computes a single output row (others stay NaN).  Returns f64 [B, Hq, n]."""
+    only=(b, hq) computes a single output row (others stay NaN).  Returns f64 [B, Hq, n].
+    resid_k / resid_v: uint16 [B, cap, Hkv, n] bf16 bits of the uncompressed residual window,
+    resid_lens[b] of whose tokens follow the compressed ones of sequence b."""
     B, Hq, n = q_bf16.shape
     page_table = np.ascontiguousarray(page_table, dtype=np.int32)
     seq_lens = np.ascontiguousarray(seq_lens, dtype=np.int32)
     out = np.full((B, Hq, n), np.nan, dtype=np.float64)
     Wmax = mean_q.shape[1] if mean_q is not None else 0
     ob, oh = (-1, -1) if only is None else only
+    cap = 0
+    if resid_k is not None:
+        resid_lens = np.ascontiguousarray(resid_lens, dtype=np.int32)
+        cap = int(resid_k.shape[1])
     lib().dqo_attention(C.byref(TK), C.byref(TV), _p(q_bf16), _p(k_cont), _p(v_cont), _p(mean_q),
                         _p(mean_scale), C.c_int(Wmax), _p(page_table), C.c_int(page_table.shape[1]),
                         _p(seq_lens), C.c_int(B), C.c_int(Hq), C.c_int(Hkv), C.c_double(sm_scale),
-                        _p(out), C.c_int(ob), C.c_int(oh))
+                        _p(out), C.c_int(ob), C.c_int(oh), _p(resid_k), _p(resid_v), _p(resid_lens),
+                        C.c_int(cap))
     return out

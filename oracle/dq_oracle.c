@@ -580,12 +580,17 @@ void dqo_decode_tokens(const dqo_table *T, const uint8_t *cont, const int8_t *me
  * and KV head g = hq / (Hq/Hkv): logits = sm_scale * <q', khat_t>, softmax over
  * t < seq_len, out' = sum a_t vhat_t; q' = Hq/sqrt(n) when keys are rotated and
  * out = H out'/sqrt(n) when values were rotated by the encoder.
+ * Residual window (Sec. 5.1: the most recent tokens are kept in BF16): when resid_k is
+ * given, sequence b has resid_lens[b] further tokens stored uncompressed and unrotated,
+ * bf16 [B][resid_cap][Hkv][n]; they join the same softmax with logits sm_scale * <q, k_t>
+ * and contribute a_t v_t to the (unrotated) output.
  * only_b/only_hq >= 0 restrict the work to one (b, hq) (others are left untouched). */
 void dqo_attention(const dqo_table *TK, const dqo_table *TV, const uint16_t *q_bf16,
                    const uint8_t *k_cont, const uint8_t *v_cont, const int8_t *mean_q,
                    const float *mean_scale, int Wmax, const int32_t *page_table, int max_pages,
                    const int32_t *seq_lens, int B, int Hq, int Hkv, double sm_scale, double *out,
-                   int only_b, int only_hq)
+                   int only_b, int only_hq, const uint16_t *resid_k, const uint16_t *resid_v,
+                   const int32_t *resid_lens, int resid_cap)
 {
     int n = TK->n, G = Hq / Hkv;
 #pragma omp parallel for schedule(dynamic, 1) collapse(2)
@@ -593,15 +598,16 @@ void dqo_attention(const dqo_table *TK, const dqo_table *TV, const uint16_t *q_b
         for (int g = 0; g < Hkv; ++g) {
             if (only_b >= 0 && b != only_b) continue;
             if (only_hq >= 0 && only_hq / G != g) continue;
-            int len = seq_lens[b];
-            if (len <= 0) {
+            int len = seq_lens[b] > 0 ? seq_lens[b] : 0;
+            int rlen = (resid_k && resid_lens[b] > 0) ? resid_lens[b] : 0;
+            if (len + rlen <= 0) {
                 for (int hq = g * G; hq < (g + 1) * G; ++hq)
                     for (int j = 0; j < n; ++j) out[((size_t)b * Hq + hq) * n + j] = 0.0;
                 continue;
             }
-            float *kh = (float *)malloc((size_t)len * n * sizeof(float));
-            float *vh = (float *)malloc((size_t)len * n * sizeof(float));
-            double *lg = (double *)malloc((size_t)len * sizeof(double));
+            float *kh = (float *)malloc((size_t)(len + 1) * n * sizeof(float));
+            float *vh = (float *)malloc((size_t)(len + 1) * n * sizeof(float));
+            double *lg = (double *)malloc((size_t)(len + rlen) * sizeof(double));
             uint8_t sym[DQO_MAX_N];
             for (int t = 0; t < len; ++t) {
                 int slot = page_table[(size_t)b * max_pages + t / DQO_PAGE] * DQO_PAGE + t % DQO_PAGE;
@@ -618,9 +624,9 @@ void dqo_attention(const dqo_table *TK, const dqo_table *TV, const uint16_t *q_b
             }
             for (int hq = g * G; hq < (g + 1) * G; ++hq) {
                 if (only_hq >= 0 && hq != only_hq) continue;
-                double qr[DQO_MAX_N], acc[DQO_MAX_N];
+                double qraw[DQO_MAX_N], qr[DQO_MAX_N], acc[DQO_MAX_N], racc[DQO_MAX_N];
                 for (int j = 0; j < n; ++j)
-                    qr[j] = (double)dqo_bf16_to_f32(q_bf16[((size_t)b * Hq + hq) * n + j]);
+                    qr[j] = qraw[j] = (double)dqo_bf16_to_f32(q_bf16[((size_t)b * Hq + hq) * n + j]);
                 if (TK->rotate) dqo_fwht_f64(qr, n);
                 double mxl = -INFINITY;
                 for (int t = 0; t < len; ++t) {
@@ -629,16 +635,28 @@ void dqo_attention(const dqo_table *TK, const dqo_table *TV, const uint16_t *q_b
                     lg[t] = sm_scale * d;
                     if (lg[t] > mxl) mxl = lg[t];
                 }
+                for (int t = 0; t < rlen; ++t) {
+                    const uint16_t *kr = resid_k + (((size_t)b * resid_cap + t) * Hkv + g) * n;
+                    double d = 0.0;
+                    for (int j = 0; j < n; ++j) d += qraw[j] * (double)dqo_bf16_to_f32(kr[j]);
+                    lg[len + t] = sm_scale * d;
+                    if (lg[len + t] > mxl) mxl = lg[len + t];
+                }
                 double den = 0.0;
-                for (int j = 0; j < n; ++j) acc[j] = 0.0;
+                for (int j = 0; j < n; ++j) { acc[j] = 0.0; racc[j] = 0.0; }
                 for (int t = 0; t < len; ++t) {
                     double a = exp(lg[t] - mxl);
                     den += a;
                     for (int j = 0; j < n; ++j) acc[j] += a * (double)vh[(size_t)t * n + j];
                 }
-                for (int j = 0; j < n; ++j) acc[j] /= den;
-                if (TV->rotate) dqo_fwht_f64(acc, n);
-                for (int j = 0; j < n; ++j) out[((size_t)b * Hq + hq) * n + j] = acc[j];
+                for (int t = 0; t < rlen; ++t) {
+                    const uint16_t *vr = resid_v + (((size_t)b * resid_cap + t) * Hkv + g) * n;
+                    double a = exp(lg[len + t] - mxl);
+                    den += a;
+                    for (int j = 0; j < n; ++j) racc[j] += a * (double)dqo_bf16_to_f32(vr[j]);
+                }
+                if (TV->rotate) dqo_fwht_f64(acc, n);   /* compressed part back to the unrotated domain */
+                for (int j = 0; j < n; ++j) out[((size_t)b * Hq + hq) * n + j] = (acc[j] + racc[j]) / den;
             }
             free(kh); free(vh); free(lg);
         }

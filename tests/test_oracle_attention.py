@@ -213,3 +213,45 @@ def test_workload_generators_are_seeded_and_shaped():
     assert workloads.make_config(1).k_rec == 36 and workloads.make_config(3).seq_lens == [131072]
     c4f = workloads.make_config(4)
     assert c4f.batch == 128 and min(c4f.seq_lens) >= 512 and max(c4f.seq_lens) <= 16384
+
+
+def test_residual_window_equals_attention_over_mixed_cache(small):
+    """BF16 residual window (Sec. 5.1): uncompressed recent tokens join the same softmax.
+    Checked against library softmax over [dequantised compressed tokens ; raw residual tokens]."""
+    w, tk, tv, kc, vc, mq, ms, sk, sv = small
+    cfg = w.cfg
+    seq_id, pos, slot = (t.numpy() for t in (w.seq_id, w.pos, w.slot))
+    H = hadamard(128) / math.sqrt(128)
+    _, kdq = oracle.decode_tokens(tk, kc, seq_id, pos, slot, cfg.hkv, mq, ms)
+    _, vdq = oracle.decode_tokens(tv, vc, seq_id, pos, slot, cfg.hkv)
+    rng = np.random.default_rng(3)
+    cap = 128
+    rk = torch.randn((cfg.batch, cap, cfg.hkv, 128), generator=torch.Generator().manual_seed(1)).to(torch.bfloat16)
+    rv = torch.randn((cfg.batch, cap, cfg.hkv, 128), generator=torch.Generator().manual_seed(2)).to(torch.bfloat16)
+    rlens = np.array([128, 0, 37], np.int32)
+    sm = 1.0 / math.sqrt(128)
+    out = oracle.attention(tk, tv, workloads.bf16_bits(w.q), kc, vc, mq, ms, w.page_table.numpy(),
+                           w.seq_lens.numpy(), cfg.hkv, sm, resid_k=workloads.bf16_bits(rk),
+                           resid_v=workloads.bf16_bits(rv), resid_lens=rlens)
+    q = w.q.float().numpy().astype(np.float64)
+    for b in range(cfg.batch):
+        sel = seq_id == b
+        for hq in (0, 7, 30):
+            g = hq // (cfg.hq // cfg.hkv)
+            k_all = np.concatenate([kdq[sel, g].astype(np.float64) @ H,          # back to the raw domain
+                                    rk[b, :rlens[b], g].double().numpy()])
+            v_all = np.concatenate([vdq[sel, g].astype(np.float64) @ H, rv[b, :rlens[b], g].double().numpy()])
+            a = softmax(sm * (k_all @ q[b, hq]))
+            assert np.allclose(out[b, hq], a @ v_all, rtol=1e-9, atol=1e-11)
+    # no residual tokens -> identical to the plain call; only residual tokens -> plain bf16 attention
+    base = oracle.attention(tk, tv, workloads.bf16_bits(w.q), kc, vc, mq, ms, w.page_table.numpy(),
+                            w.seq_lens.numpy(), cfg.hkv, sm)
+    zero = oracle.attention(tk, tv, workloads.bf16_bits(w.q), kc, vc, mq, ms, w.page_table.numpy(),
+                            w.seq_lens.numpy(), cfg.hkv, sm, resid_k=workloads.bf16_bits(rk),
+                            resid_v=workloads.bf16_bits(rv), resid_lens=np.zeros(3, np.int32))
+    assert np.array_equal(base, zero)
+    only = oracle.attention(tk, tv, workloads.bf16_bits(w.q), kc, vc, mq, ms, w.page_table.numpy(),
+                            np.zeros(3, np.int32), cfg.hkv, sm, resid_k=workloads.bf16_bits(rk),
+                            resid_v=workloads.bf16_bits(rv), resid_lens=np.array([5, 0, 128], np.int32))
+    a = softmax(sm * (rk[2, :, 1].double().numpy() @ q[2, 5]))
+    assert np.allclose(only[2, 5], a @ rv[2, :, 1].double().numpy(), rtol=1e-10) and not only[1].any()
