@@ -135,6 +135,23 @@ int dq_decode_attention(const dq_tables *tk, const dq_tables *tv, const void *q_
                         float sm_scale, void *out_bf16, float *out_f32, void *workspace,
                         size_t workspace_bytes, void *cuda_stream);
 
+/* Decode-step attention with a BF16 residual window (Sec. 5.1 "Implementation details": the
+ * most recent 128 tokens are retained in BF16).  As dq_decode_attention, plus per sequence
+ * resid_lens[b] <= resid_cap further tokens that follow the seq_lens[b] compressed ones and are
+ * stored uncompressed and unrotated:
+ *   resid_k_bf16, resid_v_bf16   device bf16 [B][resid_cap][Hkv][128]
+ *   resid_lens                   device int32 [B]
+ * They join the same softmax (logits sm_scale * q.k) and contribute a_t v_t to the output.  When
+ * a window fills, the caller encodes its 128 tokens with dq_encode_tokens(DQ_MEAN_COMPUTE): the
+ * window then gets its own channel mean.  All three pointers NULL = dq_decode_attention. */
+int dq_decode_attention_residual(const dq_tables *tk, const dq_tables *tv, const void *q_bf16,
+                                 const uint8_t *k_cont, const uint8_t *v_cont, const int8_t *k_mean_q,
+                                 const float *k_mean_scale, int max_windows, const int32_t *page_table,
+                                 int max_pages, const int32_t *seq_lens, const void *resid_k_bf16,
+                                 const void *resid_v_bf16, const int32_t *resid_lens, int resid_cap, int B,
+                                 int Hq, int Hkv, float sm_scale, void *out_bf16, float *out_f32,
+                                 void *workspace, size_t workspace_bytes, void *cuda_stream);
+
 /* dq_decode_attention for callers that must not allocate (the paper has no counterpart: this
  * is a packaging variant of the same kernels, not part of the method).
  *

@@ -94,13 +94,19 @@ static int check_attn_common(const void* q, const int32_t* page_table, int max_p
     return DQ_OK;
 }
 
-int dq_decode_attention(const dq_tables* tk, const dq_tables* tv, const void* q_bf16,
-                        const uint8_t* k_cont, const uint8_t* v_cont, const int8_t* k_mean_q,
-                        const float* k_mean_scale, int max_windows, const int32_t* page_table,
-                        int max_pages, const int32_t* seq_lens, int B, int Hq, int Hkv, float sm_scale,
-                        void* out_bf16, float* out_f32, void* workspace, size_t workspace_bytes,
-                        void* cuda_stream) {
+int dq_decode_attention_residual(const dq_tables* tk, const dq_tables* tv, const void* q_bf16,
+                                 const uint8_t* k_cont, const uint8_t* v_cont, const int8_t* k_mean_q,
+                                 const float* k_mean_scale, int max_windows, const int32_t* page_table,
+                                 int max_pages, const int32_t* seq_lens, const void* resid_k_bf16,
+                                 const void* resid_v_bf16, const int32_t* resid_lens, int resid_cap, int B, int Hq,
+                                 int Hkv, float sm_scale, void* out_bf16, float* out_f32, void* workspace,
+                                 size_t workspace_bytes, void* cuda_stream) {
     if (!tk || !tv || !k_cont || !v_cont) return DQ_ERR_ARG;
+    if (resid_k_bf16 || resid_v_bf16 || resid_lens) {
+        if (!resid_k_bf16 || !resid_v_bf16 || !resid_lens || resid_cap <= 0) return DQ_ERR_ARG;
+        if ((reinterpret_cast<uintptr_t>(resid_k_bf16) & 7u) || (reinterpret_cast<uintptr_t>(resid_v_bf16) & 7u))
+            return DQ_ERR_ARG;
+    }
     int rc = check_attn_common(q_bf16, page_table, max_pages, seq_lens, B, Hq, Hkv, out_bf16, out_f32,
                                workspace, workspace_bytes);
     if (rc != DQ_OK) return rc;
@@ -118,9 +124,21 @@ int dq_decode_attention(const dq_tables* tk, const dq_tables* tv, const void* q_
     a.out_bf16 = out_bf16; a.out_f32 = out_f32; a.workspace = workspace;
     a.max_windows = max_windows; a.max_pages = max_pages;
     a.B = B; a.Hq = Hq; a.Hkv = Hkv; a.sm_scale = sm_scale;
+    a.resid_k = resid_k_bf16; a.resid_v = resid_v_bf16; a.resid_lens = resid_lens; a.resid_cap = resid_cap;
     const cudaError_t e = dq_launch_attention(tk->dev, tv->dev, a, static_cast<cudaStream_t>(cuda_stream));
     if (e != cudaSuccess) return cuda_fail(e, "decode attention");
     return DQ_OK;
+}
+
+int dq_decode_attention(const dq_tables* tk, const dq_tables* tv, const void* q_bf16,
+                        const uint8_t* k_cont, const uint8_t* v_cont, const int8_t* k_mean_q,
+                        const float* k_mean_scale, int max_windows, const int32_t* page_table,
+                        int max_pages, const int32_t* seq_lens, int B, int Hq, int Hkv, float sm_scale,
+                        void* out_bf16, float* out_f32, void* workspace, size_t workspace_bytes,
+                        void* cuda_stream) {
+    return dq_decode_attention_residual(tk, tv, q_bf16, k_cont, v_cont, k_mean_q, k_mean_scale, max_windows,
+                                        page_table, max_pages, seq_lens, nullptr, nullptr, nullptr, 0, B, Hq, Hkv,
+                                        sm_scale, out_bf16, out_f32, workspace, workspace_bytes, cuda_stream);
 }
 
 int dq_decode_attention_static(const dq_tables* tk, const dq_tables* tv, const void* q_bf16,
@@ -158,6 +176,7 @@ int dq_decode_attention_static(const dq_tables* tk, const dq_tables* tv, const v
     a.out_bf16 = out_bf16; a.out_f32 = out_f32; a.workspace = scratch;
     a.max_windows = max_windows; a.max_pages = max_pages;
     a.B = B; a.Hq = Hq; a.Hkv = Hkv; a.sm_scale = sm_scale;
+    a.resid_k = nullptr; a.resid_v = nullptr; a.resid_lens = nullptr; a.resid_cap = 0;
     e = dq_launch_attention_static(tk->dev, tv->dev, a, static_cast<cudaStream_t>(cuda_stream));
     if (e != cudaSuccess) return cuda_fail(e, "decode attention (static scratch)");
     return DQ_OK;

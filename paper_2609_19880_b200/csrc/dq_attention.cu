@@ -99,6 +99,10 @@ struct AttnParams {
     int max_windows, windows, max_pages, B, Hq, Hkv, G, item_tokens, rotate_q, rotate_out, has_mean;
     float scale_log2;   // sm_scale * log2(e)
     unsigned hkv_magic; // ceil(2^32 / Hkv), 0 when Hkv = 1
+    const uint16_t* resid_k;      // bf16 [B][resid_cap][Hkv][128], nullable: uncompressed recent tokens
+    const uint16_t* resid_v;
+    const int32_t* resid_lens;    // [B]
+    int resid_cap;
 };
 
 // ------------------------------------------------------------------ prepare
@@ -552,13 +556,17 @@ dq_attention_kernel(const __grid_constant__ DqDevTable TK, const __grid_constant
 
 // One CTA of 8 warps per (sequence, query head): warp w merges partials w*4 .. w*4+3, w*4+32 ...
 // with a running maximum, the warps are merged through shared memory, warp 0 normalises,
-// applies the inverse rotation and stores.
+// applies the inverse rotation and stores.  With a BF16 residual window (Sec. 5.1: the most
+// recent tokens stay uncompressed) the 8 warps also split those tokens: logits q.k and
+// sum a_t v_t in the unrotated domain, merged with the un-rotated compressed part by the same
+// log-sum-exp rule.
 __global__ void __launch_bounds__(256)
 dq_attn_combine_kernel(AttnParams p) {
     pdl_launch_dependents();
     pdl_wait_prior_grid();
     __shared__ float s_acc[8][kN];
-    __shared__ float s_mlo[8][4];
+    __shared__ float s_racc[8][kN];
+    __shared__ float s_mlo[8][8];
     const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
     const int wid = blockIdx.x;
     const int b = wid / p.Hq, hq = wid % p.Hq;
@@ -592,29 +600,85 @@ dq_attn_combine_kernel(AttnParams p) {
         }
         m_run = m_new;
     }
+    // residual window: tokens w*8 .. w*8+7, then + 64, ...
+    float racc[4] = {0.f, 0.f, 0.f, 0.f}, rl = 0.f, rm = -INFINITY;
+    const int rlen = p.resid_k ? min(max(p.resid_lens[b], 0), p.resid_cap) : 0;
+    if (rlen > 0) {
+        const int h = hq / p.G;
+        const uint2 qraw = *reinterpret_cast<const uint2*>(p.q + (size_t)wid * kN + 4 * lane);
+        const float q0 = bf16_bits_to_float(qraw.x & 0xffffu), q1 = bf16_bits_to_float(qraw.x >> 16);
+        const float q2 = bf16_bits_to_float(qraw.y & 0xffffu), q3 = bf16_bits_to_float(qraw.y >> 16);
+        for (int t0 = 8 * w; t0 < rlen; t0 += 64) {
+            uint2 kr[8], vr[8];
+            float d[8];
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                const size_t off = (((size_t)b * p.resid_cap + min(t0 + u, rlen - 1)) * p.Hkv + h) * kN + 4 * lane;
+                kr[u] = *reinterpret_cast<const uint2*>(p.resid_k + off);
+                vr[u] = *reinterpret_cast<const uint2*>(p.resid_v + off);
+            }
+#pragma unroll
+            for (int u = 0; u < 8; ++u)
+                d[u] = fmaf(q0, bf16_bits_to_float(kr[u].x & 0xffffu),
+                       fmaf(q1, bf16_bits_to_float(kr[u].x >> 16),
+                       fmaf(q2, bf16_bits_to_float(kr[u].y & 0xffffu), q3 * bf16_bits_to_float(kr[u].y >> 16))));
+#pragma unroll
+            for (int s = 16; s >= 1; s >>= 1)
+#pragma unroll
+                for (int u = 0; u < 8; ++u) d[u] += __shfl_xor_sync(kFullMask, d[u], s);
+            float m_new = rm;
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                d[u] = (t0 + u < rlen) ? d[u] * p.scale_log2 : -INFINITY;
+                m_new = fmaxf(m_new, d[u]);
+            }
+            const float keep = exp2f(rm - m_new);
+#pragma unroll
+            for (int e = 0; e < 4; ++e) racc[e] *= keep;
+            rl *= keep;
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                const float pr = exp2f(d[u] - m_new);
+                rl += pr;
+                racc[0] = fmaf(pr, bf16_bits_to_float(vr[u].x & 0xffffu), racc[0]);
+                racc[1] = fmaf(pr, bf16_bits_to_float(vr[u].x >> 16), racc[1]);
+                racc[2] = fmaf(pr, bf16_bits_to_float(vr[u].y & 0xffffu), racc[2]);
+                racc[3] = fmaf(pr, bf16_bits_to_float(vr[u].y >> 16), racc[3]);
+            }
+            rm = m_new;
+        }
+    }
     *reinterpret_cast<float4*>(&s_acc[w][4 * lane]) = make_float4(acc[0], acc[1], acc[2], acc[3]);
-    if (lane == 0) { s_mlo[w][0] = m_run; s_mlo[w][1] = lsum; s_mlo[w][2] = osum; }
+    *reinterpret_cast<float4*>(&s_racc[w][4 * lane]) = make_float4(racc[0], racc[1], racc[2], racc[3]);
+    if (lane == 0) { s_mlo[w][0] = m_run; s_mlo[w][1] = lsum; s_mlo[w][2] = osum; s_mlo[w][3] = rm; s_mlo[w][4] = rl; }
     __syncthreads();
     if (w != 0) return;
     float mx = -INFINITY;
 #pragma unroll
-    for (int i = 0; i < 8; ++i) mx = fmaxf(mx, s_mlo[i][0]);
+    for (int i = 0; i < 8; ++i) mx = fmaxf(mx, fmaxf(s_mlo[i][0], s_mlo[i][3]));
     acc[0] = acc[1] = acc[2] = acc[3] = 0.f;
+    racc[0] = racc[1] = racc[2] = racc[3] = 0.f;
     lsum = osum = 0.f;
     if (mx != -INFINITY) {
 #pragma unroll
         for (int i = 0; i < 8; ++i) {
-            const float sc = exp2f(s_mlo[i][0] - mx);
+            const float sc = exp2f(s_mlo[i][0] - mx), rsc = exp2f(s_mlo[i][3] - mx);
             const float4 v = *reinterpret_cast<const float4*>(&s_acc[i][4 * lane]);
+            const float4 r = *reinterpret_cast<const float4*>(&s_racc[i][4 * lane]);
             acc[0] = fmaf(v.x, sc, acc[0]); acc[1] = fmaf(v.y, sc, acc[1]);
             acc[2] = fmaf(v.z, sc, acc[2]); acc[3] = fmaf(v.w, sc, acc[3]);
+            racc[0] = fmaf(r.x, rsc, racc[0]); racc[1] = fmaf(r.y, rsc, racc[1]);
+            racc[2] = fmaf(r.z, rsc, racc[2]); racc[3] = fmaf(r.w, rsc, racc[3]);
             lsum = fmaf(s_mlo[i][1], sc, lsum);
+            lsum = fmaf(s_mlo[i][4], rsc, lsum);
             osum = fmaf(s_mlo[i][2], sc, osum);
         }
         const float inv = 1.0f / lsum;
 #pragma unroll
         for (int e = 0; e < 4; ++e) acc[e] = (acc[e] + osum) * inv;
-        if (p.rotate_out) warp_fwht128(acc, lane);
+        if (p.rotate_out) warp_fwht128(acc, lane);          // compressed part back to the unrotated domain
+#pragma unroll
+        for (int e = 0; e < 4; ++e) acc[e] = fmaf(racc[e], inv, acc[e]);
     }
     if (p.out_f32)
         *reinterpret_cast<float4*>(p.out_f32 + (size_t)wid * kN + 4 * lane) = make_float4(acc[0], acc[1], acc[2], acc[3]);
@@ -880,6 +944,8 @@ cudaError_t dq_launch_attention(const DqDevTable& tk, const DqDevTable& tv, cons
     p.rotate_q = tk.rotate; p.rotate_out = tv.rotate; p.has_mean = tk.has_mean;
     p.scale_log2 = a.sm_scale * 1.4426950408889634f;
     p.hkv_magic = a.Hkv > 1 ? (unsigned)((0x100000000ull + a.Hkv - 1) / a.Hkv) : 0u;
+    p.resid_k = static_cast<const uint16_t*>(a.resid_k); p.resid_v = static_cast<const uint16_t*>(a.resid_v);
+    p.resid_lens = a.resid_lens; p.resid_cap = a.resid_cap;
 
     const int heads = a.B * a.Hq;
     const long long prep_warps = (long long)heads * (1 + (p.has_mean ? (p.windows + kPrepWindows - 1) / kPrepWindows : 0));
@@ -924,6 +990,7 @@ cudaError_t dq_launch_bf16_attention(const DqAttnArgs& a, const void* k_pages, c
     p.rotate_q = 0; p.rotate_out = 0;
     p.scale_log2 = a.sm_scale * 1.4426950408889634f;
     p.hkv_magic = 0;
+    p.resid_k = nullptr; p.resid_v = nullptr; p.resid_lens = nullptr; p.resid_cap = 0;
     const int heads = a.B * a.Hq;
     dq_attn_prepare_kernel<<<(heads + 7) / 8, 256, 0, st>>>(p);
     cudaError_t e = cudaGetLastError();

@@ -61,6 +61,10 @@ struct DqAttnArgs {
     void* workspace;
     int max_windows, max_pages, B, Hq, Hkv;
     float sm_scale;
+    const void* resid_k;        // bf16 [B][resid_cap][Hkv][128], nullable
+    const void* resid_v;
+    const int32_t* resid_lens;  // [B]
+    int resid_cap;
 };
 size_t dq_attn_workspace_bytes(int B, int Hq, int max_pages);
 cudaError_t dq_launch_attention(const DqDevTable& tk, const DqDevTable& tv, const DqAttnArgs& a,

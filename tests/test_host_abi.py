@@ -97,6 +97,15 @@ def test_calls_validate_before_launch(L):
     assert call(wsb=ws - 1) == -4
     assert call(mq=n) == -1 and call(mw=0) == -1       # key tables with a mean need the mean arrays
     assert call(kc=C.c_void_p(0x1001)) == -1           # containers must be 16-byte aligned
+    def call_r(rk=fake, rv=fake, rl=fake, cap=128, **kw):
+        d = dict(a); d.update(kw)
+        return L.dq_decode_attention_residual(
+            *[d[k] for k in ("tk", "tv", "q", "kc", "vc", "mq", "ms", "mw", "pt", "mp", "sl")], rk, rv, rl, cap,
+            *[d[k] for k in ("B", "Hq", "Hkv", "sm", "ob", "of", "ws", "wsb", "st")])
+
+    # a residual window needs all three arrays, a positive capacity and 8-byte aligned rows
+    assert call_r(rv=n) == -1 and call_r(rl=n) == -1 and call_r(rk=n) == -1 and call_r(cap=0) == -1
+    assert call_r(rk=C.c_void_p(0x1004)) == -1 and call_r(wsb=ws - 1) == -4 and call_r(q=n) == -1
     assert L.dq_decode_tokens(tk.handle, n, n, n, 0, n, n, fake, 4, 8, fake, n, n) == -1
     assert L.dq_bf16_decode_attention(fake, n, fake, fake, 8, fake, 2, 32, 8, C.c_float(0.1), fake, fake, ws, n) == -1
 
