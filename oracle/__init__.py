@@ -185,10 +185,13 @@ def window_means(k_bf16: np.ndarray, seq_id, pos, mean_q: np.ndarray, mean_scale
 
 def encode_tokens(T: Table, x_bf16: np.ndarray, seq_id, pos, slot, cont: np.ndarray,
                   mean_q=None, mean_scale=None):
-    """x_bf16: uint16 [T, Hkv, n]; cont: uint8 [pages, Hkv, 16, rec] updated in place.
+    """x_bf16: uint16 [T, Hkv, d]; cont: uint8 [pages, Hkv / hs, 16, rec] updated in place, where
+    hs = T.n / d heads share one stream (hs = 1: per token-head; hs = Hkv: per token).
     Returns stats uint32[4]."""
     T_tok, Hkv, n = x_bf16.shape
-    assert n == T.n and cont.dtype == np.uint8 and cont.shape[-1] == T.rec
+    hs = max(1, T.n // n)
+    assert T.n == hs * n and Hkv % hs == 0 and (hs == 1 or n == 128)
+    assert cont.dtype == np.uint8 and cont.shape[-1] == T.rec and cont.shape[1] == Hkv // hs
     seq_id = np.ascontiguousarray(seq_id, dtype=np.int32)
     pos = np.ascontiguousarray(pos, dtype=np.int32)
     slot = np.ascontiguousarray(slot, dtype=np.int32)
@@ -201,13 +204,16 @@ def encode_tokens(T: Table, x_bf16: np.ndarray, seq_id, pos, slot, cont: np.ndar
 
 def decode_tokens(T: Table, cont: np.ndarray, seq_id, pos, slot, Hkv: int, mean_q=None,
                   mean_scale=None, want_dequant: bool = True):
-    """Returns (symbols uint8 [T, Hkv, n], dequant f32 [T, Hkv, n] in the rotated domain)."""
+    """Returns (symbols uint8 [T, Hkv, d], dequant f32 [T, Hkv, d] in the rotated domain);
+    d = min(T.n, 128)."""
     seq_id = np.ascontiguousarray(seq_id, dtype=np.int32)
     pos = np.ascontiguousarray(pos, dtype=np.int32)
     slot = np.ascontiguousarray(slot, dtype=np.int32)
     T_tok = slot.shape[0]
-    sym = np.zeros((T_tok, Hkv, T.n), dtype=np.uint8)
-    deq = np.zeros((T_tok, Hkv, T.n), dtype=np.float32) if want_dequant else None
+    d = min(T.n, 128)
+    assert cont.shape[1] == Hkv // max(1, T.n // d)
+    sym = np.zeros((T_tok, Hkv, d), dtype=np.uint8)
+    deq = np.zeros((T_tok, Hkv, d), dtype=np.float32) if want_dequant else None
     Wmax = mean_q.shape[1] if mean_q is not None else 0
     lib().dqo_decode_tokens(C.byref(T), _p(cont), _p(mean_q), _p(mean_scale), C.c_int(Wmax),
                             _p(seq_id), _p(pos), _p(slot), C.c_int(T_tok), C.c_int(Hkv), _p(sym),

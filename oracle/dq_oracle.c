@@ -20,8 +20,13 @@
  *
  * Where the paper is silent the numerical contract below fixes one reading (the
  * same list is in the design notes of the repository):
- *   - a stream is the n values of one (token, KV head); sigma = 32, L = 2^23,
- *     32-bit state, byte-wise renormalisation (Algorithm 2 reads bytes);
+ *   - a stream is the n values of one (token, KV head); a table with n > 128
+ *     describes the paper's default grouping instead (Sec. 5.1: a token is
+ *     quantised as a single group): the stream spans n/128 consecutive KV heads
+ *     of a token, each head rotated and mean-centred on its own, one (s, o) pair
+ *     and one container for the whole group;
+ *   - sigma = 32, L = 2^23, 32-bit state, byte-wise renormalisation (Algorithm 2
+ *     reads bytes);
  *   - the record is [s fp16][o fp16][state u32 LE][payload bytes][zero padding];
  *   - the probability of level m is the N(0,1) mass of its cell on a grid that
  *     spans +-E[max of n normals], cells clipped to that span;
@@ -52,6 +57,7 @@
 #define DQO_SIGMA 32       /* bits of final state stored in the record             */
 #define DQO_WINDOW 128     /* tokens per channel-mean window                       */
 #define DQO_PAGE 16        /* tokens per physical page                             */
+#define DQO_HEAD 128       /* head dimension of the token-level entry points       */
 
 typedef struct {
     int M, n, rec, C, B;           /* levels, stream length, record bytes, C=rec-4, B=8C-32 */
@@ -352,7 +358,7 @@ void dqo_rans_decode(const uint8_t *payload, int cap, int n, const dqo_table *T,
 void dqo_encode_stream(const float *z, const dqo_table *T, uint8_t *rec, uint32_t *stats,
                        uint8_t *sym_out)
 {
-    int n = T->n, M = T->M, per = n / 32;
+    int n = T->n, M = T->M;
     uint8_t m[DQO_MAX_N];
     uint16_t s16 = 0, o16 = 0;
     const int64_t budget = (int64_t)T->B * 65536;
@@ -363,26 +369,33 @@ void dqo_encode_stream(const float *z, const dqo_table *T, uint8_t *rec, uint32_
         float o = mn;                                  /* FitMinMax, Eq. (affine_token) */
         float s = (mx - mn) / (float)(M - 1);
         dqo_drift(z, n, s, o, T, m);                   /* first Drift                   */
-        /* Refit: least squares of z on m.  Sums in binary64; each of 32 lanes adds
-         * its n/32 consecutive elements in order, then an xor-butterfly 16,8,4,2,1. */
+        /* Refit: least squares of z on m.  Sums in binary64 in a fixed order.  A block is
+         * the whole stream when n <= 128, else 128 consecutive values (one head): within a
+         * block each of 32 lanes adds its consecutive elements in order, then an
+         * xor-butterfly 16,8,4,2,1 joins the lanes; block sums are added in block order. */
         int64_t Sm = 0, Smm = 0;
-        double lz[32], lmz[32];
-        for (int l = 0; l < 32; ++l) {
-            double a = 0.0, b = 0.0;
-            for (int e = 0; e < per; ++e) {
-                int j = l * per + e;
-                if (e == 0) { a = (double)z[j]; b = (double)m[j] * (double)z[j]; }
-                else { a = a + (double)z[j]; b = b + (double)m[j] * (double)z[j]; }
-                Sm += m[j]; Smm += (int64_t)m[j] * m[j];
+        double Sz = 0.0, Smz = 0.0;
+        int blk = n > DQO_HEAD ? DQO_HEAD : n, bper = blk / 32;
+        for (int b0 = 0; b0 < n; b0 += blk) {
+            double lz[32], lmz[32];
+            for (int l = 0; l < 32; ++l) {
+                double a = 0.0, b = 0.0;
+                for (int e = 0; e < bper; ++e) {
+                    int j = b0 + l * bper + e;
+                    if (e == 0) { a = (double)z[j]; b = (double)m[j] * (double)z[j]; }
+                    else { a = a + (double)z[j]; b = b + (double)m[j] * (double)z[j]; }
+                    Sm += m[j]; Smm += (int64_t)m[j] * m[j];
+                }
+                lz[l] = a; lmz[l] = b;
             }
-            lz[l] = a; lmz[l] = b;
+            for (int d = 16; d >= 1; d >>= 1) {
+                double tz[32], tmz[32];
+                for (int l = 0; l < 32; ++l) { tz[l] = lz[l] + lz[l ^ d]; tmz[l] = lmz[l] + lmz[l ^ d]; }
+                memcpy(lz, tz, sizeof tz); memcpy(lmz, tmz, sizeof tmz);
+            }
+            if (b0 == 0) { Sz = lz[0]; Smz = lmz[0]; }
+            else { Sz = Sz + lz[0]; Smz = Smz + lmz[0]; }
         }
-        for (int d = 16; d >= 1; d >>= 1) {
-            double tz[32], tmz[32];
-            for (int l = 0; l < 32; ++l) { tz[l] = lz[l] + lz[l ^ d]; tmz[l] = lmz[l] + lmz[l ^ d]; }
-            memcpy(lz, tz, sizeof tz); memcpy(lmz, tmz, sizeof tmz);
-        }
-        double Sz = lz[0], Smz = lmz[0];
         int64_t den = (int64_t)n * Smm - Sm * Sm;
         double sd = (double)s, od = (double)o;
         if (den != 0) {
@@ -492,36 +505,48 @@ void dqo_window_means(const uint16_t *k_bf16, int T_tok, int Hkv, int n, const i
 
 /* ------------------------------------------------------------ token encoder */
 
-static size_t dqo_rec_offset(int slot, int h, int Hkv, int rec)
+/* Streams per token and head dimension seen by the token-level entry points: a table with
+ * n <= 128 has one stream per (token, KV head); n = hs * 128 has one stream per group of hs
+ * consecutive KV heads (hs = Hkv: the whole token, the paper's default). */
+static int dqo_heads_per_stream(const dqo_table *T) { return T->n > DQO_HEAD ? T->n / DQO_HEAD : 1; }
+static int dqo_head_dim(const dqo_table *T) { return T->n > DQO_HEAD ? DQO_HEAD : T->n; }
+
+/* containers are laid out [page, stream group, 16, rec] */
+static size_t dqo_rec_offset(int slot, int grp, int groups, int rec)
 {
-    return (((size_t)(slot / DQO_PAGE) * Hkv + h) * DQO_PAGE + (size_t)(slot % DQO_PAGE)) * rec;
+    return (((size_t)(slot / DQO_PAGE) * groups + grp) * DQO_PAGE + (size_t)(slot % DQO_PAGE)) * rec;
 }
 
 /* Encode T_tok tokens of one tensor kind (Fig. 1 pipeline: Hadamard, mean removal
- * for keys, affine grid, drift, rANS).  x_bf16 is [T, Hkv, n]; containers are laid
- * out [page, Hkv, 16, rec] and addressed by slot = page * 16 + index in page. */
+ * for keys, affine grid, drift, rANS).  x_bf16 is [T, Hkv, d]; each head is rotated (and,
+ * for keys, centred on its window mean) on its own; the hs heads of a stream group are
+ * concatenated in head order.  Containers are addressed by slot = page * 16 + index in page. */
 void dqo_encode_tokens(const dqo_table *T, const uint16_t *x_bf16, int T_tok, int Hkv,
                        const int32_t *seq_id, const int32_t *pos, const int32_t *slot,
                        uint8_t *cont, const int8_t *mean_q, const float *mean_scale, int Wmax,
                        uint32_t *stats)
 {
-    int n = T->n;
+    int d = dqo_head_dim(T), hs = dqo_heads_per_stream(T), groups = Hkv / hs;
     uint32_t st[4] = {0, 0, 0, 0};
 #pragma omp parallel
     {
         uint32_t lst[4] = {0, 0, 0, 0};
 #pragma omp for schedule(static)
-        for (int64_t th = 0; th < (int64_t)T_tok * Hkv; ++th) {
-            int t = (int)(th / Hkv), h = (int)(th % Hkv);
+        for (int64_t tg = 0; tg < (int64_t)T_tok * groups; ++tg) {
+            int t = (int)(tg / groups), grp = (int)(tg % groups);
             float z[DQO_MAX_N];
-            for (int j = 0; j < n; ++j) z[j] = dqo_bf16_to_f32(x_bf16[((size_t)t * Hkv + h) * n + j]);
-            if (T->rotate) dqo_fwht_f32(z, n);
-            if (T->has_mean) {
-                size_t mi = ((size_t)seq_id[t] * Wmax + pos[t] / DQO_WINDOW) * Hkv + h;
-                float sc = mean_scale[mi];
-                for (int j = 0; j < n; ++j) z[j] = z[j] - sc * (float)mean_q[mi * n + j];
+            for (int k = 0; k < hs; ++k) {
+                int h = grp * hs + k;
+                float *zh = z + k * d;
+                for (int j = 0; j < d; ++j) zh[j] = dqo_bf16_to_f32(x_bf16[((size_t)t * Hkv + h) * d + j]);
+                if (T->rotate) dqo_fwht_f32(zh, d);
+                if (T->has_mean) {
+                    size_t mi = ((size_t)seq_id[t] * Wmax + pos[t] / DQO_WINDOW) * Hkv + h;
+                    float sc = mean_scale[mi];
+                    for (int j = 0; j < d; ++j) zh[j] = zh[j] - sc * (float)mean_q[mi * d + j];
+                }
             }
-            dqo_encode_stream(z, T, cont + dqo_rec_offset(slot[t], h, Hkv, T->rec), lst, NULL);
+            dqo_encode_stream(z, T, cont + dqo_rec_offset(slot[t], grp, groups, T->rec), lst, NULL);
         }
 #pragma omp critical
         {
@@ -537,40 +562,45 @@ void dqo_encode_tokens(const dqo_table *T, const uint16_t *x_bf16, int T_tok, in
 
 /* ------------------------------------------------------------ token decoder */
 
-/* Decode one record: symbols and dequantised values in the rotated domain,
- * xhat_j = fma(m_j, s, o) (+ mu_j for keys), Appendix A. */
-static void dqo_decode_record(const dqo_table *T, const uint8_t *rec, const int8_t *mq, float msc,
-                              uint8_t *sym, float *xhat)
+/* Decode one record: all n symbols of the stream and (nullable) the dequantised values in
+ * the rotated domain, xhat_j = fma(m_j, s, o), Appendix A (the key mean is added by the
+ * callers, per head). */
+static void dqo_decode_record(const dqo_table *T, const uint8_t *rec, uint8_t *sym, float *xhat)
 {
     int n = T->n;
     uint16_t s16 = (uint16_t)(rec[0] | (rec[1] << 8)), o16 = (uint16_t)(rec[2] | (rec[3] << 8));
     float s = dqo_f16_to_f32(s16), o = dqo_f16_to_f32(o16);
     dqo_rans_decode(rec + 4, T->C, n, T, sym, NULL);
     if (!xhat) return;
-    for (int j = 0; j < n; ++j) {
-        float v = fmaf((float)sym[j], s, o);
-        if (mq) v = v + msc * (float)mq[j];
-        xhat[j] = v;
-    }
+    for (int j = 0; j < n; ++j) xhat[j] = fmaf((float)sym[j], s, o);
 }
 
+/* symbols / dequant are [T, Hkv, d] */
 void dqo_decode_tokens(const dqo_table *T, const uint8_t *cont, const int8_t *mean_q,
                        const float *mean_scale, int Wmax, const int32_t *seq_id,
                        const int32_t *pos, const int32_t *slot, int T_tok, int Hkv,
                        uint8_t *symbols, float *dequant)
 {
-    int n = T->n;
+    int d = dqo_head_dim(T), hs = dqo_heads_per_stream(T), groups = Hkv / hs;
 #pragma omp parallel for schedule(static)
-    for (int64_t th = 0; th < (int64_t)T_tok * Hkv; ++th) {
-        int t = (int)(th / Hkv), h = (int)(th % Hkv);
-        const int8_t *mq = NULL;
-        float msc = 0.0f;
-        if (T->has_mean && mean_q) {
-            size_t mi = ((size_t)seq_id[t] * Wmax + pos[t] / DQO_WINDOW) * Hkv + h;
-            mq = mean_q + mi * n; msc = mean_scale[mi];
+    for (int64_t tg = 0; tg < (int64_t)T_tok * groups; ++tg) {
+        int t = (int)(tg / groups), grp = (int)(tg % groups);
+        uint8_t sym[DQO_MAX_N];
+        float xh[DQO_MAX_N];
+        dqo_decode_record(T, cont + dqo_rec_offset(slot[t], grp, groups, T->rec), sym, xh);
+        for (int k = 0; k < hs; ++k) {
+            int h = grp * hs + k;
+            size_t dst = ((size_t)t * Hkv + h) * d;
+            for (int j = 0; j < d; ++j) symbols[dst + j] = sym[k * d + j];
+            if (!dequant) continue;
+            if (T->has_mean && mean_q) {
+                size_t mi = ((size_t)seq_id[t] * Wmax + pos[t] / DQO_WINDOW) * Hkv + h;
+                float msc = mean_scale[mi];
+                for (int j = 0; j < d; ++j)
+                    dequant[dst + j] = xh[k * d + j] + msc * (float)mean_q[mi * d + j];
+            } else
+                for (int j = 0; j < d; ++j) dequant[dst + j] = xh[k * d + j];
         }
-        dqo_decode_record(T, cont + dqo_rec_offset(slot[t], h, Hkv, T->rec), mq, msc,
-                          symbols + (size_t)th * n, dequant ? dequant + (size_t)th * n : NULL);
     }
 }
 
@@ -592,7 +622,8 @@ void dqo_attention(const dqo_table *TK, const dqo_table *TV, const uint16_t *q_b
                    int only_b, int only_hq, const uint16_t *resid_k, const uint16_t *resid_v,
                    const int32_t *resid_lens, int resid_cap)
 {
-    int n = TK->n, G = Hq / Hkv;
+    int n = dqo_head_dim(TK), G = Hq / Hkv;   /* n: head dimension from here on */
+    int hsk = dqo_heads_per_stream(TK), hsv = dqo_heads_per_stream(TV);
 #pragma omp parallel for schedule(dynamic, 1) collapse(2)
     for (int b = 0; b < B; ++b)
         for (int g = 0; g < Hkv; ++g) {
@@ -609,18 +640,20 @@ void dqo_attention(const dqo_table *TK, const dqo_table *TV, const uint16_t *q_b
             float *vh = (float *)malloc((size_t)(len + 1) * n * sizeof(float));
             double *lg = (double *)malloc((size_t)(len + rlen) * sizeof(double));
             uint8_t sym[DQO_MAX_N];
+            float xh[DQO_MAX_N];
             for (int t = 0; t < len; ++t) {
                 int slot = page_table[(size_t)b * max_pages + t / DQO_PAGE] * DQO_PAGE + t % DQO_PAGE;
-                const int8_t *mq = NULL;
-                float msc = 0.0f;
+                /* the stream that holds head g is decoded whole; head g's slice is kept */
+                dqo_decode_record(TK, k_cont + dqo_rec_offset(slot, g / hsk, Hkv / hsk, TK->rec), sym, xh);
+                for (int j = 0; j < n; ++j) kh[(size_t)t * n + j] = xh[(g % hsk) * n + j];
                 if (TK->has_mean) {
                     size_t mi = ((size_t)b * Wmax + t / DQO_WINDOW) * Hkv + g;
-                    mq = mean_q + mi * n; msc = mean_scale[mi];
+                    float msc = mean_scale[mi];
+                    for (int j = 0; j < n; ++j)
+                        kh[(size_t)t * n + j] = kh[(size_t)t * n + j] + msc * (float)mean_q[mi * n + j];
                 }
-                dqo_decode_record(TK, k_cont + dqo_rec_offset(slot, g, Hkv, TK->rec), mq, msc, sym,
-                                  kh + (size_t)t * n);
-                dqo_decode_record(TV, v_cont + dqo_rec_offset(slot, g, Hkv, TV->rec), NULL, 0.0f, sym,
-                                  vh + (size_t)t * n);
+                dqo_decode_record(TV, v_cont + dqo_rec_offset(slot, g / hsv, Hkv / hsv, TV->rec), sym, xh);
+                for (int j = 0; j < n; ++j) vh[(size_t)t * n + j] = xh[(g % hsv) * n + j];
             }
             for (int hq = g * G; hq < (g + 1) * G; ++hq) {
                 if (only_hq >= 0 && hq != only_hq) continue;
