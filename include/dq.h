@@ -22,6 +22,17 @@
  *   - Containers live in pages of 16 tokens: uint8 [num_pages][Hkv][16][rec_bytes].
  *     slot = page * 16 + index-in-page.  A record's address follows from (slot, head)
  *     alone (fixed stride, Sec. 4.1).
+ *   - Token-wide streams (Sec. 5.1 "Implementation details": each token is quantised as a
+ *     single group; 331 / 231-byte containers, 8 / 6 levels): tables built with
+ *     heads_per_stream = hs > 1 describe streams of hs * 128 values, the hs consecutive KV
+ *     heads of a token, each head rotated (and, for keys, centred on its window mean) on its
+ *     own, with one (s, o) pair, one rANS state and one record per stream.  Their records
+ *     (same field order, rec_bytes = floor(bits_per_elem * hs * 128 / 8)) are stored
+ *     word-interleaved per page so that the 16 tokens of a page advance through memory
+ *     together: uint8 [num_pages][Hkv / hs][rec_words][16][4], rec_words = ceil(rec_bytes / 4);
+ *     byte i of the record of (page, group, token-in-page t) sits at
+ *     ((page * (Hkv / hs) + group) * rec_words + i / 4) * 64 + t * 4 + i % 4; bytes past
+ *     rec_bytes in the last word are zero.
  *   - Key channel means: one per (sequence, window of 128 positions, KV head):
  *     int8 [S][max_windows][Hkv][128] and float scale [S][max_windows][Hkv];
  *     mean_j = scale * q_j, in the Hadamard-rotated domain.
@@ -53,7 +64,9 @@ extern "C" {
 #define DQ_HEAD_DIM 128
 #define DQ_PAGE_TOKENS 16
 #define DQ_WINDOW_TOKENS 128
-#define DQ_MAX_REC_BYTES 160
+#define DQ_MAX_REC_BYTES 160      /* per token-head records                            */
+#define DQ_MAX_WIDE_REC_BYTES 1024 /* records of streams that span several heads        */
+#define DQ_MAX_STREAM_HEADS 8     /* heads per stream (1024 values)                    */
 #define DQ_MAX_GROUP 8           /* query heads per KV head                           */
 
 #define DQ_MEAN_COMPUTE 0
@@ -68,6 +81,9 @@ typedef struct {
                        table has entropy <= B/128 and passes the feasibility test. */
     int has_mean;   /* 1: streams had a window mean removed (keys); 0: values          */
     int rotate;     /* 1: the library applies the per-head Hadamard rotation (Sec. 4.2) */
+    int heads_per_stream; /* 0 or 1: one stream per (token, KV head); hs in 2..8: one stream per
+                       hs consecutive KV heads of a token (hs = Hkv: the paper's token-wide
+                       default, Sec. 5.1).  The model's n is then hs * 128. */
 } dq_table_opts;
 
 typedef struct {
@@ -78,13 +94,15 @@ typedef struct {
     float r[DQ_MAX_LEVELS];        /* -log2(f/256), bits (Algorithm 1) */
     uint32_t R[DQ_MAX_LEVELS];     /* ceil(r * 65536)                  */
     uint32_t lut[256];             /* f << 24 | (fp16 bits of level) << 8 | (z - c) */
+    int heads_per_stream;          /* >= 1                                           */
+    int rec_words;                 /* ceil(rec_bytes / 4): words per record in the interleaved layout */
 } dq_table_info;
 
 /* Probability model and rANS tables of one tensor kind (Sec. 3.1 "Entropy Coding",
  * Sec. 4.2 last paragraph, Sec. 4.4 "Distribution sharpening").  The probability of level
- * m is the N(0,1) mass of its cell on an M-level grid spanning +-E[max of 128 normals];
- * frequencies are integers summing to 256.  Host only; needs no GPU.
- * Returns DQ_ERR_INFEASIBLE when 128 * R[mstar] > 65536 * B.  *out is set only on DQ_OK. */
+ * m is the N(0,1) mass of its cell on an M-level grid spanning +-E[max of n normals], n the
+ * stream length (128, or hs * 128); frequencies are integers summing to 256.  Host only; needs
+ * no GPU.  Returns DQ_ERR_INFEASIBLE when n * R[mstar] > 65536 * B.  *out is set only on DQ_OK. */
 int dq_build_tables(int levels, double bits_per_elem, const dq_table_opts *opts, dq_tables **out);
 void dq_free_tables(dq_tables *t);
 int dq_tables_info(const dq_tables *t, dq_table_info *out);
@@ -107,7 +125,10 @@ int dq_tables_info(const dq_tables *t, dq_table_info *out);
  *   status           device uint32[4], nullable, accumulated (not cleared): [0] streams that
  *                    fell back to the all-central assignment, [1] constant streams,
  *                    [2] rejected refits, [3] max record bytes used (atomicMax).
- * Errors: DQ_ERR_ARG for null / negative arguments, DQ_ERR_CUDA on launch failure. */
+ * With token-wide tables (heads_per_stream = hs > 1; both tables must agree, Hkv % hs == 0) one
+ * CTA of hs warps encodes a stream and the containers use the interleaved layout.
+ * Errors: DQ_ERR_ARG for null / negative arguments, DQ_ERR_UNSUPPORTED for mismatched
+ * heads_per_stream, DQ_ERR_CUDA on launch failure. */
 int dq_encode_tokens(const dq_tables *tk, const dq_tables *tv, const void *k_bf16,
                      const void *v_bf16, int T, int Hkv, const int32_t *seq_id,
                      const int32_t *pos, const int32_t *slot, uint8_t *k_cont, uint8_t *v_cont,

@@ -53,6 +53,11 @@ int dq_encode_tokens(const dq_tables* tk, const dq_tables* tv, const void* k_bf1
     const bool k_mean = tk && tk->info.has_mean;
     if (k_mean && (!k_mean_q || !k_mean_scale || max_windows <= 0)) return DQ_ERR_ARG;
     if (tv && tv->info.has_mean) return DQ_ERR_UNSUPPORTED;  // only keys carry window means
+    {
+        const int hs = tk ? tk->info.heads_per_stream : tv->info.heads_per_stream;
+        if (tk && tv && tk->info.heads_per_stream != tv->info.heads_per_stream) return DQ_ERR_UNSUPPORTED;
+        if (Hkv % hs != 0) return DQ_ERR_ARG;
+    }
     if ((k_bf16 && (reinterpret_cast<uintptr_t>(k_bf16) & 7u)) ||
         (v_bf16 && (reinterpret_cast<uintptr_t>(v_bf16) & 7u)) ||
         (k_mean && (reinterpret_cast<uintptr_t>(k_mean_q) & 3u)))

@@ -45,12 +45,64 @@ dq_decode_tokens_kernel(const __grid_constant__ DqDevTable T, const uint8_t* __r
     }
 }
 
+// Token-wide streams: one thread per (token, group of hs heads), record read from the
+// word-interleaved page layout; symbols / dequantised values are written per head.
+__global__ void __launch_bounds__(128)
+dq_decode_tokens_wide_kernel(const __grid_constant__ DqDevTable T, const uint8_t* __restrict__ cont,
+                             const int8_t* __restrict__ mean_q, const float* __restrict__ mean_scale,
+                             int Wmax, const int32_t* __restrict__ seq_id, const int32_t* __restrict__ pos,
+                             const int32_t* __restrict__ slot, int n_tok, int Hkv,
+                             uint8_t* __restrict__ symbols, float* __restrict__ dequant) {
+    const int groups = Hkv / T.hs;
+    const long long sid = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (sid >= (long long)n_tok * groups) return;
+    const int t = (int)(sid / groups), grp = (int)(sid % groups);
+    const int sl = slot[t];
+    const uint8_t* blk = cont + ((size_t)(sl / DQ_PAGE_TOKENS) * groups + grp) * ((size_t)T.rec_words * 64) +
+                         (size_t)(sl % DQ_PAGE_TOKENS) * 4;
+    auto byte_at = [&](int i) -> uint32_t { return blk[(size_t)(i >> 2) * 64 + (i & 3)]; };
+    const float s = __half2float(__ushort_as_half((unsigned short)(byte_at(0) | (byte_at(1) << 8))));
+    const float o = __half2float(__ushort_as_half((unsigned short)(byte_at(2) | (byte_at(3) << 8))));
+    uint32_t x = byte_at(4) | (byte_at(5) << 8) | (byte_at(6) << 16) | (byte_at(7) << 24);
+    int ptr = 8;
+    for (int k = 0; k < T.hs; ++k) {
+        const int h = grp * T.hs + k;
+        const int8_t* mq = nullptr;
+        float msc = 0.f;
+        if (T.has_mean && mean_q) {
+            const size_t mi = ((size_t)seq_id[t] * Wmax + pos[t] / DQ_WINDOW_TOKENS) * Hkv + h;
+            mq = mean_q + mi * DQ_HEAD_DIM;
+            msc = mean_scale[mi];
+        }
+        const size_t dst = ((size_t)t * Hkv + h) * DQ_HEAD_DIM;
+        for (int j = 0; j < DQ_HEAD_DIM; ++j) {
+            const uint32_t e = T.lut[x & 255u];
+            x = (e >> 24) * (x >> 8) + (e & 255u);
+            if (x < (1u << 23) && ptr < T.rec) x = (x << 8) | byte_at(ptr++);
+            const float lvl = __half2float(__ushort_as_half((unsigned short)((e >> 8) & 0xffffu)));
+            if (symbols) symbols[dst + j] = (uint8_t)(int)lvl;
+            if (dequant) {
+                float v = __fmaf_rn(lvl, s, o);
+                if (mq) v = __fadd_rn(v, __fmul_rn(msc, (float)mq[j]));
+                dequant[dst + j] = v;
+            }
+        }
+    }
+}
+
 }  // namespace
 
 cudaError_t dq_launch_decode_tokens(const DqDevTable& t, const uint8_t* cont, const int8_t* mean_q,
                                     const float* mean_scale, int max_windows, const int32_t* seq_id,
                                     const int32_t* pos, const int32_t* slot, int T, int Hkv,
                                     uint8_t* symbols, float* dequant, cudaStream_t st) {
+    if (t.hs > 1) {
+        const long long ns = (long long)T * (Hkv / t.hs);
+        if (ns == 0) return cudaSuccess;
+        dq_decode_tokens_wide_kernel<<<(unsigned)((ns + 127) / 128), 128, 0, st>>>(
+            t, cont, mean_q, mean_scale, max_windows, seq_id, pos, slot, T, Hkv, symbols, dequant);
+        return cudaGetLastError();
+    }
     const long long n = (long long)T * Hkv;
     if (n == 0) return cudaSuccess;
     dq_decode_tokens_kernel<<<(unsigned)((n + 127) / 128), 128, 0, st>>>(

@@ -342,6 +342,305 @@ dq_encode_kernel(const __grid_constant__ DqDevTable TK, const __grid_constant__ 
     }
 }
 
+
+// ------------------------------------------------------- token-wide streams (hs heads)
+
+// Cross-warp pieces of a stream that spans hs heads: one CTA per stream, warp w holds head w
+// (4 values per lane, as above).  Reductions over the stream go warp -> shared slot -> CTA
+// barrier; slots are double-buffered by call parity so one barrier per reduction suffices.
+struct WideShared {
+    float fmax[2][DQ_MAX_STREAM_HEADS], fmin[2][DQ_MAX_STREAM_HEADS];
+    uint32_t len[2][DQ_MAX_STREAM_HEADS];
+    double sa[DQ_MAX_STREAM_HEADS], sb[DQ_MAX_STREAM_HEADS];
+    int sm[DQ_MAX_STREAM_HEADS], smm[DQ_MAX_STREAM_HEADS];
+};
+
+// Function Drift of Algorithm 1 for a stream held by hs warps; same arithmetic as drift_m, with
+// the extrema of D and the code length taken over the whole stream.
+template <int M>
+__device__ __noinline__ uint32_t drift_wide_m(const EncTable& T, WideShared& W, int hs, int wib, uint32_t& parity,
+                                              float z0, float z1, float z2, float z3, float s, float o,
+                                              uint32_t& sym_packed) {
+    const float z[4] = {z0, z1, z2, z3};
+    const int lane = threadIdx.x & 31;
+    float tm[M], rm[M];
+    uint32_t Rm[M];
+#pragma unroll
+    for (int m = 0; m < M; ++m) {
+        tm[m] = __fmaf_rn((float)m, s, o);
+        rm[m] = T.r[m];
+        Rm[m] = T.R[m];
+    }
+    float D[4][M];
+    float maxD = -INFINITY, minD = INFINITY;
+#pragma unroll
+    for (int e = 0; e < 4; ++e)
+#pragma unroll
+        for (int m = 0; m < M; ++m) {
+            const float d = __fsub_rn(z[e], tm[m]);
+            D[e][m] = __fmul_rn(d, d);
+            maxD = fmaxf(maxD, D[e][m]);
+            minD = fminf(minD, D[e][m]);
+        }
+#pragma unroll
+    for (int d = 16; d >= 1; d >>= 1) {
+        maxD = fmaxf(maxD, __shfl_xor_sync(kFull, maxD, d));
+        minD = fminf(minD, __shfl_xor_sync(kFull, minD, d));
+    }
+    if (lane == 0) { W.fmax[parity][wib] = maxD; W.fmin[parity][wib] = minD; }
+    __syncthreads();
+    for (int w = 0; w < hs; ++w) { maxD = fmaxf(maxD, W.fmax[parity][w]); minD = fminf(minD, W.fmin[parity][w]); }
+    parity ^= 1u;
+    const uint32_t budget = (uint32_t)T.budget_bits << 16;
+    float lam_hi = __fmul_rn(8.0f, __fsub_rn(maxD, minD));
+    float lam_lo = __fmul_rn(lam_hi, 0x1p-40f);
+    uint32_t len = 0, sym[4] = {0u, 0u, 0u, 0u};
+#pragma unroll 1
+    for (int it = 0; it <= 12; ++it) {
+        const float lam = (it < 12) ? __fsqrt_rn(__fmul_rn(lam_lo, lam_hi)) : lam_hi;
+        uint32_t cost_sum = 0;
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            float c[M];
+            uint32_t idx[M];
+#pragma unroll
+            for (int m = 0; m < M; ++m) { c[m] = __fmaf_rn(lam, rm[m], D[e][m]); idx[m] = (uint32_t)m; }
+#pragma unroll
+            for (int w = 1; w < M; w <<= 1)
+#pragma unroll
+                for (int m = 0; m + w < M; m += 2 * w)
+                    if (c[m + w] < c[m]) { c[m] = c[m + w]; idx[m] = idx[m + w]; }
+            sym[e] = idx[0];
+            uint32_t Rsel = Rm[0];
+#pragma unroll
+            for (int m = 1; m < M; ++m) Rsel = (idx[0] == (uint32_t)m) ? Rm[m] : Rsel;
+            cost_sum += Rsel;
+        }
+        const uint32_t wl = __reduce_add_sync(kFull, cost_sum);
+        if (lane == 0) W.len[parity][wib] = wl;
+        __syncthreads();
+        len = 0;
+        for (int w = 0; w < hs; ++w) len += W.len[parity][w];
+        parity ^= 1u;
+        if (it < 12) {
+            if (len <= budget) lam_hi = lam; else lam_lo = lam;
+        }
+    }
+    sym_packed = sym[0] | (sym[1] << 8) | (sym[2] << 16) | (sym[3] << 24);
+    return len;
+}
+
+__device__ __forceinline__ uint32_t drift_wide(const EncTable& T, WideShared& W, int hs, int wib, uint32_t& parity,
+                                               const float (&z)[4], float s, float o, uint32_t (&sym)[4]) {
+    uint32_t packed = 0, len = 0;
+    switch (T.M) {   // uniform across the CTA
+#define DQ_DRIFT_CASE(M_) case M_: len = drift_wide_m<M_>(T, W, hs, wib, parity, z[0], z[1], z[2], z[3], s, o, packed); break;
+        DQ_DRIFT_CASE(2) DQ_DRIFT_CASE(3) DQ_DRIFT_CASE(4) DQ_DRIFT_CASE(5) DQ_DRIFT_CASE(6) DQ_DRIFT_CASE(7)
+        DQ_DRIFT_CASE(8) DQ_DRIFT_CASE(9) DQ_DRIFT_CASE(10) DQ_DRIFT_CASE(11) DQ_DRIFT_CASE(12) DQ_DRIFT_CASE(13)
+        DQ_DRIFT_CASE(14) DQ_DRIFT_CASE(15) DQ_DRIFT_CASE(16)
+#undef DQ_DRIFT_CASE
+        default: break;
+    }
+#pragma unroll
+    for (int e = 0; e < 4; ++e) sym[e] = (packed >> (8 * e)) & 0xffu;
+    return len;
+}
+
+// One CTA of hs warps per stream (token, group of hs KV heads); warp w owns head group * hs + w,
+// lane l its elements 4l .. 4l+3 (stream positions 128 w + 4 l + e).  blockIdx.y selects the
+// tensor kind.  The record goes to the word-interleaved page layout.
+__global__ void __launch_bounds__(DQ_MAX_STREAM_HEADS * 32)
+dq_encode_wide_kernel(const __grid_constant__ DqDevTable TK, const __grid_constant__ DqDevTable TV,
+                      const DqEncodeArgs a) {
+    __shared__ EncTable T;
+    __shared__ WideShared W;
+    __shared__ uint8_t s_bytes[DQ_MAX_WIDE_REC_BYTES];
+    __shared__ __align__(4) uint8_t s_sym[DQ_MAX_STREAM_HEADS * kN];
+    __shared__ uint32_t s_final[2];   // final state, bytes emitted
+    dqdev::pdl_launch_dependents();
+    const bool is_v = a.do_k ? (blockIdx.y == 1) : true;
+    if (threadIdx.x < DQ_MAX_LEVELS) {
+        const int i = threadIdx.x;
+        T.r[i] = is_v ? TV.r[i] : TK.r[i];
+        T.R[i] = is_v ? TV.R[i] : TK.R[i];
+        T.rcp[i] = is_v ? TV.enc_rcp[i] : TK.enc_rcp[i];
+        const uint32_t aux = is_v ? TV.enc_aux[i] : TK.enc_aux[i];
+        T.bias[i] = aux & 1023u;
+        T.cmpl[i] = (aux >> 10) & 511u;
+        T.rsh[i] = aux >> 19;
+        T.thr[i] = (256u - ((aux >> 10) & 511u)) << 23;
+    }
+    if (threadIdx.x == 0) {
+        T.M = is_v ? TV.M : TK.M; T.rec = is_v ? TV.rec : TK.rec; T.mstar = is_v ? TV.mstar : TK.mstar;
+        T.budget_bits = is_v ? TV.budget_bits : TK.budget_bits;
+        T.has_mean = is_v ? TV.has_mean : TK.has_mean; T.rotate = is_v ? TV.rotate : TK.rotate;
+    }
+    __syncthreads();
+    dqdev::pdl_wait_prior_grid();
+    const int lane = threadIdx.x & 31, wib = threadIdx.x >> 5;
+    const int hs = blockDim.x >> 5, Hkv = a.Hkv, groups = Hkv / hs;
+    const int n = hs * kN;
+    const int t = (int)(blockIdx.x / groups), grp = (int)(blockIdx.x % groups), h = grp * hs + wib;
+    const uint16_t* x = static_cast<const uint16_t*>(is_v ? a.v_bf16 : a.k_bf16);
+    uint8_t* cont = is_v ? a.v_cont : a.k_cont;
+    const int rec_words = (T.rec + 3) >> 2;
+    uint32_t parity = 0;
+
+    float z[4];
+    {
+        const uint2 raw = *reinterpret_cast<const uint2*>(x + ((size_t)t * Hkv + h) * kN + 4 * lane);
+        z[0] = bf16_bits_to_float(raw.x & 0xffffu); z[1] = bf16_bits_to_float(raw.x >> 16);
+        z[2] = bf16_bits_to_float(raw.y & 0xffffu); z[3] = bf16_bits_to_float(raw.y >> 16);
+    }
+    if (T.rotate) warp_fwht128(z, lane);
+    if (T.has_mean) {  // remove the (dequantised) windowed channel mean of this head, Sec. 4.2
+        const int ps = a.pos[t], w = ps / DQ_WINDOW_TOKENS;
+        const size_t mi = ((size_t)a.seq_id[t] * a.max_windows + w) * Hkv + h;
+        uint32_t q4;
+        float sc;
+        if (a.mean_mode == DQ_MEAN_REUSE && ps % DQ_WINDOW_TOKENS == 0) {
+            q4 = 0u; sc = 0.f;   // first position of a window: carry the previous window's mean forward
+            if (w > 0) {
+                const size_t src = mi - (size_t)Hkv;
+                q4 = *reinterpret_cast<const uint32_t*>(a.mean_q + src * kN + 4 * lane);
+                sc = a.mean_scale[src];
+            }
+            *reinterpret_cast<uint32_t*>(a.mean_q + mi * kN + 4 * lane) = q4;
+            if (lane == 0) a.mean_scale[mi] = sc;
+        } else {
+            sc = a.mean_scale[mi];
+            q4 = *reinterpret_cast<const uint32_t*>(a.mean_q + mi * kN + 4 * lane);
+        }
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            const float q = (float)(int)(int8_t)((q4 >> (8 * e)) & 0xffu);
+            z[e] = __fsub_rn(z[e], __fmul_rn(sc, q));
+        }
+    }
+    float mx = fmaxf(fmaxf(z[0], z[1]), fmaxf(z[2], z[3]));
+    float mn = fminf(fminf(z[0], z[1]), fminf(z[2], z[3]));
+#pragma unroll
+    for (int d = 16; d >= 1; d >>= 1) {
+        mx = fmaxf(mx, __shfl_xor_sync(kFull, mx, d));
+        mn = fminf(mn, __shfl_xor_sync(kFull, mn, d));
+    }
+    if (lane == 0) { W.fmax[parity][wib] = mx; W.fmin[parity][wib] = mn; }
+    __syncthreads();
+    for (int w = 0; w < hs; ++w) { mx = fmaxf(mx, W.fmax[parity][w]); mn = fminf(mn, W.fmin[parity][w]); }
+    parity ^= 1u;
+
+    uint32_t sym[4];
+    __half s16 = __ushort_as_half(0), o16 = __ushort_as_half(0);
+    bool degenerate = !(mx > mn);
+    uint32_t st_fallback = 0, st_refit = 0;
+    if (!degenerate) {   // uniform across the CTA: mx and mn are stream-wide
+        const float o = mn;                                         // FitMinMax, Eq. (affine_token)
+        const float s = __fdiv_rn(__fsub_rn(mx, mn), (float)(T.M - 1));
+        drift_wide(T, W, hs, wib, parity, z, s, o, sym);
+        // Refit: head sums as in the per-head encoder (lane order, then xor butterfly), added in head order
+        double sa = (double)z[0], sb = __dmul_rn((double)sym[0], (double)z[0]);
+        int sm = (int)sym[0], smm = (int)(sym[0] * sym[0]);
+#pragma unroll
+        for (int e = 1; e < 4; ++e) {
+            sa = __dadd_rn(sa, (double)z[e]);
+            sb = __dadd_rn(sb, __dmul_rn((double)sym[e], (double)z[e]));
+            sm += (int)sym[e];
+            smm += (int)(sym[e] * sym[e]);
+        }
+#pragma unroll
+        for (int d = 16; d >= 1; d >>= 1) {
+            sa = __dadd_rn(sa, __shfl_xor_sync(kFull, sa, d));
+            sb = __dadd_rn(sb, __shfl_xor_sync(kFull, sb, d));
+        }
+        sm = __reduce_add_sync(kFull, sm);
+        smm = __reduce_add_sync(kFull, smm);
+        if (lane == 0) { W.sa[wib] = sa; W.sb[wib] = sb; W.sm[wib] = sm; W.smm[wib] = smm; }
+        __syncthreads();
+        sa = W.sa[0]; sb = W.sb[0];
+        long long Sm = W.sm[0], Smm = W.smm[0];
+        for (int w = 1; w < hs; ++w) {
+            sa = __dadd_rn(sa, W.sa[w]);
+            sb = __dadd_rn(sb, W.sb[w]);
+            Sm += W.sm[w]; Smm += W.smm[w];
+        }
+        const long long den = (long long)n * Smm - Sm * Sm;
+        double sd = (double)s, od = (double)o;
+        if (den != 0) {
+            sd = __ddiv_rn(__dsub_rn(__dmul_rn((double)n, sb), __dmul_rn((double)Sm, sa)), (double)den);
+            od = __ddiv_rn(__dsub_rn(sa, __dmul_rn(sd, (double)Sm)), (double)n);
+        }
+        s16 = __double2half(sd);                                    // fp16 metadata
+        o16 = __double2half(od);
+        float sf = __half2float(s16), of = __half2float(o16);
+        if (!(isfinite(sf) && sf > 0.0f && isfinite(of))) {
+            s16 = __float2half_rn(s);
+            o16 = __float2half_rn(o);
+            sf = __half2float(s16); of = __half2float(o16);
+            st_refit = 1;
+        }
+        if (!(sf > 0.0f)) degenerate = true;
+        else {
+            const uint32_t len = drift_wide(T, W, hs, wib, parity, z, sf, of, sym);   // second Drift, fp16 grid
+            if (len > ((uint32_t)T.budget_bits << 16)) {
+#pragma unroll
+                for (int e = 0; e < 4; ++e) sym[e] = (uint32_t)T.mstar;
+                st_fallback = 1;
+            }
+        }
+    }
+    if (degenerate) {
+        s16 = __ushort_as_half(0);
+        o16 = __float2half_rn(mn);
+#pragma unroll
+        for (int e = 0; e < 4; ++e) sym[e] = (uint32_t)T.mstar;
+    }
+
+    // rANS by warp 0 over the whole stream, symbols n-1 .. 0 (Eq. rans Enc); every lane carries the
+    // same state, lane 0 records the bytes.
+    *reinterpret_cast<uint32_t*>(&s_sym[wib * kN + 4 * lane]) = sym[0] | (sym[1] << 8) | (sym[2] << 16) | (sym[3] << 24);
+    __syncthreads();
+    if (wib == 0) {
+        uint32_t xs = kL;
+        int k = 0;
+        const uint32_t bytes_addr = dqdev::smem_addr(s_bytes);
+#pragma unroll 8
+        for (int j = n - 1; j >= 0; --j) {
+            const uint32_t m = s_sym[j];
+            const uint32_t rcp = T.rcp[m], rsh = T.rsh[m], bias = T.bias[m], cmpl = T.cmpl[m], thr = T.thr[m];
+            if (xs >= thr) {
+                // the budget test keeps k < rec - 8; the bound only guards shared memory
+                if (lane == 0 && k < DQ_MAX_WIDE_REC_BYTES) asm volatile("st.shared.u8 [%0], %1;" ::"r"(bytes_addr + k), "r"(xs & 0xffu));
+                ++k;
+                xs >>= 8;
+            }
+            xs = (__umulhi(xs, rcp) >> rsh) * cmpl + (xs + bias);
+        }
+        if (lane == 0) { s_final[0] = xs; s_final[1] = (uint32_t)k; }
+    }
+    __syncthreads();
+    asm volatile("" ::: "memory");
+    const uint32_t xs = s_final[0];
+    const int k = (int)s_final[1];
+    const uint32_t hdr0 = (uint32_t)__half_as_ushort(s16) | ((uint32_t)__half_as_ushort(o16) << 16);
+    const int sl = a.slot[t];
+    uint8_t* blk = cont + ((size_t)(sl / DQ_PAGE_TOKENS) * groups + grp) * ((size_t)rec_words * 64) +
+                   (size_t)(sl % DQ_PAGE_TOKENS) * 4;
+    const int used = min(8 + k, T.rec);
+    for (int i = threadIdx.x; i < rec_words * 4; i += blockDim.x) {
+        uint8_t v = 0;
+        if (i < 4) v = (uint8_t)(hdr0 >> (8 * i));
+        else if (i < 8) v = (uint8_t)(xs >> (8 * (i - 4)));
+        else if (i < used) v = s_bytes[k - 1 - (i - 8)];
+        blk[(size_t)(i >> 2) * 64 + (i & 3)] = v;
+    }
+    if (a.status && threadIdx.x == 0) {
+        if (st_fallback) atomicAdd(a.status + 0, 1u);
+        if (degenerate) atomicAdd(a.status + 1, 1u);
+        if (st_refit) atomicAdd(a.status + 2, 1u);
+        atomicMax(a.status + 3, (uint32_t)(8 + k));
+    }
+}
+
 }  // namespace
 
 cudaError_t dq_launch_means(const DqDevTable& tk, const void* k_bf16, int T, int Hkv,
@@ -359,6 +658,9 @@ cudaError_t dq_launch_means(const DqDevTable& tk, const void* k_bf16, int T, int
 cudaError_t dq_launch_encode(const DqDevTable& tk, const DqDevTable& tv, const DqEncodeArgs& a, cudaStream_t st) {
     const long long warps = (long long)a.T * a.Hkv;
     if (warps == 0 || (!a.do_k && !a.do_v)) return cudaSuccess;
+    if (tk.hs > 1)   // token-wide streams: one CTA of hs warps per stream
+        return dq_launch_pdl(dq_encode_wide_kernel, dim3((unsigned)(warps / tk.hs), (a.do_k && a.do_v) ? 2 : 1),
+                             dim3(tk.hs * 32), 0, st, tk, tv, a);
     const unsigned blocks = (unsigned)((warps + kEncWarps - 1) / kEncWarps);
     return dq_launch_pdl(dq_encode_kernel, dim3(blocks, (a.do_k && a.do_v) ? 2 : 1), dim3(kEncWarps * 32), 0, st, tk, tv, a);
 }

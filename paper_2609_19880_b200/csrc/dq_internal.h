@@ -9,7 +9,8 @@
 // (constant bank), so building tables needs no device memory.
 struct DqDevTable {
     int M, rec, mstar, budget_bits;
-    int has_mean, rotate, pad0, pad1;
+    int has_mean, rotate;
+    int hs, rec_words;           // heads per stream (>= 1); words per record (interleaved layout, hs > 1)
     uint32_t enc_rcp[DQ_MAX_LEVELS];  // encoder, Eq. rans Enc by reciprocal: floor(x / f) = umulhi(x, rcp) >> rsh
     uint32_t enc_aux[DQ_MAX_LEVELS];  // bias | (256 - f) << 10 | rsh << 19, bias = c (+ 255 when f = 1)
     float r[DQ_MAX_LEVELS];      // ideal cost in bits     (Algorithm 1)

@@ -98,7 +98,7 @@ void finish(dq_table_info& t) {
 }
 
 bool all_central_fits(const dq_table_info& t) {
-    return (int64_t)t.head_dim * t.R[t.mstar] <= (int64_t)t.budget_bits * 65536;
+    return (int64_t)t.head_dim * t.heads_per_stream * t.R[t.mstar] <= (int64_t)t.budget_bits * 65536;
 }
 
 double table_entropy(const dq_table_info& t) {
@@ -117,16 +117,20 @@ int dq_host_build(int levels, double bits_per_elem, const dq_table_opts* opts, d
     if (opts->head_dim != DQ_HEAD_DIM) return DQ_ERR_UNSUPPORTED;
     if (levels < 2 || !(bits_per_elem > 0.0) || !std::isfinite(bits_per_elem)) return DQ_ERR_ARG;
     if (levels > DQ_MAX_LEVELS) return DQ_ERR_UNSUPPORTED;
-    const int n = DQ_HEAD_DIM;
+    if (opts->heads_per_stream < 0 || opts->heads_per_stream > DQ_MAX_STREAM_HEADS) return DQ_ERR_UNSUPPORTED;
+    const int hs = opts->heads_per_stream > 1 ? opts->heads_per_stream : 1;
+    const int n = DQ_HEAD_DIM * hs;   // stream length: the model's n (Sec. 4.2, last paragraph)
     const double rec_d = std::floor(bits_per_elem * n / 8.0 + 1e-9);
-    if (rec_d > DQ_MAX_REC_BYTES) return DQ_ERR_UNSUPPORTED;
+    if (rec_d > (hs > 1 ? DQ_MAX_WIDE_REC_BYTES : DQ_MAX_REC_BYTES)) return DQ_ERR_UNSUPPORTED;
     const int rec = (int)rec_d;
     if (rec < 9) return DQ_ERR_INFEASIBLE;  // header alone is 8 bytes
 
     dq_table_info& t = out->info;
     std::memset(out, 0, sizeof *out);
     t.levels = levels;
-    t.head_dim = n;
+    t.head_dim = DQ_HEAD_DIM;
+    t.heads_per_stream = hs;
+    t.rec_words = (rec + 3) / 4;
     t.rec_bytes = rec;
     t.container_bytes = rec - 4;              // Eq. (budget): C bytes hold state + payload
     t.budget_bits = 8 * t.container_bytes - 32;  // B = 8C - sigma, sigma = 32
@@ -157,6 +161,8 @@ int dq_host_build(int levels, double bits_per_elem, const dq_table_opts* opts, d
     d.budget_bits = t.budget_bits;
     d.has_mean = t.has_mean;
     d.rotate = t.rotate;
+    d.hs = hs;
+    d.rec_words = t.rec_words;
     for (int m = 0; m < levels; ++m) {
         // Enc(x, m) = floor(x / f) 2^p + x mod f + c = x + c + floor(x / f) (2^p - f); the quotient of a
         // 31-bit x by f comes from one high multiply with rcp = ceil(2^(31 + s) / f), s = ceil(log2 f),

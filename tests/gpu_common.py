@@ -97,3 +97,59 @@ def check_attention(out_bf16, out_f32, ref, rows=None):
         assert e32 <= 2e-3, (b, h, e32)
         assert np.all(np.abs(o16[b, h] - r) <= 2e-3 * scale + 2.0 ** -8 * np.abs(r)), (b, h)
     return worst
+
+
+# ---- token-wide streams (heads_per_stream = hs > 1): the library stores records word-interleaved
+# per page, uint8 [pages][groups][rec_words][16][4]; the oracle keeps [pages][groups][16][rec].
+
+def wide_tables(cfg, hs, k_rec=335, v_rec=235, k_levels=8, v_levels=6, alpha=1.4):
+    n = 128 * hs
+    tk = dq.dq_build_tables(k_levels, k_rec * 8 / n, alpha=alpha, has_mean=True, rotate=True, heads_per_stream=hs)
+    tv = dq.dq_build_tables(v_levels, v_rec * 8 / n, alpha=alpha, has_mean=False, rotate=True, heads_per_stream=hs)
+    ok = oracle.build_table(k_levels, n, k_rec, alpha, has_mean=True, rotate=True)
+    ov = oracle.build_table(v_levels, n, v_rec, alpha, has_mean=False, rotate=True)
+    assert tk.info().rec_bytes == k_rec and tv.info().rec_bytes == v_rec
+    return tk, tv, ok, ov
+
+
+def to_interleaved(cont: np.ndarray) -> np.ndarray:
+    """[pages][groups][16][rec] -> [pages][groups][rec_words][16][4] (zero padded)."""
+    P, Gr, _, rec = cont.shape
+    rw = (rec + 3) // 4
+    pad = np.zeros((P, Gr, 16, rw * 4), np.uint8)
+    pad[..., :rec] = cont
+    return np.ascontiguousarray(pad.reshape(P, Gr, 16, rw, 4).transpose(0, 1, 3, 2, 4))
+
+
+def from_interleaved(cw: np.ndarray, rec: int) -> np.ndarray:
+    P, Gr, rw, _, _ = cw.shape
+    flat = cw.transpose(0, 1, 3, 2, 4).reshape(P, Gr, 16, rw * 4)
+    assert not flat[..., rec:].any()          # alignment bytes stay zero
+    return np.ascontiguousarray(flat[..., :rec])
+
+
+class WideGpuCache:
+    def __init__(self, w, tk, tv, hs, dev="cuda"):
+        cfg = w.cfg
+        gr = cfg.hkv // hs
+        self.k_cont = torch.zeros((w.num_pages, gr, tk.info().rec_words, 16, 4), dtype=torch.uint8, device=dev)
+        self.v_cont = torch.zeros((w.num_pages, gr, tv.info().rec_words, 16, 4), dtype=torch.uint8, device=dev)
+        self.mean_q = torch.zeros((cfg.batch, w.max_windows, cfg.hkv, 128), dtype=torch.int8, device=dev)
+        self.mean_scale = torch.zeros((cfg.batch, w.max_windows, cfg.hkv), dtype=torch.float32, device=dev)
+        self.status = torch.zeros(4, dtype=torch.uint32, device=dev)
+
+
+def oracle_encode_wide(w, ok, ov, hs, sel=None):
+    cfg = w.cfg
+    idx = slice(None) if sel is None else sel
+    kb = workloads.bf16_bits(w.k[idx])
+    vb = workloads.bf16_bits(w.v[idx])
+    seq_id, pos, slot = (t[idx].cpu().numpy() for t in (w.seq_id, w.pos, w.slot))
+    mq = np.zeros((cfg.batch, w.max_windows, cfg.hkv, 128), np.int8)
+    ms = np.zeros((cfg.batch, w.max_windows, cfg.hkv), np.float32)
+    oracle.window_means(kb, seq_id, pos, mq, ms, 0)
+    kc = np.zeros((w.num_pages, cfg.hkv // hs, 16, ok.rec), np.uint8)
+    vc = np.zeros((w.num_pages, cfg.hkv // hs, 16, ov.rec), np.uint8)
+    sk = oracle.encode_tokens(ok, kb, seq_id, pos, slot, kc, mq, ms)
+    sv = oracle.encode_tokens(ov, vb, seq_id, pos, slot, vc)
+    return kc, vc, mq, ms, sk, sv

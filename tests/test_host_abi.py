@@ -49,6 +49,33 @@ def test_tables_equal_oracle(L, M, rec, alpha):
         assert lvl == float(o.lut_m[z])
 
 
+@pytest.mark.parametrize("M,hs,rec,alpha", [(8, 8, 335, 1.4), (6, 8, 235, 1.4), (11, 8, 235, 1.4), (6, 2, 86, 1.4),
+                                            (16, 8, 600, -1.0), (4, 4, 150, 0.0)])
+def test_token_wide_tables_equal_oracle(L, M, hs, rec, alpha):
+    """heads_per_stream = hs: the model's n is hs * 128 (Sec. 5.1: one group per token)."""
+    n = 128 * hs
+    t = dq.dq_build_tables(M, rec * 8 / n, alpha=alpha, has_mean=False, rotate=True, heads_per_stream=hs)
+    i = t.info()
+    o = oracle.build_table(M, n, rec, alpha)
+    assert (i.levels, i.rec_bytes, i.container_bytes, i.budget_bits, i.mstar) == (M, rec, o.C, o.B, o.mstar)
+    assert (i.heads_per_stream, i.rec_words, i.head_dim) == (hs, (rec + 3) // 4, 128)
+    assert abs(i.alpha - o.alpha) < 1e-12
+    assert [i.f[m] for m in range(M)] == o.freqs() and [i.R[m] for m in range(M)] == [o.R[m] for m in range(M)]
+    for z in range(256):
+        assert i.lut[z] >> 24 == o.lut_f[z] and i.lut[z] & 255 == o.lut_d[z]
+
+
+def test_token_wide_feasibility_boundary(L):
+    """Table 2: at the 231-byte value container 11 levels fit and 12 do not."""
+    dq.dq_build_tables(11, 235 * 8 / 1024, heads_per_stream=8)
+    with pytest.raises(dq.DqError) as e:
+        dq.dq_build_tables(12, 235 * 8 / 1024, heads_per_stream=8)
+    assert e.value.code == -2
+    with pytest.raises(dq.DqError) as e:
+        dq.dq_build_tables(8, 2.6, heads_per_stream=9)
+    assert e.value.code == -3
+
+
 def test_record_size_from_bits(L):
     for bits, rec in [(2.25, 36), (2.625, 42), (1.8125, 29), (4.6875, 75), (2.26, 36), (3.0, 48)]:
         assert dq.dq_build_tables(3, bits).info().rec_bytes == rec == oracle.rec_bytes(bits, 128)
