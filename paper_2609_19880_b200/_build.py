@@ -16,6 +16,7 @@ _SOURCES = [
     ("dq_api.cu", []),
     ("dq_decode_tokens.cu", []),
     ("dq_attention.cu", []),
+    ("dq_attention_wide.cu", []),
     ("dq_encode.cu", ["-fmad=false"]),
 ]
 _COMMON = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",

@@ -116,6 +116,8 @@ int dq_decode_attention_residual(const dq_tables* tk, const dq_tables* tv, const
                                workspace, workspace_bytes);
     if (rc != DQ_OK) return rc;
     if (tv->info.has_mean) return DQ_ERR_UNSUPPORTED;
+    if (tk->info.heads_per_stream != tv->info.heads_per_stream) return DQ_ERR_UNSUPPORTED;
+    if (Hkv % tk->info.heads_per_stream != 0) return DQ_ERR_ARG;
     if (tk->info.has_mean && (!k_mean_q || !k_mean_scale || max_windows <= 0)) return DQ_ERR_ARG;
     if (tk->info.has_mean && (long long)max_windows * DQ_WINDOW_TOKENS < (long long)max_pages * DQ_PAGE_TOKENS)
         return DQ_ERR_ARG;  // every addressable position needs a window slot

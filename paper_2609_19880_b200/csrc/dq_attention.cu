@@ -25,23 +25,16 @@
 #include <cuda_bf16.h>
 #include <cuda_fp16.h>
 
-#include "dq_device.cuh"
-#include "dq_internal.h"
+#include "dq_attention_common.cuh"
 
 using namespace dqdev;
+using namespace dqattn;
 
 namespace {
 
-constexpr int kN = DQ_HEAD_DIM;
-constexpr int kChunk = 32;             // tokens per warp per item
 constexpr int kTileStride = 48;        // bytes per token row of a [32 tok][16 ch] fp16 tile; the
                                        // 16 pad bytes of the K tile rows hold (sK, oK, sV, oV)
 constexpr int kTileBytes = kChunk * kTileStride;
-constexpr int kQ16Stride = 272;        // bytes per row of the fp16 q' operand (128 halves + pad)
-constexpr int kQ16Bytes = 16 * kQ16Stride;
-constexpr int kPartial = 132;          // floats per partial record: 128 acc, m, l, off, pad
-constexpr int kORow = 132;             // floats per head row of a warp's output slot
-constexpr int kMaxWarps = 16;
 constexpr int kKTail = 32;             // bytes after a warp's K records: q'.mean of its window, per head
 
 struct Item {
@@ -78,32 +71,6 @@ __host__ __device__ inline Layout make_layout(int nw, int rec_k, int rec_v, int 
     L.total = o + 256;  // slack: a malformed record may be over-read by up to 136 + 8 bytes
     return L;
 }
-
-struct AttnParams {
-    const uint16_t* q;
-    const uint8_t* k_cont;
-    const uint8_t* v_cont;
-    const int8_t* mean_q;
-    const float* mean_scale;
-    const int32_t* page_table;
-    const int32_t* seq_lens;
-    int* counter;
-    int* prefix;        // [B + 1] blocks before sequence b
-    float* qrot;        // [B][Hq][128]              rotated q (bf16 baseline reads q itself)
-    uint16_t* q16;      // [B][Hkv][16][128] halves  fp16 hi (rows g) / lo (rows 8 + g) of q'
-    float* qsum;        // [B][Hq]                   sum_j q'_j
-    float* qmu;         // [B][Hq][windows]          sum_j q'_j mean_j of every window
-    float* partial;     // [blocks][Hq][kPartial]
-    void* out_bf16;
-    float* out_f32;
-    int max_windows, windows, max_pages, B, Hq, Hkv, G, item_tokens, rotate_q, rotate_out, has_mean;
-    float scale_log2;   // sm_scale * log2(e)
-    unsigned hkv_magic; // ceil(2^32 / Hkv), 0 when Hkv = 1
-    const uint16_t* resid_k;      // bf16 [B][resid_cap][Hkv][128], nullable: uncompressed recent tokens
-    const uint16_t* resid_v;
-    const int32_t* resid_lens;    // [B]
-    int resid_cap;
-};
 
 // ------------------------------------------------------------------ prepare
 
@@ -197,12 +164,6 @@ dq_attn_prepare_kernel(AttnParams p) {
 
 // --------------------------------------------------------------------- main
 
-__device__ __forceinline__ uint32_t dp4a_u32(uint32_t a, uint32_t b, uint32_t c) {
-    uint32_t d;
-    asm("dp4a.u32.u32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
-    return d;
-}
-
 // Decode 16 symbols of one stream (Algorithm 2) and pack their levels as 8 fp16x2 words.
 //   x    rANS state;  ptr  shared-memory byte address of the next renormalisation byte
 //   lut  shared address of this lane's column of the 32-way replicated table: entry z at
@@ -234,19 +195,6 @@ __device__ __forceinline__ void decode16(uint32_t& x, uint32_t& ptr, uint32_t lu
         packed[2 * q4] = __byte_perm(e[0], e[1], 0x6521u);
         packed[2 * q4 + 1] = __byte_perm(e[2], e[3], 0x6521u);
     }
-}
-
-__device__ __forceinline__ uint32_t pack_half2(float a, float b) {
-    const __half2 h = __floats2half2_rn(a, b);
-    return *reinterpret_cast<const uint32_t*>(&h);
-}
-
-__device__ __forceinline__ void sts128(uint32_t addr, const uint32_t* v) {
-    asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};\n" ::"r"(addr), "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3])
-                 : "memory");
-}
-__device__ __forceinline__ void sts32f(uint32_t addr, float v) {
-    asm volatile("st.shared.f32 [%0], %1;\n" ::"r"(addr), "f"(v) : "memory");
 }
 
 // One pass over the 128 channels, 16 at a time.  With DO_K the K streams of the current item
@@ -916,12 +864,18 @@ cudaError_t dq_launch_attention(const DqDevTable& tk, const DqDevTable& tv, cons
     }
     int nw = kMaxWarps;
     const int G = a.Hq / a.Hkv;
+    const bool wide = tk.hs > 1;   // token-wide streams: main kernel of dq_attention_wide.cu
     Layout L = make_layout(nw, tk.rec, tv.rec, a.B, G);
-    while (L.total > smem_max && nw > 4) {
-        nw -= 2;
-        L = make_layout(nw, tk.rec, tv.rec, a.B, G);
+    if (wide) {
+        nw = dq_attn_wide_pick_warps(tk, tv, a.B, G, smem_max);
+        if (nw == 0) return cudaErrorInvalidConfiguration;
+    } else {
+        while (L.total > smem_max && nw > 4) {
+            nw -= 2;
+            L = make_layout(nw, tk.rec, tv.rec, a.B, G);
+        }
+        if (L.total > smem_max) return cudaErrorInvalidConfiguration;
     }
-    if (L.total > smem_max) return cudaErrorInvalidConfiguration;
 
     const WsLayout w = ws_layout(a.B, a.Hq, a.max_pages);
     uint8_t* ws = static_cast<uint8_t*>(a.workspace);
@@ -944,6 +898,8 @@ cudaError_t dq_launch_attention(const DqDevTable& tk, const DqDevTable& tv, cons
     p.rotate_q = tk.rotate; p.rotate_out = tv.rotate; p.has_mean = tk.has_mean;
     p.scale_log2 = a.sm_scale * 1.4426950408889634f;
     p.hkv_magic = a.Hkv > 1 ? (unsigned)((0x100000000ull + a.Hkv - 1) / a.Hkv) : 0u;
+    p.hs = tk.hs; p.groups = a.Hkv / tk.hs;
+    if (wide) p.hkv_magic = p.groups > 1 ? (unsigned)((0x100000000ull + p.groups - 1) / p.groups) : 0u;
     p.resid_k = static_cast<const uint16_t*>(a.resid_k); p.resid_v = static_cast<const uint16_t*>(a.resid_v);
     p.resid_lens = a.resid_lens; p.resid_cap = a.resid_cap;
 
@@ -951,8 +907,10 @@ cudaError_t dq_launch_attention(const DqDevTable& tk, const DqDevTable& tv, cons
     const long long prep_warps = (long long)heads * (1 + (p.has_mean ? (p.windows + kPrepWindows - 1) / kPrepWindows : 0));
     cudaError_t e = dq_launch_pdl(dq_attn_prepare_kernel, dim3((unsigned)((prep_warps + 7) / 8)), dim3(256), 0, st, p);
     if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(dq_attention_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, L.total);
-    if (e != cudaSuccess) return e;
+    if (!wide) {
+        e = cudaFuncSetAttribute(dq_attention_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, L.total);
+        if (e != cudaSuccess) return e;
+    }
     const bool prof = g_prof_on && g_prof_count < kProfRing && (g_prof_calls++ % g_prof_period) == 0;
     if (prof) {
         if (!g_prof_made[g_prof_count]) {
@@ -962,7 +920,8 @@ cudaError_t dq_launch_attention(const DqDevTable& tk, const DqDevTable& tv, cons
         }
         cudaEventRecord(g_prof_ev[g_prof_count][0], st);
     }
-    e = dq_launch_pdl(dq_attention_kernel, dim3(sm_count), dim3(nw * 32), (size_t)L.total, st, tk, tv, p);
+    if (wide) e = dq_launch_attention_wide_main(tk, tv, p, nw, sm_count, st);
+    else e = dq_launch_pdl(dq_attention_kernel, dim3(sm_count), dim3(nw * 32), (size_t)L.total, st, tk, tv, p);
     if (e != cudaSuccess) return e;
     if (prof) cudaEventRecord(g_prof_ev[g_prof_count++][1], st);
     return dq_launch_pdl(dq_attn_combine_kernel, dim3(heads), dim3(256), 0, st, p);
@@ -990,6 +949,7 @@ cudaError_t dq_launch_bf16_attention(const DqAttnArgs& a, const void* k_pages, c
     p.rotate_q = 0; p.rotate_out = 0;
     p.scale_log2 = a.sm_scale * 1.4426950408889634f;
     p.hkv_magic = 0;
+    p.hs = 1; p.groups = a.Hkv;
     p.resid_k = nullptr; p.resid_v = nullptr; p.resid_lens = nullptr; p.resid_cap = 0;
     const int heads = a.B * a.Hq;
     dq_attn_prepare_kernel<<<(heads + 7) / 8, 256, 0, st>>>(p);

@@ -98,3 +98,101 @@ def test_encoder_degenerate_and_fallback_streams():
     assert np.array_equal(gc.from_interleaved(_np(cache.v_cont), ov.rec), vc)
     st = _np(cache.status)
     assert st[1] == sk[1] + sv[1] >= 1 and st[0] == sk[0] + sv[0]
+
+
+# --------------------------------------------------------------- attention
+
+def _oracle_attention(w, ok, ov, kc, vc, mq, ms, seq_lens, **kw):
+    return oracle.attention(ok, ov, workloads.bf16_bits(w.q), kc, vc, mq, ms, _np(w.page_table), _np(seq_lens),
+                            w.cfg.hkv, gc.SM_SCALE, **kw)
+
+
+@pytest.mark.parametrize("name", list(CASES))
+def test_attention_matches_oracle(name):
+    cfg, w, hs, tk, tv, ok, ov = _setup(name)
+    cache = gc.WideGpuCache(w, tk, tv, hs)
+    gc.gpu_encode(w, tk, tv, cache)
+    out, out32 = gc.gpu_attention(w, tk, tv, cache)
+    kc = gc.from_interleaved(_np(cache.k_cont), ok.rec)
+    vc = gc.from_interleaved(_np(cache.v_cont), ov.rec)
+    ref = _oracle_attention(w, ok, ov, kc, vc, _np(cache.mean_q), _np(cache.mean_scale), w.seq_lens)
+    worst = gc.check_attention(out, out32, ref)
+    assert worst < 2e-4
+    out_b, out32_b = gc.gpu_attention(w, tk, tv, cache)
+    assert torch.equal(out, out_b) and torch.equal(out32, out32_b)   # run-to-run identical
+
+
+def test_attention_edge_lengths():
+    """Empty sequences, single tokens, lengths around page / warp / item boundaries (items are
+    15 warps x 32 tokens = 480 tokens at this shape)."""
+    lens_all = [0, 1, 15, 16, 17, 31, 32, 33, 479, 480, 481, 600, 959, 960, 961]
+    cfg = _cfg(4, batch=len(lens_all), seq_lens=[961] * len(lens_all))
+    w = workloads.generate(cfg, device="cuda")
+    tk, tv, ok, ov = gc.wide_tables(cfg, 8)
+    cache = gc.WideGpuCache(w, tk, tv, 8)
+    gc.gpu_encode(w, tk, tv, cache)
+    lens = torch.tensor(lens_all, dtype=torch.int32, device="cuda")
+    out, out32 = gc.gpu_attention(w, tk, tv, cache, seq_lens=lens)
+    kc = gc.from_interleaved(_np(cache.k_cont), ok.rec)
+    vc = gc.from_interleaved(_np(cache.v_cont), ov.rec)
+    ref = _oracle_attention(w, ok, ov, kc, vc, _np(cache.mean_q), _np(cache.mean_scale), lens)
+    gc.check_attention(out, out32, ref)
+    assert not out[0].any()
+
+
+def test_lagging_streams_take_the_global_path():
+    """Keys whose streams stop consuming bytes early (constant tokens between ordinary ones) fall
+    far behind their warp's ring and must be served from global memory with the same result."""
+    cfg, w, hs, tk, tv, ok, ov = _setup("paper_default")
+    w.k[5:400:7] = 0.0
+    w.v[9:400:11] = 0.0
+    cache = gc.WideGpuCache(w, tk, tv, hs)
+    gc.gpu_encode(w, tk, tv, cache)
+    out, out32 = gc.gpu_attention(w, tk, tv, cache)
+    kc = gc.from_interleaved(_np(cache.k_cont), ok.rec)
+    vc = gc.from_interleaved(_np(cache.v_cont), ov.rec)
+    ref = _oracle_attention(w, ok, ov, kc, vc, _np(cache.mean_q), _np(cache.mean_scale), w.seq_lens)
+    gc.check_attention(out, out32, ref)
+
+
+def test_corrupted_records_stay_in_bounds():
+    """Random bytes in place of records: the kernel must finish and write finite-or-not numbers
+    without touching memory outside its buffers (states and pointers are data-dependent)."""
+    cfg, w, hs, tk, tv, ok, ov = _setup("ragged_shuffled")
+    cache = gc.WideGpuCache(w, tk, tv, hs)
+    g = torch.Generator(device="cuda").manual_seed(5)
+    cache.k_cont.copy_(torch.randint(0, 256, cache.k_cont.shape, generator=g, device="cuda", dtype=torch.uint8))
+    cache.v_cont.copy_(torch.randint(0, 256, cache.v_cont.shape, generator=g, device="cuda", dtype=torch.uint8))
+    canary = torch.full((1 << 20,), 0x5A, dtype=torch.uint8, device="cuda")
+    out, out32 = gc.gpu_attention(w, tk, tv, cache)
+    torch.cuda.synchronize()
+    assert bool((canary == 0x5A).all())
+    # and the library still works afterwards
+    gc.gpu_encode(w, tk, tv, cache)
+    out, out32 = gc.gpu_attention(w, tk, tv, cache)
+    assert torch.isfinite(out32).all()
+
+
+def test_paper_default_with_residual_window():
+    """The paper's serving configuration: token-wide 331 / 231-byte containers, 8 / 6 levels, plus
+    the most recent tokens in BF16."""
+    cfg, w, hs, tk, tv, ok, ov = _setup("paper_default")
+    cache = gc.WideGpuCache(w, tk, tv, hs)
+    gc.gpu_encode(w, tk, tv, cache)
+    gen = torch.Generator(device="cuda").manual_seed(11)
+    rk, rv = workloads.make_kv(cfg, cfg.batch * 128, gen, torch.device("cuda"), w.k_offsets, w.k_gain)
+    rk = rk.view(cfg.batch, 128, cfg.hkv, 128).contiguous()
+    rv = rv.view(cfg.batch, 128, cfg.hkv, 128).contiguous()
+    rl = torch.tensor([128, 5, 77], dtype=torch.int32, device="cuda")
+    out = torch.empty((cfg.batch, cfg.hq, 128), dtype=torch.bfloat16, device="cuda")
+    out32 = torch.empty((cfg.batch, cfg.hq, 128), dtype=torch.float32, device="cuda")
+    ws = torch.empty(dq.dq_decode_workspace_bytes(cfg.batch, cfg.hq, w.page_table.shape[1]), dtype=torch.uint8,
+                     device="cuda")
+    dq.dq_decode_attention_residual(tk, tv, w.q, cache.k_cont, cache.v_cont, cache.mean_q, cache.mean_scale,
+                                    w.page_table, w.seq_lens, rk, rv, rl, cfg.hkv, gc.SM_SCALE, out, ws, out32)
+    torch.cuda.synchronize()
+    kc = gc.from_interleaved(_np(cache.k_cont), ok.rec)
+    vc = gc.from_interleaved(_np(cache.v_cont), ov.rec)
+    ref = _oracle_attention(w, ok, ov, kc, vc, _np(cache.mean_q), _np(cache.mean_scale), w.seq_lens,
+                            resid_k=workloads.bf16_bits(rk), resid_v=workloads.bf16_bits(rv), resid_lens=_np(rl))
+    gc.check_attention(out, out32, ref)
