@@ -3,7 +3,7 @@
 cache (2.26 bits/element), with the encoder on the step's new tokens.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
-                    [--config 2|3|4|5] [--budget 2.26]
+                    [--config 2|3|4|5] [--budget 2.26] [--streams head|token]
 
 One *step* = one decode step of the whole hot path: encode one new token per sequence (K and
 V: Hadamard, mean removal, drift, rANS) into the cache, then decode-step attention over every
@@ -104,7 +104,18 @@ class ClockSampler(threading.Thread):
 
 # --------------------------------------------------------------------------- CPU oracle leg
 
-def oracle_step_runner(cfg_idx: int, budget: float):
+def stream_setup(cfg, streams: str):
+    """Record sizes, level counts and heads per stream of the run: the benchmark's per token-head
+    streams at the requested budget, or the paper's default grouping (one stream per token:
+    335 / 235-byte records = 331 / 231-byte containers, 8 / 6 levels)."""
+    if streams == "token":
+        hs = cfg.hkv
+        assert hs <= 8, "a token-wide stream holds at most 1024 values"
+        return dict(hs=hs, k_rec=335 * hs // 8, v_rec=235 * hs // 8, k_levels=8, v_levels=6, alpha=1.4)
+    return dict(hs=1, k_rec=cfg.k_rec, v_rec=cfg.v_rec, k_levels=cfg.k_levels, v_levels=cfg.v_levels, alpha=cfg.alpha)
+
+
+def oracle_step_runner(cfg_idx: int, budget: float, streams: str = "head"):
     """Builds the bounded oracle sample (sequence 0 of the workload, all KV heads) and returns
     (step function, KV tokens per step, description).  GPU-free."""
     import numpy as np
@@ -114,15 +125,16 @@ def oracle_step_runner(cfg_idx: int, budget: float):
     cfg = workloads.make_config(cfg_idx, budget=budget)
     cfg.batch, cfg.seq_lens = 1, [min(cfg.seq_lens[0], 8192)]
     w = workloads.generate(cfg, device="cpu")
-    ok = oracle.build_table(cfg.k_levels, 128, cfg.k_rec, cfg.alpha, has_mean=True, rotate=True)
-    ov = oracle.build_table(cfg.v_levels, 128, cfg.v_rec, cfg.alpha, has_mean=False, rotate=True)
+    st = stream_setup(cfg, streams)
+    ok = oracle.build_table(st["k_levels"], 128 * st["hs"], st["k_rec"], st["alpha"], has_mean=True, rotate=True)
+    ov = oracle.build_table(st["v_levels"], 128 * st["hs"], st["v_rec"], st["alpha"], has_mean=False, rotate=True)
     kb, vb, qb = workloads.bf16_bits(w.k), workloads.bf16_bits(w.v), workloads.bf16_bits(w.q)
     seq_id, pos, slot = (t.numpy() for t in (w.seq_id, w.pos, w.slot))
     mq = np.zeros((1, w.max_windows, cfg.hkv, 128), np.int8)
     ms = np.zeros((1, w.max_windows, cfg.hkv), np.float32)
     oracle.window_means(kb, seq_id, pos, mq, ms, 0)
-    kc = np.zeros((w.num_pages, cfg.hkv, 16, ok.rec), np.uint8)
-    vc = np.zeros((w.num_pages, cfg.hkv, 16, ov.rec), np.uint8)
+    kc = np.zeros((w.num_pages, cfg.hkv // st["hs"], 16, ok.rec), np.uint8)
+    vc = np.zeros((w.num_pages, cfg.hkv // st["hs"], 16, ov.rec), np.uint8)
     oracle.encode_tokens(ok, kb, seq_id, pos, slot, kc, mq, ms)
     oracle.encode_tokens(ov, vb, seq_id, pos, slot, vc)
     last = slice(cfg.total_tokens - 1, cfg.total_tokens)
@@ -140,8 +152,8 @@ def oracle_step_runner(cfg_idx: int, budget: float):
     return step, cfg.seq_lens[0], desc, oracle.num_threads()
 
 
-def time_oracle(cfg_idx, budget, budget_s=10.0, max_steps=1000, warmup=1):
-    step, toks, desc, cores = oracle_step_runner(cfg_idx, budget)
+def time_oracle(cfg_idx, budget, budget_s=10.0, max_steps=1000, warmup=1, streams="head"):
+    step, toks, desc, cores = oracle_step_runner(cfg_idx, budget, streams)
     for _ in range(warmup):
         step()
     n, t0 = 0, time.perf_counter()
@@ -159,7 +171,7 @@ def run_reference(args):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
-    step, toks, desc, cores = oracle_step_runner(args.config, args.budget)
+    step, toks, desc, cores = oracle_step_runner(args.config, args.budget, args.streams)
     for _ in range(max(args.warmup, 1)):
         step()
     t0 = time.perf_counter()
@@ -219,18 +231,29 @@ def run_ours(args):
     cfg = workloads.make_config(args.config, budget=args.budget)
     w = workloads.generate(cfg, device=dev)
     B, Hq, Hkv = cfg.batch, cfg.hq, cfg.hkv
-    tk = dq.dq_build_tables(cfg.k_levels, cfg.bits_k, alpha=cfg.alpha, has_mean=True, rotate=True)
-    tv = dq.dq_build_tables(cfg.v_levels, cfg.bits_v, alpha=cfg.alpha, has_mean=False, rotate=True)
+    st = stream_setup(cfg, args.streams)
+    hs, k_rec, v_rec = st["hs"], st["k_rec"], st["v_rec"]
+    n_stream = 128 * hs
+    tk = dq.dq_build_tables(st["k_levels"], k_rec * 8 / n_stream, alpha=st["alpha"], has_mean=True, rotate=True,
+                            heads_per_stream=hs)
+    tv = dq.dq_build_tables(st["v_levels"], v_rec * 8 / n_stream, alpha=st["alpha"], has_mean=False, rotate=True,
+                            heads_per_stream=hs)
+    assert tk.info().rec_bytes == k_rec and tv.info().rec_bytes == v_rec
     sm_scale = 1.0 / math.sqrt(128.0)
 
     token_heads = cfg.total_tokens * Hkv
-    cache_bytes = token_heads * (cfg.k_rec + cfg.v_rec) + B * w.max_windows * Hkv * 132
+    # bytes one token-head occupies in the cache (token-wide records are padded to whole words)
+    k_b = k_rec if hs == 1 else 4 * tk.info().rec_words / hs
+    v_b = v_rec if hs == 1 else 4 * tv.info().rec_words / hs
+    cache_bytes = int(token_heads * (k_b + v_b)) + B * w.max_windows * Hkv * 132
     copies = max(2, math.ceil(2.2 * L2_BYTES / cache_bytes)) if cache_bytes < 2 * L2_BYTES else 1
 
     def new_cache():
         return dict(
-            k=torch.zeros((w.num_pages, Hkv, 16, cfg.k_rec), dtype=torch.uint8, device=dev),
-            v=torch.zeros((w.num_pages, Hkv, 16, cfg.v_rec), dtype=torch.uint8, device=dev),
+            k=torch.zeros((w.num_pages, Hkv, 16, k_rec) if hs == 1 else (w.num_pages, Hkv // hs, tk.info().rec_words, 16, 4),
+                          dtype=torch.uint8, device=dev),
+            v=torch.zeros((w.num_pages, Hkv, 16, v_rec) if hs == 1 else (w.num_pages, Hkv // hs, tv.info().rec_words, 16, 4),
+                          dtype=torch.uint8, device=dev),
             mq=torch.zeros((B, w.max_windows, Hkv, 128), dtype=torch.int8, device=dev),
             ms=torch.zeros((B, w.max_windows, Hkv), dtype=torch.float32, device=dev))
 
@@ -348,25 +371,25 @@ def run_ours(args):
     # ---- roofline of the dominant kernel (fused decode attention)
     k_ms = statistics.mean(kern_ms) if kern_ms else None
     symbols = token_heads * 256.0
-    comp_bytes = token_heads * (cfg.k_rec + cfg.v_rec + 1.0)   # records + amortised INT8 mean byte
+    comp_bytes = token_heads * (k_b + v_b + 1.0)   # records + amortised INT8 mean byte
     roofline = None
     extra = {}
     if args.traffic_bytes is None:
         # ncu, config 2: dram__bytes_read + write = 37.62 MB for 524288 token-heads at 42 + 29 byte records;
         # the kernel reads every record once, so traffic grows with the records' bytes
-        args.traffic_bytes = 37.62e6 * (token_heads * (cfg.k_rec + cfg.v_rec + 1.0)) / (524288 * 72.0)
+        args.traffic_bytes = 37.62e6 * (token_heads * (k_b + v_b + 1.0)) / (524288 * 72.0)
     if k_ms:
         alu_peak = SM_COUNT * LANES_PER_SM_CLK * sm_max_mhz * 1e6 / 1e9          # G lane-ops / s
         alu_ach = symbols * ALU_OPS_PER_SYMBOL / (k_ms * 1e-3) / 1e9
         gbs = comp_bytes / (k_ms * 1e-3) / 1e9
         roofline = {"bound": "alu", "achieved": alu_ach, "peak": alu_peak, "unit": "Gop/s (int32 lane ops)",
                     "frac": alu_ach / alu_peak, "traffic": args.traffic_bytes,
-                    "kernel": "dq_attention_kernel", "kernel_ms": k_ms, "launches_timed": len(kern_ms),
+                    "kernel": "dq_attention_kernel" if hs == 1 else "dq_attention_wide_kernel", "kernel_ms": k_ms, "launches_timed": len(kern_ms),
                     "peak_source": f"148 SM x 128 lanes x {sm_max_mhz:.0f} MHz ({peak_kind} clocks)",
                     "ops_per_symbol": ALU_OPS_PER_SYMBOL}
         extra = {"hbm": {"bound": "hbm", "achieved": gbs, "peak": hbm_peak, "unit": "GB/s", "frac": gbs / hbm_peak,
                          "frac_of_8TBps": gbs / 8000.0, "peak_source": peak_kind,
-                         "bytes_per_token_head": cfg.k_rec + cfg.v_rec + 1},
+                         "bytes_per_token_head": k_b + v_b + 1},
                  "kernel_token_heads_per_s": token_heads / (k_ms * 1e-3),
                  "kernel_symbols_per_s": symbols / (k_ms * 1e-3)}
 
@@ -401,17 +424,19 @@ def run_ours(args):
 
     cpu = None
     if world == 1 and not args.no_cpu_baseline:
-        cpu = time_oracle(args.config, args.budget)
+        cpu = time_oracle(args.config, args.budget, streams=args.streams)
 
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
         "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "u32 rANS state / f16 mma, f32 accumulate", "data": "synthetic",
-        "config": {"workload": cfg.name, "batch": B, "q_heads": Hq, "kv_heads": Hkv, "head_dim": 128,
+        "config": {"workload": cfg.name + ("" if hs == 1 else "_tokenwide"), "batch": B, "q_heads": Hq, "kv_heads": Hkv, "head_dim": 128,
                    "context": cfg.seq_lens if len(set(cfg.seq_lens)) > 1 and B <= 8 else
                    {"min": min(cfg.seq_lens), "max": max(cfg.seq_lens), "sum": kv_tokens},
-                   "bits_per_elem": args.budget, "k_rec_bytes": cfg.k_rec, "v_rec_bytes": cfg.v_rec,
-                   "k_levels": cfg.k_levels, "v_levels": cfg.v_levels,
+                   "bits_per_elem": args.budget if hs == 1 else round((k_b + v_b + 1.0) * 8 / 256, 3),
+                   "streams": "per token-head (128 values)" if hs == 1 else f"per token ({n_stream} values)",
+                   "k_rec_bytes": k_rec, "v_rec_bytes": v_rec,
+                   "k_levels": st["k_levels"], "v_levels": st["v_levels"],
                    "step": "encode 1 new token per sequence + decode attention over the whole cache",
                    "l2": f"{copies} rotating copies of the cache ({copies * cache_bytes / 2**20:.0f} MiB > 126 MiB L2)",
                    "parallelism": "replicas only" if world > 1 else "single GPU"},
@@ -419,7 +444,7 @@ def run_ours(args):
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
         "gpu_launches": launches_per_step * args.steps, "clocks": clocks,
         "encoder": {"token_heads_per_s": 2 * token_heads / (enc_ms * 1e-3), "prefill_ms": enc_ms,
-                    "streams": 2 * token_heads},
+                    "streams": 2 * token_heads // hs},
         "bf16_baseline": bf16,
     }
     line.update(extra)
@@ -436,6 +461,9 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--config", type=int, default=2, choices=[2, 3, 4, 5])
     ap.add_argument("--budget", type=float, default=2.26)
+    ap.add_argument("--streams", default="head", choices=["head", "token"],
+                    help="head: one stream per (token, KV head), the benchmark's configuration; token: the paper's "
+                         "default grouping, one 335 / 235-byte record per token, 8 / 6 levels")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--profile-only", action="store_true",
                     help="warm-up and timed steps only (for profiler captures); prints a short line")
