@@ -41,7 +41,8 @@ def build(force: bool = False, verbose: bool = False) -> str:
         s = os.path.join(_CSRC, src)
         o = os.path.join(obj_dir, src.replace(".cu", ".o"))
         if force or _newer(o, [s] + headers):
-            cmd = [nvcc] + _COMMON + extra + (["-Xptxas", "-v"] if verbose else []) + ["-c", s, "-o", o]
+            cmd = [nvcc] + _COMMON + extra + os.environ.get("DQ_NVCC_EXTRA", "").split() + \
+                  (["-Xptxas", "-v"] if verbose else []) + ["-c", s, "-o", o]
             subprocess.run(cmd, check=True)
         objs.append(o)
     if force or _newer(LIB_PATH, objs):

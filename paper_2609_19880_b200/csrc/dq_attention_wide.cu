@@ -29,6 +29,7 @@ constexpr int kRingK = kRowsK * 128, kRingV = kRowsV * 128;
 constexpr int kTile = 1024;                    // [32 tok][16 ch] fp16, 32-byte rows, halves swizzled by (row >> 2) & 1
 constexpr int kFillRows = 12;                  // rows fetched when a stream starts (header + 40 bytes)
 constexpr int kAhead = 10;                     // rows kept beyond the fastest lane's word index
+constexpr int kWideWarps = 15;                 // most warps per CTA (480 threads leave 136 registers each)
 
 struct Item {
     int b, grp, blk, len, bg, valid;
@@ -56,7 +57,7 @@ __host__ __device__ inline WLayout make_wlayout(int nw, int B, int G) {
     L.off_prefix = o; o += align16w((2 * B + 1) * 4);
     L.off_qsum = o; o += 2 * DQ_MAX_GROUP * 4;
     L.off_red = o; o += (kMaxWarps + 2) * DQ_MAX_GROUP * 4;
-    L.off_pages = o; o += kMaxWarps * 3 * 2 * 4 + 16;
+    L.off_pages = o; o += kMaxWarps * 4 * 2 * 4 + 16;   // per warp: page ids of 4 items in flight; prev rows
     L.off_qmu = o; o += nw * 2 * DQ_MAX_GROUP * 4;
     L.total = o;
     return L;
@@ -64,25 +65,16 @@ __host__ __device__ inline WLayout make_wlayout(int nw, int B, int G) {
 
 // Decode 16 symbols of one stream (Algorithm 2) out of the warp's ring and pack their levels as
 // 8 fp16x2 words.  ptr is the index of the next renormalisation byte within the record; the
-// 4-byte window is reloaded every 4 symbols from ring rows (ptr >> 2) and (ptr >> 2) + 1, or,
-// for a lane outside the ring's range (`fast` false), from the record in global memory
-// (gcol: this lane's word 0; consecutive words are 16 words apart).
+// 4-byte window is reloaded every 4 symbols from ring rows (ptr >> 2) and (ptr >> 2) + 1.
 template <int ROWS>
 __device__ __forceinline__ void decode16_ring(uint32_t& x, uint32_t& ptr, uint32_t ring_lane, uint32_t lut, uint32_t one,
-                                              uint32_t (&packed)[8], bool fast, const uint32_t* gcol, int rec_words) {
+                                              uint32_t (&packed)[8]) {
     constexpr uint32_t kMask = (uint32_t)(ROWS - 1) << 7;
 #pragma unroll
     for (int q4 = 0; q4 < 4; ++q4) {
         const uint32_t t = ptr << 5;   // (word index) * 128 + junk below bit 7
-        uint32_t lo, hi;
-        if (fast) {
-            lo = lds32(ring_lane + (t & kMask));
-            hi = lds32(ring_lane + ((t + 128u) & kMask));
-        } else {
-            const int wi = min((int)(ptr >> 2), rec_words - 2);
-            lo = __ldg(gcol + (size_t)wi * 16);
-            hi = __ldg(gcol + (size_t)wi * 16 + 16);
-        }
+        const uint32_t lo = lds32(ring_lane + (t & kMask));
+        const uint32_t hi = lds32(ring_lane + ((t + 128u) & kMask));
         const uint32_t win = __funnelshift_r(lo, hi, ptr << 3);
         uint32_t sel = 0x2104u;
         uint32_t e[4];
@@ -102,33 +94,77 @@ __device__ __forceinline__ void decode16_ring(uint32_t& x, uint32_t& ptr, uint32
     }
 }
 
+// The same 16 symbols for a warp in which some lane lags too far behind the ring: such a lane
+// (`fast` false) takes its window words from the record in global memory (col: its word 0;
+// consecutive words are 16 words apart).  Rare, kept out of line.
+struct Decoded16 {
+    uint32_t packed[8];
+    uint32_t x, ptr;
+};
+__device__ __noinline__ Decoded16 decode16_mixed(uint32_t x, uint32_t ptr, uint32_t ring_lane, uint32_t ring_mask,
+                                                 uint32_t lut, bool fast, const uint32_t* col, int rec_words) {
+    Decoded16 r;
+    for (int q4 = 0; q4 < 4; ++q4) {
+        const uint32_t t = ptr << 5;
+        uint32_t lo, hi;
+        if (fast) {
+            lo = lds32(ring_lane + (t & ring_mask));
+            hi = lds32(ring_lane + ((t + 128u) & ring_mask));
+        } else {
+            const int wi = min((int)(ptr >> 2), rec_words - 2);
+            lo = __ldg(col + (size_t)wi * 16);
+            hi = __ldg(col + (size_t)wi * 16 + 16);
+        }
+        uint32_t win = __funnelshift_r(lo, hi, ptr << 3);
+        uint32_t e[4];
+        for (int i = 0; i < 4; ++i) {
+            e[i] = lds32(lut + ((x & 255u) << 7));
+            x = (e[i] >> 24) * (x >> 8) + (e[i] & 255u);
+            if (x < (1u << 23)) {   // at most one byte per symbol
+                x = (x << 8) | (win & 255u);
+                win >>= 8;
+                ++ptr;
+            }
+        }
+        r.packed[2 * q4] = __byte_perm(e[0], e[1], 0x6521u);
+        r.packed[2 * q4 + 1] = __byte_perm(e[2], e[3], 0x6521u);
+    }
+    r.x = x; r.ptr = ptr;
+    return r;
+}
+
 // State of one tensor kind's streams in a warp.
 struct Chain {
     uint32_t x, ptr;        // rANS state, next byte index within the record (per lane)
     uint32_t E;             // ring holds rows [.., E) (warp-uniform)
-    uint32_t src16;         // per lane: source of its 16-byte piece of row 0, in 16-byte units
-    const uint32_t* gcol;   // per lane: word 0 of its own record (global)
+    uint32_t src16;         // per lane: source of its 16-byte piece of row 0, in 16-byte units from the container base
     bool active;            // lane's token exists
     bool copy_ok;           // lane's piece belongs to a page that holds tokens of the sequence
 };
 
 // Extend the ring to kAhead rows beyond the fastest lane (call with all earlier copies landed
 // and the warp converged); returns whether this lane may read the ring during the next tile.
+// A tile consumes at most 16 bytes, so at most 5 rows (40 pieces, two per lane) are due.
 template <int ROWS>
-__device__ __forceinline__ bool ring_advance(Chain& c, uint32_t ring, const uint8_t* cont, int rec_words, int lane) {
+__device__ __forceinline__ bool ring_advance(Chain& c, uint32_t ring_piece, const uint8_t* cont, int rec_words, int lane) {
     const uint32_t wi = c.ptr >> 2;
     const uint32_t wmax = __reduce_max_sync(kFullMask, c.active ? wi : 0u);
-    const uint32_t Enew = min(wmax + (uint32_t)kAhead, (uint32_t)rec_words);
-    if (Enew > c.E) {   // warp-uniform; at most 5 rows = 40 pieces
-        uint32_t row = c.E + (uint32_t)(lane >> 3);
-        if (row < Enew && c.copy_ok)
-            cp_async16(ring + ((row & (ROWS - 1)) << 7) + ((lane & 7) << 4), cont + (size_t)(c.src16 + row * 4u) * 16);
-        row += 4;
-        if (row < Enew && c.copy_ok)
-            cp_async16(ring + ((row & (ROWS - 1)) << 7) + ((lane & 7) << 4), cont + (size_t)(c.src16 + row * 4u) * 16);
-        c.E = Enew;
-    }
-    return !c.active || (wi + ROWS >= c.E);
+    const uint32_t Enew = max(c.E, min(wmax + (uint32_t)kAhead, (uint32_t)rec_words));
+    uint32_t row = c.E + (uint32_t)(lane >> 3);
+    if (row < Enew && c.copy_ok)
+        cp_async16(ring_piece + ((row & (ROWS - 1)) << 7), cont + (size_t)(c.src16 + row * 4u) * 16);
+    row += 4;
+    if (row < Enew && c.copy_ok)
+        cp_async16(ring_piece + ((row & (ROWS - 1)) << 7), cont + (size_t)(c.src16 + row * 4u) * 16);
+    c.E = Enew;
+    return !c.active || (wi + ROWS >= Enew);
+}
+
+// Word 0 of this lane's own record (global): the container block of its page starts at 64 times
+// the src16 / 4 of the lane whose piece lies in that page (lane 0 or 4).
+__device__ __forceinline__ const uint32_t* own_column(const Chain& c, const uint8_t* cont, int lane) {
+    const uint32_t blk64 = __shfl_sync(kFullMask, c.src16, (lane >> 4) * 4) >> 2;
+    return reinterpret_cast<const uint32_t*>(cont + (size_t)blk64 * 64) + (lane & 15);
 }
 
 // One step: 128 channels (one head), 16 at a time; K streams of the current step's head and V
@@ -147,17 +183,35 @@ __device__ __forceinline__ void wide_pass(Chain& ck, Chain& cv, uint32_t ringk, 
     const uint32_t st_lo = lane * 32 + (((lane >> 2) & 1) << 4), st_hi = lane * 32 + ((((lane >> 2) & 1) ^ 1) << 4);
     const uint32_t o_addr = obuf + ((2 * (lane & 3)) * kORow + (lane >> 2)) * 4;
     const uint32_t ringk_lane = ringk + lane * 4, ringv_lane = ringv + lane * 4;
+    const uint32_t ringk_piece = ringk + ((lane & 7) << 4), ringv_piece = ringv + ((lane & 7) << 4);
 #pragma unroll 1
     for (int cg = 0; cg < 8; ++cg) {
         cp_async_wait<0>();
         __syncwarp();
         bool fk = true, fv = true;
-        if (DO_K) fk = ring_advance<kRowsK>(ck, ringk, k_cont, rwk, lane);
-        if (DO_V) fv = ring_advance<kRowsV>(cv, ringv, v_cont, rwv, lane);
+        if (DO_K) fk = ring_advance<kRowsK>(ck, ringk_piece, k_cont, rwk, lane);
+        if (DO_V) fv = ring_advance<kRowsV>(cv, ringv_piece, v_cont, rwv, lane);
         cp_async_commit();
         uint32_t pk[8], pv[8];
-        if (DO_K) decode16_ring<kRowsK>(ck.x, ck.ptr, ringk_lane, lutk, one, pk, fk, ck.gcol, rwk);
-        if (DO_V) decode16_ring<kRowsV>(cv.x, cv.ptr, ringv_lane, lutv, one, pv, fv, cv.gcol, rwv);
+        if (__all_sync(kFullMask, fk && fv)) {
+            if (DO_K) decode16_ring<kRowsK>(ck.x, ck.ptr, ringk_lane, lutk, one, pk);
+            if (DO_V) decode16_ring<kRowsV>(cv.x, cv.ptr, ringv_lane, lutv, one, pv);
+        } else {   // some lane lags behind its ring: that lane reads global memory (rare, out of line)
+            if (DO_K) {
+                const Decoded16 r = decode16_mixed(ck.x, ck.ptr, ringk_lane, (uint32_t)(kRowsK - 1) << 7, lutk, fk,
+                                                   own_column(ck, k_cont, lane), rwk);
+#pragma unroll
+                for (int i = 0; i < 8; ++i) pk[i] = r.packed[i];
+                ck.x = r.x; ck.ptr = r.ptr;
+            }
+            if (DO_V) {
+                const Decoded16 r = decode16_mixed(cv.x, cv.ptr, ringv_lane, (uint32_t)(kRowsV - 1) << 7, lutv, fv,
+                                                   own_column(cv, v_cont, lane), rwv);
+#pragma unroll
+                for (int i = 0; i < 8; ++i) pv[i] = r.packed[i];
+                cv.x = r.x; cv.ptr = r.ptr;
+            }
+        }
         if (DO_K) { sts128(ktile + st_lo, pk); sts128(ktile + st_hi, pk + 4); }
         if (DO_V) { sts128(vtile + st_lo, pv); sts128(vtile + st_hi, pv + 4); }
         __syncwarp();
@@ -188,7 +242,7 @@ __device__ __forceinline__ void wide_pass(Chain& ck, Chain& cv, uint32_t ringk, 
     }
 }
 
-__global__ void __launch_bounds__(kMaxWarps * 32, 1)
+__global__ void __launch_bounds__(kWideWarps * 32, 1)
 dq_attention_wide_kernel(const __grid_constant__ DqDevTable TK, const __grid_constant__ DqDevTable TV,
                          const AttnParams p) {
     extern __shared__ __align__(128) uint8_t smem[];
@@ -245,12 +299,12 @@ dq_attention_wide_kernel(const __grid_constant__ DqDevTable TK, const __grid_con
         }
         return it;
     };
-    int* my_pages = reinterpret_cast<int*>(smem + L.off_pages) + warp * 6;
-    long long* s_prev_row = reinterpret_cast<long long*>(smem + L.off_pages + kMaxWarps * 24);
+    int* my_pages = reinterpret_cast<int*>(smem + L.off_pages) + warp * 8;
+    long long* s_prev_row = reinterpret_cast<long long*>(smem + L.off_pages + kMaxWarps * 32);
     auto fetch_pages = [&](int n, const Item& it) {
         const int tok0 = (it.blk * nw + warp) * kChunk;
         if (it.valid && tok0 < it.len && lane < 2 && tok0 + 16 * lane < it.len)
-            cp_async4(smem_addr(my_pages + (n % 3) * 2 + lane),
+            cp_async4(smem_addr(my_pages + (n & 3) * 2 + lane),
                       p.page_table + (size_t)it.b * p.max_pages + (tok0 >> 4) + lane);
     };
     // q' operand, sum of q' and q'.mean of this warp's window for (item, head): what a step's
@@ -268,7 +322,7 @@ dq_attention_wide_kernel(const __grid_constant__ DqDevTable TK, const __grid_con
             cp_async4(my_qmu + ((s & 1) * DQ_MAX_GROUP + lane) * 4,
                       p.qmu + ((size_t)it.b * p.Hq + (size_t)h * G + lane) * p.windows + tok0 / DQ_WINDOW_TOKENS);
     };
-    // Start the streams of item `it` (ring slot n % 3 of the page ids) for one tensor kind:
+    // Start the streams of item `it` (slot n mod 4 of the page ids) for one tensor kind:
     // per-lane sources and the first rows of the ring.  The caller has made sure nobody still
     // reads the ring.
     auto start_chain = [&](Chain& c, int n, const Item& it, const uint8_t* cont, int rec_words, uint32_t ring, int rows) {
@@ -277,14 +331,9 @@ dq_attention_wide_kernel(const __grid_constant__ DqDevTable TK, const __grid_con
         const int pslot = (lane >> 2) & 1;     // page of this lane's 16-byte piece (tokens 4 (lane & 7) ..)
         c.copy_ok = it.valid && tok0 + 16 * pslot < it.len;
         c.src16 = 0u;
-        c.gcol = reinterpret_cast<const uint32_t*>(cont);
         if (c.copy_ok) {
-            const unsigned pg = (unsigned)my_pages[(n % 3) * 2 + pslot];
+            const unsigned pg = (unsigned)my_pages[(n & 3) * 2 + pslot];
             c.src16 = (pg * (unsigned)groups + (unsigned)it.grp) * (unsigned)rec_words * 4u + (unsigned)(lane & 3);
-        }
-        if (c.active) {
-            const size_t pg = (size_t)my_pages[(n % 3) * 2 + (lane >> 4)];
-            c.gcol = reinterpret_cast<const uint32_t*>(cont + (pg * groups + it.grp) * ((size_t)rec_words * 64)) + (lane & 15);
         }
         const int fill = min(kFillRows, rec_words);
         if (c.copy_ok)
@@ -298,7 +347,7 @@ dq_attention_wide_kernel(const __grid_constant__ DqDevTable TK, const __grid_con
 
     Chain ck, cv;
     ck.x = cv.x = 1u << 23; ck.ptr = cv.ptr = 8u; ck.E = cv.E = 0u; ck.src16 = cv.src16 = 0u;
-    ck.gcol = cv.gcol = nullptr; ck.active = cv.active = false; ck.copy_ok = cv.copy_ok = false;
+    ck.active = cv.active = false; ck.copy_ok = cv.copy_ok = false;
 
     // prologue: page ids of items 0 and 1, K ring and step loads of (item 0, head 0)
     int hint = 0;
@@ -318,8 +367,8 @@ dq_attention_wide_kernel(const __grid_constant__ DqDevTable TK, const __grid_con
     int nK = 0, kK = 0;                // K chain: item index of this CTA, head within the group
     bool have_prev = false;            // a V step is pending (the previous step had a K step)
     int kV = 0;                        // head of the pending V step
-    Item vit = cur;                    // item of the pending V step
-    vit.valid = 0;
+    bool wv = false;                   // this warp holds tokens of the pending V step's item
+    int nwv = 0;                       // warps that hold tokens of that item
     uint32_t hk = 0u, hv = 0u, xv_next = 1u << 23;   // headers (s, o as fp16 pairs) of the K item's tokens; V start state
     uint32_t pb_hi[2][2] = {{0u, 0u}, {0u, 0u}}, pb_lo[2][2] = {{0u, 0u}, {0u, 0u}};
 
@@ -339,7 +388,7 @@ dq_attention_wide_kernel(const __grid_constant__ DqDevTable TK, const __grid_con
         cp_async_commit();
 
         // streams that start with this step
-        if (have_prev && kV == 0) {          // V streams of `vit` (their first rows were fetched after the last pass)
+        if (have_prev && kV == 0) {          // V streams of the pending item (their first rows were fetched after the last pass)
             cv.x = xv_next;
         }
         const int tok0 = (cur.blk * nw + warp) * kChunk;
@@ -347,7 +396,7 @@ dq_attention_wide_kernel(const __grid_constant__ DqDevTable TK, const __grid_con
             hk = lds32(ringk + lane * 4);
             ck.x = lds32(ringk + 128 + lane * 4);
             if (ck.active) {                  // V header of the same tokens: needed for this item's weights
-                const size_t pg = (size_t)my_pages[(nK % 3) * 2 + (lane >> 4)];
+                const size_t pg = (size_t)my_pages[(nK & 3) * 2 + (lane >> 4)];
                 const uint32_t* vcol = reinterpret_cast<const uint32_t*>(p.v_cont + (pg * groups + cur.grp) * ((size_t)rwv * 64)) + (lane & 15);
                 hv = __ldg(vcol);
                 xv_next = __ldg(vcol + 16);
@@ -358,13 +407,16 @@ dq_attention_wide_kernel(const __grid_constant__ DqDevTable TK, const __grid_con
         float sacc[4][4];
 #pragma unroll
         for (int i = 0; i < 4; ++i) { sacc[i][0] = sacc[i][1] = sacc[i][2] = sacc[i][3] = 0.f; }
-        if (cur.valid && have_prev)
+        // a warp whose 32 tokens lie beyond the sequence end skips the decode (its logits are masked,
+        // its output slot is left out of the merge)
+        const bool wk = cur.valid && tok0 < cur.len;
+        if (wk && wv)
             wide_pass<true, true>(ck, cv, ringk, ringv, p.k_cont, p.v_cont, rwk, rwv, my_lutk, my_lutv, one, ktile, vtile, q16,
                                   my_obuf, lane, G, sacc, pb_hi, pb_lo);
-        else if (cur.valid)
+        else if (wk)
             wide_pass<true, false>(ck, cv, ringk, ringv, p.k_cont, p.v_cont, rwk, rwv, my_lutk, my_lutv, one, ktile, vtile, q16,
                                    my_obuf, lane, G, sacc, pb_hi, pb_lo);
-        else
+        else if (wv)
             wide_pass<false, true>(ck, cv, ringk, ringv, p.k_cont, p.v_cont, rwk, rwv, my_lutk, my_lutv, one, ktile, vtile, q16,
                                    my_obuf, lane, G, sacc, pb_hi, pb_lo);
 
@@ -422,7 +474,7 @@ dq_attention_wide_kernel(const __grid_constant__ DqDevTable TK, const __grid_con
                 const int g = e / 130, col = e - g * 130;
                 const int src = col < kN ? col : lcol + (col - kN);
                 float sum = 0.f;
-                for (int w = 0; w < nw; ++w) sum += obuf_all[(w * G + g) * kORow + src];
+                for (int w = 0; w < nwv; ++w) sum += obuf_all[(w * G + g) * kORow + src];
                 float* dst = p.partial + ((size_t)s_prev_row[(s + 1) & 1] + g) * kPartial;
                 if (col < kN) dst[col] = sum;
                 else dst[col + 1] = sum;
@@ -433,7 +485,8 @@ dq_attention_wide_kernel(const __grid_constant__ DqDevTable TK, const __grid_con
         // ------------------------------------------ softmax weights of this step, scaled by the step maximum
         have_prev = cur.valid;
         kV = kK;
-        vit = cur;
+        wv = wk;
+        nwv = min(nw, (cur.len - cur.blk * nw * kChunk + kChunk - 1) / kChunk);
         if (cur.valid) {
             float m_item = -INFINITY;
             for (int w = 0; w < nw; ++w) m_item = fmaxf(m_item, red_m[w * DQ_MAX_GROUP + g_row]);
@@ -473,14 +526,14 @@ dq_attention_wide_kernel(const __grid_constant__ DqDevTable TK, const __grid_con
         }
     }
     cp_async_wait<0>();
-    (void)hint; (void)vit;
+    (void)hint;
 }
 
 }  // namespace
 
 int dq_attn_wide_pick_warps(const DqDevTable& tk, const DqDevTable& tv, int B, int G, int smem_max) {
     (void)tk; (void)tv;
-    for (int nw = kMaxWarps; nw >= 4; --nw)
+    for (int nw = kWideWarps; nw >= 4; --nw)
         if (make_wlayout(nw, B, G).total <= smem_max) return nw;
     return 0;
 }
