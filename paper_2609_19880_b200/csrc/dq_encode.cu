@@ -343,6 +343,45 @@ dq_encode_kernel(const __grid_constant__ DqDevTable TK, const __grid_constant__ 
 }
 
 
+// rANS encode of one stream by one warp (Eq. rans Enc on symbols n-1 .. 0 so that decoding runs
+// forward).  Every lane carries the same state; lane 0 records the emitted bytes (in emission
+// order) at `bytes_addr` in shared memory.  The per-symbol table entries do not depend on the
+// state, so they are fetched four symbols ahead of the serial state chain.
+//   ent[m] = {rcp, bias | (256 - f) << 10 | rsh << 19}
+__device__ __forceinline__ void rans_encode_warp(const uint2* ent, const uint8_t* sym, int n, uint32_t bytes_addr,
+                                                 int cap, int lane, uint32_t& xs_out, int& k_out) {
+    uint32_t xs = kL;
+    int k = 0;
+    const uint32_t* sym4 = reinterpret_cast<const uint32_t*>(sym);
+    uint2 cur[4], nxt[4];
+    {
+        const uint32_t m4 = sym4[n / 4 - 1];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) nxt[i] = ent[(m4 >> (8 * i)) & 255u];
+    }
+#pragma unroll 1
+    for (int j4 = n / 4 - 1; j4 >= 0; --j4) {
+#pragma unroll
+        for (int i = 0; i < 4; ++i) cur[i] = nxt[i];
+        if (j4 > 0) {
+            const uint32_t m4 = sym4[j4 - 1];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) nxt[i] = ent[(m4 >> (8 * i)) & 255u];
+        }
+#pragma unroll
+        for (int i = 3; i >= 0; --i) {
+            const uint32_t aux = cur[i].y, cmpl = (aux >> 10) & 511u;
+            const bool emit = xs >= ((256u - cmpl) << 23);   // at most once: xs < 2^31 <= 2^8 * (f << 23)
+            if (emit && lane == 0 && k < cap) asm volatile("st.shared.u8 [%0], %1;" ::"r"(bytes_addr + k), "r"(xs & 0xffu));
+            k += emit ? 1 : 0;
+            xs = emit ? (xs >> 8) : xs;
+            xs = (__umulhi(xs, cur[i].x) >> (aux >> 19)) * cmpl + (xs + (aux & 1023u));
+        }
+    }
+    xs_out = xs;
+    k_out = k;
+}
+
 // ------------------------------------------------------- token-wide streams (hs heads)
 
 // Cross-warp pieces of a stream that spans hs heads: one CTA per stream, warp w holds head w
@@ -353,6 +392,7 @@ struct WideShared {
     uint32_t len[2][DQ_MAX_STREAM_HEADS];
     double sa[DQ_MAX_STREAM_HEADS], sb[DQ_MAX_STREAM_HEADS];
     int sm[DQ_MAX_STREAM_HEADS], smm[DQ_MAX_STREAM_HEADS];
+    uint2 ent[DQ_MAX_LEVELS];   // rANS encode entries {rcp, bias | (256 - f) << 10 | rsh << 19}
 };
 
 // Function Drift of Algorithm 1 for a stream held by hs warps; same arithmetic as drift_m, with
@@ -446,46 +486,37 @@ __device__ __forceinline__ uint32_t drift_wide(const EncTable& T, WideShared& W,
     return len;
 }
 
-// One CTA of hs warps per stream (token, group of hs KV heads); warp w owns head group * hs + w,
-// lane l its elements 4l .. 4l+3 (stream positions 128 w + 4 l + e).  blockIdx.y selects the
-// tensor kind.  The record goes to the word-interleaved page layout.
-__global__ void __launch_bounds__(DQ_MAX_STREAM_HEADS * 32)
-dq_encode_wide_kernel(const __grid_constant__ DqDevTable TK, const __grid_constant__ DqDevTable TV,
-                      const DqEncodeArgs a) {
-    __shared__ EncTable T;
-    __shared__ WideShared W;
-    __shared__ uint8_t s_bytes[DQ_MAX_WIDE_REC_BYTES];
-    __shared__ __align__(4) uint8_t s_sym[DQ_MAX_STREAM_HEADS * kN];
-    __shared__ uint32_t s_final[2];   // final state, bytes emitted
-    dqdev::pdl_launch_dependents();
-    const bool is_v = a.do_k ? (blockIdx.y == 1) : true;
+// Table fields of one tensor kind into shared memory (first 16 threads + thread 0).
+__device__ __forceinline__ void load_wide_table(EncTable& T, WideShared& W, const DqDevTable& TK, const DqDevTable& TV,
+                                                bool is_v) {
     if (threadIdx.x < DQ_MAX_LEVELS) {
         const int i = threadIdx.x;
         T.r[i] = is_v ? TV.r[i] : TK.r[i];
         T.R[i] = is_v ? TV.R[i] : TK.R[i];
-        T.rcp[i] = is_v ? TV.enc_rcp[i] : TK.enc_rcp[i];
-        const uint32_t aux = is_v ? TV.enc_aux[i] : TK.enc_aux[i];
-        T.bias[i] = aux & 1023u;
-        T.cmpl[i] = (aux >> 10) & 511u;
-        T.rsh[i] = aux >> 19;
-        T.thr[i] = (256u - ((aux >> 10) & 511u)) << 23;
+        W.ent[i] = make_uint2(is_v ? TV.enc_rcp[i] : TK.enc_rcp[i], is_v ? TV.enc_aux[i] : TK.enc_aux[i]);
     }
     if (threadIdx.x == 0) {
         T.M = is_v ? TV.M : TK.M; T.rec = is_v ? TV.rec : TK.rec; T.mstar = is_v ? TV.mstar : TK.mstar;
         T.budget_bits = is_v ? TV.budget_bits : TK.budget_bits;
         T.has_mean = is_v ? TV.has_mean : TK.has_mean; T.rotate = is_v ? TV.rotate : TK.rotate;
     }
-    __syncthreads();
-    dqdev::pdl_wait_prior_grid();
-    const int lane = threadIdx.x & 31, wib = threadIdx.x >> 5;
-    const int hs = blockDim.x >> 5, Hkv = a.Hkv, groups = Hkv / hs;
-    const int n = hs * kN;
-    const int t = (int)(blockIdx.x / groups), grp = (int)(blockIdx.x % groups), h = grp * hs + wib;
-    const uint16_t* x = static_cast<const uint16_t*>(is_v ? a.v_bf16 : a.k_bf16);
-    uint8_t* cont = is_v ? a.v_cont : a.k_cont;
-    const int rec_words = (T.rec + 3) >> 2;
-    uint32_t parity = 0;
+}
 
+struct WideQuantised {
+    uint32_t hdr0;      // s fp16 | o fp16 << 16
+    uint32_t flags;     // 1: all-central fallback, 2: constant stream, 4: refit rejected
+};
+
+// Steps 1-6 of Algorithm 1 for the stream (token t, group grp) held by the CTA's hs warps
+// (warp w owns head grp * hs + w, lane l its elements 4l .. 4l+3 = stream positions
+// 128 w + 4 l + e): rotation, mean removal, min-max grid, drift, refit, fp16 metadata, second
+// drift.  The final symbols go to s_sym (visible to the whole CTA on return).
+__device__ __forceinline__ WideQuantised wide_quantise(const EncTable& T, WideShared& W, const DqEncodeArgs& a,
+                                                       bool is_v, int t, int grp, uint8_t* s_sym, uint32_t& parity) {
+    const int lane = threadIdx.x & 31, wib = threadIdx.x >> 5;
+    const int hs = blockDim.x >> 5, Hkv = a.Hkv, h = grp * hs + wib;
+    const int n = hs * kN;
+    const uint16_t* x = static_cast<const uint16_t*>(is_v ? a.v_bf16 : a.k_bf16);
     float z[4];
     {
         const uint2 raw = *reinterpret_cast<const uint2*>(x + ((size_t)t * Hkv + h) * kN + 4 * lane);
@@ -532,7 +563,7 @@ dq_encode_wide_kernel(const __grid_constant__ DqDevTable TK, const __grid_consta
     uint32_t sym[4];
     __half s16 = __ushort_as_half(0), o16 = __ushort_as_half(0);
     bool degenerate = !(mx > mn);
-    uint32_t st_fallback = 0, st_refit = 0;
+    uint32_t flags = 0;
     if (!degenerate) {   // uniform across the CTA: mx and mn are stream-wide
         const float o = mn;                                         // FitMinMax, Eq. (affine_token)
         const float s = __fdiv_rn(__fsub_rn(mx, mn), (float)(T.M - 1));
@@ -554,6 +585,7 @@ dq_encode_wide_kernel(const __grid_constant__ DqDevTable TK, const __grid_consta
         }
         sm = __reduce_add_sync(kFull, sm);
         smm = __reduce_add_sync(kFull, smm);
+        __syncthreads();   // the previous stream's readers of W.sa .. are done
         if (lane == 0) { W.sa[wib] = sa; W.sb[wib] = sb; W.sm[wib] = sm; W.smm[wib] = smm; }
         __syncthreads();
         sa = W.sa[0]; sb = W.sb[0];
@@ -576,7 +608,7 @@ dq_encode_wide_kernel(const __grid_constant__ DqDevTable TK, const __grid_consta
             s16 = __float2half_rn(s);
             o16 = __float2half_rn(o);
             sf = __half2float(s16); of = __half2float(o16);
-            st_refit = 1;
+            flags |= 4u;
         }
         if (!(sf > 0.0f)) degenerate = true;
         else {
@@ -584,7 +616,7 @@ dq_encode_wide_kernel(const __grid_constant__ DqDevTable TK, const __grid_consta
             if (len > ((uint32_t)T.budget_bits << 16)) {
 #pragma unroll
                 for (int e = 0; e < 4; ++e) sym[e] = (uint32_t)T.mstar;
-                st_fallback = 1;
+                flags |= 1u;
             }
         }
     }
@@ -593,52 +625,115 @@ dq_encode_wide_kernel(const __grid_constant__ DqDevTable TK, const __grid_consta
         o16 = __float2half_rn(mn);
 #pragma unroll
         for (int e = 0; e < 4; ++e) sym[e] = (uint32_t)T.mstar;
+        flags |= 2u;
     }
-
-    // rANS by warp 0 over the whole stream, symbols n-1 .. 0 (Eq. rans Enc); every lane carries the
-    // same state, lane 0 records the bytes.
     *reinterpret_cast<uint32_t*>(&s_sym[wib * kN + 4 * lane]) = sym[0] | (sym[1] << 8) | (sym[2] << 16) | (sym[3] << 24);
     __syncthreads();
-    if (wib == 0) {
-        uint32_t xs = kL;
-        int k = 0;
-        const uint32_t bytes_addr = dqdev::smem_addr(s_bytes);
-#pragma unroll 8
-        for (int j = n - 1; j >= 0; --j) {
-            const uint32_t m = s_sym[j];
-            const uint32_t rcp = T.rcp[m], rsh = T.rsh[m], bias = T.bias[m], cmpl = T.cmpl[m], thr = T.thr[m];
-            if (xs >= thr) {
-                // the budget test keeps k < rec - 8; the bound only guards shared memory
-                if (lane == 0 && k < DQ_MAX_WIDE_REC_BYTES) asm volatile("st.shared.u8 [%0], %1;" ::"r"(bytes_addr + k), "r"(xs & 0xffu));
-                ++k;
-                xs >>= 8;
-            }
-            xs = (__umulhi(xs, rcp) >> rsh) * cmpl + (xs + bias);
-        }
-        if (lane == 0) { s_final[0] = xs; s_final[1] = (uint32_t)k; }
-    }
-    __syncthreads();
-    asm volatile("" ::: "memory");
-    const uint32_t xs = s_final[0];
-    const int k = (int)s_final[1];
-    const uint32_t hdr0 = (uint32_t)__half_as_ushort(s16) | ((uint32_t)__half_as_ushort(o16) << 16);
-    const int sl = a.slot[t];
-    uint8_t* blk = cont + ((size_t)(sl / DQ_PAGE_TOKENS) * groups + grp) * ((size_t)rec_words * 64) +
-                   (size_t)(sl % DQ_PAGE_TOKENS) * 4;
-    const int used = min(8 + k, T.rec);
+    WideQuantised r;
+    r.hdr0 = (uint32_t)__half_as_ushort(s16) | ((uint32_t)__half_as_ushort(o16) << 16);
+    r.flags = flags;
+    return r;
+}
+
+// Record of one stream into the word-interleaved page layout (all threads of the CTA).
+__device__ __forceinline__ void write_wide_record(uint8_t* cont, int groups, int grp, int rec, int slot, uint32_t hdr0,
+                                                  uint32_t xs, int k, const uint8_t* bytes) {
+    const int rec_words = (rec + 3) >> 2;
+    uint8_t* blk = cont + ((size_t)(slot / DQ_PAGE_TOKENS) * groups + grp) * ((size_t)rec_words * 64) +
+                   (size_t)(slot % DQ_PAGE_TOKENS) * 4;
+    const int used = min(8 + k, rec);   // the budget test keeps 8 + k <= rec
     for (int i = threadIdx.x; i < rec_words * 4; i += blockDim.x) {
         uint8_t v = 0;
         if (i < 4) v = (uint8_t)(hdr0 >> (8 * i));
         else if (i < 8) v = (uint8_t)(xs >> (8 * (i - 4)));
-        else if (i < used) v = s_bytes[k - 1 - (i - 8)];
+        else if (i < used) v = bytes[k - 1 - (i - 8)];   // emitted last = read first
         blk[(size_t)(i >> 2) * 64 + (i & 3)] = v;
     }
-    if (a.status && threadIdx.x == 0) {
-        if (st_fallback) atomicAdd(a.status + 0, 1u);
-        if (degenerate) atomicAdd(a.status + 1, 1u);
-        if (st_refit) atomicAdd(a.status + 2, 1u);
-        atomicMax(a.status + 3, (uint32_t)(8 + k));
+}
+
+__device__ __forceinline__ void add_status(uint32_t* status, uint32_t flags, int k) {
+    if (!status) return;
+    if (flags & 1u) atomicAdd(status + 0, 1u);
+    if (flags & 2u) atomicAdd(status + 1, 1u);
+    if (flags & 4u) atomicAdd(status + 2, 1u);
+    atomicMax(status + 3, (uint32_t)(8 + k));
+}
+
+// One CTA of hs warps per stream (token, group of hs KV heads): lowest latency, used when a
+// call holds few streams (a decode step).  blockIdx.y selects the tensor kind.
+__global__ void __launch_bounds__(DQ_MAX_STREAM_HEADS * 32)
+dq_encode_wide_kernel(const __grid_constant__ DqDevTable TK, const __grid_constant__ DqDevTable TV,
+                      const DqEncodeArgs a) {
+    __shared__ EncTable T;
+    __shared__ __align__(16) WideShared W;
+    __shared__ uint8_t s_bytes[DQ_MAX_WIDE_REC_BYTES];
+    __shared__ __align__(4) uint8_t s_sym[DQ_MAX_STREAM_HEADS * kN];
+    __shared__ uint32_t s_final[2];   // final state, bytes emitted
+    dqdev::pdl_launch_dependents();
+    const bool is_v = a.do_k ? (blockIdx.y == 1) : true;
+    load_wide_table(T, W, TK, TV, is_v);
+    __syncthreads();
+    dqdev::pdl_wait_prior_grid();
+    const int lane = threadIdx.x & 31, wib = threadIdx.x >> 5;
+    const int hs = blockDim.x >> 5, groups = a.Hkv / hs;
+    const int t = (int)(blockIdx.x / groups), grp = (int)(blockIdx.x % groups);
+    uint32_t parity = 0;
+    const WideQuantised q = wide_quantise(T, W, a, is_v, t, grp, s_sym, parity);
+    if (wib == 0) {
+        uint32_t xs;
+        int k;
+        rans_encode_warp(W.ent, s_sym, hs * kN, dqdev::smem_addr(s_bytes), DQ_MAX_WIDE_REC_BYTES, lane, xs, k);
+        if (lane == 0) { s_final[0] = xs; s_final[1] = (uint32_t)k; }
     }
+    __syncthreads();
+    asm volatile("" ::: "memory");
+    write_wide_record(is_v ? a.v_cont : a.k_cont, groups, grp, T.rec, a.slot[t], q.hdr0, s_final[0], (int)s_final[1], s_bytes);
+    if (threadIdx.x == 0) add_status(a.status, q.flags, (int)s_final[1]);
+}
+
+// Throughput variant for calls with many streams (prefill, a window's bulk encode): a CTA takes
+// kBatch consecutive streams; its hs warps quantise them one after the other, then every warp
+// entropy-codes whole streams on its own, so the serial rANS chains of kBatch streams run side
+// by side instead of leaving hs - 1 warps idle.
+constexpr int kBatch = 8;
+__global__ void __launch_bounds__(DQ_MAX_STREAM_HEADS * 32, 2)
+dq_encode_wide_batch_kernel(const __grid_constant__ DqDevTable TK, const __grid_constant__ DqDevTable TV,
+                            const DqEncodeArgs a) {
+    __shared__ EncTable T;
+    __shared__ __align__(16) WideShared W;
+    __shared__ uint8_t s_bytes[kBatch][DQ_MAX_WIDE_REC_BYTES];
+    __shared__ __align__(4) uint8_t s_sym[kBatch][DQ_MAX_STREAM_HEADS * kN];
+    __shared__ uint32_t s_hdr[kBatch], s_flags[kBatch], s_xs[kBatch], s_k[kBatch];
+    dqdev::pdl_launch_dependents();
+    const bool is_v = a.do_k ? (blockIdx.y == 1) : true;
+    load_wide_table(T, W, TK, TV, is_v);
+    __syncthreads();
+    dqdev::pdl_wait_prior_grid();
+    const int lane = threadIdx.x & 31, wib = threadIdx.x >> 5;
+    const int hs = blockDim.x >> 5, groups = a.Hkv / hs;
+    const long long total = (long long)a.T * groups;
+    const long long first = (long long)blockIdx.x * kBatch;
+    const int ns = (int)min((long long)kBatch, total - first);
+    uint32_t parity = 0;
+    for (int i = 0; i < ns; ++i) {
+        const long long sid = first + i;
+        const WideQuantised q = wide_quantise(T, W, a, is_v, (int)(sid / groups), (int)(sid % groups), s_sym[i], parity);
+        if (threadIdx.x == 0) { s_hdr[i] = q.hdr0; s_flags[i] = q.flags; }
+    }
+    for (int i = wib; i < ns; i += hs) {
+        uint32_t xs;
+        int k;
+        rans_encode_warp(W.ent, s_sym[i], hs * kN, dqdev::smem_addr(s_bytes[i]), DQ_MAX_WIDE_REC_BYTES, lane, xs, k);
+        if (lane == 0) { s_xs[i] = xs; s_k[i] = (uint32_t)k; }
+    }
+    __syncthreads();
+    asm volatile("" ::: "memory");
+    for (int i = 0; i < ns; ++i) {
+        const long long sid = first + i;
+        write_wide_record(is_v ? a.v_cont : a.k_cont, groups, (int)(sid % groups), T.rec, a.slot[(int)(sid / groups)], s_hdr[i],
+                          s_xs[i], (int)s_k[i], s_bytes[i]);
+    }
+    if (threadIdx.x < ns) add_status(a.status, s_flags[threadIdx.x], (int)s_k[threadIdx.x]);
 }
 
 }  // namespace
@@ -658,9 +753,14 @@ cudaError_t dq_launch_means(const DqDevTable& tk, const void* k_bf16, int T, int
 cudaError_t dq_launch_encode(const DqDevTable& tk, const DqDevTable& tv, const DqEncodeArgs& a, cudaStream_t st) {
     const long long warps = (long long)a.T * a.Hkv;
     if (warps == 0 || (!a.do_k && !a.do_v)) return cudaSuccess;
-    if (tk.hs > 1)   // token-wide streams: one CTA of hs warps per stream
-        return dq_launch_pdl(dq_encode_wide_kernel, dim3((unsigned)(warps / tk.hs), (a.do_k && a.do_v) ? 2 : 1),
+    if (tk.hs > 1) {   // token-wide streams: CTAs of hs warps; few streams: one per CTA, many: kBatch per CTA
+        const long long streams = warps / tk.hs;
+        const dim3 kinds_y(1, (a.do_k && a.do_v) ? 2 : 1);
+        if (streams < 4LL * 148 * kBatch)
+            return dq_launch_pdl(dq_encode_wide_kernel, dim3((unsigned)streams, kinds_y.y), dim3(tk.hs * 32), 0, st, tk, tv, a);
+        return dq_launch_pdl(dq_encode_wide_batch_kernel, dim3((unsigned)((streams + kBatch - 1) / kBatch), kinds_y.y),
                              dim3(tk.hs * 32), 0, st, tk, tv, a);
+    }
     const unsigned blocks = (unsigned)((warps + kEncWarps - 1) / kEncWarps);
     return dq_launch_pdl(dq_encode_kernel, dim3(blocks, (a.do_k && a.do_v) ? 2 : 1), dim3(kEncWarps * 32), 0, st, tk, tv, a);
 }
