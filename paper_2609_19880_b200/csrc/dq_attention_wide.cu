@@ -35,32 +35,24 @@ struct Item {
     int b, grp, blk, len, bg, valid;
 };
 
-struct WLayout {
-    int off_lutk, off_lutv, off_ringk, off_ringv, off_tiles, off_obuf, off_q16, off_prefix, off_qsum, off_red,
-        off_pages, off_qmu, total;
-    int warp_obuf_bytes;
-};
+// Shared-memory layout.  Everything the decode loop touches sits at a compile-time offset from
+// the CTA's base or from the warp's own region, so the addresses cost no registers.
+constexpr int kOffLutK = 0, kOffLutV = kOffLutK + 256 * 32 * 4;
+constexpr int kOffQ16 = kOffLutV + 256 * 32 * 4;                       // [2] fp16 q' operand
+constexpr int kOffQsum = kOffQ16 + 2 * kQ16Bytes;                      // [2][8] sum of q'
+constexpr int kOffRed = kOffQsum + 2 * DQ_MAX_GROUP * 4;               // [warp][head] maxima, [2][head] step maxima
+constexpr int kOffPages = kOffRed + (kMaxWarps + 2) * DQ_MAX_GROUP * 4;   // per warp: page ids of 4 items in flight
+constexpr int kOffPrevRow = kOffPages + kMaxWarps * 4 * 2 * 4;         // [2] partial row of the pending V step
+constexpr int kOffWarp = (kOffPrevRow + 16 + 127) & ~127;              // per-warp regions
+constexpr int kWRingK = 0, kWRingV = kWRingK + kRingK, kWTileK = kWRingV + kRingV, kWTileV = kWTileK + kTile;
+constexpr int kWQmu = kWTileV + kTile;                                 // [2][8] q'.mean of the warp's window
+constexpr int kWObuf = kWQmu + 2 * DQ_MAX_GROUP * 4;                   // [G][kORow] output slot
 
+__host__ __device__ inline int warp_stride(int G) { return kWObuf + G * kORow * 4; }
 __host__ __device__ inline int align16w(int x) { return (x + 15) & ~15; }
-
-__host__ __device__ inline WLayout make_wlayout(int nw, int B, int G) {
-    WLayout L;
-    L.warp_obuf_bytes = G * kORow * 4;
-    int o = 0;
-    L.off_lutk = o; o += 256 * 32 * 4;
-    L.off_lutv = o; o += 256 * 32 * 4;
-    L.off_ringk = o; o += nw * kRingK;
-    L.off_ringv = o; o += nw * kRingV;
-    L.off_tiles = o; o += nw * 2 * kTile;
-    L.off_obuf = o; o += nw * L.warp_obuf_bytes;
-    L.off_q16 = o; o += 2 * kQ16Bytes;
-    L.off_prefix = o; o += align16w((2 * B + 1) * 4);
-    L.off_qsum = o; o += 2 * DQ_MAX_GROUP * 4;
-    L.off_red = o; o += (kMaxWarps + 2) * DQ_MAX_GROUP * 4;
-    L.off_pages = o; o += kMaxWarps * 4 * 2 * 4 + 16;   // per warp: page ids of 4 items in flight; prev rows
-    L.off_qmu = o; o += nw * 2 * DQ_MAX_GROUP * 4;
-    L.total = o;
-    return L;
+// total bytes: fixed part, nw warp regions, then the per-sequence block prefix sums and lengths
+__host__ __device__ inline int wide_smem_bytes(int nw, int B, int G) {
+    return kOffWarp + nw * warp_stride(G) + align16w((2 * B + 1) * 4);
 }
 
 // Decode 16 symbols of one stream (Algorithm 2) out of the warp's ring and pack their levels as
@@ -250,17 +242,16 @@ dq_attention_wide_kernel(const __grid_constant__ DqDevTable TK, const __grid_con
     const int nthreads = blockDim.x, nw = nthreads >> 5;
     const int G = p.G, hs = p.hs, groups = p.groups;
     const int rwk = TK.rec_words, rwv = TV.rec_words;
-    const WLayout L = make_wlayout(nw, p.B, G);
     const uint32_t sbase = smem_addr(smem);
+    const int wstride = warp_stride(G);
 
-    uint32_t* lutk = reinterpret_cast<uint32_t*>(smem + L.off_lutk);
-    uint32_t* lutv = reinterpret_cast<uint32_t*>(smem + L.off_lutv);
-    int* prefix = reinterpret_cast<int*>(smem + L.off_prefix);
+    uint32_t* lutk = reinterpret_cast<uint32_t*>(smem + kOffLutK);
+    uint32_t* lutv = reinterpret_cast<uint32_t*>(smem + kOffLutV);
+    int* prefix = reinterpret_cast<int*>(smem + kOffWarp + nw * wstride);
     int* s_len = prefix + (p.B + 1);
-    float* qsum = reinterpret_cast<float*>(smem + L.off_qsum);      // [2][8]
-    float* red_m = reinterpret_cast<float*>(smem + L.off_red);      // [warp][head] chunk maxima
+    float* qsum = reinterpret_cast<float*>(smem + kOffQsum);        // [2][8]
+    float* red_m = reinterpret_cast<float*>(smem + kOffRed);        // [warp][head] chunk maxima
     float* red_M = red_m + kMaxWarps * DQ_MAX_GROUP;                // [2][head] step maxima
-    float* obuf_all = reinterpret_cast<float*>(smem + L.off_obuf);  // [warp][head][kORow]
 
     pdl_launch_dependents();
     for (int i = tid; i < 256 * 32; i += nthreads) {
@@ -275,11 +266,10 @@ dq_attention_wide_kernel(const __grid_constant__ DqDevTable TK, const __grid_con
     __syncthreads();
     const int total_items = prefix[p.B] * groups;
 
-    const uint32_t my_lutk = sbase + L.off_lutk + lane * 4, my_lutv = sbase + L.off_lutv + lane * 4;
-    const uint32_t ringk = sbase + L.off_ringk + warp * kRingK, ringv = sbase + L.off_ringv + warp * kRingV;
-    const uint32_t ktile = sbase + L.off_tiles + warp * 2 * kTile, vtile = ktile + kTile;
-    const uint32_t my_obuf = sbase + L.off_obuf + warp * L.warp_obuf_bytes;
-    const uint32_t my_qmu = sbase + L.off_qmu + warp * (2 * DQ_MAX_GROUP * 4);
+    const uint32_t my_lutk = sbase + kOffLutK + lane * 4, my_lutv = sbase + kOffLutV + lane * 4;
+    const uint32_t wb = sbase + kOffWarp + warp * wstride;   // this warp's region
+    const uint32_t ringk = wb + kWRingK, ringv = wb + kWRingV, ktile = wb + kWTileK, vtile = wb + kWTileV;
+    const uint32_t my_obuf = wb + kWObuf, my_qmu = wb + kWQmu;
     const uint32_t one = (sbase >> 31) | 1u;
     const int g_row = lane >> 2, qd = lane & 3;
 
@@ -299,8 +289,8 @@ dq_attention_wide_kernel(const __grid_constant__ DqDevTable TK, const __grid_con
         }
         return it;
     };
-    int* my_pages = reinterpret_cast<int*>(smem + L.off_pages) + warp * 8;
-    long long* s_prev_row = reinterpret_cast<long long*>(smem + L.off_pages + kMaxWarps * 32);
+    int* my_pages = reinterpret_cast<int*>(smem + kOffPages) + warp * 8;
+    long long* s_prev_row = reinterpret_cast<long long*>(smem + kOffPrevRow);
     auto fetch_pages = [&](int n, const Item& it) {
         const int tok0 = (it.blk * nw + warp) * kChunk;
         if (it.valid && tok0 < it.len && lane < 2 && tok0 + 16 * lane < it.len)
@@ -314,9 +304,9 @@ dq_attention_wide_kernel(const __grid_constant__ DqDevTable TK, const __grid_con
         const int h = it.grp * hs + k;
         const uint16_t* qsrc = p.q16 + ((size_t)it.b * p.Hkv + h) * 16 * kN;
         for (int i = tid; i < 16 * 16; i += nthreads)
-            cp_async16(sbase + L.off_q16 + (s & 1) * kQ16Bytes + (i >> 4) * kQ16Stride + (i & 15) * 16, qsrc + i * 8);
+            cp_async16(sbase + kOffQ16 + (s & 1) * kQ16Bytes + (i >> 4) * kQ16Stride + (i & 15) * 16, qsrc + i * 8);
         if (tid < G)
-            cp_async4(sbase + L.off_qsum + ((s & 1) * DQ_MAX_GROUP + tid) * 4, p.qsum + (size_t)it.b * p.Hq + (size_t)h * G + tid);
+            cp_async4(sbase + kOffQsum + ((s & 1) * DQ_MAX_GROUP + tid) * 4, p.qsum + (size_t)it.b * p.Hq + (size_t)h * G + tid);
         const int tok0 = (it.blk * nw + warp) * kChunk;
         if (p.has_mean && tok0 < it.len && lane < G)
             cp_async4(my_qmu + ((s & 1) * DQ_MAX_GROUP + lane) * 4,
@@ -369,7 +359,7 @@ dq_attention_wide_kernel(const __grid_constant__ DqDevTable TK, const __grid_con
     int kV = 0;                        // head of the pending V step
     bool wv = false;                   // this warp holds tokens of the pending V step's item
     int nwv = 0;                       // warps that hold tokens of that item
-    uint32_t hk = 0u, hv = 0u, xv_next = 1u << 23;   // headers (s, o as fp16 pairs) of the K item's tokens; V start state
+    uint32_t hk = 0u, hv = 0u;        // headers (s, o as fp16 pairs) of the K item's tokens
     uint32_t pb_hi[2][2] = {{0u, 0u}, {0u, 0u}}, pb_lo[2][2] = {{0u, 0u}, {0u, 0u}};
 
     for (int s = 0;; ++s) {
@@ -388,10 +378,9 @@ dq_attention_wide_kernel(const __grid_constant__ DqDevTable TK, const __grid_con
         cp_async_commit();
 
         // streams that start with this step
-        if (have_prev && kV == 0) {          // V streams of the pending item (their first rows were fetched after the last pass)
-            cv.x = xv_next;
-        }
-        const int tok0 = (cur.blk * nw + warp) * kChunk;
+        if (have_prev && kV == 0)            // V streams of the pending item: state from ring row 1 (fetched after the last pass)
+            cv.x = lds32(ringv + 128 + lane * 4);
+        int tok0 = (cur.blk * nw + warp) * kChunk;
         if (cur.valid && kK == 0) {          // K streams of `cur`: header and state from ring rows 0, 1
             hk = lds32(ringk + lane * 4);
             ck.x = lds32(ringk + 128 + lane * 4);
@@ -399,17 +388,16 @@ dq_attention_wide_kernel(const __grid_constant__ DqDevTable TK, const __grid_con
                 const size_t pg = (size_t)my_pages[(nK & 3) * 2 + (lane >> 4)];
                 const uint32_t* vcol = reinterpret_cast<const uint32_t*>(p.v_cont + (pg * groups + cur.grp) * ((size_t)rwv * 64)) + (lane & 15);
                 hv = __ldg(vcol);
-                xv_next = __ldg(vcol + 16);
             }
         }
 
-        const uint32_t q16 = sbase + L.off_q16 + (s & 1) * kQ16Bytes;
+        const uint32_t q16 = sbase + kOffQ16 + (s & 1) * kQ16Bytes;
         float sacc[4][4];
 #pragma unroll
         for (int i = 0; i < 4; ++i) { sacc[i][0] = sacc[i][1] = sacc[i][2] = sacc[i][3] = 0.f; }
         // a warp whose 32 tokens lie beyond the sequence end skips the decode (its logits are masked,
         // its output slot is left out of the merge)
-        const bool wk = cur.valid && tok0 < cur.len;
+        bool wk = cur.valid && tok0 < cur.len;
         if (wk && wv)
             wide_pass<true, true>(ck, cv, ringk, ringv, p.k_cont, p.v_cont, rwk, rwv, my_lutk, my_lutv, one, ktile, vtile, q16,
                                   my_obuf, lane, G, sacc, pb_hi, pb_lo);
@@ -419,6 +407,13 @@ dq_attention_wide_kernel(const __grid_constant__ DqDevTable TK, const __grid_con
         else if (wv)
             wide_pass<false, true>(ck, cv, ringk, ringv, p.k_cont, p.v_cont, rwk, rwv, my_lutk, my_lutv, one, ktile, vtile, q16,
                                    my_obuf, lane, G, sacc, pb_hi, pb_lo);
+
+        // The item descriptors are derived again rather than kept in registers across the pass.
+        cur = item_of(nK, hint);
+        nxt = cur;
+        if (last_head) nxt = item_of(nK + 1, cur.b);
+        tok0 = (cur.blk * nw + warp) * kChunk;
+        wk = cur.valid && tok0 < cur.len;
 
         // streams that ended with this pass hand their ring to the next item's streams
         cp_async_wait<0>();
@@ -474,7 +469,8 @@ dq_attention_wide_kernel(const __grid_constant__ DqDevTable TK, const __grid_con
                 const int g = e / 130, col = e - g * 130;
                 const int src = col < kN ? col : lcol + (col - kN);
                 float sum = 0.f;
-                for (int w = 0; w < nwv; ++w) sum += obuf_all[(w * G + g) * kORow + src];
+                for (int w = 0; w < nwv; ++w)
+                    sum += reinterpret_cast<const float*>(smem + kOffWarp + w * wstride + kWObuf)[g * kORow + src];
                 float* dst = p.partial + ((size_t)s_prev_row[(s + 1) & 1] + g) * kPartial;
                 if (col < kN) dst[col] = sum;
                 else dst[col + 1] = sum;
@@ -534,14 +530,14 @@ dq_attention_wide_kernel(const __grid_constant__ DqDevTable TK, const __grid_con
 int dq_attn_wide_pick_warps(const DqDevTable& tk, const DqDevTable& tv, int B, int G, int smem_max) {
     (void)tk; (void)tv;
     for (int nw = kWideWarps; nw >= 4; --nw)
-        if (make_wlayout(nw, B, G).total <= smem_max) return nw;
+        if (wide_smem_bytes(nw, B, G) <= smem_max) return nw;
     return 0;
 }
 
 cudaError_t dq_launch_attention_wide_main(const DqDevTable& tk, const DqDevTable& tv, const AttnParams& p, int nw,
                                           int sm_count, cudaStream_t st) {
-    const WLayout L = make_wlayout(nw, p.B, p.G);
-    cudaError_t e = cudaFuncSetAttribute(dq_attention_wide_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, L.total);
+    const int smem_bytes = wide_smem_bytes(nw, p.B, p.G);
+    cudaError_t e = cudaFuncSetAttribute(dq_attention_wide_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes);
     if (e != cudaSuccess) return e;
-    return dq_launch_pdl(dq_attention_wide_kernel, dim3(sm_count), dim3(nw * 32), (size_t)L.total, st, tk, tv, p);
+    return dq_launch_pdl(dq_attention_wide_kernel, dim3(sm_count), dim3(nw * 32), (size_t)smem_bytes, st, tk, tv, p);
 }
