@@ -56,18 +56,20 @@ __host__ __device__ inline Layout make_layout(int nw, int rec_k, int rec_v, int 
     L.stage_v = align16(kChunk * rec_v);
     L.warp_tile_bytes = 2 * kTileBytes;             // K tile (+ per-token metadata), V tile
     L.warp_obuf_bytes = G * kORow * 4;              // this warp's O[g][channel], l, off
+    // compile-time offsets first (the decode loop's addresses then cost no registers), sizes that
+    // depend on the launch after them
     int o = 0;
     L.off_lutk = o; o += 256 * 32 * 4;
     L.off_lutv = o; o += 256 * 32 * 4;
-    L.off_prefix = o; o += align16((2 * B + 1) * 4);   // block prefix sums, sequence lengths
     L.off_q16 = o; o += 2 * kQ16Bytes;
     L.off_qsum = o; o += 2 * DQ_MAX_GROUP * 4;
     L.off_red = o; o += (kMaxWarps + 2) * DQ_MAX_GROUP * 4;
     L.off_pages = o; o += kMaxWarps * 3 * 2 * 4 + 16;   // per warp: page ids of 3 items in flight; prev row
-    L.off_kst = o; o += 2 * nw * L.stage_k;
-    L.off_vst = o; o += 2 * nw * L.stage_v;
     L.off_tiles = o; o += nw * L.warp_tile_bytes;
     L.off_obuf = o; o += nw * L.warp_obuf_bytes;
+    L.off_kst = o; o += 2 * nw * L.stage_k;
+    L.off_vst = o; o += 2 * nw * L.stage_v;
+    L.off_prefix = o; o += align16((2 * B + 1) * 4);   // block prefix sums, sequence lengths
     L.total = o + 256;  // slack: a malformed record may be over-read by up to 136 + 8 bytes
     return L;
 }
@@ -384,10 +386,11 @@ dq_attention_kernel(const __grid_constant__ DqDevTable TK, const __grid_constant
         __syncthreads();   // q' operand of `cur` visible; last iteration's merge reads are done
 
         // ------------------------------------------ K streams of `cur`, V streams of `prev`
-        const int tok0 = (cur.blk * nw + warp) * kChunk;
-        const uint32_t kst = sbase + L.off_kst + ((n & 1) * nw + warp) * L.stage_k;
+        int tok0 = (cur.blk * nw + warp) * kChunk;
+        uint32_t kst = sbase + L.off_kst + ((n & 1) * nw + warp) * L.stage_k;
         const uint32_t vst_prev = sbase + L.off_vst + (((n + 1) & 1) * nw + warp) * L.stage_v;
-        const uint32_t rk = kst + lane * TK.rec, rvp = vst_prev + lane * TV.rec;
+        uint32_t rk = kst + lane * TK.rec;
+        const uint32_t rvp = vst_prev + lane * TV.rec;
         const uint32_t q16 = sbase + L.off_q16 + (n & 1) * kQ16Bytes;
         float sacc[4][4];
 #pragma unroll
@@ -406,6 +409,10 @@ dq_attention_kernel(const __grid_constant__ DqDevTable TK, const __grid_constant
         }
 
         // ------------------------------------------ logits of `cur` and this warp's maximum (base 2)
+        cur = item_of(n, hint);   // derived again rather than kept in registers across the pass
+        tok0 = (cur.blk * nw + warp) * kChunk;
+        kst = sbase + L.off_kst + ((n & 1) * nw + warp) * L.stage_k;
+        rk = kst + lane * TK.rec;
         float lg[4][2], sv_t[4][2], ov_t[4][2];
         if (cur.valid) {
             cp_async_wait<0>();   // the V records of `cur` (header needed now) have landed
