@@ -37,10 +37,11 @@ def _host(cache):
     return dict(kc=_np(cache.k_cont), vc=_np(cache.v_cont), mq=_np(cache.mean_q), ms=_np(cache.mean_scale))
 
 
-def _check_encoder_sample(w, ok, ov, host, rng, n_windows=6):
+def _check_encoder_sample(w, ok, ov, host, rng, n_windows=6, groups=None):
     """Oracle re-encodes a few whole (sequence, window) runs (into compact containers of its
     own) and compares their records and window means with what the GPU wrote."""
     cfg = w.cfg
+    groups = cfg.hkv if groups is None else groups     # streams per token
     seq_id, pos, slot = _np(w.seq_id), _np(w.pos), _np(w.slot)
     starts = np.concatenate([[0], np.cumsum(cfg.seq_lens)[:-1]])
     picked = set()
@@ -58,8 +59,8 @@ def _check_encoder_sample(w, ok, ov, host, rng, n_windows=6):
         mq = np.zeros((cfg.batch, w.max_windows, cfg.hkv, 128), np.int8)
         ms = np.zeros((cfg.batch, w.max_windows, cfg.hkv), np.float32)
         oracle.window_means(kb, seq_id[lo:hi], pos[lo:hi], mq, ms, 0)
-        kc = np.zeros(((n + 15) // 16, cfg.hkv, 16, ok.rec), np.uint8)
-        vc = np.zeros(((n + 15) // 16, cfg.hkv, 16, ov.rec), np.uint8)
+        kc = np.zeros(((n + 15) // 16, groups, 16, ok.rec), np.uint8)
+        vc = np.zeros(((n + 15) // 16, groups, 16, ov.rec), np.uint8)
         oracle.encode_tokens(ok, kb, seq_id[lo:hi], pos[lo:hi], compact, kc, mq, ms)
         oracle.encode_tokens(ov, vb, seq_id[lo:hi], pos[lo:hi], compact, vc)
         sl = slot[lo:hi]
@@ -206,3 +207,36 @@ def test_config5_encode_decode_loop_full():
     ref_rows = oracle.attention(ok, ov, workloads.bf16_bits(w.q), kc, vc, _np(cache.mean_q), _np(cache.mean_scale),
                                 _np(w.page_table), _np(final), cfg.hkv, gc.SM_SCALE, only=(b0, 3))
     gc.check_attention(out, out32, ref_rows, rows=[(b0, 3)])     # the loop's own last output
+
+
+# ------------------------------------------------ token-wide streams at full size
+
+def _run_config_wide(cfg, seed, hs=8):
+    """The paper's default grouping (one 335 / 235-byte record per token, 8 / 6 levels) on a full
+    benchmark shape: same sampled checks, containers compared after undoing the page interleave."""
+    rng = np.random.default_rng(seed)
+    w = workloads.generate(cfg, device="cuda")
+    tk, tv, ok, ov = gc.wide_tables(cfg, hs)
+    cache = gc.WideGpuCache(w, tk, tv, hs)
+    gc.gpu_encode(w, tk, tv, cache)
+    torch.cuda.synchronize()
+    st = _np(cache.status)
+    assert st[0] == 0 and st[3] <= max(ok.rec, ov.rec)
+    host = dict(kc=gc.from_interleaved(_np(cache.k_cont), ok.rec), vc=gc.from_interleaved(_np(cache.v_cont), ov.rec),
+                mq=_np(cache.mean_q), ms=_np(cache.mean_scale))
+    _check_encoder_sample(w, ok, ov, host, rng, n_windows=4, groups=cfg.hkv // hs)
+    _check_decoder_sample(w, tk, tv, ok, ov, cache, host, rng, n_tokens=128)
+    _check_attention_sample(w, tk, tv, ok, ov, cache, host, rng)
+    return w, tk, tv, ok, ov, cache
+
+
+def test_config2_token_wide_full():
+    cfg = workloads.make_config(2)
+    assert cfg.total_tokens == 65536 and cfg.hkv == 8
+    _run_config_wide(cfg, 12)
+
+
+def test_config4_ragged_paged_token_wide_full():
+    cfg = workloads.make_config(4)
+    assert cfg.batch == 128 and cfg.shuffle_pages
+    _run_config_wide(cfg, 14)
