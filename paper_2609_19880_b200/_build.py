@@ -9,6 +9,8 @@ _CSRC = os.path.join(_PKG, "csrc")
 _INC = os.path.join(os.path.dirname(_PKG), "include")
 LIB_PATH = os.path.join(_PKG, "libdquant.so")
 
+# Extra nvcc flags for every translation unit can be given in the environment variable
+# DQ_NVCC_EXTRA (e.g. "-Xptxas -v" variants while tuning).
 # (source, extra flags).  The encoder is compiled without FMA contraction: its records must be
 # reproducible bit for bit, every rounding is written out explicitly.
 _SOURCES = [
