@@ -173,6 +173,25 @@ int dq_decode_attention_residual(const dq_tables *tk, const dq_tables *tv, const
                                  int Hq, int Hkv, float sm_scale, void *out_bf16, float *out_f32,
                                  void *workspace, size_t workspace_bytes, void *cuda_stream);
 
+/* Attention for q_len query tokens per sequence in one pass over the cache (speculative
+ * decoding, short chunks of prefill); the paper's kernel is the q_len = 1 case (Sec. 4.5).
+ *   q_bf16, out_*   [B][q_len][Hq][128]
+ *   seq_lens, resid_lens   count every token of the sequence including the q_len newest ones, whose
+ *                   K/V the caller has already stored (compressed, or in the BF16 window).  Query token
+ *                   i (0 = oldest) sees the first seq_lens[b] + resid_lens[b] - (q_len - 1 - i) tokens of
+ *                   the sequence: all compressed tokens come before all window tokens.
+ *   workspace       >= dq_decode_workspace_bytes(B, Hq * q_len, max_pages)
+ * The q_len * (Hq / Hkv) rows of a KV head share one decode of its streams, so the cost is that of
+ * q_len = 1; q_len * (Hq / Hkv) must be <= 8 (DQ_ERR_UNSUPPORTED otherwise: split the call).
+ * resid_* may be NULL (no window). */
+int dq_decode_attention_multi(const dq_tables *tk, const dq_tables *tv, const void *q_bf16, int q_len,
+                              const uint8_t *k_cont, const uint8_t *v_cont, const int8_t *k_mean_q,
+                              const float *k_mean_scale, int max_windows, const int32_t *page_table,
+                              int max_pages, const int32_t *seq_lens, const void *resid_k_bf16,
+                              const void *resid_v_bf16, const int32_t *resid_lens, int resid_cap, int B,
+                              int Hq, int Hkv, float sm_scale, void *out_bf16, float *out_f32,
+                              void *workspace, size_t workspace_bytes, void *cuda_stream);
+
 /* dq_decode_attention for callers that must not allocate (the paper has no counterpart: this
  * is a packaging variant of the same kernels, not part of the method).
  *

@@ -24,6 +24,7 @@ ERRORS = {0: "DQ_OK", -1: "DQ_ERR_ARG", -2: "DQ_ERR_INFEASIBLE", -3: "DQ_ERR_UNS
 
 EXPORTS = ["dq_build_tables", "dq_free_tables", "dq_tables_info", "dq_encode_tokens",
            "dq_decode_workspace_bytes", "dq_decode_attention", "dq_decode_attention_residual",
+           "dq_decode_attention_multi",
            "dq_decode_attention_static", "dq_decode_tokens",
            "dq_bf16_decode_attention", "dq_profile_enable", "dq_profile_read", "dq_strerror",
            "dq_last_cuda_error"]
@@ -77,6 +78,9 @@ def lib():
         L.dq_decode_attention_residual.restype = i32
         L.dq_decode_attention_residual.argtypes = [vp, vp, vp, vp, vp, vp, vp, i32, vp, i32, vp, vp, vp, vp, i32,
                                                    i32, i32, i32, f32, vp, vp, vp, sz, vp]
+        L.dq_decode_attention_multi.restype = i32
+        L.dq_decode_attention_multi.argtypes = [vp, vp, vp, i32, vp, vp, vp, vp, i32, vp, i32, vp, vp, vp, vp, i32,
+                                                i32, i32, i32, f32, vp, vp, vp, sz, vp]
         L.dq_decode_attention_static.restype = i32
         L.dq_decode_attention_static.argtypes = [vp, vp, vp, vp, vp, vp, vp, i32, vp, i32, vp, i32, i32, i32, f32,
                                                  vp, vp, vp]
@@ -195,6 +199,22 @@ def dq_decode_attention_residual(tk, tv, q_bf16, k_cont, v_cont, k_mean_q, k_mea
         _ptr(resid_lens), int(resid_k.shape[1]), B, Hq, int(Hkv), float(sm_scale), _ptr(out_bf16), _ptr(out_f32),
         _ptr(workspace), int(workspace.numel() * workspace.element_size()), _stream(stream))
     _check(rc, "dq_decode_attention_residual")
+
+
+def dq_decode_attention_multi(tk, tv, q_bf16, k_cont, v_cont, k_mean_q, k_mean_scale, page_table, seq_lens,
+                              Hkv: int, sm_scale: float, out_bf16, workspace, out_f32=None, resid_k=None,
+                              resid_v=None, resid_lens=None, stream=None):
+    """q bf16 [B, q_len, Hq, 128] -> out bf16 [B, q_len, Hq, 128]: q_len query tokens per sequence share
+    one pass over the cache; seq_lens (+ resid_lens) include the q_len newest tokens."""
+    B, q_len, Hq = int(q_bf16.shape[0]), int(q_bf16.shape[1]), int(q_bf16.shape[2])
+    max_windows = int(k_mean_q.shape[1]) if k_mean_q is not None else 0
+    rc = lib().dq_decode_attention_multi(
+        tk.handle, tv.handle, _ptr(q_bf16), q_len, _ptr(k_cont), _ptr(v_cont), _ptr(k_mean_q), _ptr(k_mean_scale),
+        max_windows, _ptr(page_table), int(page_table.shape[1]), _ptr(seq_lens), _ptr(resid_k), _ptr(resid_v),
+        _ptr(resid_lens), int(resid_k.shape[1]) if resid_k is not None else 0, B, Hq, int(Hkv), float(sm_scale),
+        _ptr(out_bf16), _ptr(out_f32), _ptr(workspace), int(workspace.numel() * workspace.element_size()),
+        _stream(stream))
+    _check(rc, "dq_decode_attention_multi")
 
 
 STATIC_SCRATCH_BYTES = 4 << 20

@@ -99,14 +99,16 @@ static int check_attn_common(const void* q, const int32_t* page_table, int max_p
     return DQ_OK;
 }
 
-int dq_decode_attention_residual(const dq_tables* tk, const dq_tables* tv, const void* q_bf16,
-                                 const uint8_t* k_cont, const uint8_t* v_cont, const int8_t* k_mean_q,
-                                 const float* k_mean_scale, int max_windows, const int32_t* page_table,
-                                 int max_pages, const int32_t* seq_lens, const void* resid_k_bf16,
-                                 const void* resid_v_bf16, const int32_t* resid_lens, int resid_cap, int B, int Hq,
-                                 int Hkv, float sm_scale, void* out_bf16, float* out_f32, void* workspace,
-                                 size_t workspace_bytes, void* cuda_stream) {
+int dq_decode_attention_multi(const dq_tables* tk, const dq_tables* tv, const void* q_bf16, int q_len,
+                              const uint8_t* k_cont, const uint8_t* v_cont, const int8_t* k_mean_q,
+                              const float* k_mean_scale, int max_windows, const int32_t* page_table,
+                              int max_pages, const int32_t* seq_lens, const void* resid_k_bf16,
+                              const void* resid_v_bf16, const int32_t* resid_lens, int resid_cap, int B, int Hq,
+                              int Hkv, float sm_scale, void* out_bf16, float* out_f32, void* workspace,
+                              size_t workspace_bytes, void* cuda_stream) {
     if (!tk || !tv || !k_cont || !v_cont) return DQ_ERR_ARG;
+    if (q_len < 1) return DQ_ERR_ARG;
+    if (Hkv > 0 && Hq > 0 && Hq % Hkv == 0 && (long long)q_len * (Hq / Hkv) > DQ_MAX_GROUP) return DQ_ERR_UNSUPPORTED;
     if (resid_k_bf16 || resid_v_bf16 || resid_lens) {
         if (!resid_k_bf16 || !resid_v_bf16 || !resid_lens || resid_cap <= 0) return DQ_ERR_ARG;
         if ((reinterpret_cast<uintptr_t>(resid_k_bf16) & 7u) || (reinterpret_cast<uintptr_t>(resid_v_bf16) & 7u))
@@ -115,6 +117,7 @@ int dq_decode_attention_residual(const dq_tables* tk, const dq_tables* tv, const
     int rc = check_attn_common(q_bf16, page_table, max_pages, seq_lens, B, Hq, Hkv, out_bf16, out_f32,
                                workspace, workspace_bytes);
     if (rc != DQ_OK) return rc;
+    if (workspace_bytes < dq_attn_workspace_bytes(B, Hq * q_len, max_pages)) return DQ_ERR_WORKSPACE;
     if (tv->info.has_mean) return DQ_ERR_UNSUPPORTED;
     if (tk->info.heads_per_stream != tv->info.heads_per_stream) return DQ_ERR_UNSUPPORTED;
     if (Hkv % tk->info.heads_per_stream != 0) return DQ_ERR_ARG;
@@ -132,9 +135,22 @@ int dq_decode_attention_residual(const dq_tables* tk, const dq_tables* tv, const
     a.max_windows = max_windows; a.max_pages = max_pages;
     a.B = B; a.Hq = Hq; a.Hkv = Hkv; a.sm_scale = sm_scale;
     a.resid_k = resid_k_bf16; a.resid_v = resid_v_bf16; a.resid_lens = resid_lens; a.resid_cap = resid_cap;
+    a.q_len = q_len;
     const cudaError_t e = dq_launch_attention(tk->dev, tv->dev, a, static_cast<cudaStream_t>(cuda_stream));
     if (e != cudaSuccess) return cuda_fail(e, "decode attention");
     return DQ_OK;
+}
+
+int dq_decode_attention_residual(const dq_tables* tk, const dq_tables* tv, const void* q_bf16,
+                                 const uint8_t* k_cont, const uint8_t* v_cont, const int8_t* k_mean_q,
+                                 const float* k_mean_scale, int max_windows, const int32_t* page_table,
+                                 int max_pages, const int32_t* seq_lens, const void* resid_k_bf16,
+                                 const void* resid_v_bf16, const int32_t* resid_lens, int resid_cap, int B, int Hq,
+                                 int Hkv, float sm_scale, void* out_bf16, float* out_f32, void* workspace,
+                                 size_t workspace_bytes, void* cuda_stream) {
+    return dq_decode_attention_multi(tk, tv, q_bf16, 1, k_cont, v_cont, k_mean_q, k_mean_scale, max_windows, page_table,
+                                     max_pages, seq_lens, resid_k_bf16, resid_v_bf16, resid_lens, resid_cap, B, Hq, Hkv,
+                                     sm_scale, out_bf16, out_f32, workspace, workspace_bytes, cuda_stream);
 }
 
 int dq_decode_attention(const dq_tables* tk, const dq_tables* tv, const void* q_bf16,
@@ -184,6 +200,7 @@ int dq_decode_attention_static(const dq_tables* tk, const dq_tables* tv, const v
     a.max_windows = max_windows; a.max_pages = max_pages;
     a.B = B; a.Hq = Hq; a.Hkv = Hkv; a.sm_scale = sm_scale;
     a.resid_k = nullptr; a.resid_v = nullptr; a.resid_lens = nullptr; a.resid_cap = 0;
+    a.q_len = 1;
     e = dq_launch_attention_static(tk->dev, tv->dev, a, static_cast<cudaStream_t>(cuda_stream));
     if (e != cudaSuccess) return cuda_fail(e, "decode attention (static scratch)");
     return DQ_OK;

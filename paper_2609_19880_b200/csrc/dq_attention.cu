@@ -90,7 +90,7 @@ dq_attn_prepare_kernel(AttnParams p) {
     const int wgroups = p.has_mean ? (p.windows + kPrepWindows - 1) / kPrepWindows : 0;
     if (wid < (long long)heads * (1 + wgroups)) {
         const int head = (int)(wid % heads), win = (int)(wid / heads) - 1;
-        const uint2 raw = *reinterpret_cast<const uint2*>(p.q + (size_t)head * kN + 4 * lane);
+        const uint2 raw = *reinterpret_cast<const uint2*>(p.q + qo_row(p, head / p.Hq, head % p.Hq) * kN + 4 * lane);
         float v[4] = {bf16_bits_to_float(raw.x & 0xffffu), bf16_bits_to_float(raw.x >> 16),
                       bf16_bits_to_float(raw.y & 0xffffu), bf16_bits_to_float(raw.y >> 16)};
         if (p.rotate_q) warp_fwht128(v, lane);
@@ -427,6 +427,10 @@ dq_attention_kernel(const __grid_constant__ DqDevTable TK, const __grid_constant
                 asm volatile("st.shared.v4.f32 [%0], {%1,%2,%3,%4};\n" ::"r"(ktile + lane * kTileStride + 32), "f"(sK),
                              "f"(oK), "f"(sV), "f"(oV) : "memory");
             }
+            // tokens this thread's row may see: a query token that is not the last one stops earlier; tokens
+            // of a BF16 residual window come after the compressed ones and absorb the offset first
+            int row_len = cur.len;
+            if (p.q_len > 1) row_len -= max(0, row_offset(p, g_row) - (p.resid_lens ? max(p.resid_lens[cur.b], 0) : 0));
             float qmu = 0.f, qs = 0.f;   // q' . window mean and sum of q', for the head row this thread owns
             if (g_row < G) {
                 qs = qsum[(n & 1) * DQ_MAX_GROUP + g_row];
@@ -443,7 +447,7 @@ dq_attention_kernel(const __grid_constant__ DqDevTable TK, const __grid_constant
                     asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4];\n"
                                  : "=f"(m4.x), "=f"(m4.y), "=f"(m4.z), "=f"(m4.w) : "r"(ktile + tk * kTileStride + 32));
                     const float S = sacc[i][u] + sacc[i][2 + u];
-                    const bool ok = tok0 + tk < cur.len;
+                    const bool ok = tok0 + tk < row_len;
                     lg[i][u] = ok ? p.scale_log2 * fmaf(m4.x, S, fmaf(m4.y, qs, qmu)) : -INFINITY;
                     sv_t[i][u] = ok ? m4.z : 0.f;
                     ov_t[i][u] = ok ? m4.w : 0.f;
@@ -557,10 +561,12 @@ dq_attn_combine_kernel(AttnParams p) {
     }
     // residual window: tokens w*8 .. w*8+7, then + 64, ...
     float racc[4] = {0.f, 0.f, 0.f, 0.f}, rl = 0.f, rm = -INFINITY;
-    const int rlen = p.resid_k ? min(max(p.resid_lens[b], 0), p.resid_cap) : 0;
+    const size_t io_row = qo_row(p, b, hq);
+    int rlen = p.resid_k ? min(max(p.resid_lens[b], 0), p.resid_cap) : 0;
+    rlen = max(0, rlen - row_offset(p, hq % p.G));   // an earlier query token sees fewer of the newest tokens
     if (rlen > 0) {
         const int h = hq / p.G;
-        const uint2 qraw = *reinterpret_cast<const uint2*>(p.q + (size_t)wid * kN + 4 * lane);
+        const uint2 qraw = *reinterpret_cast<const uint2*>(p.q + io_row * kN + 4 * lane);
         const float q0 = bf16_bits_to_float(qraw.x & 0xffffu), q1 = bf16_bits_to_float(qraw.x >> 16);
         const float q2 = bf16_bits_to_float(qraw.y & 0xffffu), q3 = bf16_bits_to_float(qraw.y >> 16);
         for (int t0 = 8 * w; t0 < rlen; t0 += 64) {
@@ -636,13 +642,13 @@ dq_attn_combine_kernel(AttnParams p) {
         for (int e = 0; e < 4; ++e) acc[e] = fmaf(racc[e], inv, acc[e]);
     }
     if (p.out_f32)
-        *reinterpret_cast<float4*>(p.out_f32 + (size_t)wid * kN + 4 * lane) = make_float4(acc[0], acc[1], acc[2], acc[3]);
+        *reinterpret_cast<float4*>(p.out_f32 + io_row * kN + 4 * lane) = make_float4(acc[0], acc[1], acc[2], acc[3]);
     if (p.out_bf16) {
         const __nv_bfloat162 lo = __floats2bfloat162_rn(acc[0], acc[1]), hi = __floats2bfloat162_rn(acc[2], acc[3]);
         uint2 wv;
         wv.x = *reinterpret_cast<const uint32_t*>(&lo);
         wv.y = *reinterpret_cast<const uint32_t*>(&hi);
-        *reinterpret_cast<uint2*>(reinterpret_cast<uint16_t*>(p.out_bf16) + (size_t)wid * kN + 4 * lane) = wv;
+        *reinterpret_cast<uint2*>(reinterpret_cast<uint16_t*>(p.out_bf16) + io_row * kN + 4 * lane) = wv;
     }
 }
 
@@ -870,7 +876,8 @@ cudaError_t dq_launch_attention(const DqDevTable& tk, const DqDevTable& tv, cons
         if (e != cudaSuccess) return e;
     }
     int nw = kMaxWarps;
-    const int G = a.Hq / a.Hkv;
+    const int q_len = a.q_len > 1 ? a.q_len : 1;
+    const int G1 = a.Hq / a.Hkv, G = G1 * q_len;   // rows per KV head
     const bool wide = tk.hs > 1;   // token-wide streams: main kernel of dq_attention_wide.cu
     Layout L = make_layout(nw, tk.rec, tv.rec, a.B, G);
     if (wide) {
@@ -884,7 +891,7 @@ cudaError_t dq_launch_attention(const DqDevTable& tk, const DqDevTable& tv, cons
         if (L.total > smem_max) return cudaErrorInvalidConfiguration;
     }
 
-    const WsLayout w = ws_layout(a.B, a.Hq, a.max_pages);
+    const WsLayout w = ws_layout(a.B, a.Hq * q_len, a.max_pages);
     uint8_t* ws = static_cast<uint8_t*>(a.workspace);
     AttnParams p;
     p.q = static_cast<const uint16_t*>(a.q_bf16);
@@ -900,7 +907,8 @@ cudaError_t dq_launch_attention(const DqDevTable& tk, const DqDevTable& tv, cons
     p.partial = reinterpret_cast<float*>(ws + w.off_partial);
     p.out_bf16 = a.out_bf16; p.out_f32 = a.out_f32;
     p.max_windows = a.max_windows; p.windows = windows_for(a.max_pages); p.max_pages = a.max_pages;
-    p.B = a.B; p.Hq = a.Hq; p.Hkv = a.Hkv; p.G = G;
+    p.B = a.B; p.Hq = a.Hq * q_len; p.Hkv = a.Hkv; p.G = G;
+    p.q_len = q_len; p.G1 = G1; p.Hq1 = a.Hq;
     p.item_tokens = nw * kChunk;
     p.rotate_q = tk.rotate; p.rotate_out = tv.rotate; p.has_mean = tk.has_mean;
     p.scale_log2 = a.sm_scale * 1.4426950408889634f;
@@ -910,7 +918,7 @@ cudaError_t dq_launch_attention(const DqDevTable& tk, const DqDevTable& tv, cons
     p.resid_k = static_cast<const uint16_t*>(a.resid_k); p.resid_v = static_cast<const uint16_t*>(a.resid_v);
     p.resid_lens = a.resid_lens; p.resid_cap = a.resid_cap;
 
-    const int heads = a.B * a.Hq;
+    const int heads = a.B * a.Hq * q_len;
     const long long prep_warps = (long long)heads * (1 + (p.has_mean ? (p.windows + kPrepWindows - 1) / kPrepWindows : 0));
     cudaError_t e = dq_launch_pdl(dq_attn_prepare_kernel, dim3((unsigned)((prep_warps + 7) / 8)), dim3(256), 0, st, p);
     if (e != cudaSuccess) return e;
@@ -957,6 +965,7 @@ cudaError_t dq_launch_bf16_attention(const DqAttnArgs& a, const void* k_pages, c
     p.scale_log2 = a.sm_scale * 1.4426950408889634f;
     p.hkv_magic = 0;
     p.hs = 1; p.groups = a.Hkv;
+    p.q_len = 1; p.G1 = p.G; p.Hq1 = a.Hq;
     p.resid_k = nullptr; p.resid_v = nullptr; p.resid_lens = nullptr; p.resid_cap = 0;
     const int heads = a.B * a.Hq;
     dq_attn_prepare_kernel<<<(heads + 7) / 8, 256, 0, st>>>(p);

@@ -434,6 +434,8 @@ dq_attention_wide_kernel(const __grid_constant__ DqDevTable TK, const __grid_con
                 asm volatile("st.shared.v4.f32 [%0], {%1,%2,%3,%4};\n" ::"r"(ktile + lane * 16), "f"(sK), "f"(oK), "f"(sV),
                              "f"(oV) : "memory");
             }
+            int row_len = cur.len;   // tokens this thread's row may see (earlier query tokens stop earlier)
+            if (p.q_len > 1) row_len -= max(0, row_offset(p, g_row) - (p.resid_lens ? max(p.resid_lens[cur.b], 0) : 0));
             float qmu = 0.f, qs = 0.f;
             if (g_row < G) {
                 qs = qsum[(s & 1) * DQ_MAX_GROUP + g_row];
@@ -450,7 +452,7 @@ dq_attention_wide_kernel(const __grid_constant__ DqDevTable TK, const __grid_con
                     asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4];\n"
                                  : "=f"(m4.x), "=f"(m4.y), "=f"(m4.z), "=f"(m4.w) : "r"(ktile + tk * 16));
                     const float S = sacc[i][u] + sacc[i][2 + u];
-                    const bool ok = tok0 + tk < cur.len;
+                    const bool ok = tok0 + tk < row_len;
                     lg[i][u] = ok ? p.scale_log2 * fmaf(m4.x, S, fmaf(m4.y, qs, qmu)) : -INFINITY;
                     sv_t[i][u] = ok ? m4.z : 0.f;
                     ov_t[i][u] = ok ? m4.w : 0.f;

@@ -66,6 +66,7 @@ struct DqAttnArgs {
     const void* resid_v;
     const int32_t* resid_lens;  // [B]
     int resid_cap;
+    int q_len;                  // query tokens per sequence (q and out are [B][q_len][Hq][128]); 0 or 1: one
 };
 size_t dq_attn_workspace_bytes(int B, int Hq, int max_pages);
 cudaError_t dq_launch_attention(const DqDevTable& tk, const DqDevTable& tv, const DqAttnArgs& a,
