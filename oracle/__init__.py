@@ -170,23 +170,48 @@ def encode_stream(z: np.ndarray, T: Table):
     return rec, sym, st
 
 
+ROPE_NONE, ROPE_HALF, ROPE_PAIRS = 0, 1, 2
+
+
+def rope_f32(x: np.ndarray, cs: np.ndarray, sn: np.ndarray, style: int) -> np.ndarray:
+    """Rotary embedding of one head vector (binary32); cs / sn: d/2 entries of this position."""
+    y = np.ascontiguousarray(x, dtype=np.float32).copy()
+    cs = np.ascontiguousarray(cs, dtype=np.float32)
+    sn = np.ascontiguousarray(sn, dtype=np.float32)
+    lib().dqo_rope_f32(_p(y), C.c_int(y.shape[0]), _p(cs), _p(sn), C.c_int(style))
+    return y
+
+
+def _rope_args(rope, d):
+    if rope is None:
+        return None, None, 0
+    cs, sn, style = rope
+    cs = np.ascontiguousarray(cs, dtype=np.float32)
+    sn = np.ascontiguousarray(sn, dtype=np.float32)
+    assert cs.shape == sn.shape and cs.shape[1] == d // 2 and style in (ROPE_HALF, ROPE_PAIRS)
+    return cs, sn, style
+
+
 def window_means(k_bf16: np.ndarray, seq_id, pos, mean_q: np.ndarray, mean_scale: np.ndarray,
-                 mode: int, rotate: bool = True):
+                 mode: int, rotate: bool = True, rope=None):
     """k_bf16: uint16 [T, Hkv, n] (bf16 bits).  mean_q int8 [S, Wmax, Hkv, n] and
     mean_scale f32 [S, Wmax, Hkv] are updated in place."""
     T_tok, Hkv, n = k_bf16.shape
     Wmax = mean_q.shape[1]
     seq_id = np.ascontiguousarray(seq_id, dtype=np.int32)
     pos = np.ascontiguousarray(pos, dtype=np.int32)
+    cs, sn, style = _rope_args(rope, n)
+    assert style == 0 or int(pos.max(initial=0)) < cs.shape[0]
     lib().dqo_window_means(_p(k_bf16), C.c_int(T_tok), C.c_int(Hkv), C.c_int(n), _p(seq_id), _p(pos),
                            _p(mean_q), _p(mean_scale), C.c_int(Wmax), C.c_int(mode),
-                           C.c_int(int(rotate)))
+                           C.c_int(int(rotate)), _p(cs), _p(sn), C.c_int(style))
 
 
 def encode_tokens(T: Table, x_bf16: np.ndarray, seq_id, pos, slot, cont: np.ndarray,
-                  mean_q=None, mean_scale=None):
+                  mean_q=None, mean_scale=None, rope=None):
     """x_bf16: uint16 [T, Hkv, d]; cont: uint8 [pages, Hkv / hs, 16, rec] updated in place, where
     hs = T.n / d heads share one stream (hs = 1: per token-head; hs = Hkv: per token).
+    rope = (cos f32 [positions, d/2], sin, style): x holds keys before their rotary embedding.
     Returns stats uint32[4]."""
     T_tok, Hkv, n = x_bf16.shape
     hs = max(1, T.n // n)
@@ -197,8 +222,11 @@ def encode_tokens(T: Table, x_bf16: np.ndarray, seq_id, pos, slot, cont: np.ndar
     slot = np.ascontiguousarray(slot, dtype=np.int32)
     Wmax = mean_q.shape[1] if mean_q is not None else 0
     st = np.zeros(4, dtype=np.uint32)
+    cs, sn, style = _rope_args(rope, n)
+    assert style == 0 or int(pos.max(initial=0)) < cs.shape[0]
     lib().dqo_encode_tokens(C.byref(T), _p(x_bf16), C.c_int(T_tok), C.c_int(Hkv), _p(seq_id), _p(pos),
-                            _p(slot), _p(cont), _p(mean_q), _p(mean_scale), C.c_int(Wmax), _p(st))
+                            _p(slot), _p(cont), _p(mean_q), _p(mean_scale), C.c_int(Wmax), _p(st),
+                            _p(cs), _p(sn), C.c_int(style))
     return st
 
 

@@ -434,6 +434,25 @@ void dqo_encode_stream(const float *z, const dqo_table *T, uint8_t *rec, uint32_
     if (sym_out) memcpy(sym_out, m, (size_t)n);
 }
 
+/* ------------------------------------------------------- rotary embedding */
+
+/* Rotary position embedding of one head vector x[d] in binary32 (keys only; applied before the
+ * Hadamard rotation when the caller hands over keys that have not been rotated yet).  cs / sn are
+ * the caller's tables for this token's position, d/2 entries each.  style 1 pairs element j with
+ * j + d/2 (the "rotate half" convention), style 2 pairs 2j with 2j + 1:
+ *   (a, b) -> (a cos_j - b sin_j, b cos_j + a sin_j), each product and each sum rounded once. */
+void dqo_rope_f32(float *x, int d, const float *cs, const float *sn, int style)
+{
+    int half = d / 2;
+    for (int j = 0; j < half; ++j) {
+        int ia = style == 1 ? j : 2 * j, ib = style == 1 ? j + half : 2 * j + 1;
+        float a = x[ia], b = x[ib];
+        float ac = a * cs[j], bs = b * sn[j], bc = b * cs[j], as = a * sn[j];
+        x[ia] = ac - bs;
+        x[ib] = bc + as;
+    }
+}
+
 /* ----------------------------------------------------------- window means */
 
 static void dqo_quantise_mean(float *mu, int n, int8_t *q, float *scale)
@@ -462,7 +481,7 @@ static void dqo_quantise_mean(float *mu, int n, int8_t *q, float *scale)
  *   (q, scale) into its own window slot (window 0: zeros); nothing else changes. */
 void dqo_window_means(const uint16_t *k_bf16, int T_tok, int Hkv, int n, const int32_t *seq_id,
                       const int32_t *pos, int8_t *mean_q, float *mean_scale, int Wmax, int mode,
-                      int rotate)
+                      int rotate, const float *rope_cos, const float *rope_sin, int rope_style)
 {
     if (mode == 1) {
         for (int t = 0; t < T_tok; ++t) {
@@ -488,13 +507,15 @@ void dqo_window_means(const uint16_t *k_bf16, int T_tok, int Hkv, int n, const i
         int w = pos[t0] / DQO_WINDOW;
         float inv = 1.0f / (float)(t1 - t0);
         for (int h = 0; h < Hkv; ++h) {
-            float mu[DQO_MAX_N];
-            for (int j = 0; j < n; ++j) {
-                float acc = 0.0f;
-                for (int t = t0; t < t1; ++t)
-                    acc = acc + dqo_bf16_to_f32(k_bf16[((size_t)t * Hkv + h) * n + j]);
-                mu[j] = acc * inv;
+            float mu[DQO_MAX_N], acc[DQO_MAX_N], kt[DQO_MAX_N];
+            for (int j = 0; j < n; ++j) acc[j] = 0.0f;
+            for (int t = t0; t < t1; ++t) {   /* sequential binary32 sum over the run, per channel */
+                for (int j = 0; j < n; ++j) kt[j] = dqo_bf16_to_f32(k_bf16[((size_t)t * Hkv + h) * n + j]);
+                if (rope_style)
+                    dqo_rope_f32(kt, n, rope_cos + (size_t)pos[t] * (n / 2), rope_sin + (size_t)pos[t] * (n / 2), rope_style);
+                for (int j = 0; j < n; ++j) acc[j] = acc[j] + kt[j];
             }
+            for (int j = 0; j < n; ++j) mu[j] = acc[j] * inv;
             if (rotate) dqo_fwht_f32(mu, n);
             size_t dst = ((size_t)seq_id[t0] * Wmax + w) * Hkv + h;
             dqo_quantise_mean(mu, n, mean_q + dst * n, mean_scale + dst);
@@ -524,7 +545,7 @@ static size_t dqo_rec_offset(int slot, int grp, int groups, int rec)
 void dqo_encode_tokens(const dqo_table *T, const uint16_t *x_bf16, int T_tok, int Hkv,
                        const int32_t *seq_id, const int32_t *pos, const int32_t *slot,
                        uint8_t *cont, const int8_t *mean_q, const float *mean_scale, int Wmax,
-                       uint32_t *stats)
+                       uint32_t *stats, const float *rope_cos, const float *rope_sin, int rope_style)
 {
     int d = dqo_head_dim(T), hs = dqo_heads_per_stream(T), groups = Hkv / hs;
     uint32_t st[4] = {0, 0, 0, 0};
@@ -539,6 +560,8 @@ void dqo_encode_tokens(const dqo_table *T, const uint16_t *x_bf16, int T_tok, in
                 int h = grp * hs + k;
                 float *zh = z + k * d;
                 for (int j = 0; j < d; ++j) zh[j] = dqo_bf16_to_f32(x_bf16[((size_t)t * Hkv + h) * d + j]);
+                if (rope_style)   /* keys handed over before their rotary embedding */
+                    dqo_rope_f32(zh, d, rope_cos + (size_t)pos[t] * (d / 2), rope_sin + (size_t)pos[t] * (d / 2), rope_style);
                 if (T->rotate) dqo_fwht_f32(zh, d);
                 if (T->has_mean) {
                     size_t mi = ((size_t)seq_id[t] * Wmax + pos[t] / DQO_WINDOW) * Hkv + h;
