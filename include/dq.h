@@ -72,6 +72,9 @@ extern "C" {
 #define DQ_MEAN_COMPUTE 0
 #define DQ_MEAN_REUSE 1
 
+#define DQ_ROPE_HALF 1           /* rotary pairs (j, j + 64): the "rotate half" convention */
+#define DQ_ROPE_PAIRS 2          /* rotary pairs (2j, 2j + 1)                              */
+
 typedef struct dq_tables dq_tables; /* opaque, immutable after build, host memory */
 
 typedef struct {
@@ -134,6 +137,22 @@ int dq_encode_tokens(const dq_tables *tk, const dq_tables *tv, const void *k_bf1
                      const int32_t *pos, const int32_t *slot, uint8_t *k_cont, uint8_t *v_cont,
                      int8_t *k_mean_q, float *k_mean_scale, int max_windows, int mean_mode,
                      uint32_t *status, void *cuda_stream);
+
+/* dq_encode_tokens for keys handed over before their rotary position embedding, so that the
+ * embedded keys never exist in bf16 (the paper encodes post-RoPE keys, Sec. 5.1; it does not
+ * describe this fusion): k_bf16 is rotated in binary32 by the angle tables of each token's
+ * position, then goes through the same pipeline (Hadamard, window mean, grid, drift, rANS);
+ * window means (DQ_MEAN_COMPUTE) are those of the embedded keys.  Values are untouched.
+ *   rope_cos, rope_sin   device float [positions][64], 16-byte aligned, positions > every pos[t]:
+ *                        cos / sin of position * frequency j (the caller owns the frequency rule)
+ *   rope_style           DQ_ROPE_HALF or DQ_ROPE_PAIRS; 0 (with NULL tables) = dq_encode_tokens
+ * Per pair (a, b): (a cos - b sin, b cos + a sin), every product and sum rounded once. */
+int dq_encode_tokens_rope(const dq_tables *tk, const dq_tables *tv, const void *k_bf16,
+                          const void *v_bf16, int T, int Hkv, const int32_t *seq_id,
+                          const int32_t *pos, const int32_t *slot, uint8_t *k_cont, uint8_t *v_cont,
+                          int8_t *k_mean_q, float *k_mean_scale, int max_windows, int mean_mode,
+                          const float *rope_cos, const float *rope_sin, int rope_style,
+                          uint32_t *status, void *cuda_stream);
 
 /* Bytes of scratch dq_decode_attention needs (split-K partials and a work counter). */
 size_t dq_decode_workspace_bytes(int B, int Hq, int max_pages);

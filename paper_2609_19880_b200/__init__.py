@@ -22,7 +22,7 @@ MEAN_REUSE = 1
 ERRORS = {0: "DQ_OK", -1: "DQ_ERR_ARG", -2: "DQ_ERR_INFEASIBLE", -3: "DQ_ERR_UNSUPPORTED",
           -4: "DQ_ERR_WORKSPACE", -5: "DQ_ERR_CUDA"}
 
-EXPORTS = ["dq_build_tables", "dq_free_tables", "dq_tables_info", "dq_encode_tokens",
+EXPORTS = ["dq_build_tables", "dq_free_tables", "dq_tables_info", "dq_encode_tokens", "dq_encode_tokens_rope",
            "dq_decode_workspace_bytes", "dq_decode_attention", "dq_decode_attention_residual",
            "dq_decode_attention_multi",
            "dq_decode_attention_static", "dq_decode_tokens",
@@ -70,6 +70,9 @@ def lib():
         L.dq_tables_info.argtypes = [vp, C.POINTER(TableInfo)]
         L.dq_encode_tokens.restype = i32
         L.dq_encode_tokens.argtypes = [vp, vp, vp, vp, i32, i32, vp, vp, vp, vp, vp, vp, vp, i32, i32, vp, vp]
+        L.dq_encode_tokens_rope.restype = i32
+        L.dq_encode_tokens_rope.argtypes = [vp, vp, vp, vp, i32, i32, vp, vp, vp, vp, vp, vp, vp, i32, i32, vp, vp, i32,
+                                            vp, vp]
         L.dq_decode_workspace_bytes.restype = sz
         L.dq_decode_workspace_bytes.argtypes = [i32, i32, i32]
         L.dq_decode_attention.restype = i32
@@ -156,16 +159,24 @@ def dq_tables_info(t: Tables) -> TableInfo:
     return t.info()
 
 
+ROPE_HALF, ROPE_PAIRS = 1, 2
+
+
 def dq_encode_tokens(tk, tv, k_bf16, v_bf16, seq_id, pos, slot, k_cont, v_cont, k_mean_q=None,
-                     k_mean_scale=None, mean_mode: int = MEAN_COMPUTE, status=None, stream=None):
-    """K/V bf16 [T, Hkv, 128] -> containers (+ window means).  All tensors on the device."""
+                     k_mean_scale=None, mean_mode: int = MEAN_COMPUTE, status=None, stream=None, rope=None):
+    """K/V bf16 [T, Hkv, 128] -> containers (+ window means).  All tensors on the device.
+    rope = (cos f32 [positions, 64], sin, style): keys are given before their rotary embedding."""
     ref = k_bf16 if k_bf16 is not None else v_bf16
     T, Hkv = int(ref.shape[0]), int(ref.shape[1])
     max_windows = int(k_mean_q.shape[1]) if k_mean_q is not None else 0
-    rc = lib().dq_encode_tokens(tk.handle if tk else None, tv.handle if tv else None, _ptr(k_bf16), _ptr(v_bf16),
-                                T, Hkv, _ptr(seq_id), _ptr(pos), _ptr(slot), _ptr(k_cont), _ptr(v_cont),
-                                _ptr(k_mean_q), _ptr(k_mean_scale), max_windows, int(mean_mode), _ptr(status),
-                                _stream(stream))
+    common = (tk.handle if tk else None, tv.handle if tv else None, _ptr(k_bf16), _ptr(v_bf16),
+              T, Hkv, _ptr(seq_id), _ptr(pos), _ptr(slot), _ptr(k_cont), _ptr(v_cont),
+              _ptr(k_mean_q), _ptr(k_mean_scale), max_windows, int(mean_mode))
+    if rope is None:
+        rc = lib().dq_encode_tokens(*common, _ptr(status), _stream(stream))
+    else:
+        cs, sn, style = rope
+        rc = lib().dq_encode_tokens_rope(*common, _ptr(cs), _ptr(sn), int(style), _ptr(status), _stream(stream))
     _check(rc, "dq_encode_tokens")
 
 

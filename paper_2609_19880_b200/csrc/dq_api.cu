@@ -41,11 +41,14 @@ int dq_tables_info(const dq_tables* t, dq_table_info* out) {
     return DQ_OK;
 }
 
-int dq_encode_tokens(const dq_tables* tk, const dq_tables* tv, const void* k_bf16, const void* v_bf16,
-                     int T, int Hkv, const int32_t* seq_id, const int32_t* pos, const int32_t* slot,
-                     uint8_t* k_cont, uint8_t* v_cont, int8_t* k_mean_q, float* k_mean_scale,
-                     int max_windows, int mean_mode, uint32_t* status, void* cuda_stream) {
+int dq_encode_tokens_rope(const dq_tables* tk, const dq_tables* tv, const void* k_bf16, const void* v_bf16,
+                          int T, int Hkv, const int32_t* seq_id, const int32_t* pos, const int32_t* slot,
+                          uint8_t* k_cont, uint8_t* v_cont, int8_t* k_mean_q, float* k_mean_scale,
+                          int max_windows, int mean_mode, const float* rope_cos, const float* rope_sin,
+                          int rope_style, uint32_t* status, void* cuda_stream) {
     if (T < 0 || Hkv <= 0 || (!tk && !tv)) return DQ_ERR_ARG;
+    if (rope_style != 0 && rope_style != DQ_ROPE_HALF && rope_style != DQ_ROPE_PAIRS) return DQ_ERR_ARG;
+    if (rope_style != 0 && (!rope_cos || !rope_sin || !aligned16(rope_cos) || !aligned16(rope_sin))) return DQ_ERR_ARG;
     if (!seq_id || !pos || !slot) return DQ_ERR_ARG;
     if (tk && (!k_bf16 || !k_cont)) return DQ_ERR_ARG;
     if (tv && (!v_bf16 || !v_cont)) return DQ_ERR_ARG;
@@ -67,7 +70,7 @@ int dq_encode_tokens(const dq_tables* tk, const dq_tables* tv, const void* k_bf1
     cudaError_t e;
     if (k_mean && mean_mode == DQ_MEAN_COMPUTE) {
         e = dq_launch_means(tk->dev, k_bf16, T, Hkv, seq_id, pos, k_mean_q, k_mean_scale, max_windows,
-                            mean_mode, st);
+                            mean_mode, rope_cos, rope_sin, rope_style, st);
         if (e != cudaSuccess) return cuda_fail(e, "window means");
     }
     // keys and values go through one launch; in DQ_MEAN_REUSE mode the encoder warp of a
@@ -77,9 +80,18 @@ int dq_encode_tokens(const dq_tables* tk, const dq_tables* tv, const void* k_bf1
     a.k_cont = k_cont; a.v_cont = v_cont; a.mean_q = k_mean_q; a.mean_scale = k_mean_scale;
     a.status = status; a.T = T; a.Hkv = Hkv; a.max_windows = max_windows; a.mean_mode = mean_mode;
     a.do_k = tk ? 1 : 0; a.do_v = tv ? 1 : 0;
+    a.rope_cos = rope_cos; a.rope_sin = rope_sin; a.rope_style = rope_style;
     e = dq_launch_encode(tk ? tk->dev : tv->dev, tv ? tv->dev : tk->dev, a, st);
     if (e != cudaSuccess) return cuda_fail(e, "encode");
     return DQ_OK;
+}
+
+int dq_encode_tokens(const dq_tables* tk, const dq_tables* tv, const void* k_bf16, const void* v_bf16,
+                     int T, int Hkv, const int32_t* seq_id, const int32_t* pos, const int32_t* slot,
+                     uint8_t* k_cont, uint8_t* v_cont, int8_t* k_mean_q, float* k_mean_scale,
+                     int max_windows, int mean_mode, uint32_t* status, void* cuda_stream) {
+    return dq_encode_tokens_rope(tk, tv, k_bf16, v_bf16, T, Hkv, seq_id, pos, slot, k_cont, v_cont, k_mean_q,
+                                 k_mean_scale, max_windows, mean_mode, nullptr, nullptr, 0, status, cuda_stream);
 }
 
 size_t dq_decode_workspace_bytes(int B, int Hq, int max_pages) {

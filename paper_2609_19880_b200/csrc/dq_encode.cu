@@ -17,6 +17,33 @@ constexpr uint32_t kL = 1u << 23;  // lower bound of the rANS state interval
 using dqdev::bf16_bits_to_float;
 using dqdev::warp_fwht128;  // per-head Hadamard rotation (Sec. 4.2), 4 values per lane
 
+// Rotary position embedding of a head vector held 4 values per lane (element 4 lane + e), in
+// binary32 with every product and sum rounded once.  DQ_ROPE_HALF pairs element j with j + 64
+// (the partner sits in lane ^ 16), DQ_ROPE_PAIRS pairs 2j with 2j + 1 (same lane).
+// cs / sn: this position's 64 cosines / sines.
+__device__ __forceinline__ void warp_rope128(float (&v)[4], int lane, const float* cs, const float* sn, int style) {
+    if (style == DQ_ROPE_HALF) {
+        const float4 c = *reinterpret_cast<const float4*>(cs + 4 * (lane & 15));
+        const float4 s = *reinterpret_cast<const float4*>(sn + 4 * (lane & 15));
+        const float cc[4] = {c.x, c.y, c.z, c.w}, ss[4] = {s.x, s.y, s.z, s.w};
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            const float other = __shfl_xor_sync(kFull, v[e], 16);
+            // lanes 0-15 hold a: a cos - b sin; lanes 16-31 hold b: b cos + a sin
+            const float mine = __fmul_rn(v[e], cc[e]), cross = __fmul_rn(other, ss[e]);
+            v[e] = (lane < 16) ? __fsub_rn(mine, cross) : __fadd_rn(mine, cross);
+        }
+    } else {
+        const float2 c = *reinterpret_cast<const float2*>(cs + 2 * lane);
+        const float2 s = *reinterpret_cast<const float2*>(sn + 2 * lane);
+        const float a0 = v[0], b0 = v[1], a1 = v[2], b1 = v[3];
+        v[0] = __fsub_rn(__fmul_rn(a0, c.x), __fmul_rn(b0, s.x));
+        v[1] = __fadd_rn(__fmul_rn(b0, c.x), __fmul_rn(a0, s.x));
+        v[2] = __fsub_rn(__fmul_rn(a1, c.y), __fmul_rn(b1, s.y));
+        v[3] = __fadd_rn(__fmul_rn(b1, c.y), __fmul_rn(a1, s.y));
+    }
+}
+
 // ------------------------------------------------------------------ window means
 
 // DQ_MEAN_COMPUTE.  A run is a maximal range of consecutive call tokens with the same
@@ -26,7 +53,8 @@ using dqdev::warp_fwht128;  // per-head Hadamard rotation (Sec. 4.2), 4 values p
 __global__ void __launch_bounds__(256)
 dq_means_compute_kernel(const uint16_t* __restrict__ k, int T, int Hkv, int rotate,
                         const int32_t* __restrict__ seq_id, const int32_t* __restrict__ pos,
-                        int8_t* __restrict__ mean_q, float* __restrict__ mean_scale, int Wmax) {
+                        int8_t* __restrict__ mean_q, float* __restrict__ mean_scale, int Wmax,
+                        const float* __restrict__ rope_cos, const float* __restrict__ rope_sin, int rope_style) {
     const int lane = threadIdx.x & 31;
     const long long wid = (long long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
     if (wid >= (long long)T * Hkv) return;
@@ -38,10 +66,11 @@ dq_means_compute_kernel(const uint16_t* __restrict__ k, int T, int Hkv, int rota
     for (; t < T; ++t) {
         if (t > t0 && !(seq_id[t] == s && pos[t] / DQ_WINDOW_TOKENS == w)) break;
         const uint2 raw = *reinterpret_cast<const uint2*>(k + ((size_t)t * Hkv + h) * kN + 4 * lane);
-        acc[0] = __fadd_rn(acc[0], bf16_bits_to_float(raw.x & 0xffffu));
-        acc[1] = __fadd_rn(acc[1], bf16_bits_to_float(raw.x >> 16));
-        acc[2] = __fadd_rn(acc[2], bf16_bits_to_float(raw.y & 0xffffu));
-        acc[3] = __fadd_rn(acc[3], bf16_bits_to_float(raw.y >> 16));
+        float kt[4] = {bf16_bits_to_float(raw.x & 0xffffu), bf16_bits_to_float(raw.x >> 16),
+                       bf16_bits_to_float(raw.y & 0xffffu), bf16_bits_to_float(raw.y >> 16)};
+        if (rope_style) warp_rope128(kt, lane, rope_cos + (size_t)pos[t] * 64, rope_sin + (size_t)pos[t] * 64, rope_style);
+#pragma unroll
+        for (int e = 0; e < 4; ++e) acc[e] = __fadd_rn(acc[e], kt[e]);
     }
     const float inv = __fdiv_rn(1.0f, (float)(t - t0));
 #pragma unroll
@@ -209,6 +238,8 @@ dq_encode_kernel(const __grid_constant__ DqDevTable TK, const __grid_constant__ 
         z[0] = bf16_bits_to_float(raw.x & 0xffffu); z[1] = bf16_bits_to_float(raw.x >> 16);
         z[2] = bf16_bits_to_float(raw.y & 0xffffu); z[3] = bf16_bits_to_float(raw.y >> 16);
     }
+    if (!is_v && a.rope_style)
+        warp_rope128(z, lane, a.rope_cos + (size_t)a.pos[t] * 64, a.rope_sin + (size_t)a.pos[t] * 64, a.rope_style);
     if (T.rotate) warp_fwht128(z, lane);
     if (T.has_mean) {  // remove the (dequantised) windowed channel mean, Sec. 4.2
         const int ps = a.pos[t], w = ps / DQ_WINDOW_TOKENS;
@@ -523,6 +554,8 @@ __device__ __forceinline__ WideQuantised wide_quantise(const EncTable& T, WideSh
         z[0] = bf16_bits_to_float(raw.x & 0xffffu); z[1] = bf16_bits_to_float(raw.x >> 16);
         z[2] = bf16_bits_to_float(raw.y & 0xffffu); z[3] = bf16_bits_to_float(raw.y >> 16);
     }
+    if (!is_v && a.rope_style)
+        warp_rope128(z, lane, a.rope_cos + (size_t)a.pos[t] * 64, a.rope_sin + (size_t)a.pos[t] * 64, a.rope_style);
     if (T.rotate) warp_fwht128(z, lane);
     if (T.has_mean) {  // remove the (dequantised) windowed channel mean of this head, Sec. 4.2
         const int ps = a.pos[t], w = ps / DQ_WINDOW_TOKENS;
@@ -740,13 +773,14 @@ dq_encode_wide_batch_kernel(const __grid_constant__ DqDevTable TK, const __grid_
 
 cudaError_t dq_launch_means(const DqDevTable& tk, const void* k_bf16, int T, int Hkv,
                             const int32_t* seq_id, const int32_t* pos, int8_t* mean_q,
-                            float* mean_scale, int max_windows, int mode, cudaStream_t st) {
+                            float* mean_scale, int max_windows, int mode, const float* rope_cos,
+                            const float* rope_sin, int rope_style, cudaStream_t st) {
     const long long warps = (long long)T * Hkv;
     if (warps == 0) return cudaSuccess;
     const unsigned blocks = (unsigned)((warps + 7) / 8);
     if (mode != DQ_MEAN_COMPUTE) return cudaSuccess;  // carry-forward is done by the encoder warps
     dq_means_compute_kernel<<<blocks, 256, 0, st>>>((const uint16_t*)k_bf16, T, Hkv, tk.rotate, seq_id, pos,
-                                                    mean_q, mean_scale, max_windows);
+                                                    mean_q, mean_scale, max_windows, rope_cos, rope_sin, rope_style);
     return cudaGetLastError();
 }
 

@@ -29,7 +29,8 @@ int dq_host_build(int levels, double bits_per_elem, const dq_table_opts* opts, d
 // kernels' host launchers (each returns a cudaError_t from the launch)
 cudaError_t dq_launch_means(const DqDevTable& tk, const void* k_bf16, int T, int Hkv,
                             const int32_t* seq_id, const int32_t* pos, int8_t* mean_q,
-                            float* mean_scale, int max_windows, int mode, cudaStream_t st);
+                            float* mean_scale, int max_windows, int mode, const float* rope_cos,
+                            const float* rope_sin, int rope_style, cudaStream_t st);
 struct DqEncodeArgs {
     const void* k_bf16;
     const void* v_bf16;
@@ -42,6 +43,9 @@ struct DqEncodeArgs {
     float* mean_scale;
     uint32_t* status;
     int T, Hkv, max_windows, mean_mode, do_k, do_v;
+    const float* rope_cos;   // [positions][64], nullable: keys are handed over before their rotary embedding
+    const float* rope_sin;
+    int rope_style;          // 0 none, DQ_ROPE_HALF, DQ_ROPE_PAIRS
 };
 cudaError_t dq_launch_encode(const DqDevTable& tk, const DqDevTable& tv, const DqEncodeArgs& a, cudaStream_t st);
 cudaError_t dq_launch_decode_tokens(const DqDevTable& t, const uint8_t* cont, const int8_t* mean_q,
