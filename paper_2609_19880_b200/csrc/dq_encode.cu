@@ -199,7 +199,10 @@ constexpr int kEncWarps = 8;
 
 // One warp per stream (token, KV head); lane l owns elements 4l .. 4l+3.  blockIdx.y selects
 // the tensor kind when keys and values are encoded by one launch.
-__global__ void __launch_bounds__(kEncWarps * 32)
+// MINB CTAs per SM: 2 leaves every thread 128 registers (lowest latency: the single-token step), 4 trades a
+// few spills for twice the resident warps (throughput: prefill, bulk encodes).
+template <int MINB>
+__global__ void __launch_bounds__(kEncWarps * 32, MINB)
 dq_encode_kernel(const __grid_constant__ DqDevTable TK, const __grid_constant__ DqDevTable TV,
                  const DqEncodeArgs a) {
     __shared__ EncTable T;
@@ -729,7 +732,10 @@ dq_encode_wide_kernel(const __grid_constant__ DqDevTable TK, const __grid_consta
 // entropy-codes whole streams on its own, so the serial rANS chains of kBatch streams run side
 // by side instead of leaving hs - 1 warps idle.
 constexpr int kBatch = 8;
-__global__ void __launch_bounds__(DQ_MAX_STREAM_HEADS * 32, 2)
+#ifndef DQ_ENCW_MINB
+#define DQ_ENCW_MINB 3
+#endif
+__global__ void __launch_bounds__(DQ_MAX_STREAM_HEADS * 32, DQ_ENCW_MINB)
 dq_encode_wide_batch_kernel(const __grid_constant__ DqDevTable TK, const __grid_constant__ DqDevTable TV,
                             const DqEncodeArgs a) {
     __shared__ EncTable T;
@@ -796,5 +802,7 @@ cudaError_t dq_launch_encode(const DqDevTable& tk, const DqDevTable& tv, const D
                              dim3(tk.hs * 32), 0, st, tk, tv, a);
     }
     const unsigned blocks = (unsigned)((warps + kEncWarps - 1) / kEncWarps);
-    return dq_launch_pdl(dq_encode_kernel, dim3(blocks, (a.do_k && a.do_v) ? 2 : 1), dim3(kEncWarps * 32), 0, st, tk, tv, a);
+    if (warps >= 4LL * 148 * kEncWarps * 4)   // enough streams to fill the GPU at 4 CTAs per SM several times
+        return dq_launch_pdl(dq_encode_kernel<4>, dim3(blocks, (a.do_k && a.do_v) ? 2 : 1), dim3(kEncWarps * 32), 0, st, tk, tv, a);
+    return dq_launch_pdl(dq_encode_kernel<2>, dim3(blocks, (a.do_k && a.do_v) ? 2 : 1), dim3(kEncWarps * 32), 0, st, tk, tv, a);
 }
