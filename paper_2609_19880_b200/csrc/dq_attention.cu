@@ -43,7 +43,7 @@ struct Item {
 
 struct Layout {
     int stage_k, stage_v;               // bytes of one warp's K (+ tail) / V record buffer
-    int off_lutk, off_lutv, off_prefix, off_q16, off_qsum, off_red, off_pages, off_kst, off_vst, off_tiles,
+    int off_lutk, off_lutv, off_prefix, off_q16, off_qsum, off_red, off_pages, off_items, off_kst, off_vst, off_tiles,
         off_obuf, total;
     int warp_tile_bytes, warp_obuf_bytes;
 };
@@ -65,6 +65,7 @@ __host__ __device__ inline Layout make_layout(int nw, int rec_k, int rec_v, int 
     L.off_qsum = o; o += 2 * DQ_MAX_GROUP * 4;
     L.off_red = o; o += (kMaxWarps + 2) * DQ_MAX_GROUP * 4;
     L.off_pages = o; o += kMaxWarps * 3 * 2 * 4 + 16;   // per warp: page ids of 3 items in flight; prev row
+    L.off_items = o; o += 4 * 32;                       // descriptors of the items n .. n + 3 of this CTA
     L.off_tiles = o; o += nw * L.warp_tile_bytes;
     L.off_obuf = o; o += nw * L.warp_obuf_bytes;
     L.off_kst = o; o += 2 * nw * L.stage_k;
@@ -287,10 +288,11 @@ dq_attention_kernel(const __grid_constant__ DqDevTable TK, const __grid_constant
     const uint32_t one = (sbase >> 31) | 1u;
     const int g_row = lane >> 2, qd = lane & 3;
 
-    // Items are dealt round-robin to the CTAs; every thread derives the descriptor itself from
-    // the tables in shared memory, so no broadcast or global atomic sits on the critical path.
-    // (Item indices of one CTA grow with n, so the sequence is found by walking forward from `hint`,
-    // the sequence of an earlier item.)
+    // Items are dealt round-robin to the CTAs.  Thread 0 derives the descriptor of item n + 3 while the
+    // CTA works on item n and leaves it in a ring of four in shared memory; everybody else reads the
+    // descriptors it needs (n, n + 1, n + 2) after the next CTA barrier, so neither a global atomic nor
+    // the search sits on the critical path.  (Item indices of one CTA grow with n, so the sequence is
+    // found by walking forward from `hint`, the sequence of an earlier item.)
     auto item_of = [&](int n, int hint) {
         Item it;
         it.valid = 0; it.b = hint; it.h = it.blk = it.len = it.bg = 0; it.pad0 = it.pad1 = 0;
@@ -353,19 +355,27 @@ dq_attention_kernel(const __grid_constant__ DqDevTable TK, const __grid_constant
         }
     };
 
+    Item* s_items = reinterpret_cast<Item*>(smem + L.off_items);
+    int hint = 0;   // thread 0: sequence of the newest descriptor, the search start for the next one
+    if (tid == 0) {
+        for (int n = 0; n < 3; ++n) {
+            const Item it = item_of(n, hint);
+            s_items[n] = it;
+            hint = it.b;
+        }
+    }
+    __syncthreads();
     // prologue: page ids of items 0 and 1, then the K records of item 0
-    int hint = 0;   // sequence of the current item: search start for later items
     {
-        const Item i0 = item_of(0, 0);
+        const Item i0 = s_items[0];
         fetch_pages(0, i0);
-        fetch_pages(1, item_of(1, i0.b));
+        fetch_pages(1, s_items[1]);
         cp_async_commit();
         cp_async_wait<0>();
         __syncwarp();
         Item none = i0; none.valid = 0;
         issue_loads(0, i0, 0, none);
         cp_async_commit();
-        hint = i0.b;
     }
 
     // state carried from the item whose V streams are still to be decoded
@@ -373,17 +383,20 @@ dq_attention_kernel(const __grid_constant__ DqDevTable TK, const __grid_constant
     uint32_t pb_hi[2][2] = {{0u, 0u}, {0u, 0u}}, pb_lo[2][2] = {{0u, 0u}, {0u, 0u}};
 
     for (int n = 0;; ++n) {
-        Item cur = item_of(n, hint);
+        Item cur = s_items[n & 3];
         if (!cur.valid && !have_prev) break;
-        hint = cur.b;
         {   // records of item n + 1 (its page ids arrived last iteration), page ids of item n + 2
-            const Item nxt = item_of(n + 1, cur.b);
-            issue_loads(n + 1, nxt, n, cur);
-            fetch_pages(n + 2, item_of(n + 2, nxt.b));
+            issue_loads(n + 1, s_items[(n + 1) & 3], n, cur);
+            fetch_pages(n + 2, s_items[(n + 2) & 3]);
             cp_async_commit();
         }
         cp_async_wait<1>();
         __syncthreads();   // q' operand of `cur` visible; last iteration's merge reads are done
+        if (tid == 0) {    // slot of item n - 1, which nobody reads any more
+            const Item it = item_of(n + 3, hint);
+            s_items[(n + 3) & 3] = it;
+            hint = it.b;
+        }
 
         // ------------------------------------------ K streams of `cur`, V streams of `prev`
         int tok0 = (cur.blk * nw + warp) * kChunk;
@@ -409,7 +422,7 @@ dq_attention_kernel(const __grid_constant__ DqDevTable TK, const __grid_constant
         }
 
         // ------------------------------------------ logits of `cur` and this warp's maximum (base 2)
-        cur = item_of(n, hint);   // derived again rather than kept in registers across the pass
+        cur = s_items[n & 3];   // read again rather than kept in registers across the pass
         tok0 = (cur.blk * nw + warp) * kChunk;
         kst = sbase + L.off_kst + ((n & 1) * nw + warp) * L.stage_k;
         rk = kst + lane * TK.rec;
