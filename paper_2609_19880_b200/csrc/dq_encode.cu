@@ -197,44 +197,18 @@ __device__ __forceinline__ uint32_t drift(const EncTable& T, const float (&z)[4]
 
 constexpr int kEncWarps = 8;
 
-// One warp per stream (token, KV head); lane l owns elements 4l .. 4l+3.  blockIdx.y selects
-// the tensor kind when keys and values are encoded by one launch.
-// MINB CTAs per SM: 2 leaves every thread 128 registers (lowest latency: the single-token step), 4 trades a
-// few spills for twice the resident warps (throughput: prefill, bulk encodes).
-template <int MINB>
-__global__ void __launch_bounds__(kEncWarps * 32, MINB)
-dq_encode_kernel(const __grid_constant__ DqDevTable TK, const __grid_constant__ DqDevTable TV,
-                 const DqEncodeArgs a) {
-    __shared__ EncTable T;
-    __shared__ uint8_t s_bytes[kEncWarps][DQ_MAX_REC_BYTES];
-    __shared__ __align__(4) uint8_t s_sym[kEncWarps][kN];
-    dqdev::pdl_launch_dependents();
-    const bool is_v = a.do_k ? (blockIdx.y == 1) : true;
-    if (threadIdx.x < DQ_MAX_LEVELS) {
-        const int i = threadIdx.x;
-        T.r[i] = is_v ? TV.r[i] : TK.r[i];
-        T.R[i] = is_v ? TV.R[i] : TK.R[i];
-        T.rcp[i] = is_v ? TV.enc_rcp[i] : TK.enc_rcp[i];
-        const uint32_t aux = is_v ? TV.enc_aux[i] : TK.enc_aux[i];
-        T.bias[i] = aux & 1023u;
-        T.cmpl[i] = (aux >> 10) & 511u;
-        T.rsh[i] = aux >> 19;
-        T.thr[i] = (256u - ((aux >> 10) & 511u)) << 23;
-    }
-    if (threadIdx.x == 0) {
-        T.M = is_v ? TV.M : TK.M; T.rec = is_v ? TV.rec : TK.rec; T.mstar = is_v ? TV.mstar : TK.mstar;
-        T.budget_bits = is_v ? TV.budget_bits : TK.budget_bits;
-        T.has_mean = is_v ? TV.has_mean : TK.has_mean; T.rotate = is_v ? TV.rotate : TK.rotate;
-    }
-    __syncthreads();
-    dqdev::pdl_wait_prior_grid();   // inputs and the cache may be written / read by the previous kernel
-    const int lane = threadIdx.x & 31, wib = threadIdx.x >> 5;
-    const long long wid = (long long)blockIdx.x * kEncWarps + wib;
-    if (wid >= (long long)a.T * a.Hkv) return;
-    const int t = (int)(wid / a.Hkv), h = (int)(wid % a.Hkv), Hkv = a.Hkv;
-    const uint16_t* x = static_cast<const uint16_t*>(is_v ? a.v_bf16 : a.k_bf16);
-    uint8_t* cont = is_v ? a.v_cont : a.k_cont;
+struct StreamQuantised {
+    uint32_t hdr0;      // s fp16 | o fp16 << 16
+    uint32_t flags;     // 1: all-central fallback, 2: constant stream, 4: refit rejected
+    uint32_t sym;       // this lane's four symbols, one per byte
+};
 
+// Steps 1-6 of Algorithm 1 for the stream (token t, KV head h) by one warp: rotation (and rotary
+// embedding when asked), mean removal, min-max grid, drift, refit, fp16 metadata, second drift.
+__device__ __forceinline__ StreamQuantised quantise_stream(const EncTable& T, const DqEncodeArgs& a, bool is_v, int t, int h,
+                                                           int lane) {
+    const int Hkv = a.Hkv;
+    const uint16_t* x = static_cast<const uint16_t*>(is_v ? a.v_bf16 : a.k_bf16);
     float z[4];
     {
         const uint2 raw = *reinterpret_cast<const uint2*>(x + ((size_t)t * Hkv + h) * kN + 4 * lane);
@@ -334,9 +308,54 @@ dq_encode_kernel(const __grid_constant__ DqDevTable TK, const __grid_constant__ 
         for (int e = 0; e < 4; ++e) sym[e] = (uint32_t)T.mstar;
     }
 
+    StreamQuantised r;
+    r.hdr0 = (uint32_t)__half_as_ushort(s16) | ((uint32_t)__half_as_ushort(o16) << 16);
+    r.flags = st_fallback | (degenerate ? 2u : 0u) | (st_refit << 2);
+    r.sym = sym[0] | (sym[1] << 8) | (sym[2] << 16) | (sym[3] << 24);
+    return r;
+}
+
+// One warp per stream (token, KV head); lane l owns elements 4l .. 4l+3.  blockIdx.y selects
+// the tensor kind when keys and values are encoded by one launch.
+// MINB CTAs per SM: 2 leaves every thread 128 registers (lowest latency: the single-token step), 4 trades a
+// few spills for twice the resident warps (throughput: prefill, bulk encodes).
+template <int MINB>
+__global__ void __launch_bounds__(kEncWarps * 32, MINB)
+dq_encode_kernel(const __grid_constant__ DqDevTable TK, const __grid_constant__ DqDevTable TV,
+                 const DqEncodeArgs a) {
+    __shared__ EncTable T;
+    __shared__ uint8_t s_bytes[kEncWarps][DQ_MAX_REC_BYTES];
+    __shared__ __align__(4) uint8_t s_sym[kEncWarps][kN];
+    dqdev::pdl_launch_dependents();
+    const bool is_v = a.do_k ? (blockIdx.y == 1) : true;
+    if (threadIdx.x < DQ_MAX_LEVELS) {
+        const int i = threadIdx.x;
+        T.r[i] = is_v ? TV.r[i] : TK.r[i];
+        T.R[i] = is_v ? TV.R[i] : TK.R[i];
+        T.rcp[i] = is_v ? TV.enc_rcp[i] : TK.enc_rcp[i];
+        const uint32_t aux = is_v ? TV.enc_aux[i] : TK.enc_aux[i];
+        T.bias[i] = aux & 1023u;
+        T.cmpl[i] = (aux >> 10) & 511u;
+        T.rsh[i] = aux >> 19;
+        T.thr[i] = (256u - ((aux >> 10) & 511u)) << 23;
+    }
+    if (threadIdx.x == 0) {
+        T.M = is_v ? TV.M : TK.M; T.rec = is_v ? TV.rec : TK.rec; T.mstar = is_v ? TV.mstar : TK.mstar;
+        T.budget_bits = is_v ? TV.budget_bits : TK.budget_bits;
+        T.has_mean = is_v ? TV.has_mean : TK.has_mean; T.rotate = is_v ? TV.rotate : TK.rotate;
+    }
+    __syncthreads();
+    dqdev::pdl_wait_prior_grid();   // inputs and the cache may be written / read by the previous kernel
+    const int lane = threadIdx.x & 31, wib = threadIdx.x >> 5;
+    const long long wid = (long long)blockIdx.x * kEncWarps + wib;
+    if (wid >= (long long)a.T * a.Hkv) return;
+    const int t = (int)(wid / a.Hkv), h = (int)(wid % a.Hkv), Hkv = a.Hkv;
+    uint8_t* cont = is_v ? a.v_cont : a.k_cont;
+
+    const StreamQuantised sq = quantise_stream(T, a, is_v, t, h, lane);
     // rANS, Eq. (rans) Enc on symbols 127 .. 0 so that decoding runs forward.  Every lane
     // carries the same state (the symbols come from shared memory); lane 0 records the bytes.
-    *reinterpret_cast<uint32_t*>(&s_sym[wib][4 * lane]) = sym[0] | (sym[1] << 8) | (sym[2] << 16) | (sym[3] << 24);
+    *reinterpret_cast<uint32_t*>(&s_sym[wib][4 * lane]) = sq.sym;
     __syncwarp();
     uint32_t xs = kL;
     int k = 0;
@@ -356,7 +375,7 @@ dq_encode_kernel(const __grid_constant__ DqDevTable TK, const __grid_constant__ 
     }
     __syncwarp();
     asm volatile("" ::: "memory");
-    const uint32_t hdr0 = (uint32_t)__half_as_ushort(s16) | ((uint32_t)__half_as_ushort(o16) << 16);
+    const uint32_t hdr0 = sq.hdr0;
     const int sl = a.slot[t];
     uint8_t* rec = cont + (((size_t)(sl / DQ_PAGE_TOKENS) * Hkv + h) * DQ_PAGE_TOKENS +
                            (size_t)(sl % DQ_PAGE_TOKENS)) * T.rec;
@@ -369,13 +388,108 @@ dq_encode_kernel(const __grid_constant__ DqDevTable TK, const __grid_constant__ 
         rec[i] = v;
     }
     if (a.status && lane == 0) {
-        if (st_fallback) atomicAdd(a.status + 0, 1u);
-        if (degenerate) atomicAdd(a.status + 1, 1u);
-        if (st_refit) atomicAdd(a.status + 2, 1u);
+        if (sq.flags & 1u) atomicAdd(a.status + 0, 1u);
+        if (sq.flags & 2u) atomicAdd(a.status + 1, 1u);
+        if (sq.flags & 4u) atomicAdd(a.status + 2, 1u);
         atomicMax(a.status + 3, (uint32_t)(8 + k));
     }
 }
 
+
+// Throughput variant for calls with many streams: a CTA of 8 warps takes 32 consecutive streams.
+// Each warp quantises 4 of them (steps 1-6 of Algorithm 1, as above) and leaves the symbols in
+// shared memory; then ONE warp entropy-codes all 32 streams at once, lane = stream, so the serial
+// rANS chain costs one instruction stream per 32 streams instead of one per stream with 32
+// redundant lanes.  Symbols are stored [position][stream] and emitted bytes [byte index][stream] so
+// that the lanes of that warp touch consecutive bytes.
+#ifndef DQ_B32_MINB
+#define DQ_B32_MINB 4
+#endif
+constexpr int kB32 = 32;                 // streams per CTA
+constexpr int kB32SymStride = 36;        // bytes per position row (32 streams + pad against bank conflicts)
+template <int MINB>
+__global__ void __launch_bounds__(kEncWarps * 32, MINB)
+dq_encode_batch32_kernel(const __grid_constant__ DqDevTable TK, const __grid_constant__ DqDevTable TV,
+                         const DqEncodeArgs a) {
+    __shared__ EncTable T;
+    __shared__ __align__(4) uint8_t s_symT[kN * kB32SymStride];
+    __shared__ uint8_t s_bytesT[DQ_MAX_REC_BYTES * kB32];
+    __shared__ uint32_t s_hdr[kB32], s_xs[kB32], s_k[kB32];
+    __shared__ unsigned long long s_rec[kB32];   // record addresses
+    dqdev::pdl_launch_dependents();
+    const bool is_v = a.do_k ? (blockIdx.y == 1) : true;
+    if (threadIdx.x < DQ_MAX_LEVELS) {
+        const int i = threadIdx.x;
+        T.r[i] = is_v ? TV.r[i] : TK.r[i];
+        T.R[i] = is_v ? TV.R[i] : TK.R[i];
+        T.rcp[i] = is_v ? TV.enc_rcp[i] : TK.enc_rcp[i];
+        const uint32_t aux = is_v ? TV.enc_aux[i] : TK.enc_aux[i];
+        T.bias[i] = aux & 1023u;
+        T.cmpl[i] = (aux >> 10) & 511u;
+        T.rsh[i] = aux >> 19;
+        T.thr[i] = (256u - ((aux >> 10) & 511u)) << 23;
+    }
+    if (threadIdx.x == 0) {
+        T.M = is_v ? TV.M : TK.M; T.rec = is_v ? TV.rec : TK.rec; T.mstar = is_v ? TV.mstar : TK.mstar;
+        T.budget_bits = is_v ? TV.budget_bits : TK.budget_bits;
+        T.has_mean = is_v ? TV.has_mean : TK.has_mean; T.rotate = is_v ? TV.rotate : TK.rotate;
+    }
+    __syncthreads();
+    dqdev::pdl_wait_prior_grid();
+    const int lane = threadIdx.x & 31, wib = threadIdx.x >> 5;
+    const long long total = (long long)a.T * a.Hkv;
+    const long long first = (long long)blockIdx.x * kB32;
+    const int ns = (int)min((long long)kB32, total - first);
+    uint8_t* cont = is_v ? a.v_cont : a.k_cont;
+
+    for (int i = wib; i < ns; i += kEncWarps) {   // quantise: warp w takes streams w, w + 8, ...
+        const long long wid = first + i;
+        const int t = (int)(wid / a.Hkv), h = (int)(wid % a.Hkv);
+        const StreamQuantised sq = quantise_stream(T, a, is_v, t, h, lane);
+#pragma unroll
+        for (int e = 0; e < 4; ++e) s_symT[(4 * lane + e) * kB32SymStride + i] = (uint8_t)(sq.sym >> (8 * e));
+        if (lane == 0) {
+            s_hdr[i] = sq.hdr0;
+            const int sl = a.slot[t];
+            s_rec[i] = (unsigned long long)(cont + (((size_t)(sl / DQ_PAGE_TOKENS) * a.Hkv + h) * DQ_PAGE_TOKENS +
+                                                    (size_t)(sl % DQ_PAGE_TOKENS)) * T.rec);
+            if (a.status) {
+                if (sq.flags & 1u) atomicAdd(a.status + 0, 1u);
+                if (sq.flags & 2u) atomicAdd(a.status + 1, 1u);
+                if (sq.flags & 4u) atomicAdd(a.status + 2, 1u);
+            }
+        }
+    }
+    __syncthreads();
+    if (wib == 0 && lane < ns) {   // rANS, Eq. (rans) Enc on symbols 127 .. 0; lane = stream
+        uint32_t xs = kL, k = 0;
+#pragma unroll 4
+        for (int j = kN - 1; j >= 0; --j) {
+            const uint32_t m = s_symT[j * kB32SymStride + lane];
+            const uint32_t rcp = T.rcp[m], rsh = T.rsh[m], bias = T.bias[m], cmpl = T.cmpl[m], thr = T.thr[m];
+            if (xs >= thr) {   // at most once: xs < 2^31 <= 2^8 * (f << 23)
+                if (k < DQ_MAX_REC_BYTES) s_bytesT[k * kB32 + lane] = (uint8_t)xs;   // the budget test keeps k < rec - 8
+                ++k;
+                xs >>= 8;
+            }
+            xs = (__umulhi(xs, rcp) >> rsh) * cmpl + (xs + bias);
+        }
+        s_xs[lane] = xs;
+        s_k[lane] = k;
+        if (a.status) atomicMax(a.status + 3, 8u + k);
+    }
+    __syncthreads();
+    const int rec = T.rec;
+    for (int idx = threadIdx.x; idx < ns * rec; idx += blockDim.x) {   // records out: 8 + k bytes, then zeros
+        const int si = idx / rec, i = idx - si * rec;
+        const int k = (int)s_k[si], used = min(8 + k, rec);
+        uint8_t v = 0;
+        if (i < 4) v = (uint8_t)(s_hdr[si] >> (8 * i));
+        else if (i < 8) v = (uint8_t)(s_xs[si] >> (8 * (i - 4)));
+        else if (i < used) v = s_bytesT[(k - 1 - (i - 8)) * kB32 + si];   // emitted last = read first
+        reinterpret_cast<uint8_t*>(s_rec[si])[i] = v;
+    }
+}
 
 // rANS encode of one stream by one warp (Eq. rans Enc on symbols n-1 .. 0 so that decoding runs
 // forward).  Every lane carries the same state; lane 0 records the emitted bytes (in emission
@@ -546,7 +660,8 @@ struct WideQuantised {
 // 128 w + 4 l + e): rotation, mean removal, min-max grid, drift, refit, fp16 metadata, second
 // drift.  The final symbols go to s_sym (visible to the whole CTA on return).
 __device__ __forceinline__ WideQuantised wide_quantise(const EncTable& T, WideShared& W, const DqEncodeArgs& a,
-                                                       bool is_v, int t, int grp, uint8_t* s_sym, uint32_t& parity) {
+                                                       bool is_v, int t, int grp, uint8_t* s_sym, int sym_stride,
+                                                       uint32_t& parity) {
     const int lane = threadIdx.x & 31, wib = threadIdx.x >> 5;
     const int hs = blockDim.x >> 5, Hkv = a.Hkv, h = grp * hs + wib;
     const int n = hs * kN;
@@ -663,7 +778,9 @@ __device__ __forceinline__ WideQuantised wide_quantise(const EncTable& T, WideSh
         for (int e = 0; e < 4; ++e) sym[e] = (uint32_t)T.mstar;
         flags |= 2u;
     }
-    *reinterpret_cast<uint32_t*>(&s_sym[wib * kN + 4 * lane]) = sym[0] | (sym[1] << 8) | (sym[2] << 16) | (sym[3] << 24);
+    // symbol of stream position j goes to s_sym[j * sym_stride]
+#pragma unroll
+    for (int e = 0; e < 4; ++e) s_sym[(wib * kN + 4 * lane + e) * sym_stride] = (uint8_t)sym[e];
     __syncthreads();
     WideQuantised r;
     r.hdr0 = (uint32_t)__half_as_ushort(s16) | ((uint32_t)__half_as_ushort(o16) << 16);
@@ -714,7 +831,7 @@ dq_encode_wide_kernel(const __grid_constant__ DqDevTable TK, const __grid_consta
     const int hs = blockDim.x >> 5, groups = a.Hkv / hs;
     const int t = (int)(blockIdx.x / groups), grp = (int)(blockIdx.x % groups);
     uint32_t parity = 0;
-    const WideQuantised q = wide_quantise(T, W, a, is_v, t, grp, s_sym, parity);
+    const WideQuantised q = wide_quantise(T, W, a, is_v, t, grp, s_sym, 1, parity);
     if (wib == 0) {
         uint32_t xs;
         int k;
@@ -728,49 +845,75 @@ dq_encode_wide_kernel(const __grid_constant__ DqDevTable TK, const __grid_consta
 }
 
 // Throughput variant for calls with many streams (prefill, a window's bulk encode): a CTA takes
-// kBatch consecutive streams; its hs warps quantise them one after the other, then every warp
-// entropy-codes whole streams on its own, so the serial rANS chains of kBatch streams run side
-// by side instead of leaving hs - 1 warps idle.
-constexpr int kBatch = 8;
+// 32 consecutive streams; its hs warps quantise them one after the other, then one warp
+// entropy-codes all 32 at once, lane = stream (symbols stored [position][stream], emitted bytes
+// [byte index][stream]), so the serial rANS chain is paid once per 32 streams.
+constexpr int kWB = 32;              // streams per CTA
+constexpr int kWBSymStride = 36;     // bytes per position row
+__host__ __device__ inline int wide_batch_smem(int hs, int rec) { return hs * kN * kWBSymStride + ((rec + 3) & ~3) * kWB; }
+
 #ifndef DQ_ENCW_MINB
 #define DQ_ENCW_MINB 3
 #endif
 __global__ void __launch_bounds__(DQ_MAX_STREAM_HEADS * 32, DQ_ENCW_MINB)
 dq_encode_wide_batch_kernel(const __grid_constant__ DqDevTable TK, const __grid_constant__ DqDevTable TV,
                             const DqEncodeArgs a) {
+    extern __shared__ __align__(16) uint8_t dyn[];
     __shared__ EncTable T;
     __shared__ __align__(16) WideShared W;
-    __shared__ uint8_t s_bytes[kBatch][DQ_MAX_WIDE_REC_BYTES];
-    __shared__ __align__(4) uint8_t s_sym[kBatch][DQ_MAX_STREAM_HEADS * kN];
-    __shared__ uint32_t s_hdr[kBatch], s_flags[kBatch], s_xs[kBatch], s_k[kBatch];
+    __shared__ uint32_t s_hdr[kWB], s_flags[kWB], s_xs[kWB], s_k[kWB];
     dqdev::pdl_launch_dependents();
     const bool is_v = a.do_k ? (blockIdx.y == 1) : true;
     load_wide_table(T, W, TK, TV, is_v);
     __syncthreads();
     dqdev::pdl_wait_prior_grid();
     const int lane = threadIdx.x & 31, wib = threadIdx.x >> 5;
-    const int hs = blockDim.x >> 5, groups = a.Hkv / hs;
+    const int hs = blockDim.x >> 5, groups = a.Hkv / hs, n = hs * kN;
+    uint8_t* s_symT = dyn;                                   // [n][kWBSymStride]
+    uint8_t* s_bytesT = dyn + n * kWBSymStride;              // [rec][kWB]
+    const int cap = (T.rec + 3) & ~3;
     const long long total = (long long)a.T * groups;
-    const long long first = (long long)blockIdx.x * kBatch;
-    const int ns = (int)min((long long)kBatch, total - first);
+    const long long first = (long long)blockIdx.x * kWB;
+    const int ns = (int)min((long long)kWB, total - first);
     uint32_t parity = 0;
     for (int i = 0; i < ns; ++i) {
         const long long sid = first + i;
-        const WideQuantised q = wide_quantise(T, W, a, is_v, (int)(sid / groups), (int)(sid % groups), s_sym[i], parity);
+        const WideQuantised q = wide_quantise(T, W, a, is_v, (int)(sid / groups), (int)(sid % groups), s_symT + i,
+                                              kWBSymStride, parity);
         if (threadIdx.x == 0) { s_hdr[i] = q.hdr0; s_flags[i] = q.flags; }
     }
-    for (int i = wib; i < ns; i += hs) {
-        uint32_t xs;
-        int k;
-        rans_encode_warp(W.ent, s_sym[i], hs * kN, dqdev::smem_addr(s_bytes[i]), DQ_MAX_WIDE_REC_BYTES, lane, xs, k);
-        if (lane == 0) { s_xs[i] = xs; s_k[i] = (uint32_t)k; }
+    if (wib == 0 && lane < ns) {   // rANS, Eq. (rans) Enc on symbols n-1 .. 0; lane = stream
+        uint32_t xs = kL, k = 0;
+#pragma unroll 4
+        for (int j = n - 1; j >= 0; --j) {
+            const uint32_t m = s_symT[j * kWBSymStride + lane];
+            const uint2 e = W.ent[m];
+            const uint32_t cmpl = (e.y >> 10) & 511u;
+            if (xs >= ((256u - cmpl) << 23)) {   // at most once: xs < 2^31 <= 2^8 * (f << 23)
+                if ((int)k < cap) s_bytesT[k * kWB + lane] = (uint8_t)xs;   // the budget test keeps k < rec - 8
+                ++k;
+                xs >>= 8;
+            }
+            xs = (__umulhi(xs, e.x) >> (e.y >> 19)) * cmpl + (xs + (e.y & 1023u));
+        }
+        s_xs[lane] = xs;
+        s_k[lane] = k;
     }
     __syncthreads();
-    asm volatile("" ::: "memory");
-    for (int i = 0; i < ns; ++i) {
-        const long long sid = first + i;
-        write_wide_record(is_v ? a.v_cont : a.k_cont, groups, (int)(sid % groups), T.rec, a.slot[(int)(sid / groups)], s_hdr[i],
-                          s_xs[i], (int)s_k[i], s_bytes[i]);
+    const int rec = T.rec, rec_words = (rec + 3) >> 2;
+    uint8_t* cont = is_v ? a.v_cont : a.k_cont;
+    for (int idx = threadIdx.x; idx < ns * rec_words * 4; idx += blockDim.x) {
+        const int si = idx / (rec_words * 4), i = idx - si * rec_words * 4;
+        const long long sid = first + si;
+        const int sl = a.slot[(int)(sid / groups)], grp = (int)(sid % groups);
+        const int k = (int)s_k[si], used = min(8 + k, rec);
+        uint8_t v = 0;
+        if (i < 4) v = (uint8_t)(s_hdr[si] >> (8 * i));
+        else if (i < 8) v = (uint8_t)(s_xs[si] >> (8 * (i - 4)));
+        else if (i < used) v = s_bytesT[(k - 1 - (i - 8)) * kWB + si];   // emitted last = read first
+        uint8_t* blk = cont + ((size_t)(sl / DQ_PAGE_TOKENS) * groups + grp) * ((size_t)rec_words * 64) +
+                       (size_t)(sl % DQ_PAGE_TOKENS) * 4;
+        blk[(size_t)(i >> 2) * 64 + (i & 3)] = v;
     }
     if (threadIdx.x < ns) add_status(a.status, s_flags[threadIdx.x], (int)s_k[threadIdx.x]);
 }
@@ -793,16 +936,20 @@ cudaError_t dq_launch_means(const DqDevTable& tk, const void* k_bf16, int T, int
 cudaError_t dq_launch_encode(const DqDevTable& tk, const DqDevTable& tv, const DqEncodeArgs& a, cudaStream_t st) {
     const long long warps = (long long)a.T * a.Hkv;
     if (warps == 0 || (!a.do_k && !a.do_v)) return cudaSuccess;
-    if (tk.hs > 1) {   // token-wide streams: CTAs of hs warps; few streams: one per CTA, many: kBatch per CTA
+    if (tk.hs > 1) {   // token-wide streams: CTAs of hs warps; few streams: one per CTA, many: 32 per CTA
         const long long streams = warps / tk.hs;
         const dim3 kinds_y(1, (a.do_k && a.do_v) ? 2 : 1);
-        if (streams < 4LL * 148 * kBatch)
+        if (streams < 3LL * 148 * kWB)
             return dq_launch_pdl(dq_encode_wide_kernel, dim3((unsigned)streams, kinds_y.y), dim3(tk.hs * 32), 0, st, tk, tv, a);
-        return dq_launch_pdl(dq_encode_wide_batch_kernel, dim3((unsigned)((streams + kBatch - 1) / kBatch), kinds_y.y),
-                             dim3(tk.hs * 32), 0, st, tk, tv, a);
+        const int smem = wide_batch_smem(tk.hs, tk.rec > tv.rec ? tk.rec : tv.rec);
+        const cudaError_t e = cudaFuncSetAttribute(dq_encode_wide_batch_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+        if (e != cudaSuccess) return e;
+        return dq_launch_pdl(dq_encode_wide_batch_kernel, dim3((unsigned)((streams + kWB - 1) / kWB), kinds_y.y),
+                             dim3(tk.hs * 32), (size_t)smem, st, tk, tv, a);
     }
     const unsigned blocks = (unsigned)((warps + kEncWarps - 1) / kEncWarps);
-    if (warps >= 4LL * 148 * kEncWarps * 4)   // enough streams to fill the GPU at 4 CTAs per SM several times
-        return dq_launch_pdl(dq_encode_kernel<4>, dim3(blocks, (a.do_k && a.do_v) ? 2 : 1), dim3(kEncWarps * 32), 0, st, tk, tv, a);
+    if (warps >= 4LL * 148 * kB32 * 4)   // enough streams to fill the GPU at 4 CTAs per SM several times
+        return dq_launch_pdl(dq_encode_batch32_kernel<DQ_B32_MINB>, dim3((unsigned)((warps + kB32 - 1) / kB32), (a.do_k && a.do_v) ? 2 : 1),
+                             dim3(kEncWarps * 32), 0, st, tk, tv, a);
     return dq_launch_pdl(dq_encode_kernel<2>, dim3(blocks, (a.do_k && a.do_v) ? 2 : 1), dim3(kEncWarps * 32), 0, st, tk, tv, a);
 }
