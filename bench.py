@@ -297,25 +297,23 @@ def run_ours(args):
         # stays at its configured length) and the window restarts.
         rk = torch.zeros((B, 128, Hkv, 128), dtype=torch.bfloat16, device=dev)
         rv = torch.zeros_like(rk)
-        rl = [torch.full((B,), r, dtype=torch.int32, device=dev) for r in range(129)]
+        rl = torch.zeros(B, dtype=torch.int32, device=dev)     # tokens in the window, kept on the device
         win_idx = torch.cat([torch.arange(int(e) - 128, int(e)) for e in torch.cumsum(lens, 0)]).to(dev)
         win_seq, win_pos, win_slot = (t[win_idx].contiguous() for t in (w.seq_id, w.pos, w.slot))
 
         def step(i, q=w.q, nk=new_k, nv=new_v):
             c = caches[i % copies]
-            r = state["r"]
-            rk[:, r].copy_(nk)
-            rv[:, r].copy_(nv)
-            r += 1
+            dq.dq_window_append(nk, nv, rk, rv, rl)
+            state["r"] += 1
             dq.dq_decode_attention_residual(tk, tv, q, c["k"], c["v"], c["mq"], c["ms"], w.page_table, w.seq_lens,
-                                            rk, rv, rl[r], Hkv, sm_scale, out, ws)
-            if r == 128:
+                                            rk, rv, rl, Hkv, sm_scale, out, ws)
+            if state["r"] == 128:
                 dq.dq_encode_tokens(tk, tv, rk.view(B * 128, Hkv, 128), rv.view(B * 128, Hkv, 128), win_seq, win_pos,
                                     win_slot, c["k"], c["v"], c["mq"], c["ms"], dq.MEAN_COMPUTE)
+                rl.zero_()
                 state["closes"] += 1
-                r = 0
-            state["r"] = r
-        launches_per_step = 3 + 3.0 / 128   # prepare, fused attention, combine; means + K/V encode per 128 steps
+                state["r"] = 0
+        launches_per_step = 4 + 3.0 / 128   # window append, prepare, fused attention, combine; means + K/V encode per 128 steps
         step_desc = ("append the new token to a 128-token BF16 window + decode attention over the compressed cache "
                      "and the window; a full window is encoded in bulk (once per 128 steps)")
 

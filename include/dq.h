@@ -192,6 +192,16 @@ int dq_decode_attention_residual(const dq_tables *tk, const dq_tables *tv, const
                                  int Hq, int Hkv, float sm_scale, void *out_bf16, float *out_f32,
                                  void *workspace, size_t workspace_bytes, void *cuda_stream);
 
+/* Appends one new token per sequence to the BF16 residual window and counts it (the serving
+ * policy of Sec. 5.1: new tokens enter the window; when it holds resid_cap tokens the caller encodes
+ * them with dq_encode_tokens(DQ_MEAN_COMPUTE) and resets resid_lens[b] to 0).
+ *   k_bf16, v_bf16               device bf16 [B][Hkv][128], 16-byte aligned: the new tokens
+ *   resid_k_bf16, resid_v_bf16   device bf16 [B][resid_cap][Hkv][128], 16-byte aligned
+ *   resid_lens                   device int32 [B], read and incremented; a sequence whose window is
+ *                                full (or whose count is negative) is left unchanged */
+int dq_window_append(const void *k_bf16, const void *v_bf16, void *resid_k_bf16, void *resid_v_bf16,
+                     int32_t *resid_lens, int resid_cap, int B, int Hkv, void *cuda_stream);
+
 /* Attention for q_len query tokens per sequence in one pass over the cache (speculative
  * decoding, short chunks of prefill); the paper's kernel is the q_len = 1 case (Sec. 4.5).
  *   q_bf16, out_*   [B][q_len][Hq][128]

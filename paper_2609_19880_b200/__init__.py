@@ -24,7 +24,7 @@ ERRORS = {0: "DQ_OK", -1: "DQ_ERR_ARG", -2: "DQ_ERR_INFEASIBLE", -3: "DQ_ERR_UNS
 
 EXPORTS = ["dq_build_tables", "dq_free_tables", "dq_tables_info", "dq_encode_tokens", "dq_encode_tokens_rope",
            "dq_decode_workspace_bytes", "dq_decode_attention", "dq_decode_attention_residual",
-           "dq_decode_attention_multi",
+           "dq_decode_attention_multi", "dq_window_append",
            "dq_decode_attention_static", "dq_decode_tokens",
            "dq_bf16_decode_attention", "dq_profile_enable", "dq_profile_read", "dq_strerror",
            "dq_last_cuda_error"]
@@ -84,6 +84,8 @@ def lib():
         L.dq_decode_attention_multi.restype = i32
         L.dq_decode_attention_multi.argtypes = [vp, vp, vp, i32, vp, vp, vp, vp, i32, vp, i32, vp, vp, vp, vp, i32,
                                                 i32, i32, i32, f32, vp, vp, vp, sz, vp]
+        L.dq_window_append.restype = i32
+        L.dq_window_append.argtypes = [vp, vp, vp, vp, vp, i32, i32, i32, vp]
         L.dq_decode_attention_static.restype = i32
         L.dq_decode_attention_static.argtypes = [vp, vp, vp, vp, vp, vp, vp, i32, vp, i32, vp, i32, i32, i32, f32,
                                                  vp, vp, vp]
@@ -226,6 +228,13 @@ def dq_decode_attention_multi(tk, tv, q_bf16, k_cont, v_cont, k_mean_q, k_mean_s
         _ptr(out_bf16), _ptr(out_f32), _ptr(workspace), int(workspace.numel() * workspace.element_size()),
         _stream(stream))
     _check(rc, "dq_decode_attention_multi")
+
+
+def dq_window_append(k_bf16, v_bf16, resid_k, resid_v, resid_lens, stream=None):
+    """New tokens bf16 [B, Hkv, 128] -> BF16 window [B, cap, Hkv, 128] at position resid_lens[b]; resid_lens += 1."""
+    B, Hkv = int(k_bf16.shape[0]), int(k_bf16.shape[1])
+    _check(lib().dq_window_append(_ptr(k_bf16), _ptr(v_bf16), _ptr(resid_k), _ptr(resid_v), _ptr(resid_lens),
+                                  int(resid_k.shape[1]), B, Hkv, _stream(stream)), "dq_window_append")
 
 
 STATIC_SCRATCH_BYTES = 4 << 20

@@ -252,6 +252,17 @@ int dq_bf16_decode_attention(const void* q_bf16, const void* k_bf16_pages, const
     return DQ_OK;
 }
 
+int dq_window_append(const void* k_bf16, const void* v_bf16, void* resid_k_bf16, void* resid_v_bf16,
+                     int32_t* resid_lens, int resid_cap, int B, int Hkv, void* cuda_stream) {
+    if (!k_bf16 || !v_bf16 || !resid_k_bf16 || !resid_v_bf16 || !resid_lens) return DQ_ERR_ARG;
+    if (B < 0 || Hkv <= 0 || resid_cap <= 0) return DQ_ERR_ARG;
+    if (!aligned16(k_bf16) || !aligned16(v_bf16) || !aligned16(resid_k_bf16) || !aligned16(resid_v_bf16)) return DQ_ERR_ARG;
+    const cudaError_t e = dq_launch_window_append(k_bf16, v_bf16, resid_k_bf16, resid_v_bf16, resid_lens, resid_cap, B, Hkv,
+                                                  static_cast<cudaStream_t>(cuda_stream));
+    if (e != cudaSuccess) return cuda_fail(e, "window append");
+    return DQ_OK;
+}
+
 void dq_profile_enable(int on) { dq_attn_profile_enable(on); }
 
 int dq_profile_read(float* ms_out, int max_records) {

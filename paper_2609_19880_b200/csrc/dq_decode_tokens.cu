@@ -90,7 +90,35 @@ dq_decode_tokens_wide_kernel(const __grid_constant__ DqDevTable T, const uint8_t
     }
 }
 
+// BF16 residual window (Sec. 5.1: the most recent tokens stay uncompressed): append one new
+// token per sequence at position resid_lens[b] and count it.  One CTA per sequence; a full
+// window is left unchanged.
+__global__ void __launch_bounds__(256)
+dq_window_append_kernel(const uint4* __restrict__ k_new, const uint4* __restrict__ v_new, uint4* __restrict__ resid_k,
+                        uint4* __restrict__ resid_v, int32_t* __restrict__ resid_lens, int cap, int Hkv) {
+    const int b = blockIdx.x;
+    const int r = resid_lens[b];
+    __syncthreads();   // every thread has read the count before thread 0 advances it
+    if (r < 0 || r >= cap) return;
+    const int row16 = Hkv * (DQ_HEAD_DIM * 2 / 16);   // 16-byte pieces of one token's K (or V)
+    const size_t dst = ((size_t)b * cap + r) * row16, src = (size_t)b * row16;
+    for (int i = threadIdx.x; i < row16; i += blockDim.x) {
+        resid_k[dst + i] = k_new[src + i];
+        resid_v[dst + i] = v_new[src + i];
+    }
+    if (threadIdx.x == 0) resid_lens[b] = r + 1;
+}
+
 }  // namespace
+
+cudaError_t dq_launch_window_append(const void* k_new, const void* v_new, void* resid_k, void* resid_v,
+                                    int32_t* resid_lens, int cap, int B, int Hkv, cudaStream_t st) {
+    if (B == 0) return cudaSuccess;
+    dq_window_append_kernel<<<B, 256, 0, st>>>(static_cast<const uint4*>(k_new), static_cast<const uint4*>(v_new),
+                                               static_cast<uint4*>(resid_k), static_cast<uint4*>(resid_v), resid_lens,
+                                               cap, Hkv);
+    return cudaGetLastError();
+}
 
 cudaError_t dq_launch_decode_tokens(const DqDevTable& t, const uint8_t* cont, const int8_t* mean_q,
                                     const float* mean_scale, int max_windows, const int32_t* seq_id,

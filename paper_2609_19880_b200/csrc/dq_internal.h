@@ -53,6 +53,9 @@ cudaError_t dq_launch_decode_tokens(const DqDevTable& t, const uint8_t* cont, co
                                     const int32_t* pos, const int32_t* slot, int T, int Hkv,
                                     uint8_t* symbols, float* dequant, cudaStream_t st);
 
+cudaError_t dq_launch_window_append(const void* k_new, const void* v_new, void* resid_k, void* resid_v,
+                                    int32_t* resid_lens, int cap, int B, int Hkv, cudaStream_t st);
+
 struct DqAttnArgs {
     const void* q_bf16;
     const uint8_t* k_cont;

@@ -167,3 +167,24 @@ def test_sliding_window_policy_loop():
     out, out32 = _attend(w, tk, tv, cache, lens.cuda(), rk, rv, rl.cuda())
     ref = _reference(w, ok, ov, cache, lens.cuda(), rk, rv, rl.cuda())
     gc.check_attention(out, out32, ref)
+
+
+def test_window_append_matches_indexing():
+    """dq_window_append writes the new token at position resid_lens[b], counts it, and leaves full windows alone."""
+    B, Hkv, cap = 5, 8, 8
+    g = torch.Generator(device="cuda").manual_seed(1)
+    rk = torch.randn((B, cap, Hkv, 128), generator=g, device="cuda").to(torch.bfloat16)
+    rv = torch.randn((B, cap, Hkv, 128), generator=g, device="cuda").to(torch.bfloat16)
+    rl = torch.tensor([0, 3, 7, 8, 5], dtype=torch.int32, device="cuda")
+    want_k, want_v, want_l = rk.clone(), rv.clone(), rl.clone()
+    for step in range(3):
+        nk = torch.randn((B, Hkv, 128), generator=g, device="cuda").to(torch.bfloat16)
+        nv = torch.randn((B, Hkv, 128), generator=g, device="cuda").to(torch.bfloat16)
+        dq.dq_window_append(nk, nv, rk, rv, rl)
+        for b in range(B):
+            r = int(want_l[b])
+            if r < cap:
+                want_k[b, r], want_v[b, r] = nk[b], nv[b]
+                want_l[b] = r + 1
+        torch.cuda.synchronize()
+        assert torch.equal(rk, want_k) and torch.equal(rv, want_v) and torch.equal(rl, want_l)
