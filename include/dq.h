@@ -209,9 +209,10 @@ int dq_window_append(const void *k_bf16, const void *v_bf16, void *resid_k_bf16,
  *                   K/V the caller has already stored (compressed, or in the BF16 window).  Query token
  *                   i (0 = oldest) sees the first seq_lens[b] + resid_lens[b] - (q_len - 1 - i) tokens of
  *                   the sequence: all compressed tokens come before all window tokens.
- *   workspace       >= dq_decode_workspace_bytes(B, Hq * q_len, max_pages)
- * The q_len * (Hq / Hkv) rows of a KV head share one decode of its streams, so the cost is that of
- * q_len = 1; q_len * (Hq / Hkv) must be <= 8 (DQ_ERR_UNSUPPORTED otherwise: split the call).
+ *   workspace       >= dq_decode_workspace_bytes(B, Hq * min(q_len, 8 / (Hq / Hkv)), max_pages)
+ * Up to 8 (query token, head) rows of a KV head share one decode of its streams: while
+ * q_len * (Hq / Hkv) <= 8 the cost is that of q_len = 1; more query tokens are handled in
+ * ceil(q_len / (8 / (Hq / Hkv))) passes over the cache inside this call.
  * resid_* may be NULL (no window). */
 int dq_decode_attention_multi(const dq_tables *tk, const dq_tables *tv, const void *q_bf16, int q_len,
                               const uint8_t *k_cont, const uint8_t *v_cont, const int8_t *k_mean_q,

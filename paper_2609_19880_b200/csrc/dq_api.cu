@@ -120,7 +120,6 @@ int dq_decode_attention_multi(const dq_tables* tk, const dq_tables* tv, const vo
                               size_t workspace_bytes, void* cuda_stream) {
     if (!tk || !tv || !k_cont || !v_cont) return DQ_ERR_ARG;
     if (q_len < 1) return DQ_ERR_ARG;
-    if (Hkv > 0 && Hq > 0 && Hq % Hkv == 0 && (long long)q_len * (Hq / Hkv) > DQ_MAX_GROUP) return DQ_ERR_UNSUPPORTED;
     if (resid_k_bf16 || resid_v_bf16 || resid_lens) {
         if (!resid_k_bf16 || !resid_v_bf16 || !resid_lens || resid_cap <= 0) return DQ_ERR_ARG;
         if ((reinterpret_cast<uintptr_t>(resid_k_bf16) & 7u) || (reinterpret_cast<uintptr_t>(resid_v_bf16) & 7u))
@@ -129,7 +128,11 @@ int dq_decode_attention_multi(const dq_tables* tk, const dq_tables* tv, const vo
     int rc = check_attn_common(q_bf16, page_table, max_pages, seq_lens, B, Hq, Hkv, out_bf16, out_f32,
                                workspace, workspace_bytes);
     if (rc != DQ_OK) return rc;
-    if (workspace_bytes < dq_attn_workspace_bytes(B, Hq * q_len, max_pages)) return DQ_ERR_WORKSPACE;
+    {   // one pass holds DQ_MAX_GROUP rows per KV head; more query tokens take more passes over the same scratch
+        const int per_pass = DQ_MAX_GROUP / (Hq / Hkv);
+        const int pass_tokens = q_len < per_pass ? q_len : per_pass;
+        if (workspace_bytes < dq_attn_workspace_bytes(B, Hq * pass_tokens, max_pages)) return DQ_ERR_WORKSPACE;
+    }
     if (tv->info.has_mean) return DQ_ERR_UNSUPPORTED;
     if (tk->info.heads_per_stream != tv->info.heads_per_stream) return DQ_ERR_UNSUPPORTED;
     if (Hkv % tk->info.heads_per_stream != 0) return DQ_ERR_ARG;

@@ -443,7 +443,7 @@ dq_attention_kernel(const __grid_constant__ DqDevTable TK, const __grid_constant
             // tokens this thread's row may see: a query token that is not the last one stops earlier; tokens
             // of a BF16 residual window come after the compressed ones and absorb the offset first
             int row_len = cur.len;
-            if (p.q_len > 1) row_len -= max(0, row_offset(p, g_row) - (p.resid_lens ? max(p.resid_lens[cur.b], 0) : 0));
+            if (p.q_total > 1) row_len -= max(0, row_offset(p, g_row) - (p.resid_lens ? max(p.resid_lens[cur.b], 0) : 0));
             float qmu = 0.f, qs = 0.f;   // q' . window mean and sum of q', for the head row this thread owns
             if (g_row < G) {
                 qs = qsum[(n & 1) * DQ_MAX_GROUP + g_row];
@@ -876,8 +876,9 @@ int dq_attn_profile_read(float* ms, int max_records) {
     return n;
 }
 
-cudaError_t dq_launch_attention(const DqDevTable& tk, const DqDevTable& tv, const DqAttnArgs& a,
-                                cudaStream_t st) {
+// One pass: query tokens [q_first, q_first + q_len) of the q_total given; q_len * (Hq / Hkv) <= 8.
+static cudaError_t launch_attention_pass(const DqDevTable& tk, const DqDevTable& tv, const DqAttnArgs& a, int q_total,
+                                         int q_first, int q_len, cudaStream_t st) {
     static int sm_count = 0, smem_max = 0;
     if (sm_count == 0) {
         int dev = 0;
@@ -889,7 +890,6 @@ cudaError_t dq_launch_attention(const DqDevTable& tk, const DqDevTable& tv, cons
         if (e != cudaSuccess) return e;
     }
     int nw = kMaxWarps;
-    const int q_len = a.q_len > 1 ? a.q_len : 1;
     const int G1 = a.Hq / a.Hkv, G = G1 * q_len;   // rows per KV head
     const bool wide = tk.hs > 1;   // token-wide streams: main kernel of dq_attention_wide.cu
     Layout L = make_layout(nw, tk.rec, tv.rec, a.B, G);
@@ -922,6 +922,7 @@ cudaError_t dq_launch_attention(const DqDevTable& tk, const DqDevTable& tv, cons
     p.max_windows = a.max_windows; p.windows = windows_for(a.max_pages); p.max_pages = a.max_pages;
     p.B = a.B; p.Hq = a.Hq * q_len; p.Hkv = a.Hkv; p.G = G;
     p.q_len = q_len; p.G1 = G1; p.Hq1 = a.Hq;
+    p.q_total = q_total; p.q_first = q_first;
     p.item_tokens = nw * kChunk;
     p.rotate_q = tk.rotate; p.rotate_out = tv.rotate; p.has_mean = tk.has_mean;
     p.scale_log2 = a.sm_scale * 1.4426950408889634f;
@@ -955,6 +956,20 @@ cudaError_t dq_launch_attention(const DqDevTable& tk, const DqDevTable& tv, cons
     return dq_launch_pdl(dq_attn_combine_kernel, dim3(heads), dim3(256), 0, st, p);
 }
 
+// q_len query tokens per sequence: as many passes over the cache as it takes to give every
+// (query token, head) pair of a KV head one of the 8 rows of the MMA tile.
+cudaError_t dq_launch_attention(const DqDevTable& tk, const DqDevTable& tv, const DqAttnArgs& a,
+                                cudaStream_t st) {
+    const int q_total = a.q_len > 1 ? a.q_len : 1;
+    const int per_pass = DQ_MAX_GROUP / (a.Hq / a.Hkv) > 0 ? DQ_MAX_GROUP / (a.Hq / a.Hkv) : 1;
+    for (int q_first = 0; q_first < q_total; q_first += per_pass) {
+        const int q_len = q_total - q_first < per_pass ? q_total - q_first : per_pass;
+        const cudaError_t e = launch_attention_pass(tk, tv, a, q_total, q_first, q_len, st);
+        if (e != cudaSuccess) return e;
+    }
+    return cudaSuccess;
+}
+
 cudaError_t dq_launch_bf16_attention(const DqAttnArgs& a, const void* k_pages, const void* v_pages,
                                      cudaStream_t st) {
     const WsLayout w = ws_layout(a.B, a.Hq, a.max_pages);
@@ -978,7 +993,7 @@ cudaError_t dq_launch_bf16_attention(const DqAttnArgs& a, const void* k_pages, c
     p.scale_log2 = a.sm_scale * 1.4426950408889634f;
     p.hkv_magic = 0;
     p.hs = 1; p.groups = a.Hkv;
-    p.q_len = 1; p.G1 = p.G; p.Hq1 = a.Hq;
+    p.q_len = 1; p.G1 = p.G; p.Hq1 = a.Hq; p.q_total = 1; p.q_first = 0;
     p.resid_k = nullptr; p.resid_v = nullptr; p.resid_lens = nullptr; p.resid_cap = 0;
     const int heads = a.B * a.Hq;
     dq_attn_prepare_kernel<<<(heads + 7) / 8, 256, 0, st>>>(p);

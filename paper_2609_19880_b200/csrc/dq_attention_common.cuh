@@ -41,7 +41,9 @@ struct AttnParams {
     // Several query tokens per sequence (q_len > 1): the rows of one KV head are (query token i, head g),
     // r = i * G1 + g; G = q_len * G1 rows per KV head and Hq = Hkv * G rows per sequence everywhere in the
     // workspace.  Query token i is q_len - 1 - i positions before the end of the sequence.
-    int q_len, G1, Hq1; // tokens per sequence in q; query heads per KV head and per token
+    int q_len, G1, Hq1; // query tokens of this pass; query heads per KV head and per token
+    int q_total, q_first; // tokens per sequence in q / out, and the first one this pass handles (a call with
+                        // more rows than one MMA tile holds is run as several passes)
     const uint16_t* resid_k;      // bf16 [B][resid_cap][Hkv][128], nullable: uncompressed recent tokens
     const uint16_t* resid_v;
     const int32_t* resid_lens;    // [B]
@@ -67,13 +69,15 @@ __device__ __forceinline__ void sts32f(uint32_t addr, float v) {
     asm volatile("st.shared.f32 [%0], %1;\n" ::"r"(addr), "f"(v) : "memory");
 }
 
-// Source / destination of workspace row (b, hq) in q / out, laid out [B][q_len][Hq1][128].
+// Source / destination of workspace row (b, hq) in q / out, laid out [B][q_total][Hq1][128].
 __device__ __forceinline__ size_t qo_row(const AttnParams& p, int b, int hq) {
     const int h = hq / p.G, r = hq - h * p.G, i = r / p.G1, g = r - i * p.G1;
-    return ((size_t)b * p.q_len + i) * p.Hq1 + (size_t)h * p.G1 + g;
+    return ((size_t)b * p.q_total + p.q_first + i) * p.Hq1 + (size_t)h * p.G1 + g;
 }
 // Positions before the sequence end of the query token that row r of a KV head belongs to.
-__device__ __forceinline__ int row_offset(const AttnParams& p, int r) { return r < p.G ? p.q_len - 1 - r / p.G1 : 0; }
+__device__ __forceinline__ int row_offset(const AttnParams& p, int r) {
+    return r < p.G ? p.q_total - 1 - (p.q_first + r / p.G1) : 0;
+}
 
 }  // namespace dqattn
 

@@ -435,7 +435,7 @@ dq_attention_wide_kernel(const __grid_constant__ DqDevTable TK, const __grid_con
                              "f"(oV) : "memory");
             }
             int row_len = cur.len;   // tokens this thread's row may see (earlier query tokens stop earlier)
-            if (p.q_len > 1) row_len -= max(0, row_offset(p, g_row) - (p.resid_lens ? max(p.resid_lens[cur.b], 0) : 0));
+            if (p.q_total > 1) row_len -= max(0, row_offset(p, g_row) - (p.resid_lens ? max(p.resid_lens[cur.b], 0) : 0));
             float qmu = 0.f, qs = 0.f;
             if (g_row < G) {
                 qs = qsum[(s & 1) * DQ_MAX_GROUP + g_row];

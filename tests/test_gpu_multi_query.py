@@ -99,17 +99,18 @@ def test_with_residual_window_gqa2(wide_hs):
     _run(cfg, 4, wide_hs=wide_hs, resid=[128, 2, 0, 37])
 
 
-def test_single_token_equals_plain_call_and_limits():
+def test_single_token_equals_plain_call():
     cfg = _cfg(4, batch=5, seq_lens=[200, 16, 333, 1, 1030])
     w, tk, tv, cache, q, out, out32 = _run(cfg, 1)
     w.q = q[:, 0].contiguous()
     out_p, out32_p = gc.gpu_attention(w, tk, tv, cache)
     assert torch.equal(out32[:, 0], out32_p) and torch.equal(out[:, 0], out_p)
-    q3 = torch.zeros((cfg.batch, 3, cfg.hq, 128), dtype=torch.bfloat16, device="cuda")
-    o3 = torch.empty_like(q3)
-    ws = torch.empty(dq.dq_decode_workspace_bytes(cfg.batch, cfg.hq * 3, w.page_table.shape[1]), dtype=torch.uint8,
-                     device="cuda")
-    with pytest.raises(dq.DqError) as e:   # 3 tokens x 4 heads per KV head = 12 rows > 8
-        dq.dq_decode_attention_multi(tk, tv, q3, cache.k_cont, cache.v_cont, cache.mean_q, cache.mean_scale,
-                                     w.page_table, w.seq_lens, cfg.hkv, gc.SM_SCALE, o3, ws)
-    assert e.value.code == -3
+
+
+def test_more_rows_than_one_pass_holds():
+    """5 query tokens x 4 heads per KV head = 20 rows: three passes inside one call (2 + 2 + 1 tokens);
+    and 11 tokens with one head per KV head (8 + 3), with a window."""
+    cfg = _cfg(2, batch=3, seq_lens=[600, 64, 7])
+    _run(cfg, 5, seed=21)
+    cfg = _cfg(2, batch=2, seq_lens=[530, 40], hq=8)
+    _run(cfg, 11, wide_hs=8, resid=[6, 128], seed=22)

@@ -139,8 +139,8 @@ def test_calls_validate_before_launch(L):
             d["tk"], d["tv"], d["q"], q_len, *[d[k] for k in ("kc", "vc", "mq", "ms", "mw", "pt", "mp", "sl")], n, n, n, 0,
             *[d[k] for k in ("B", "Hq", "Hkv", "sm", "ob", "of", "ws", "wsb", "st")])
 
-    # several query tokens: q_len * (Hq / Hkv) rows of a KV head must fit 8; the workspace grows with q_len
-    assert call_m(0) == -1 and call_m(3) == -3 and call_m(2, wsb=ws) == -4
+    # several query tokens: the workspace must hold one pass of min(q_len, 8 / (Hq / Hkv)) tokens
+    assert call_m(0) == -1 and call_m(2, wsb=ws) == -4 and call_m(5, wsb=dq.dq_decode_workspace_bytes(2, 64, 8) - 1) == -4
     assert call_m(2, q=n, wsb=dq.dq_decode_workspace_bytes(2, 64, 8)) == -1
     assert L.dq_decode_tokens(tk.handle, n, n, n, 0, n, n, fake, 4, 8, fake, n, n) == -1
     assert L.dq_bf16_decode_attention(fake, n, fake, fake, 8, fake, 2, 32, 8, C.c_float(0.1), fake, fake, ws, n) == -1
