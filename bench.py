@@ -282,14 +282,23 @@ def run_ours(args):
 
     state = {"r": 0, "closes": 0}
     if hs == 1:
-        def step(i, q=w.q, nk=new_k, nv=new_v):
-            c = caches[i % copies]
-            dq.dq_encode_tokens(tk, tv, nk, nv, new_seq, new_pos, new_slot, c["k"], c["v"], c["mq"], c["ms"],
-                                dq.MEAN_REUSE)
-            dq.dq_decode_attention(tk, tv, q, c["k"], c["v"], c["mq"], c["ms"], w.page_table, w.seq_lens, Hkv,
-                                   sm_scale, out, ws)
+        if args.separate_calls:
+            def step(i, q=w.q, nk=new_k, nv=new_v):
+                c = caches[i % copies]
+                dq.dq_encode_tokens(tk, tv, nk, nv, new_seq, new_pos, new_slot, c["k"], c["v"], c["mq"], c["ms"],
+                                    dq.MEAN_REUSE)
+                dq.dq_decode_attention(tk, tv, q, c["k"], c["v"], c["mq"], c["ms"], w.page_table, w.seq_lens, Hkv,
+                                       sm_scale, out, ws)
+            step_desc = "encode 1 new token per sequence + decode attention over the whole cache (two calls)"
+        else:
+            # the same work through the one-call step API: the attention kernel starts beside the encoder
+            def step(i, q=w.q, nk=new_k, nv=new_v):
+                c = caches[i % copies]
+                dq.dq_decode_step(tk, tv, nk, nv, new_slot, q, c["k"], c["v"], c["mq"], c["ms"], w.page_table,
+                                  w.seq_lens, Hkv, sm_scale, out, ws)
+            step_desc = ("encode 1 new token per sequence + decode attention over the whole cache "
+                         "(dq_decode_step: attention starts while the encoder runs)")
         launches_per_step = 4   # encode (K and V), prepare, fused attention, combine
-        step_desc = "encode 1 new token per sequence + decode attention over the whole cache"
     else:
         # The paper's serving policy (Sec. 5.1): the newest tokens stay in a 128-token BF16 window that
         # joins the attention; when the window is full its 128 tokens per sequence are encoded in one
@@ -521,6 +530,8 @@ def main():
                     help="head: one stream per (token, KV head), the benchmark's configuration; token: the paper's "
                          "default grouping, one 335 / 235-byte record per token, 8 / 6 levels")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--separate-calls", action="store_true",
+                    help="per token-head streams: dq_encode_tokens + dq_decode_attention instead of dq_decode_step")
     ap.add_argument("--no-graph", action="store_true", help="end-to-end leg: launch directly instead of replaying CUDA graphs")
     ap.add_argument("--profile-only", action="store_true",
                     help="warm-up and timed steps only (for profiler captures); prints a short line")

@@ -192,6 +192,27 @@ int dq_decode_attention_residual(const dq_tables *tk, const dq_tables *tv, const
                                  int Hq, int Hkv, float sm_scale, void *out_bf16, float *out_f32,
                                  void *workspace, size_t workspace_bytes, void *cuda_stream);
 
+/* One decode step of a layer in a single call: encode the newest token of every sequence
+ * (dq_encode_tokens with DQ_MEAN_REUSE: token b is the token at position seq_lens[b] - 1 of
+ * sequence b; sequences of length 0 have none) and attend over the whole cache including it
+ * (dq_decode_attention).  Same results as those two calls; the point is the schedule: the
+ * attention kernel starts while the encoder still runs, works through every block that does not
+ * hold a newest token first (work items come from a global counter, so the few SMs that host the
+ * encoder simply take fewer), and waits for the encoder only before the first block that does.
+ * Per token-head streams only (heads_per_stream = 1: DQ_ERR_UNSUPPORTED otherwise).
+ *   k_new_bf16, v_new_bf16   device bf16 [B][Hkv][128]
+ *   slot_new                 device int32 [B]: physical slot of each newest token
+ *   seq_lens                 device int32 [B]: lengths including the newest token
+ *   status                   as in dq_encode_tokens (nullable)
+ * Other arguments as in dq_decode_attention.  Not to be mixed on one stream with work that
+ * reads `workspace` concurrently; the first 16 bytes of the workspace carry the hand-over state. */
+int dq_decode_step(const dq_tables *tk, const dq_tables *tv, const void *k_new_bf16, const void *v_new_bf16,
+                   const int32_t *slot_new, const void *q_bf16, uint8_t *k_cont, uint8_t *v_cont,
+                   int8_t *k_mean_q, float *k_mean_scale, int max_windows, const int32_t *page_table,
+                   int max_pages, const int32_t *seq_lens, int B, int Hq, int Hkv, float sm_scale,
+                   void *out_bf16, float *out_f32, void *workspace, size_t workspace_bytes,
+                   uint32_t *status, void *cuda_stream);
+
 /* Appends one new token per sequence to the BF16 residual window and counts it (the serving
  * policy of Sec. 5.1: new tokens enter the window; when it holds resid_cap tokens the caller encodes
  * them with dq_encode_tokens(DQ_MEAN_COMPUTE) and resets resid_lens[b] to 0).

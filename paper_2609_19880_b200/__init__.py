@@ -24,7 +24,7 @@ ERRORS = {0: "DQ_OK", -1: "DQ_ERR_ARG", -2: "DQ_ERR_INFEASIBLE", -3: "DQ_ERR_UNS
 
 EXPORTS = ["dq_build_tables", "dq_free_tables", "dq_tables_info", "dq_encode_tokens", "dq_encode_tokens_rope",
            "dq_decode_workspace_bytes", "dq_decode_attention", "dq_decode_attention_residual",
-           "dq_decode_attention_multi", "dq_window_append",
+           "dq_decode_attention_multi", "dq_window_append", "dq_decode_step",
            "dq_decode_attention_static", "dq_decode_tokens",
            "dq_bf16_decode_attention", "dq_profile_enable", "dq_profile_read", "dq_strerror",
            "dq_last_cuda_error"]
@@ -84,6 +84,9 @@ def lib():
         L.dq_decode_attention_multi.restype = i32
         L.dq_decode_attention_multi.argtypes = [vp, vp, vp, i32, vp, vp, vp, vp, i32, vp, i32, vp, vp, vp, vp, i32,
                                                 i32, i32, i32, f32, vp, vp, vp, sz, vp]
+        L.dq_decode_step.restype = i32
+        L.dq_decode_step.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, i32, vp, i32, vp, i32, i32, i32, f32, vp, vp,
+                                     vp, sz, vp, vp]
         L.dq_window_append.restype = i32
         L.dq_window_append.argtypes = [vp, vp, vp, vp, vp, i32, i32, i32, vp]
         L.dq_decode_attention_static.restype = i32
@@ -228,6 +231,20 @@ def dq_decode_attention_multi(tk, tv, q_bf16, k_cont, v_cont, k_mean_q, k_mean_s
         _ptr(out_bf16), _ptr(out_f32), _ptr(workspace), int(workspace.numel() * workspace.element_size()),
         _stream(stream))
     _check(rc, "dq_decode_attention_multi")
+
+
+def dq_decode_step(tk, tv, k_new, v_new, slot_new, q_bf16, k_cont, v_cont, k_mean_q, k_mean_scale, page_table,
+                   seq_lens, Hkv: int, sm_scale: float, out_bf16, workspace, out_f32=None, status=None, stream=None):
+    """Encode the newest token of every sequence (k_new / v_new bf16 [B, Hkv, 128] at slot_new, position
+    seq_lens - 1) and attend over the whole cache, as one overlapped launch sequence."""
+    B, Hq = int(q_bf16.shape[0]), int(q_bf16.shape[1])
+    max_windows = int(k_mean_q.shape[1]) if k_mean_q is not None else 0
+    rc = lib().dq_decode_step(tk.handle, tv.handle, _ptr(k_new), _ptr(v_new), _ptr(slot_new), _ptr(q_bf16),
+                              _ptr(k_cont), _ptr(v_cont), _ptr(k_mean_q), _ptr(k_mean_scale), max_windows,
+                              _ptr(page_table), int(page_table.shape[1]), _ptr(seq_lens), B, Hq, int(Hkv),
+                              float(sm_scale), _ptr(out_bf16), _ptr(out_f32), _ptr(workspace),
+                              int(workspace.numel() * workspace.element_size()), _ptr(status), _stream(stream))
+    _check(rc, "dq_decode_step")
 
 
 def dq_window_append(k_bf16, v_bf16, resid_k, resid_v, resid_lens, stream=None):

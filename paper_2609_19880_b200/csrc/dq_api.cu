@@ -81,6 +81,7 @@ int dq_encode_tokens_rope(const dq_tables* tk, const dq_tables* tv, const void* 
     a.status = status; a.T = T; a.Hkv = Hkv; a.max_windows = max_windows; a.mean_mode = mean_mode;
     a.do_k = tk ? 1 : 0; a.do_v = tv ? 1 : 0;
     a.rope_cos = rope_cos; a.rope_sin = rope_sin; a.rope_style = rope_style;
+    a.step_seq_lens = nullptr; a.step_flags = nullptr;
     e = dq_launch_encode(tk ? tk->dev : tv->dev, tv ? tv->dev : tk->dev, a, st);
     if (e != cudaSuccess) return cuda_fail(e, "encode");
     return DQ_OK;
@@ -151,6 +152,7 @@ int dq_decode_attention_multi(const dq_tables* tk, const dq_tables* tv, const vo
     a.B = B; a.Hq = Hq; a.Hkv = Hkv; a.sm_scale = sm_scale;
     a.resid_k = resid_k_bf16; a.resid_v = resid_v_bf16; a.resid_lens = resid_lens; a.resid_cap = resid_cap;
     a.q_len = q_len;
+    a.fused = 0;
     const cudaError_t e = dq_launch_attention(tk->dev, tv->dev, a, static_cast<cudaStream_t>(cuda_stream));
     if (e != cudaSuccess) return cuda_fail(e, "decode attention");
     return DQ_OK;
@@ -216,6 +218,7 @@ int dq_decode_attention_static(const dq_tables* tk, const dq_tables* tv, const v
     a.B = B; a.Hq = Hq; a.Hkv = Hkv; a.sm_scale = sm_scale;
     a.resid_k = nullptr; a.resid_v = nullptr; a.resid_lens = nullptr; a.resid_cap = 0;
     a.q_len = 1;
+    a.fused = 0;
     e = dq_launch_attention_static(tk->dev, tv->dev, a, static_cast<cudaStream_t>(cuda_stream));
     if (e != cudaSuccess) return cuda_fail(e, "decode attention (static scratch)");
     return DQ_OK;
@@ -252,6 +255,46 @@ int dq_bf16_decode_attention(const void* q_bf16, const void* k_bf16_pages, const
     const cudaError_t e = dq_launch_bf16_attention(a, k_bf16_pages, v_bf16_pages,
                                                    static_cast<cudaStream_t>(cuda_stream));
     if (e != cudaSuccess) return cuda_fail(e, "bf16 decode attention");
+    return DQ_OK;
+}
+
+int dq_decode_step(const dq_tables* tk, const dq_tables* tv, const void* k_new_bf16, const void* v_new_bf16,
+                   const int32_t* slot_new, const void* q_bf16, uint8_t* k_cont, uint8_t* v_cont, int8_t* k_mean_q,
+                   float* k_mean_scale, int max_windows, const int32_t* page_table, int max_pages,
+                   const int32_t* seq_lens, int B, int Hq, int Hkv, float sm_scale, void* out_bf16, float* out_f32,
+                   void* workspace, size_t workspace_bytes, uint32_t* status, void* cuda_stream) {
+    if (!tk || !tv || !k_new_bf16 || !v_new_bf16 || !slot_new || !k_cont || !v_cont) return DQ_ERR_ARG;
+    int rc = check_attn_common(q_bf16, page_table, max_pages, seq_lens, B, Hq, Hkv, out_bf16, out_f32, workspace,
+                               workspace_bytes);
+    if (rc != DQ_OK) return rc;
+    if (tk->info.heads_per_stream != 1 || tv->info.heads_per_stream != 1) return DQ_ERR_UNSUPPORTED;
+    if (tv->info.has_mean) return DQ_ERR_UNSUPPORTED;
+    if (tk->info.has_mean && (!k_mean_q || !k_mean_scale || max_windows <= 0)) return DQ_ERR_ARG;
+    if (tk->info.has_mean && (long long)max_windows * DQ_WINDOW_TOKENS < (long long)max_pages * DQ_PAGE_TOKENS)
+        return DQ_ERR_ARG;
+    if (!aligned16(k_cont) || !aligned16(v_cont) || (tk->info.has_mean && !aligned16(k_mean_q))) return DQ_ERR_ARG;
+    if ((reinterpret_cast<uintptr_t>(k_new_bf16) & 7u) || (reinterpret_cast<uintptr_t>(v_new_bf16) & 7u)) return DQ_ERR_ARG;
+    if ((out_bf16 && (reinterpret_cast<uintptr_t>(out_bf16) & 7u)) || (out_f32 && !aligned16(out_f32))) return DQ_ERR_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    DqEncodeArgs e;
+    std::memset(&e, 0, sizeof e);
+    e.k_bf16 = k_new_bf16; e.v_bf16 = v_new_bf16; e.slot = slot_new;
+    e.k_cont = k_cont; e.v_cont = v_cont; e.mean_q = k_mean_q; e.mean_scale = k_mean_scale;
+    e.status = status; e.T = B; e.Hkv = Hkv; e.max_windows = max_windows; e.mean_mode = DQ_MEAN_REUSE;
+    e.do_k = 1; e.do_v = 1;
+    e.step_seq_lens = seq_lens; e.step_flags = dq_attn_workspace_flags(workspace);
+    cudaError_t ce = dq_launch_encode(tk->dev, tv->dev, e, st);
+    if (ce != cudaSuccess) return cuda_fail(ce, "decode step: encode");
+    DqAttnArgs a;
+    std::memset(&a, 0, sizeof a);
+    a.q_bf16 = q_bf16; a.k_cont = k_cont; a.v_cont = v_cont;
+    a.mean_q = k_mean_q; a.mean_scale = k_mean_scale;
+    a.page_table = page_table; a.seq_lens = seq_lens;
+    a.out_bf16 = out_bf16; a.out_f32 = out_f32; a.workspace = workspace;
+    a.max_windows = max_windows; a.max_pages = max_pages;
+    a.B = B; a.Hq = Hq; a.Hkv = Hkv; a.sm_scale = sm_scale;
+    ce = dq_launch_step(tk->dev, tv->dev, e, a, st);
+    if (ce != cudaSuccess) return cuda_fail(ce, "decode step: attention");
     return DQ_OK;
 }
 

@@ -38,7 +38,9 @@ constexpr int kTileBytes = kChunk * kTileStride;
 constexpr int kKTail = 32;             // bytes after a warp's K records: q'.mean of its window, per head
 
 struct Item {
-    int b, h, blk, len, bg, valid, pad0, pad1;
+    int b, h, blk, len, bg, valid;
+    int late;   // decode-step mode: the block holds the sequence's newest token, whose record the step's encoder writes
+    int pad1;
 };
 
 struct Layout {
@@ -70,7 +72,7 @@ __host__ __device__ inline Layout make_layout(int nw, int rec_k, int rec_v, int 
     L.off_obuf = o; o += nw * L.warp_obuf_bytes;
     L.off_kst = o; o += 2 * nw * L.stage_k;
     L.off_vst = o; o += 2 * nw * L.stage_v;
-    L.off_prefix = o; o += align16((2 * B + 1) * 4);   // block prefix sums, sequence lengths
+    L.off_prefix = o; o += align16((3 * B + 2) * 4);   // block prefix sums, sequence lengths, non-empty counts
     L.total = o + 256;  // slack: a malformed record may be over-read by up to 136 + 8 bytes
     return L;
 }
@@ -84,7 +86,9 @@ constexpr int kPrepWindows = 8;
 __global__ void __launch_bounds__(256)
 dq_attn_prepare_kernel(AttnParams p) {
     pdl_launch_dependents();
-    pdl_wait_prior_grid();   // q, the window means and seq_lens may come from the previous kernel
+    // Decode-step mode: this kernel was let go by the step's encoder after THAT kernel's wait, so everything
+    // older is complete; it must not wait for the encoder (it runs beside it) and reads nothing the encoder writes.
+    if (!p.fused) pdl_wait_prior_grid();   // q, the window means and seq_lens may come from the previous kernel
     const int lane = threadIdx.x & 31;
     const long long wid = (long long)blockIdx.x * 8 + (threadIdx.x >> 5);
     const int heads = p.B * p.Hq;
@@ -125,11 +129,19 @@ dq_attn_prepare_kernel(AttnParams p) {
             uint32_t q4[kPrepWindows];
             float msc[kPrepWindows], s[kPrepWindows];
 #pragma unroll
+            // Decode-step mode: when the newest token opens a window, the encoder is writing that window's
+            // mean right now as a copy of the previous window's (zero for window 0): read the source instead.
+            int w_open = -1;
+            if (p.fused) {
+                const int np = p.seq_lens[b] - 1;
+                if (np >= 0 && np % DQ_WINDOW_TOKENS == 0) w_open = np / DQ_WINDOW_TOKENS;
+            }
             for (int u = 0; u < kPrepWindows; ++u) {   // all loads first
                 const int w = min(win * kPrepWindows + u, p.windows - 1);
-                const size_t mi = ((size_t)b * p.max_windows + w) * p.Hkv + h;
+                const int ws = (w == w_open) ? w - 1 : w;
+                const size_t mi = ((size_t)b * p.max_windows + max(ws, 0)) * p.Hkv + h;
                 q4[u] = *reinterpret_cast<const uint32_t*>(p.mean_q + mi * kN + 4 * lane);
-                msc[u] = p.mean_scale[mi];
+                msc[u] = ws < 0 ? 0.f : p.mean_scale[mi];
             }
 #pragma unroll
             for (int u = 0; u < kPrepWindows; ++u) {
@@ -146,22 +158,38 @@ dq_attn_prepare_kernel(AttnParams p) {
                 if (lane == u && win * kPrepWindows + u < p.windows) p.qmu[(size_t)head * p.windows + win * kPrepWindows + u] = s[u];
         }
     }
-    if (blockIdx.x == 0 && threadIdx.x < 32) {  // exclusive scan of blocks per sequence
-        int carry = 0;
+    if (blockIdx.x == 0 && threadIdx.x < 32) {  // exclusive scans: blocks per sequence, non-empty sequences
+        int carry = 0, ne_carry = 0;
         for (int base = 0; base < p.B; base += 32) {
             const int b = base + lane;
             int nb = 0;
             if (b < p.B) nb = (min(max(p.seq_lens[b], 0), p.max_pages * DQ_PAGE_TOKENS) + p.item_tokens - 1) / p.item_tokens;
-            int incl = nb;
+            int incl = nb, ne = nb > 0 ? 1 : 0;
+            const int ne_self = ne;
 #pragma unroll
             for (int d = 1; d < 32; d <<= 1) {
-                const int o = __shfl_up_sync(kFullMask, incl, d);
-                if (lane >= d) incl += o;
+                const int o = __shfl_up_sync(kFullMask, incl, d), oe = __shfl_up_sync(kFullMask, ne, d);
+                if (lane >= d) { incl += o; ne += oe; }
             }
-            if (b < p.B) p.prefix[b] = carry + incl - nb;
+            if (b < p.B) { p.prefix[b] = carry + incl - nb; p.ne_before[b] = ne_carry + ne - ne_self; }
             carry += __shfl_sync(kFullMask, incl, 31);
+            ne_carry += __shfl_sync(kFullMask, ne, 31);
         }
-        if (lane == 0) { p.prefix[p.B] = carry; *p.counter = 0; }
+        if (lane == 0) { p.prefix[p.B] = carry; p.ne_before[p.B] = ne_carry; if (!p.fused) *p.counter = 0; }
+    }
+    if (p.fused) {
+        // Hand-over: when the last CTA is done, it publishes the first dynamic item index (the first three
+        // items of every attention CTA are dealt statically) and then the ready flag, and one of its threads
+        // stays to wait for the encoder, so that this kernel's end implies the encoder's.  Every other CTA
+        // leaves at once: the attention CTAs need whole SMs.
+        __threadfence();
+        __syncthreads();
+        if (threadIdx.x == 0 && atomicAdd(&p.flags[2], 1) == (int)gridDim.x - 1) {
+            p.flags[0] = 3 * p.attn_grid;
+            __threadfence();
+            atomicExch(&p.flags[1], 1);
+            pdl_wait_prior_grid();
+        }
     }
 }
 
@@ -250,6 +278,12 @@ __device__ __forceinline__ void fused_pass(uint32_t xk, uint32_t ptrk, uint32_t 
     }
 }
 
+// FUSED (decode-step mode): the kernel starts while the step's encoder still runs.  It takes the
+// prepare kernel's outputs on a ready flag instead of waiting for that kernel, pulls its work items
+// from a global counter (SMs still busy with the encoder join late and simply take fewer), leaves the
+// blocks that hold a sequence's newest token to the end of the item order, and waits for the preceding
+// kernels -- whose completion implies the encoder's -- only before the first of those blocks.
+template <bool FUSED>
 __global__ void __launch_bounds__(kMaxWarps * 32, 1)
 dq_attention_kernel(const __grid_constant__ DqDevTable TK, const __grid_constant__ DqDevTable TV,
                     const AttnParams p) {
@@ -274,10 +308,30 @@ dq_attention_kernel(const __grid_constant__ DqDevTable TK, const __grid_constant
         lutk[i] = TK.lut[i >> 5];
         lutv[i] = TV.lut[i >> 5];
     }
-    pdl_wait_prior_grid();   // everything below reads what the prepare kernel wrote
+    int* ne_before = s_len + p.B;                                   // [B + 1] (FUSED) non-empty sequences before b
+    bool waited = !FUSED;   // the preceding kernels are known to be complete
+    if (FUSED) {
+        // acquire-poll the ready flag (bounded); a CTA that gives up waits for the preceding kernels instead
+        int* s_ok = reinterpret_cast<int*>(smem + L.off_items);
+        if (tid == 0) {
+            int ok = 0;
+            for (int it = 0; it < (1 << 16) && !ok; ++it) {
+                asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(ok) : "l"(p.flags + 1) : "memory");
+                if (!ok) __nanosleep(64);
+            }
+            if (!ok) atomicAdd(p.flags + 3, 1);
+            *s_ok = ok;
+        }
+        __syncthreads();
+        if (!*s_ok) { pdl_wait_prior_grid(); waited = true; }
+        __syncthreads();
+    } else {
+        pdl_wait_prior_grid();   // everything below reads what the prepare kernel wrote
+    }
     for (int i = tid; i <= p.B; i += nthreads) {
         prefix[i] = p.prefix[i];
         if (i < p.B) s_len[i] = min(p.seq_lens[i], p.max_pages * DQ_PAGE_TOKENS);
+        if (FUSED) ne_before[i] = p.ne_before[i];
     }
     __syncthreads();
     const int total_items = prefix[p.B] * p.Hkv;
@@ -295,7 +349,7 @@ dq_attention_kernel(const __grid_constant__ DqDevTable TK, const __grid_constant
     // found by walking forward from `hint`, the sequence of an earlier item.)
     auto item_of = [&](int n, int hint) {
         Item it;
-        it.valid = 0; it.b = hint; it.h = it.blk = it.len = it.bg = 0; it.pad0 = it.pad1 = 0;
+        it.valid = 0; it.b = hint; it.h = it.blk = it.len = it.bg = 0; it.late = it.pad1 = 0;
         const unsigned idx = blockIdx.x + (unsigned)n * gridDim.x;   // < 2^31: total_items is an int
         if (idx < (unsigned)total_items) {
             it.valid = 1;
@@ -308,6 +362,42 @@ dq_attention_kernel(const __grid_constant__ DqDevTable TK, const __grid_constant
             it.blk = it.bg - prefix[b];
             it.len = s_len[b];
         }
+        return it;
+    };
+    // Decode-step mode: item order = every block that is not the last of its sequence (sequence-major),
+    // then the last blocks; the first three items of a CTA are static, the rest come from the counter.
+    int hint = 0;        // thread 0: sequence of the newest descriptor, the search start for the next one
+    int hint_late = 0;   // thread 0: search start among the last blocks
+    auto item_of_fused = [&](int n) {
+        Item it;
+        it.valid = 0; it.b = 0; it.h = it.blk = it.len = it.bg = 0; it.late = it.pad1 = 0;
+        const int n_early = (prefix[p.B] - ne_before[p.B]) * p.Hkv, n_late = ne_before[p.B] * p.Hkv;
+        unsigned r;
+        if (n < 3) r = blockIdx.x + (unsigned)n * gridDim.x;
+        else r = (unsigned)atomicAdd(p.flags + 0, 1);
+        if (r >= (unsigned)(n_early + n_late)) return it;
+        it.valid = 1;
+        if (r < (unsigned)n_early) {
+            const int bgA = p.hkv_magic ? (int)__umulhi(r, p.hkv_magic) : (int)r;   // r / Hkv
+            it.h = (int)(r - (unsigned)bgA * (unsigned)p.Hkv);
+            int b = hint;   // non-last blocks before sequence b: prefix[b] - ne_before[b]
+            while (prefix[b + 1] - ne_before[b + 1] <= bgA) ++b;
+            hint = b;
+            it.b = b;
+            it.blk = bgA - (prefix[b] - ne_before[b]);
+        } else {
+            const unsigned rl = r - (unsigned)n_early;
+            const int j = p.hkv_magic ? (int)__umulhi(rl, p.hkv_magic) : (int)rl;   // j-th non-empty sequence
+            it.h = (int)(rl - (unsigned)j * (unsigned)p.Hkv);
+            int b = hint_late;
+            while (ne_before[b + 1] <= j) ++b;
+            hint_late = b;
+            it.b = b;
+            it.blk = prefix[b + 1] - prefix[b] - 1;
+            it.late = 1;
+        }
+        it.bg = prefix[it.b] + it.blk;
+        it.len = s_len[it.b];
         return it;
     };
     // The physical page ids of this warp's 32 tokens are fetched two items ahead by cp.async into
@@ -356,9 +446,9 @@ dq_attention_kernel(const __grid_constant__ DqDevTable TK, const __grid_constant
     };
 
     Item* s_items = reinterpret_cast<Item*>(smem + L.off_items);
-    int hint = 0;   // thread 0: sequence of the newest descriptor, the search start for the next one
     if (tid == 0) {
         for (int n = 0; n < 3; ++n) {
+            if (FUSED) { s_items[n] = item_of_fused(n); continue; }
             const Item it = item_of(n, hint);
             s_items[n] = it;
             hint = it.b;
@@ -368,6 +458,7 @@ dq_attention_kernel(const __grid_constant__ DqDevTable TK, const __grid_constant
     // prologue: page ids of items 0 and 1, then the K records of item 0
     {
         const Item i0 = s_items[0];
+        if (FUSED && !waited && i0.valid && i0.late) { pdl_wait_prior_grid(); waited = true; }
         fetch_pages(0, i0);
         fetch_pages(1, s_items[1]);
         cp_async_commit();
@@ -386,6 +477,10 @@ dq_attention_kernel(const __grid_constant__ DqDevTable TK, const __grid_constant
         Item cur = s_items[n & 3];
         if (!cur.valid && !have_prev) break;
         {   // records of item n + 1 (its page ids arrived last iteration), page ids of item n + 2
+            if (FUSED && !waited && s_items[(n + 1) & 3].valid && s_items[(n + 1) & 3].late) {
+                pdl_wait_prior_grid();   // the newest tokens' records are complete from here on
+                waited = true;
+            }
             issue_loads(n + 1, s_items[(n + 1) & 3], n, cur);
             fetch_pages(n + 2, s_items[(n + 2) & 3]);
             cp_async_commit();
@@ -393,9 +488,13 @@ dq_attention_kernel(const __grid_constant__ DqDevTable TK, const __grid_constant
         cp_async_wait<1>();
         __syncthreads();   // q' operand of `cur` visible; last iteration's merge reads are done
         if (tid == 0) {    // slot of item n - 1, which nobody reads any more
-            const Item it = item_of(n + 3, hint);
-            s_items[(n + 3) & 3] = it;
-            hint = it.b;
+            if (FUSED) {
+                s_items[(n + 3) & 3] = item_of_fused(n + 3);
+            } else {
+                const Item it = item_of(n + 3, hint);
+                s_items[(n + 3) & 3] = it;
+                hint = it.b;
+            }
         }
 
         // ------------------------------------------ K streams of `cur`, V streams of `prev`
@@ -831,7 +930,7 @@ WsLayout ws_layout(int B, int Hq, int max_pages) {
     size_t o = 0;
     auto up = [](size_t x) { return (x + 15) & ~(size_t)15; };
     w.off_counter = o; o += 16;
-    w.off_prefix = o; o += up((size_t)(B + 1) * 4);
+    w.off_prefix = o; o += up((size_t)(B + 1) * 8);   // block prefix sums, then non-empty-sequence counts
     w.off_qrot = o; o += (size_t)B * Hq * kN * 4;
     w.off_q16 = o; o += (size_t)B * Hq * 16 * kN * 2;   // Hkv <= Hq rows blocks
     w.off_qsum = o; o += up((size_t)B * Hq * 4);
@@ -923,6 +1022,8 @@ static cudaError_t launch_attention_pass(const DqDevTable& tk, const DqDevTable&
     p.B = a.B; p.Hq = a.Hq * q_len; p.Hkv = a.Hkv; p.G = G;
     p.q_len = q_len; p.G1 = G1; p.Hq1 = a.Hq;
     p.q_total = q_total; p.q_first = q_first;
+    p.fused = a.fused && !wide; p.attn_grid = sm_count; p.flags = p.counter;
+    p.ne_before = p.prefix + (a.B + 1);
     p.item_tokens = nw * kChunk;
     p.rotate_q = tk.rotate; p.rotate_out = tv.rotate; p.has_mean = tk.has_mean;
     p.scale_log2 = a.sm_scale * 1.4426950408889634f;
@@ -937,7 +1038,8 @@ static cudaError_t launch_attention_pass(const DqDevTable& tk, const DqDevTable&
     cudaError_t e = dq_launch_pdl(dq_attn_prepare_kernel, dim3((unsigned)((prep_warps + 7) / 8)), dim3(256), 0, st, p);
     if (e != cudaSuccess) return e;
     if (!wide) {
-        e = cudaFuncSetAttribute(dq_attention_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, L.total);
+        e = p.fused ? cudaFuncSetAttribute(dq_attention_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, L.total)
+                    : cudaFuncSetAttribute(dq_attention_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, L.total);
         if (e != cudaSuccess) return e;
     }
     const bool prof = g_prof_on && g_prof_count < kProfRing && (g_prof_calls++ % g_prof_period) == 0;
@@ -950,7 +1052,8 @@ static cudaError_t launch_attention_pass(const DqDevTable& tk, const DqDevTable&
         cudaEventRecord(g_prof_ev[g_prof_count][0], st);
     }
     if (wide) e = dq_launch_attention_wide_main(tk, tv, p, nw, sm_count, st);
-    else e = dq_launch_pdl(dq_attention_kernel, dim3(sm_count), dim3(nw * 32), (size_t)L.total, st, tk, tv, p);
+    else if (p.fused) e = dq_launch_pdl(dq_attention_kernel<true>, dim3(sm_count), dim3(nw * 32), (size_t)L.total, st, tk, tv, p);
+    else e = dq_launch_pdl(dq_attention_kernel<false>, dim3(sm_count), dim3(nw * 32), (size_t)L.total, st, tk, tv, p);
     if (e != cudaSuccess) return e;
     if (prof) cudaEventRecord(g_prof_ev[g_prof_count++][1], st);
     return dq_launch_pdl(dq_attn_combine_kernel, dim3(heads), dim3(256), 0, st, p);
@@ -969,6 +1072,18 @@ cudaError_t dq_launch_attention(const DqDevTable& tk, const DqDevTable& tv, cons
     }
     return cudaSuccess;
 }
+
+// Decode step: the caller has just launched the step's encoder (in decode-step mode) on `st`.
+cudaError_t dq_launch_step(const DqDevTable& tk, const DqDevTable& tv, const DqEncodeArgs& enc, const DqAttnArgs& a,
+                           cudaStream_t st) {
+    (void)enc;
+    DqAttnArgs b = a;
+    b.fused = 1;
+    b.q_len = 1;
+    return dq_launch_attention(tk, tv, b, st);
+}
+
+int* dq_attn_workspace_flags(void* workspace) { return reinterpret_cast<int*>(workspace); }
 
 cudaError_t dq_launch_bf16_attention(const DqAttnArgs& a, const void* k_pages, const void* v_pages,
                                      cudaStream_t st) {
@@ -994,6 +1109,7 @@ cudaError_t dq_launch_bf16_attention(const DqAttnArgs& a, const void* k_pages, c
     p.hkv_magic = 0;
     p.hs = 1; p.groups = a.Hkv;
     p.q_len = 1; p.G1 = p.G; p.Hq1 = a.Hq; p.q_total = 1; p.q_first = 0;
+    p.fused = 0; p.attn_grid = 0; p.flags = p.counter; p.ne_before = p.prefix + (a.B + 1);
     p.resid_k = nullptr; p.resid_v = nullptr; p.resid_lens = nullptr; p.resid_cap = 0;
     const int heads = a.B * a.Hq;
     dq_attn_prepare_kernel<<<(heads + 7) / 8, 256, 0, st>>>(p);

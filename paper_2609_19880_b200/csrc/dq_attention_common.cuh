@@ -42,6 +42,12 @@ struct AttnParams {
     // r = i * G1 + g; G = q_len * G1 rows per KV head and Hq = Hkv * G rows per sequence everywhere in the
     // workspace.  Query token i is q_len - 1 - i positions before the end of the sequence.
     int q_len, G1, Hq1; // query tokens of this pass; query heads per KV head and per token
+    // Decode-step mode (dq_decode_step): the attention kernel starts while the step's encoder still runs.
+    // flags: [0] next dynamic item, [1] set when the prepare kernel's outputs are complete, [2] prepare
+    // CTAs finished, [3] times a CTA gave up polling [1].  ne_before[b]: non-empty sequences before b.
+    int fused, attn_grid;
+    int* flags;
+    int* ne_before;
     int q_total, q_first; // tokens per sequence in q / out, and the first one this pass handles (a call with
                         // more rows than one MMA tile holds is run as several passes)
     const uint16_t* resid_k;      // bf16 [B][resid_cap][Hkv][128], nullable: uncompressed recent tokens

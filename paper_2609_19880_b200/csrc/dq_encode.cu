@@ -197,6 +197,10 @@ __device__ __forceinline__ uint32_t drift(const EncTable& T, const float (&z)[4]
 
 constexpr int kEncWarps = 8;
 
+// Position and sequence of call token t (decode-step mode derives them from the sequence lengths).
+__device__ __forceinline__ int tok_pos(const DqEncodeArgs& a, int t) { return a.step_seq_lens ? a.step_seq_lens[t] - 1 : a.pos[t]; }
+__device__ __forceinline__ int tok_seq(const DqEncodeArgs& a, int t) { return a.step_seq_lens ? t : a.seq_id[t]; }
+
 struct StreamQuantised {
     uint32_t hdr0;      // s fp16 | o fp16 << 16
     uint32_t flags;     // 1: all-central fallback, 2: constant stream, 4: refit rejected
@@ -216,11 +220,11 @@ __device__ __forceinline__ StreamQuantised quantise_stream(const EncTable& T, co
         z[2] = bf16_bits_to_float(raw.y & 0xffffu); z[3] = bf16_bits_to_float(raw.y >> 16);
     }
     if (!is_v && a.rope_style)
-        warp_rope128(z, lane, a.rope_cos + (size_t)a.pos[t] * 64, a.rope_sin + (size_t)a.pos[t] * 64, a.rope_style);
+        warp_rope128(z, lane, a.rope_cos + (size_t)tok_pos(a, t) * 64, a.rope_sin + (size_t)tok_pos(a, t) * 64, a.rope_style);
     if (T.rotate) warp_fwht128(z, lane);
     if (T.has_mean) {  // remove the (dequantised) windowed channel mean, Sec. 4.2
-        const int ps = a.pos[t], w = ps / DQ_WINDOW_TOKENS;
-        const size_t mi = ((size_t)a.seq_id[t] * a.max_windows + w) * Hkv + h;
+        const int ps = tok_pos(a, t), w = ps / DQ_WINDOW_TOKENS;
+        const size_t mi = ((size_t)tok_seq(a, t) * a.max_windows + w) * Hkv + h;
         uint32_t q4;
         float sc;
         if (a.mean_mode == DQ_MEAN_REUSE && ps % DQ_WINDOW_TOKENS == 0) {
@@ -326,7 +330,10 @@ dq_encode_kernel(const __grid_constant__ DqDevTable TK, const __grid_constant__ 
     __shared__ EncTable T;
     __shared__ uint8_t s_bytes[kEncWarps][DQ_MAX_REC_BYTES];
     __shared__ __align__(4) uint8_t s_sym[kEncWarps][kN];
-    dqdev::pdl_launch_dependents();
+    // Decode-step mode: the kernels after this one start while it runs and take their own launch as proof
+    // that everything before this kernel has finished, so the trigger comes after the wait (and after the
+    // hand-over words are cleared).  Otherwise: trigger first, so that the next kernel's launch overlaps this one.
+    if (!a.step_flags) dqdev::pdl_launch_dependents();
     const bool is_v = a.do_k ? (blockIdx.y == 1) : true;
     if (threadIdx.x < DQ_MAX_LEVELS) {
         const int i = threadIdx.x;
@@ -346,9 +353,18 @@ dq_encode_kernel(const __grid_constant__ DqDevTable TK, const __grid_constant__ 
     }
     __syncthreads();
     dqdev::pdl_wait_prior_grid();   // inputs and the cache may be written / read by the previous kernel
+    if (a.step_flags) {
+        if (blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x < 4) {
+            a.step_flags[threadIdx.x] = 0;
+            __threadfence();
+        }
+        __syncthreads();
+        dqdev::pdl_launch_dependents();
+    }
     const int lane = threadIdx.x & 31, wib = threadIdx.x >> 5;
     const long long wid = (long long)blockIdx.x * kEncWarps + wib;
     if (wid >= (long long)a.T * a.Hkv) return;
+    if (tok_pos(a, (int)(wid / a.Hkv)) < 0) return;   // decode-step mode: an empty sequence has no new token
     const int t = (int)(wid / a.Hkv), h = (int)(wid % a.Hkv), Hkv = a.Hkv;
     uint8_t* cont = is_v ? a.v_cont : a.k_cont;
 
@@ -948,7 +964,7 @@ cudaError_t dq_launch_encode(const DqDevTable& tk, const DqDevTable& tv, const D
                              dim3(tk.hs * 32), (size_t)smem, st, tk, tv, a);
     }
     const unsigned blocks = (unsigned)((warps + kEncWarps - 1) / kEncWarps);
-    if (warps >= 4LL * 148 * kB32 * 4)   // enough streams to fill the GPU at 4 CTAs per SM several times
+    if (!a.step_flags && warps >= 4LL * 148 * kB32 * 4)   // enough streams to fill the GPU at 4 CTAs per SM several times
         return dq_launch_pdl(dq_encode_batch32_kernel<DQ_B32_MINB>, dim3((unsigned)((warps + kB32 - 1) / kB32), (a.do_k && a.do_v) ? 2 : 1),
                              dim3(kEncWarps * 32), 0, st, tk, tv, a);
     return dq_launch_pdl(dq_encode_kernel<2>, dim3(blocks, (a.do_k && a.do_v) ? 2 : 1), dim3(kEncWarps * 32), 0, st, tk, tv, a);

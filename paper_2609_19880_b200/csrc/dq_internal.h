@@ -46,6 +46,10 @@ struct DqEncodeArgs {
     const float* rope_cos;   // [positions][64], nullable: keys are handed over before their rotary embedding
     const float* rope_sin;
     int rope_style;          // 0 none, DQ_ROPE_HALF, DQ_ROPE_PAIRS
+    // Decode-step mode (dq_decode_step): token t is the newest token of sequence t, at position
+    // step_seq_lens[t] - 1 (sequences of length 0 have none); seq_id / pos are not read.
+    const int32_t* step_seq_lens;
+    int* step_flags;         // decode-step mode: 4 hand-over words this kernel clears for the kernels after it
 };
 cudaError_t dq_launch_encode(const DqDevTable& tk, const DqDevTable& tv, const DqEncodeArgs& a, cudaStream_t st);
 cudaError_t dq_launch_decode_tokens(const DqDevTable& t, const uint8_t* cont, const int8_t* mean_q,
@@ -74,8 +78,12 @@ struct DqAttnArgs {
     const int32_t* resid_lens;  // [B]
     int resid_cap;
     int q_len;                  // query tokens per sequence (q and out are [B][q_len][Hq][128]); 0 or 1: one
+    int fused;                  // decode-step mode: launched right after the step's encoder (see dq_decode_step)
 };
 size_t dq_attn_workspace_bytes(int B, int Hq, int max_pages);
+int* dq_attn_workspace_flags(void* workspace);   // the 4 scheduling / hand-over words at the head of a workspace
+cudaError_t dq_launch_step(const DqDevTable& tk, const DqDevTable& tv, const DqEncodeArgs& enc, const DqAttnArgs& a,
+                           cudaStream_t st);   // encode -> prepare -> attention -> combine
 cudaError_t dq_launch_attention(const DqDevTable& tk, const DqDevTable& tv, const DqAttnArgs& a,
                                 cudaStream_t st);
 cudaError_t dq_attn_static_scratch(void** out);
