@@ -196,6 +196,9 @@ __device__ __forceinline__ uint32_t drift(const EncTable& T, const float (&z)[4]
 // ---------------------------------------------------------------------- encoder
 
 constexpr int kEncWarps = 8;
+#ifndef DQ_STEP_ENC_WARPS
+#define DQ_STEP_ENC_WARPS 16
+#endif
 
 // Position and sequence of call token t (decode-step mode derives them from the sequence lengths).
 __device__ __forceinline__ int tok_pos(const DqEncodeArgs& a, int t) { return a.step_seq_lens ? a.step_seq_lens[t] - 1 : a.pos[t]; }
@@ -323,13 +326,15 @@ __device__ __forceinline__ StreamQuantised quantise_stream(const EncTable& T, co
 // the tensor kind when keys and values are encoded by one launch.
 // MINB CTAs per SM: 2 leaves every thread 128 registers (lowest latency: the single-token step), 4 trades a
 // few spills for twice the resident warps (throughput: prefill, bulk encodes).
-template <int MINB>
-__global__ void __launch_bounds__(kEncWarps * 32, MINB)
+// WARPS streams per CTA: 8 normally; the decode step uses 16 (512 threads at full register budget) so that its
+// 2 B Hkv streams occupy few SMs while the attention kernel runs on all the others.
+template <int MINB, int WARPS>
+__global__ void __launch_bounds__(WARPS * 32, MINB)
 dq_encode_kernel(const __grid_constant__ DqDevTable TK, const __grid_constant__ DqDevTable TV,
                  const DqEncodeArgs a) {
     __shared__ EncTable T;
-    __shared__ uint8_t s_bytes[kEncWarps][DQ_MAX_REC_BYTES];
-    __shared__ __align__(4) uint8_t s_sym[kEncWarps][kN];
+    __shared__ uint8_t s_bytes[WARPS][DQ_MAX_REC_BYTES];
+    __shared__ __align__(4) uint8_t s_sym[WARPS][kN];
     // Decode-step mode: the kernels after this one start while it runs and take their own launch as proof
     // that everything before this kernel has finished, so the trigger comes after the wait (and after the
     // hand-over words are cleared).  Otherwise: trigger first, so that the next kernel's launch overlaps this one.
@@ -362,7 +367,7 @@ dq_encode_kernel(const __grid_constant__ DqDevTable TK, const __grid_constant__ 
         dqdev::pdl_launch_dependents();
     }
     const int lane = threadIdx.x & 31, wib = threadIdx.x >> 5;
-    const long long wid = (long long)blockIdx.x * kEncWarps + wib;
+    const long long wid = (long long)blockIdx.x * WARPS + wib;
     if (wid >= (long long)a.T * a.Hkv) return;
     if (tok_pos(a, (int)(wid / a.Hkv)) < 0) return;   // decode-step mode: an empty sequence has no new token
     const int t = (int)(wid / a.Hkv), h = (int)(wid % a.Hkv), Hkv = a.Hkv;
@@ -967,5 +972,10 @@ cudaError_t dq_launch_encode(const DqDevTable& tk, const DqDevTable& tv, const D
     if (!a.step_flags && warps >= 4LL * 148 * kB32 * 4)   // enough streams to fill the GPU at 4 CTAs per SM several times
         return dq_launch_pdl(dq_encode_batch32_kernel<DQ_B32_MINB>, dim3((unsigned)((warps + kB32 - 1) / kB32), (a.do_k && a.do_v) ? 2 : 1),
                              dim3(kEncWarps * 32), 0, st, tk, tv, a);
-    return dq_launch_pdl(dq_encode_kernel<2>, dim3(blocks, (a.do_k && a.do_v) ? 2 : 1), dim3(kEncWarps * 32), 0, st, tk, tv, a);
+    if (a.step_flags) {   // decode step: big CTAs, so that few SMs are kept from the attention kernel
+        constexpr int kStepWarps = DQ_STEP_ENC_WARPS;
+        return dq_launch_pdl(dq_encode_kernel<1, kStepWarps>, dim3((unsigned)((warps + kStepWarps - 1) / kStepWarps), (a.do_k && a.do_v) ? 2 : 1),
+                             dim3(kStepWarps * 32), 0, st, tk, tv, a);
+    }
+    return dq_launch_pdl(dq_encode_kernel<2, kEncWarps>, dim3(blocks, (a.do_k && a.do_v) ? 2 : 1), dim3(kEncWarps * 32), 0, st, tk, tv, a);
 }
