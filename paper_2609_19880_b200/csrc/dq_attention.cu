@@ -1022,7 +1022,10 @@ static cudaError_t launch_attention_pass(const DqDevTable& tk, const DqDevTable&
     p.B = a.B; p.Hq = a.Hq * q_len; p.Hkv = a.Hkv; p.G = G;
     p.q_len = q_len; p.G1 = G1; p.Hq1 = a.Hq;
     p.q_total = q_total; p.q_first = q_first;
-    p.fused = a.fused && !wide; p.attn_grid = sm_count; p.flags = p.counter;
+    // Decode-step mode pays (dynamic item order, late wait) while the encoder's ~20 us matter: not when every
+    // CTA has dozens of items anyway (upper bound from the page-table width; the lengths live on the device).
+    const long long max_items = (long long)a.B * ((a.max_pages * DQ_PAGE_TOKENS + nw * kChunk - 1) / (nw * kChunk)) * a.Hkv;
+    p.fused = a.fused && !wide && max_items <= 32LL * sm_count; p.attn_grid = sm_count; p.flags = p.counter;
     p.ne_before = p.prefix + (a.B + 1);
     p.item_tokens = nw * kChunk;
     p.rotate_q = tk.rotate; p.rotate_out = tv.rotate; p.has_mean = tk.has_mean;
