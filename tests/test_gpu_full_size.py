@@ -240,3 +240,45 @@ def test_config4_ragged_paged_token_wide_full():
     cfg = workloads.make_config(4)
     assert cfg.batch == 128 and cfg.shuffle_pages
     _run_config_wide(cfg, 14)
+
+
+def test_config5_decode_step_full():
+    """Config 5 at full size through dq_decode_step (overlapped encoder / attention): 64 steps, every
+    step bit-identical to dq_encode_tokens + dq_decode_attention on a second cache; sampled rows of the
+    last step against the oracle."""
+    cfg = workloads.make_config(5)
+    steps = 64
+    rng = np.random.default_rng(55)
+    w = workloads.generate(cfg, device="cuda", extra_tokens_per_seq=steps)
+    tk, tv, ok, ov = gc.tables(cfg)
+    ca, cb = gc.GpuCache(w, ok.rec, ov.rec), gc.GpuCache(w, ok.rec, ov.rec)
+    gc.gpu_encode(w, tk, tv, ca)
+    for name in ("k_cont", "v_cont", "mean_q", "mean_scale"):
+        getattr(cb, name).copy_(getattr(ca, name))
+    B, Hq, Hkv = cfg.batch, cfg.hq, cfg.hkv
+    gen = torch.Generator(device="cuda").manual_seed(56)
+    lens = torch.tensor(cfg.seq_lens, dtype=torch.int32)
+    seq = torch.arange(B, dtype=torch.int32).cuda()
+    pt_cpu = w.page_table.cpu()
+    ws = torch.empty(dq.dq_decode_workspace_bytes(B, Hq, w.page_table.shape[1]), dtype=torch.uint8, device="cuda")
+    out_a = torch.empty((B, Hq, 128), dtype=torch.bfloat16, device="cuda"); out32_a = torch.empty((B, Hq, 128), dtype=torch.float32, device="cuda")
+    out_b = torch.empty_like(out_a); out32_b = torch.empty_like(out32_a)
+    for s in range(steps):
+        k1, v1 = workloads.make_kv(cfg, B, gen, torch.device("cuda"), w.k_offsets, w.k_gain)
+        lens = lens + 1
+        pos = lens - 1
+        slot = (pt_cpu[torch.arange(B), (pos // 16).long()] * 16 + pos % 16).to(torch.int32).cuda()
+        lens_d = lens.cuda()
+        dq.dq_decode_step(tk, tv, k1, v1, slot, w.q, ca.k_cont, ca.v_cont, ca.mean_q, ca.mean_scale, w.page_table, lens_d,
+                          Hkv, gc.SM_SCALE, out_a, ws, out32_a, ca.status)
+        dq.dq_encode_tokens(tk, tv, k1, v1, seq, pos.cuda(), slot, cb.k_cont, cb.v_cont, cb.mean_q, cb.mean_scale,
+                            dq.MEAN_REUSE, cb.status)
+        dq.dq_decode_attention(tk, tv, w.q, cb.k_cont, cb.v_cont, cb.mean_q, cb.mean_scale, w.page_table, lens_d, Hkv,
+                               gc.SM_SCALE, out_b, ws, out32_b)
+        if s % 8 == 7:
+            torch.cuda.synchronize()
+            assert torch.equal(out32_a, out32_b) and torch.equal(out_a, out_b), s
+    torch.cuda.synchronize()
+    assert torch.equal(ca.k_cont, cb.k_cont) and torch.equal(ca.v_cont, cb.v_cont) and torch.equal(ca.mean_q, cb.mean_q)
+    assert int(_np(ws[:16].view(torch.int32))[3]) == 0
+    _check_attention_sample(w, tk, tv, ok, ov, ca, _host(ca), rng, rows=2, seq_lens=lens.cuda())
