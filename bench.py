@@ -310,18 +310,25 @@ def run_ours(args):
         win_idx = torch.cat([torch.arange(int(e) - 128, int(e)) for e in torch.cumsum(lens, 0)]).to(dev)
         win_seq, win_pos, win_slot = (t[win_idx].contiguous() for t in (w.seq_id, w.pos, w.slot))
 
-        def step(i, q=w.q, nk=new_k, nv=new_v):
+        def step_core(i, q=w.q, nk=new_k, nv=new_v):   # the same launches every step (the counts live on the device)
             c = caches[i % copies]
             dq.dq_window_append(nk, nv, rk, rv, rl)
-            state["r"] += 1
             dq.dq_decode_attention_residual(tk, tv, q, c["k"], c["v"], c["mq"], c["ms"], w.page_table, w.seq_lens,
                                             rk, rv, rl, Hkv, sm_scale, out, ws)
+
+        def step_close(i):                             # after every 128th step: the full window becomes compressed
+            state["r"] += 1
             if state["r"] == 128:
+                c = caches[i % copies]
                 dq.dq_encode_tokens(tk, tv, rk.view(B * 128, Hkv, 128), rv.view(B * 128, Hkv, 128), win_seq, win_pos,
                                     win_slot, c["k"], c["v"], c["mq"], c["ms"], dq.MEAN_COMPUTE)
                 rl.zero_()
                 state["closes"] += 1
                 state["r"] = 0
+
+        def step(i, q=w.q, nk=new_k, nv=new_v):
+            step_core(i, q, nk, nv)
+            step_close(i)
         launches_per_step = 4 + 3.0 / 128   # window append, prepare, fused attention, combine; means + K/V encode per 128 steps
         step_desc = ("append the new token to a 128-token BF16 window + decode attention over the compressed cache "
                      "and the window; a full window is encoded in bulk (once per 128 steps)")
@@ -388,10 +395,10 @@ def run_ours(args):
     h2d = hin.numel() * 2
     d2h = hout.numel() * 2
 
-    # One CUDA graph per cache copy holds the whole step (H2D copy, the library's launches, D2H copy);
-    # the token-wide policy changes its arguments every step and is launched directly.
+    # One CUDA graph per cache copy holds the whole step (H2D copy, the library's launches, D2H copy).
     graphs, graph_note = None, "direct launches"
-    if hs == 1 and not args.no_graph:
+    core = step if hs == 1 else step_core
+    if not args.no_graph:
         try:
             torch.cuda.synchronize()
             graphs = []
@@ -399,10 +406,14 @@ def run_ours(args):
                 g = torch.cuda.CUDAGraph()
                 with torch.cuda.graph(g):
                     din.copy_(hin, non_blocking=True)
-                    step(c_i, dq_q, dk, dv)
+                    core(c_i, dq_q, dk, dv)
                     hout.copy_(out, non_blocking=True)
                 graphs.append(g)
             graph_note = f"one CUDA graph per cache copy ({copies})"
+            if hs > 1:
+                graph_note += "; the window's bulk encode every 128 steps is launched directly"
+                rl.zero_()            # the captures' warm-up runs appended tokens
+                state["r"] = 0
         except Exception as ex:   # capture is an optimisation of the launch path only
             graphs, graph_note = None, f"direct launches (graph capture failed: {type(ex).__name__})"
             torch.cuda.synchronize()
@@ -412,8 +423,10 @@ def run_ours(args):
             graphs[i % copies].replay()
         else:
             din.copy_(hin, non_blocking=True)
-            step(i, dq_q, dk, dv)
+            core(i, dq_q, dk, dv)
             hout.copy_(out, non_blocking=True)
+        if hs > 1:
+            step_close(i)
         torch.cuda.synchronize()
 
     for i in range(3):
