@@ -29,7 +29,7 @@ constexpr int kRingK = kRowsK * 128, kRingV = kRowsV * 128;
 constexpr int kTile = 1024;                    // [32 tok][16 ch] fp16, 32-byte rows, halves swizzled by (row >> 2) & 1
 constexpr int kFillRows = 12;                  // rows fetched when a stream starts (header + 40 bytes)
 constexpr int kAhead = 10;                     // rows kept beyond the fastest lane's word index
-constexpr int kWideWarps = 15;                 // most warps per CTA (480 threads leave 136 registers each)
+constexpr int kWideWarps = 15;                 // most warps per CTA: the rings of a 16th do not fit the shared memory
 
 struct Item {
     int b, grp, blk, len, bg, valid;
