@@ -345,7 +345,10 @@ def run_ours(args):
     barrier()
 
     # ---- timed region: exactly K steps, CUDA events on the launch stream
-    dq.dq_profile_enable(8)   # CUDA events around the fused kernel of every 8th step
+    # CUDA events around the fused kernel of every prof_period-th step (the events serialise that step's
+    # kernels, ~20 us each time, so they are kept sparse; at least 4 samples)
+    prof_period = max(1, min(int(os.environ.get("DQ_BENCH_PROFILE_PERIOD", "16")), args.steps // 4))
+    dq.dq_profile_enable(prof_period)
     t_wall0 = time.time()
     closes0 = state["closes"]
     e0.record()
