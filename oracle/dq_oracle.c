@@ -36,9 +36,9 @@
  * Pins (tests/test_oracle_*.py): closed-form storage accounting, the feasibility
  * boundary and NMSE curve of Table 2, rANS round trip, Shannon bound, orthonormal
  * self-inverse Hadamard, brute-force drift optimality, textbook special cases.
- * PARITY UNPINNED by the paper (defined only by this build's contract): the INT8
- * window-mean quantiser, the mean carry-forward rule for appended tokens and the
- * automatic choice of alpha.
+ * PARITY UNPINNED by the paper (defined only by this build's contract): the mean
+ * carry-forward rule for appended tokens and the automatic choice of alpha.  (The INT8
+ * window-mean quantiser is pinned to a library per-tensor quantiser.)
  */
 #define _GNU_SOURCE
 #include <math.h>

@@ -57,6 +57,30 @@ def test_window_mean_is_the_rotated_channel_mean(small):
             assert np.abs(mq[b, win]).max(axis=1).min() == 127      # scale uses the full range
 
 
+def test_window_mean_quantiser_is_symmetric_absmax_int8(small):
+    """The INT8 step is plain symmetric abs-max quantisation: against torch's per-tensor affine
+    quantiser (scale = max |mean| / 127, zero point 0, round half to even) on an independently
+    computed rotated mean.  The two means differ by binary32 summation order, so a code may differ
+    by one step where the mean sits on a rounding boundary; nothing else may differ."""
+    w, tk, tv, kc, vc, mq, ms, sk, sv = small
+    H = (hadamard(128) / math.sqrt(128)).astype(np.float64)
+    k = w.k.float().numpy().astype(np.float64)
+    seq_id, pos = w.seq_id.numpy(), w.pos.numpy()
+    total = off_by_one = 0
+    for b in range(w.cfg.batch):
+        for win in range((w.cfg.seq_lens[b] + 127) // 128):
+            sel = (seq_id == b) & (pos // 128 == win)
+            mu = (k[sel].mean(0) @ H.T).astype(np.float32)          # [Hkv, 128]
+            for h in range(w.cfg.hkv):
+                scale = float(ms[b, win, h])
+                assert abs(scale - np.abs(mu[h]).max() / 127.0) <= 2e-6 * max(scale, 1e-30) + 1e-9
+                q = torch.quantize_per_tensor(torch.from_numpy(mu[h]), scale, 0, torch.qint8).int_repr().numpy()
+                d = np.abs(q.astype(np.int32) - mq[b, win, h].astype(np.int32))
+                assert d.max() <= 1
+                total += d.size; off_by_one += int((d == 1).sum())
+    assert off_by_one <= 0.01 * total
+
+
 def test_mean_reuse_copies_previous_window():
     n, Hkv = 128, 2
     rng = np.random.default_rng(0)
