@@ -621,6 +621,9 @@ dq_attention_kernel(const __grid_constant__ DqDevTable TK, const __grid_constant
         if (tid == 0) s_prev_row[n & 1] = (long long)cur.bg * p.Hq + (long long)cur.h * G;   // read after two barriers
     }
     cp_async_wait<0>();
+    // decode-step mode: no CTA leaves before the preceding kernels are complete, so that this kernel's end
+    // implies theirs whatever the item mix was (returns at once by now)
+    if (FUSED && !waited) pdl_wait_prior_grid();
 }
 
 // ------------------------------------------------------------------ combine
