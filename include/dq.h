@@ -5,10 +5,16 @@
  * keys and values of every token in fixed-size, rANS-coded containers and decodes
  * them inside the decode-step attention kernel.  This library holds that path:
  *
- *   dq_build_tables      normal-derived rANS tables             (Sec. 3.1, 4.2, 4.4)
- *   dq_encode_tokens     K/V bf16 -> containers + window means  (Fig. 1, Algorithm 1)
- *   dq_decode_attention  q, containers -> attention output      (Algorithm 2, App. A)
- *   dq_decode_tokens     containers -> symbols / dequantised values (Algorithm 2; checks)
+ *   dq_build_tables           normal-derived rANS tables                  (Sec. 3.1, 4.2, 4.4)
+ *   dq_encode_tokens          K/V bf16 -> containers + window means       (Fig. 1, Algorithm 1)
+ *   dq_encode_tokens_rope     the same for keys handed over before their rotary embedding
+ *   dq_decode_attention       q, containers -> attention output           (Algorithm 2, App. A)
+ *   dq_decode_step            newest token encoded + attention, one overlapped launch sequence
+ *   dq_decode_attention_residual / dq_window_append
+ *                             the BF16 window of the most recent tokens   (Sec. 5.1)
+ *   dq_decode_attention_multi several query tokens per sequence in one pass over the cache
+ *   dq_decode_attention_static  dq_decode_attention without any allocation at call time
+ *   dq_decode_tokens          containers -> symbols / dequantised values  (Algorithm 2; checks)
  *   dq_bf16_decode_attention  plain bf16-cache decode attention (comparison baseline)
  *
  * Conventions
