@@ -283,6 +283,9 @@ __device__ __forceinline__ void fused_pass(uint32_t xk, uint32_t ptrk, uint32_t 
 // from a global counter (SMs still busy with the encoder join late and simply take fewer), leaves the
 // blocks that hold a sequence's newest token to the end of the item order, and waits for the preceding
 // kernels -- whose completion implies the encoder's -- only before the first of those blocks.
+#ifndef DQ_STEP_POLL_LIMIT
+#define DQ_STEP_POLL_LIMIT (1 << 16)   // polls of the ready flag (64 ns apart) before a CTA falls back to the grid wait
+#endif
 template <bool FUSED>
 __global__ void __launch_bounds__(kMaxWarps * 32, 1)
 dq_attention_kernel(const __grid_constant__ DqDevTable TK, const __grid_constant__ DqDevTable TV,
@@ -315,7 +318,7 @@ dq_attention_kernel(const __grid_constant__ DqDevTable TK, const __grid_constant
         int* s_ok = reinterpret_cast<int*>(smem + L.off_items);
         if (tid == 0) {
             int ok = 0;
-            for (int it = 0; it < (1 << 16) && !ok; ++it) {
+            for (int it = 0; it < DQ_STEP_POLL_LIMIT && !ok; ++it) {
                 asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(ok) : "l"(p.flags + 1) : "memory");
                 if (!ok) __nanosleep(64);
             }
