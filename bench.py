@@ -442,6 +442,12 @@ def run_ours(args):
     e2e_s = time.perf_counter() - t0
     e2e_s = max_over_ranks(e2e_s, world, dev)
     e2e_value = job_throughput(kv_tokens, e2e_s / args.steps, world)
+    # what came back to the host must be what a direct call computes (same inputs, same cache contents)
+    e2e_check = None
+    if hs == 1:
+        step(0)
+        torch.cuda.synchronize()
+        e2e_check = bool(torch.equal(hout, out.cpu()))
 
     if rank != 0:
         if world > 1:
@@ -522,7 +528,7 @@ def run_ours(args):
                    "parallelism": "replicas only" if world > 1 else "single GPU"},
         "roofline": roofline, "cpu_baseline": cpu,
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
-                "launch": graph_note},
+                "launch": graph_note, "output_equals_direct_call": e2e_check},
         "gpu_launches": int(round(launches_per_step * args.steps)), "clocks": clocks,
         "encoder": {"token_heads_per_s": 2 * token_heads / (enc_ms * 1e-3), "prefill_ms": enc_ms,
                     "streams": 2 * token_heads // hs},
