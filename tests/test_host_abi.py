@@ -142,6 +142,22 @@ def test_calls_validate_before_launch(L):
     # several query tokens: the workspace must hold one pass of min(q_len, 8 / (Hq / Hkv)) tokens
     assert call_m(0) == -1 and call_m(2, wsb=ws) == -4 and call_m(5, wsb=dq.dq_decode_workspace_bytes(2, 64, 8) - 1) == -4
     assert call_m(2, q=n, wsb=dq.dq_decode_workspace_bytes(2, 64, 8)) == -1
+    # decode step in one call: per token-head tables only; same checks as the two calls it stands for
+    def call_s(**kw):
+        d = dict(a); d.update(kw)
+        return L.dq_decode_step(d["tk"], d["tv"], d.get("kn", fake), d.get("vn", fake), d.get("sn", fake), d["q"], d["kc"],
+                                d["vc"], d["mq"], d["ms"], d["mw"], d["pt"], d["mp"], d["sl"], d["B"], d["Hq"], d["Hkv"],
+                                d["sm"], d["ob"], d["of"], d["ws"], d["wsb"], n, d["st"])
+
+    assert call_s(kn=n) == -1 and call_s(sn=n) == -1 and call_s(q=n) == -1 and call_s(wsb=ws - 1) == -4
+    assert call_s(kn=C.c_void_p(0x1004)) == -1 and call_s(mq=n) == -1
+    tw = dq.dq_build_tables(8, 335 * 8 / 1024, has_mean=True, heads_per_stream=8)
+    twv = dq.dq_build_tables(6, 235 * 8 / 1024, heads_per_stream=8)
+    assert call_s(tk=tw.handle, tv=twv.handle) == -3 and call_s(tk=tw.handle) == -3
+    # BF16 window append
+    assert L.dq_window_append(n, fake, fake, fake, fake, 128, 2, 8, n) == -1
+    assert L.dq_window_append(fake, fake, fake, fake, fake, 0, 2, 8, n) == -1
+    assert L.dq_window_append(fake, fake, C.c_void_p(0x1008), fake, fake, 128, 2, 8, n) == -1
     assert L.dq_decode_tokens(tk.handle, n, n, n, 0, n, n, fake, 4, 8, fake, n, n) == -1
     assert L.dq_bf16_decode_attention(fake, n, fake, fake, 8, fake, 2, 32, 8, C.c_float(0.1), fake, fake, ws, n) == -1
 
