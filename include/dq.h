@@ -38,7 +38,9 @@
  *     together: uint8 [num_pages][Hkv / hs][rec_words][16][4], rec_words = ceil(rec_bytes / 4);
  *     byte i of the record of (page, group, token-in-page t) sits at
  *     ((page * (Hkv / hs) + group) * rec_words + i / 4) * 64 + t * 4 + i % 4; bytes past
- *     rec_bytes in the last word are zero.
+ *     rec_bytes in the last word are zero.  The attention kernel addresses such an array in
+ *     16-byte units with 32 bits: one token-wide container array may span at most 64 GiB
+ *     (every page id in the page table times the page's bytes must stay below 2^36).
  *   - Key channel means: one per (sequence, window of 128 positions, KV head):
  *     int8 [S][max_windows][Hkv][128] and float scale [S][max_windows][Hkv];
  *     mean_j = scale * q_j, in the Hadamard-rotated domain.
