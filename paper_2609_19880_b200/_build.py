@@ -49,7 +49,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
         objs.append(o)
     if force or _newer(LIB_PATH, objs):
         tmp = LIB_PATH + f".{os.getpid()}.tmp"
-        subprocess.run([nvcc, "-shared", "-o", tmp] + objs, check=True)
+        subprocess.run([nvcc] + _COMMON[:2] + ["-shared", "-o", tmp] + objs, check=True)
         os.replace(tmp, LIB_PATH)
     return LIB_PATH
 

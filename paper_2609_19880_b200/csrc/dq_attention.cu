@@ -128,7 +128,6 @@ dq_attn_prepare_kernel(AttnParams p) {
         } else {
             uint32_t q4[kPrepWindows];
             float msc[kPrepWindows], s[kPrepWindows];
-#pragma unroll
             // Decode-step mode: when the newest token opens a window, the encoder is writing that window's
             // mean right now as a copy of the previous window's (zero for window 0): read the source instead.
             int w_open = -1;
@@ -136,6 +135,7 @@ dq_attn_prepare_kernel(AttnParams p) {
                 const int np = p.seq_lens[b] - 1;
                 if (np >= 0 && np % DQ_WINDOW_TOKENS == 0) w_open = np / DQ_WINDOW_TOKENS;
             }
+#pragma unroll
             for (int u = 0; u < kPrepWindows; ++u) {   // all loads first
                 const int w = min(win * kPrepWindows + u, p.windows - 1);
                 const int ws = (w == w_open) ? w - 1 : w;
