@@ -119,12 +119,12 @@ __device__ __noinline__ uint32_t drift_m(const EncTable& T, float z0, float z1, 
                                          uint32_t& sym_packed) {
     const float z[4] = {z0, z1, z2, z3};
     float tm[M], rm[M];
-    uint32_t Rm[M];
+    uint32_t Km[M];   // ceil(65536 r_m) << 8 | m: the minimum tree carries one word for length and index
 #pragma unroll
     for (int m = 0; m < M; ++m) {
         tm[m] = __fmaf_rn((float)m, s, o);
         rm[m] = T.r[m];
-        Rm[m] = T.R[m];
+        Km[m] = (T.R[m] << 8) | (uint32_t)m;
     }
     float D[4][M];
     float maxD = -INFINITY, minD = INFINITY;
@@ -153,27 +153,24 @@ __device__ __noinline__ uint32_t drift_m(const EncTable& T, float z0, float z1, 
 #pragma unroll
         for (int e = 0; e < 4; ++e) {
             float c[M];
-            uint32_t idx[M];
+            uint32_t key[M];
 #pragma unroll
-            for (int m = 0; m < M; ++m) { c[m] = __fmaf_rn(lam, rm[m], D[e][m]); idx[m] = (uint32_t)m; }
+            for (int m = 0; m < M; ++m) { c[m] = __fmaf_rn(lam, rm[m], D[e][m]); key[m] = Km[m]; }
             // pairwise minimum, the left (lower index) operand wins ties
 #pragma unroll
             for (int w = 1; w < M; w <<= 1)
 #pragma unroll
                 for (int m = 0; m + w < M; m += 2 * w)
-                    if (c[m + w] < c[m]) { c[m] = c[m + w]; idx[m] = idx[m + w]; }
-            sym[e] = idx[0];
-            uint32_t Rsel = Rm[0];
-#pragma unroll
-            for (int m = 1; m < M; ++m) Rsel = (idx[0] == (uint32_t)m) ? Rm[m] : Rsel;
-            cost_sum += Rsel;
+                    if (c[m + w] < c[m]) { c[m] = c[m + w]; key[m] = key[m + w]; }
+            sym[e] = key[0];
+            cost_sum += key[0];
         }
-        len = __reduce_add_sync(kFull, cost_sum);
+        len = __reduce_add_sync(kFull, cost_sum >> 8);   // four indices (< 16 each) stay below bit 8
         if (it < 12) {
             if (len <= budget) lam_hi = lam; else lam_lo = lam;
         }
     }
-    sym_packed = sym[0] | (sym[1] << 8) | (sym[2] << 16) | (sym[3] << 24);
+    sym_packed = (sym[0] & 0xffu) | ((sym[1] & 0xffu) << 8) | ((sym[2] & 0xffu) << 16) | (sym[3] << 24);
     return len;
 }
 
@@ -573,12 +570,12 @@ __device__ __noinline__ uint32_t drift_wide_m(const EncTable& T, WideShared& W, 
     const float z[4] = {z0, z1, z2, z3};
     const int lane = threadIdx.x & 31;
     float tm[M], rm[M];
-    uint32_t Rm[M];
+    uint32_t Km[M];   // ceil(65536 r_m) << 8 | m: the minimum tree carries one word for length and index
 #pragma unroll
     for (int m = 0; m < M; ++m) {
         tm[m] = __fmaf_rn((float)m, s, o);
         rm[m] = T.r[m];
-        Rm[m] = T.R[m];
+        Km[m] = (T.R[m] << 8) | (uint32_t)m;
     }
     float D[4][M];
     float maxD = -INFINITY, minD = INFINITY;
@@ -611,21 +608,18 @@ __device__ __noinline__ uint32_t drift_wide_m(const EncTable& T, WideShared& W, 
 #pragma unroll
         for (int e = 0; e < 4; ++e) {
             float c[M];
-            uint32_t idx[M];
+            uint32_t key[M];
 #pragma unroll
-            for (int m = 0; m < M; ++m) { c[m] = __fmaf_rn(lam, rm[m], D[e][m]); idx[m] = (uint32_t)m; }
+            for (int m = 0; m < M; ++m) { c[m] = __fmaf_rn(lam, rm[m], D[e][m]); key[m] = Km[m]; }
 #pragma unroll
             for (int w = 1; w < M; w <<= 1)
 #pragma unroll
                 for (int m = 0; m + w < M; m += 2 * w)
-                    if (c[m + w] < c[m]) { c[m] = c[m + w]; idx[m] = idx[m + w]; }
-            sym[e] = idx[0];
-            uint32_t Rsel = Rm[0];
-#pragma unroll
-            for (int m = 1; m < M; ++m) Rsel = (idx[0] == (uint32_t)m) ? Rm[m] : Rsel;
-            cost_sum += Rsel;
+                    if (c[m + w] < c[m]) { c[m] = c[m + w]; key[m] = key[m + w]; }
+            sym[e] = key[0];
+            cost_sum += key[0];
         }
-        const uint32_t wl = __reduce_add_sync(kFull, cost_sum);
+        const uint32_t wl = __reduce_add_sync(kFull, cost_sum >> 8);
         if (lane == 0) W.len[parity][wib] = wl;
         __syncthreads();
         len = 0;
@@ -635,7 +629,7 @@ __device__ __noinline__ uint32_t drift_wide_m(const EncTable& T, WideShared& W, 
             if (len <= budget) lam_hi = lam; else lam_lo = lam;
         }
     }
-    sym_packed = sym[0] | (sym[1] << 8) | (sym[2] << 16) | (sym[3] << 24);
+    sym_packed = (sym[0] & 0xffu) | ((sym[1] & 0xffu) << 8) | ((sym[2] & 0xffu) << 16) | (sym[3] << 24);
     return len;
 }
 
