@@ -61,17 +61,36 @@ dq_means_compute_kernel(const uint16_t* __restrict__ k, int T, int Hkv, int rota
     const int t0 = (int)(wid / Hkv), h = (int)(wid % Hkv);
     const int s = seq_id[t0], w = pos[t0] / DQ_WINDOW_TOKENS;
     if (t0 > 0 && seq_id[t0 - 1] == s && pos[t0 - 1] / DQ_WINDOW_TOKENS == w) return;
-    float acc[4] = {0.f, 0.f, 0.f, 0.f};
-    int t = t0;
-    for (; t < T; ++t) {
-        if (t > t0 && !(seq_id[t] == s && pos[t] / DQ_WINDOW_TOKENS == w)) break;
-        const uint2 raw = *reinterpret_cast<const uint2*>(k + ((size_t)t * Hkv + h) * kN + 4 * lane);
-        float kt[4] = {bf16_bits_to_float(raw.x & 0xffffu), bf16_bits_to_float(raw.x >> 16),
-                       bf16_bits_to_float(raw.y & 0xffffu), bf16_bits_to_float(raw.y >> 16)};
-        if (rope_style) warp_rope128(kt, lane, rope_cos + (size_t)pos[t] * 64, rope_sin + (size_t)pos[t] * 64, rope_style);
-#pragma unroll
-        for (int e = 0; e < 4; ++e) acc[e] = __fadd_rn(acc[e], kt[e]);
+    // length of the run: 32 candidates per round, lanes in parallel (the sums below stay sequential)
+    int cnt = 0;
+    for (int base = t0; base < T; base += 32) {
+        const int tt = base + lane;
+        const bool same = tt < T && seq_id[tt] == s && pos[tt] / DQ_WINDOW_TOKENS == w;
+        const unsigned m = __ballot_sync(kFull, same);
+        if (m != kFull) { cnt += __ffs((int)~m) - 1; break; }
+        cnt += 32;
     }
+    float acc[4] = {0.f, 0.f, 0.f, 0.f};
+    constexpr int kAheadLoads = 8;   // independent loads in flight; the additions keep token order
+    for (int tb = t0; tb < t0 + cnt; tb += kAheadLoads) {
+        uint2 raw[kAheadLoads];
+#pragma unroll
+        for (int u = 0; u < kAheadLoads; ++u) {
+            const int tt = min(tb + u, t0 + cnt - 1);
+            raw[u] = *reinterpret_cast<const uint2*>(k + ((size_t)tt * Hkv + h) * kN + 4 * lane);
+        }
+#pragma unroll
+        for (int u = 0; u < kAheadLoads; ++u) {
+            if (tb + u >= t0 + cnt) break;
+            float kt[4] = {bf16_bits_to_float(raw[u].x & 0xffffu), bf16_bits_to_float(raw[u].x >> 16),
+                           bf16_bits_to_float(raw[u].y & 0xffffu), bf16_bits_to_float(raw[u].y >> 16)};
+            if (rope_style)
+                warp_rope128(kt, lane, rope_cos + (size_t)pos[tb + u] * 64, rope_sin + (size_t)pos[tb + u] * 64, rope_style);
+#pragma unroll
+            for (int e = 0; e < 4; ++e) acc[e] = __fadd_rn(acc[e], kt[e]);
+        }
+    }
+    const int t = t0 + cnt;
     const float inv = __fdiv_rn(1.0f, (float)(t - t0));
 #pragma unroll
     for (int e = 0; e < 4; ++e) acc[e] = __fmul_rn(acc[e], inv);
