@@ -46,21 +46,13 @@ __device__ __forceinline__ void warp_rope128(float (&v)[4], int lane, const floa
 
 // ------------------------------------------------------------------ window means
 
-// DQ_MEAN_COMPUTE.  A run is a maximal range of consecutive call tokens with the same
-// (seq_id, pos / 128).  One warp per (run head token, KV head); warps whose token is not
-// the first of its run exit.  Sequential binary32 sum over the run, times 1/count, rotated,
-// quantised to INT8 with one scale (max |mean| / 127).
-__global__ void __launch_bounds__(256)
-dq_means_compute_kernel(const uint16_t* __restrict__ k, int T, int Hkv, int rotate,
-                        const int32_t* __restrict__ seq_id, const int32_t* __restrict__ pos,
-                        int8_t* __restrict__ mean_q, float* __restrict__ mean_scale, int Wmax,
-                        const float* __restrict__ rope_cos, const float* __restrict__ rope_sin, int rope_style) {
-    const int lane = threadIdx.x & 31;
-    const long long wid = (long long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
-    if (wid >= (long long)T * Hkv) return;
-    const int t0 = (int)(wid / Hkv), h = (int)(wid % Hkv);
+// Mean of the run that starts at call token t0, for KV head h, by one warp.
+__device__ __forceinline__ void means_of_run(const uint16_t* __restrict__ k, int T, int Hkv, int rotate,
+                                             const int32_t* __restrict__ seq_id, const int32_t* __restrict__ pos,
+                                             int8_t* __restrict__ mean_q, float* __restrict__ mean_scale, int Wmax,
+                                             const float* __restrict__ rope_cos, const float* __restrict__ rope_sin,
+                                             int rope_style, int t0, int h, int lane) {
     const int s = seq_id[t0], w = pos[t0] / DQ_WINDOW_TOKENS;
-    if (t0 > 0 && seq_id[t0 - 1] == s && pos[t0 - 1] / DQ_WINDOW_TOKENS == w) return;
     // length of the run: 32 candidates per round, lanes in parallel (the sums below stay sequential)
     int cnt = 0;
     for (int base = t0; base < T; base += 32) {
@@ -109,6 +101,36 @@ dq_means_compute_kernel(const uint16_t* __restrict__ k, int T, int Hkv, int rota
     const size_t mi = ((size_t)s * Wmax + w) * Hkv + h;
     *reinterpret_cast<uint32_t*>(mean_q + mi * kN + 4 * lane) = packed;
     if (lane == 0) mean_scale[mi] = sc;
+}
+
+// DQ_MEAN_COMPUTE.  A run is a maximal range of consecutive call tokens with the same
+// (seq_id, pos / 128).  A CTA looks at kMeansTokens consecutive call tokens, lists those that
+// start a run, and its warps take the (run, KV head) pairs in turn.  Sequential binary32 sum over
+// the run, times 1/count, rotated, quantised to INT8 with one scale (max |mean| / 127).
+constexpr int kMeansTokens = 128;
+__global__ void __launch_bounds__(256)
+dq_means_compute_kernel(const uint16_t* __restrict__ k, int T, int Hkv, int rotate,
+                        const int32_t* __restrict__ seq_id, const int32_t* __restrict__ pos,
+                        int8_t* __restrict__ mean_q, float* __restrict__ mean_scale, int Wmax,
+                        const float* __restrict__ rope_cos, const float* __restrict__ rope_sin, int rope_style) {
+    __shared__ int s_first[kMeansTokens];
+    __shared__ int s_n;
+    const int lane = threadIdx.x & 31;
+    if (threadIdx.x == 0) s_n = 0;
+    __syncthreads();
+    {
+        const long long tt = (long long)blockIdx.x * kMeansTokens + threadIdx.x;
+        if (threadIdx.x < kMeansTokens && tt < T) {
+            const int t = (int)tt;
+            const bool first = t == 0 || seq_id[t - 1] != seq_id[t] || pos[t - 1] / DQ_WINDOW_TOKENS != pos[t] / DQ_WINDOW_TOKENS;
+            if (first) s_first[atomicAdd(&s_n, 1)] = t;
+        }
+    }
+    __syncthreads();
+    const int tasks = s_n * Hkv;
+    for (int task = threadIdx.x >> 5; task < tasks; task += (int)(blockDim.x >> 5))
+        means_of_run(k, T, Hkv, rotate, seq_id, pos, mean_q, mean_scale, Wmax, rope_cos, rope_sin, rope_style,
+                     s_first[task / Hkv], task % Hkv, lane);
 }
 
 // ------------------------------------------------------------------------ drift
@@ -958,10 +980,9 @@ cudaError_t dq_launch_means(const DqDevTable& tk, const void* k_bf16, int T, int
                             const int32_t* seq_id, const int32_t* pos, int8_t* mean_q,
                             float* mean_scale, int max_windows, int mode, const float* rope_cos,
                             const float* rope_sin, int rope_style, cudaStream_t st) {
-    const long long warps = (long long)T * Hkv;
-    if (warps == 0) return cudaSuccess;
-    const unsigned blocks = (unsigned)((warps + 7) / 8);
+    if (T == 0 || Hkv == 0) return cudaSuccess;
     if (mode != DQ_MEAN_COMPUTE) return cudaSuccess;  // carry-forward is done by the encoder warps
+    const unsigned blocks = (unsigned)((T + kMeansTokens - 1) / kMeansTokens);
     dq_means_compute_kernel<<<blocks, 256, 0, st>>>((const uint16_t*)k_bf16, T, Hkv, tk.rotate, seq_id, pos,
                                                     mean_q, mean_scale, max_windows, rope_cos, rope_sin, rope_style);
     return cudaGetLastError();
