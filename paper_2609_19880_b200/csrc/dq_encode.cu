@@ -455,19 +455,24 @@ dq_encode_kernel(const __grid_constant__ DqDevTable TK, const __grid_constant__ 
 }
 
 
-// Throughput variant for calls with many streams: a CTA of 8 warps takes 32 consecutive streams.
-// Each warp quantises 4 of them (steps 1-6 of Algorithm 1, as above) and leaves the symbols in
+// Throughput variant for calls with many streams: a CTA of 4 warps takes 32 consecutive streams.
+// Each warp quantises 8 of them (steps 1-6 of Algorithm 1, as above) and leaves the symbols in
 // shared memory; then ONE warp entropy-codes all 32 streams at once, lane = stream, so the serial
 // rANS chain costs one instruction stream per 32 streams instead of one per stream with 32
 // redundant lanes.  Symbols are stored [position][stream] and emitted bytes [byte index][stream] so
-// that the lanes of that warp touch consecutive bytes.
+// that the lanes of that warp touch consecutive bytes.  Small CTAs, 8 per SM at 64 registers: the
+// other warps of a CTA idle during its rANS pass, so that pass should be a small part of a small CTA.
 #ifndef DQ_B32_MINB
-#define DQ_B32_MINB 4
+#define DQ_B32_MINB 8
+#endif
+#ifndef DQ_B32_WARPS
+#define DQ_B32_WARPS 4
 #endif
 constexpr int kB32 = 32;                 // streams per CTA
 constexpr int kB32SymStride = 36;        // bytes per position row (32 streams + pad against bank conflicts)
+constexpr int kB32Warps = DQ_B32_WARPS;
 template <int MINB>
-__global__ void __launch_bounds__(kEncWarps * 32, MINB)
+__global__ void __launch_bounds__(kB32Warps * 32, MINB)
 dq_encode_batch32_kernel(const __grid_constant__ DqDevTable TK, const __grid_constant__ DqDevTable TV,
                          const DqEncodeArgs a) {
     __shared__ EncTable T;
@@ -501,7 +506,7 @@ dq_encode_batch32_kernel(const __grid_constant__ DqDevTable TK, const __grid_con
     const int ns = (int)min((long long)kB32, total - first);
     uint8_t* cont = is_v ? a.v_cont : a.k_cont;
 
-    for (int i = wib; i < ns; i += kEncWarps) {   // quantise: warp w takes streams w, w + 8, ...
+    for (int i = wib; i < ns; i += kB32Warps) {   // quantise: warp w takes streams w, w + warps, ...
         const long long wid = first + i;
         const int t = (int)(wid / a.Hkv), h = (int)(wid % a.Hkv);
         const StreamQuantised sq = quantise_stream(T, a, is_v, t, h, lane);
@@ -1005,7 +1010,7 @@ cudaError_t dq_launch_encode(const DqDevTable& tk, const DqDevTable& tv, const D
     const unsigned blocks = (unsigned)((warps + kEncWarps - 1) / kEncWarps);
     if (!a.step_flags && warps >= 4LL * 148 * kB32 * 4)   // enough streams to fill the GPU at 4 CTAs per SM several times
         return dq_launch_pdl(dq_encode_batch32_kernel<DQ_B32_MINB>, dim3((unsigned)((warps + kB32 - 1) / kB32), (a.do_k && a.do_v) ? 2 : 1),
-                             dim3(kEncWarps * 32), 0, st, tk, tv, a);
+                             dim3(kB32Warps * 32), 0, st, tk, tv, a);
     if (a.step_flags) {   // decode step: big CTAs, so that few SMs are kept from the attention kernel
         constexpr int kStepWarps = DQ_STEP_ENC_WARPS;
         return dq_launch_pdl(dq_encode_kernel<1, kStepWarps>, dim3((unsigned)((warps + kStepWarps - 1) / kStepWarps), (a.do_k && a.do_v) ? 2 : 1),
