@@ -175,7 +175,8 @@ size_t dq_decode_workspace_bytes(int B, int Hq, int max_pages);
  *   out_bf16    device bf16 [B][Hq][128] (nullable if out_f32 is given)
  *   out_f32     device float [B][Hq][128], nullable: the result before bf16 rounding
  *   workspace   device, >= dq_decode_workspace_bytes(B, Hq, max_pages), 16-byte aligned
- * Hq must be a multiple of Hkv with Hq / Hkv <= 8 (else DQ_ERR_UNSUPPORTED). */
+ * Hq must be a multiple of Hkv with Hq / Hkv <= 8, and B <= 4096 (else DQ_ERR_UNSUPPORTED: the
+ * kernels keep the per-sequence block prefix sums in shared memory). */
 int dq_decode_attention(const dq_tables *tk, const dq_tables *tv, const void *q_bf16,
                         const uint8_t *k_cont, const uint8_t *v_cont, const int8_t *k_mean_q,
                         const float *k_mean_scale, int max_windows, const int32_t *page_table,

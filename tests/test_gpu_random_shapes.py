@@ -90,3 +90,31 @@ def test_random_shape(seed):
         ref = oracle.attention(ok, ov, workloads.bf16_bits(q[:, i]), kc, vc, mq, ms, _np(w.page_table), vis_c, Hkv,
                                gc.SM_SCALE, **kw)
         gc.check_attention(out[:, i].contiguous(), out32[:, i].contiguous(), ref)
+
+
+@pytest.mark.parametrize("wide", [False, True])
+def test_largest_batch(wide):
+    """B = 4096 (the most the attention calls accept), ragged lengths 0..20, shuffled pages."""
+    B, hkv, g = 4096, 8, 4
+    kr, vr, km, vm = workloads.BUDGETS[2.26]
+    lens = [int(x) for x in np.random.default_rng(B).integers(0, 21, size=B)]
+    cfg = workloads.Config("largest_batch", B, hkv * g, hkv, lens, 99, kr, vr, km, vm, shuffle_pages=True,
+                           v_student_t=False)
+    w = workloads.generate(cfg, device="cuda")
+    if wide:
+        tk, tv, ok, ov = gc.wide_tables(cfg, hkv, k_rec=335, v_rec=235)
+        cache = gc.WideGpuCache(w, tk, tv, hkv)
+    else:
+        tk, tv, ok, ov = gc.tables(cfg)
+        cache = gc.GpuCache(w, ok.rec, ov.rec)
+    gc.gpu_encode(w, tk, tv, cache)
+    out, out32 = gc.gpu_attention(w, tk, tv, cache)
+    torch.cuda.synchronize()
+    kc, vc, mq, ms, _, _ = gc.oracle_encode_wide(w, ok, ov, hkv) if wide else gc.oracle_encode(w, ok, ov)
+    got_k, got_v = _np(cache.k_cont), _np(cache.v_cont)
+    if wide:
+        got_k, got_v = gc.from_interleaved(got_k, ok.rec), gc.from_interleaved(got_v, ov.rec)
+    assert np.array_equal(got_k, kc) and np.array_equal(got_v, vc)
+    ref = oracle.attention(ok, ov, workloads.bf16_bits(w.q), kc, vc, mq, ms, _np(w.page_table), _np(w.seq_lens), hkv,
+                           gc.SM_SCALE)
+    gc.check_attention(out, out32, ref)
