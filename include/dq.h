@@ -138,6 +138,9 @@ int dq_tables_info(const dq_tables *t, dq_table_info *out);
  *                    [2] rejected refits, [3] max record bytes used (atomicMax).
  * With token-wide tables (heads_per_stream = hs > 1; both tables must agree, Hkv % hs == 0) one
  * CTA of hs warps encodes a stream and the containers use the interleaved layout.
+ * Calls with many streams (prefill, bulk encodes) run batch kernels that code 32 streams per CTA;
+ * the records are the same.  The environment variable DQ_ENCODE_BATCH_MIN (a stream count, read at
+ * every call) moves the size from which they are used.
  * Errors: DQ_ERR_ARG for null / negative arguments, DQ_ERR_UNSUPPORTED for mismatched
  * heads_per_stream, DQ_ERR_CUDA on launch failure. */
 int dq_encode_tokens(const dq_tables *tk, const dq_tables *tv, const void *k_bf16,

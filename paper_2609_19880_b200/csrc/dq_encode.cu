@@ -5,6 +5,8 @@
 #include <cuda_bf16.h>
 #include <cuda_fp16.h>
 
+#include <cstdlib>
+
 #include "dq_device.cuh"
 #include "dq_internal.h"
 
@@ -993,13 +995,23 @@ cudaError_t dq_launch_means(const DqDevTable& tk, const void* k_bf16, int T, int
     return cudaGetLastError();
 }
 
+// Smallest number of streams for which a call goes to the batch kernels (32 streams per CTA).  The
+// environment variable DQ_ENCODE_BATCH_MIN overrides the default (tuning; 0 sends every call there).
+static long long batch_min_streams(long long dflt) {
+    const char* e = getenv("DQ_ENCODE_BATCH_MIN");
+    if (!e || !*e) return dflt;
+    char* end = nullptr;
+    const long long v = strtoll(e, &end, 10);
+    return (end && *end == 0 && v >= 0) ? v : dflt;
+}
+
 cudaError_t dq_launch_encode(const DqDevTable& tk, const DqDevTable& tv, const DqEncodeArgs& a, cudaStream_t st) {
     const long long warps = (long long)a.T * a.Hkv;
     if (warps == 0 || (!a.do_k && !a.do_v)) return cudaSuccess;
     if (tk.hs > 1) {   // token-wide streams: CTAs of hs warps; few streams: one per CTA, many: 32 per CTA
         const long long streams = warps / tk.hs;
         const dim3 kinds_y(1, (a.do_k && a.do_v) ? 2 : 1);
-        if (streams < 3LL * 148 * kWB)
+        if (streams < batch_min_streams(3LL * 148 * kWB))
             return dq_launch_pdl(dq_encode_wide_kernel, dim3((unsigned)streams, kinds_y.y), dim3(tk.hs * 32), 0, st, tk, tv, a);
         const int smem = wide_batch_smem(tk.hs, tk.rec > tv.rec ? tk.rec : tv.rec);
         const cudaError_t e = cudaFuncSetAttribute(dq_encode_wide_batch_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
@@ -1008,7 +1020,7 @@ cudaError_t dq_launch_encode(const DqDevTable& tk, const DqDevTable& tv, const D
                              dim3(tk.hs * 32), (size_t)smem, st, tk, tv, a);
     }
     const unsigned blocks = (unsigned)((warps + kEncWarps - 1) / kEncWarps);
-    if (!a.step_flags && warps >= 4LL * 148 * kB32 * 4)   // enough streams to fill the GPU at 4 CTAs per SM several times
+    if (!a.step_flags && warps >= batch_min_streams(4LL * 148 * kB32 * 4))   // enough streams to fill the GPU several times
         return dq_launch_pdl(dq_encode_batch32_kernel<DQ_B32_MINB>, dim3((unsigned)((warps + kB32 - 1) / kB32), (a.do_k && a.do_v) ? 2 : 1),
                              dim3(kB32Warps * 32), 0, st, tk, tv, a);
     if (a.step_flags) {   // decode step: big CTAs, so that few SMs are kept from the attention kernel

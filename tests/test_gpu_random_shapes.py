@@ -118,3 +118,12 @@ def test_largest_batch(wide):
     ref = oracle.attention(ok, ov, workloads.bf16_bits(w.q), kc, vc, mq, ms, _np(w.page_table), _np(w.seq_lens), hkv,
                            gc.SM_SCALE)
     gc.check_attention(out, out32, ref)
+
+
+@pytest.mark.parametrize("seed", range(16, 28))
+def test_random_shape_through_the_batch_encoders(seed, monkeypatch):
+    """The same sweep with every encode call sent to the batch kernels (32 streams per CTA, one
+    lane per stream in the rANS pass), which calls of this size would not reach on their own:
+    ragged last CTAs, empty sequences, both stream groupings, every record against the oracle."""
+    monkeypatch.setenv("DQ_ENCODE_BATCH_MIN", "0")
+    test_random_shape(seed)
