@@ -242,13 +242,11 @@ def test_config4_ragged_paged_token_wide_full():
     _run_config_wide(cfg, 14)
 
 
-def test_config5_decode_step_full():
-    """Config 5 at full size through dq_decode_step (overlapped encoder / attention): 64 steps, every
-    step bit-identical to dq_encode_tokens + dq_decode_attention on a second cache; sampled rows of the
-    last step against the oracle."""
-    cfg = workloads.make_config(5)
-    steps = 64
-    rng = np.random.default_rng(55)
+def _step_vs_two_calls(cfg, steps, seed):
+    """`steps` decode steps through dq_decode_step on one cache and through dq_encode_tokens +
+    dq_decode_attention on a copy: bit-identical every 8th and the last step; sampled rows of the last
+    step against the oracle."""
+    rng = np.random.default_rng(seed)
     w = workloads.generate(cfg, device="cuda", extra_tokens_per_seq=steps)
     tk, tv, ok, ov = gc.tables(cfg)
     ca, cb = gc.GpuCache(w, ok.rec, ov.rec), gc.GpuCache(w, ok.rec, ov.rec)
@@ -256,7 +254,7 @@ def test_config5_decode_step_full():
     for name in ("k_cont", "v_cont", "mean_q", "mean_scale"):
         getattr(cb, name).copy_(getattr(ca, name))
     B, Hq, Hkv = cfg.batch, cfg.hq, cfg.hkv
-    gen = torch.Generator(device="cuda").manual_seed(56)
+    gen = torch.Generator(device="cuda").manual_seed(seed + 1)
     lens = torch.tensor(cfg.seq_lens, dtype=torch.int32)
     seq = torch.arange(B, dtype=torch.int32).cuda()
     pt_cpu = w.page_table.cpu()
@@ -275,9 +273,23 @@ def test_config5_decode_step_full():
                             dq.MEAN_REUSE, cb.status)
         dq.dq_decode_attention(tk, tv, w.q, cb.k_cont, cb.v_cont, cb.mean_q, cb.mean_scale, w.page_table, lens_d, Hkv,
                                gc.SM_SCALE, out_b, ws, out32_b)
-        if s % 8 == 7:
+        if s % 8 == 7 or s == steps - 1:
             torch.cuda.synchronize()
             assert torch.equal(out32_a, out32_b) and torch.equal(out_a, out_b), s
     torch.cuda.synchronize()
     assert torch.equal(ca.k_cont, cb.k_cont) and torch.equal(ca.v_cont, cb.v_cont) and torch.equal(ca.mean_q, cb.mean_q)
     _check_attention_sample(w, tk, tv, ok, ov, ca, _host(ca), rng, rows=2, seq_lens=lens.cuda())
+
+
+def test_config5_decode_step_full():
+    """Config 5 at full size through dq_decode_step: few work items, so the attention kernel starts
+    beside the encoder (ready flag, dynamic item order, late dependency wait)."""
+    _step_vs_two_calls(workloads.make_config(5), steps=64, seed=55)
+
+
+def test_config4_decode_step_full():
+    """Config 4 at full size through dq_decode_step: far more work items than the overlapped schedule
+    takes (B * blocks * Hkv > 32 per SM), so the call runs the plain kernel sequence."""
+    cfg = workloads.make_config(4)
+    assert sum((l + 511) // 512 for l in cfg.seq_lens) * cfg.hkv > 32 * 148
+    _step_vs_two_calls(cfg, steps=3, seed=44)
