@@ -217,7 +217,10 @@ int dq_decode_attention_residual(const dq_tables *tk, const dq_tables *tv, const
  *   seq_lens                 device int32 [B]: lengths including the newest token
  *   status                   as in dq_encode_tokens (nullable)
  * Other arguments as in dq_decode_attention.  Not to be mixed on one stream with work that
- * reads `workspace` concurrently; the first 16 bytes of the workspace carry the hand-over state. */
+ * reads `workspace` concurrently; the first 16 bytes of the workspace carry the hand-over state.
+ * The attention CTAs take the hand-over on a flag they poll a bounded number of times (65 536 polls,
+ * 64 ns apart; the environment variable DQ_STEP_POLL_LIMIT, read at every call, replaces the count);
+ * a CTA that gives up waits for the preceding kernels instead: same results, no overlap. */
 int dq_decode_step(const dq_tables *tk, const dq_tables *tv, const void *k_new_bf16, const void *v_new_bf16,
                    const int32_t *slot_new, const void *q_bf16, uint8_t *k_cont, uint8_t *v_cont,
                    int8_t *k_mean_q, float *k_mean_scale, int max_windows, const int32_t *page_table,

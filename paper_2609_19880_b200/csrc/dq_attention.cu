@@ -25,6 +25,8 @@
 #include <cuda_bf16.h>
 #include <cuda_fp16.h>
 
+#include <cstdlib>
+
 #include "dq_attention_common.cuh"
 
 using namespace dqdev;
@@ -286,6 +288,15 @@ __device__ __forceinline__ void fused_pass(uint32_t xk, uint32_t ptrk, uint32_t 
 #ifndef DQ_STEP_POLL_LIMIT
 #define DQ_STEP_POLL_LIMIT (1 << 16)   // polls of the ready flag (64 ns apart) before a CTA falls back to the grid wait
 #endif
+// The environment variable DQ_STEP_POLL_LIMIT (read at every call) replaces the default; 0 makes every CTA
+// take the fallback at once, which is how the tests run that path.
+static int step_poll_limit() {
+    const char* e = getenv("DQ_STEP_POLL_LIMIT");
+    if (!e || !*e) return DQ_STEP_POLL_LIMIT;
+    char* end = nullptr;
+    const long v = strtol(e, &end, 10);
+    return (end && *end == 0 && v >= 0 && v <= (1L << 24)) ? (int)v : DQ_STEP_POLL_LIMIT;
+}
 template <bool FUSED>
 __global__ void __launch_bounds__(kMaxWarps * 32, 1)
 dq_attention_kernel(const __grid_constant__ DqDevTable TK, const __grid_constant__ DqDevTable TV,
@@ -318,7 +329,7 @@ dq_attention_kernel(const __grid_constant__ DqDevTable TK, const __grid_constant
         int* s_ok = reinterpret_cast<int*>(smem + L.off_items);
         if (tid == 0) {
             int ok = 0;
-            for (int it = 0; it < DQ_STEP_POLL_LIMIT && !ok; ++it) {
+            for (int it = 0; it < p.poll_limit && !ok; ++it) {
                 asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(ok) : "l"(p.flags + 1) : "memory");
                 if (!ok) __nanosleep(64);
             }
@@ -1032,6 +1043,7 @@ static cudaError_t launch_attention_pass(const DqDevTable& tk, const DqDevTable&
     // CTA has dozens of items anyway (upper bound from the page-table width; the lengths live on the device).
     const long long max_items = (long long)a.B * ((a.max_pages * DQ_PAGE_TOKENS + nw * kChunk - 1) / (nw * kChunk)) * a.Hkv;
     p.fused = a.fused && !wide && max_items <= 32LL * sm_count; p.attn_grid = sm_count; p.flags = p.counter;
+    p.poll_limit = p.fused ? step_poll_limit() : 0;
     p.ne_before = p.prefix + (a.B + 1);
     p.item_tokens = nw * kChunk;
     p.rotate_q = tk.rotate; p.rotate_out = tv.rotate; p.has_mean = tk.has_mean;
@@ -1118,7 +1130,7 @@ cudaError_t dq_launch_bf16_attention(const DqAttnArgs& a, const void* k_pages, c
     p.hkv_magic = 0;
     p.hs = 1; p.groups = a.Hkv;
     p.q_len = 1; p.G1 = p.G; p.Hq1 = a.Hq; p.q_total = 1; p.q_first = 0;
-    p.fused = 0; p.attn_grid = 0; p.flags = p.counter; p.ne_before = p.prefix + (a.B + 1);
+    p.fused = 0; p.attn_grid = 0; p.poll_limit = 0; p.flags = p.counter; p.ne_before = p.prefix + (a.B + 1);
     p.resid_k = nullptr; p.resid_v = nullptr; p.resid_lens = nullptr; p.resid_cap = 0;
     const int heads = a.B * a.Hq;
     dq_attn_prepare_kernel<<<(heads + 7) / 8, 256, 0, st>>>(p);

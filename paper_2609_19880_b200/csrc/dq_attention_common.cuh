@@ -46,6 +46,7 @@ struct AttnParams {
     // flags: [0] next dynamic item, [1] set when the prepare kernel's outputs are complete, [2] prepare
     // CTAs finished, [3] times a CTA gave up polling [1].  ne_before[b]: non-empty sequences before b.
     int fused, attn_grid;
+    int poll_limit;   // decode-step mode: polls of the ready flag before a CTA falls back to the grid dependency wait
     int* flags;
     int* ne_before;
     int q_total, q_first; // tokens per sequence in q / out, and the first one this pass handles (a call with

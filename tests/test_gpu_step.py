@@ -108,3 +108,11 @@ def test_step_many_steps_budget_3bits():
     cfg = workloads.make_config(3, budget=3.0, scale=1 / 64)      # 64 query / 8 kv heads
     cfg.batch = 2; cfg.seq_lens = [1500, 380]
     _loop(cfg, steps=20, seed=4, check_every=7)
+
+
+def test_step_when_the_ready_flag_is_never_seen(monkeypatch):
+    """Poll limit 0: every attention CTA gives up on the ready flag at once and takes the grid
+    dependency wait instead; the step must still equal the two-call sequence and the oracle."""
+    monkeypatch.setenv("DQ_STEP_POLL_LIMIT", "0")
+    cfg = _cfg(2, batch=5, seq_lens=[511, 127, 0, 1023, 300])
+    _loop(cfg, steps=3, seed=5)
