@@ -122,7 +122,8 @@ int dq_tables_info(const dq_tables *t, dq_table_info *out);
  * mean removal (keys), min-max affine grid, drift, least-squares refit, fp16 metadata,
  * second drift, rANS.  One warp per stream.
  *   tk / tv          tables for keys / values; either may be NULL to skip that tensor
- *   k_bf16, v_bf16   device, bf16 [T][Hkv][128]
+ *   k_bf16, v_bf16   device, bf16 [T][Hkv][128]; finite values (any magnitude, subnormals included);
+ *                    a NaN or an infinity gives an unspecified (in-bounds) record
  *   seq_id, pos      device int32 [T]: sequence and position of each token
  *   slot             device int32 [T]: physical slot; distinct per token
  *   k_cont, v_cont   device, containers as laid out above; only the T records written

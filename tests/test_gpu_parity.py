@@ -233,3 +233,31 @@ def test_bf16_baseline_against_torch():
         ref = torch.einsum("ht,thd->hd", a, v)
         assert (out[b].float() - ref).abs().max() <= 0.02 * ref.abs().max()
         start += n
+
+
+@pytest.mark.parametrize("wide", [False, True])
+def test_encoder_extreme_finite_values(wide):
+    """The largest bf16 magnitudes (squares overflow: every candidate cost is infinite), subnormals
+    and negative zero: records, means and status counters as the oracle's."""
+    cfg = _small(2, batch=1, seq_lens=[48])
+    w = workloads.generate(cfg, device="cuda")
+    big = 3.38e38
+    w.v[3, 0, 5] = big; w.v[4, 1, :] = big; w.v[5, 2, ::2] = big; w.v[5, 2, 1::2] = -big
+    w.k[6, 0, 7] = big; w.k[7, 3, 1] = -big
+    w.v[13] = 1e-40; w.v[13, 0, 5] = 3e-40; w.v[14] = -0.0; w.k[16] = 1e-39; w.k[16, 1, 3] = 2e-39
+    if wide:
+        tk, tv, ok, ov = gc.wide_tables(cfg, cfg.hkv, k_rec=335, v_rec=235)
+        cache = gc.WideGpuCache(w, tk, tv, cfg.hkv)
+    else:
+        tk, tv, ok, ov = gc.tables(cfg)
+        cache = gc.GpuCache(w, ok.rec, ov.rec)
+    gc.gpu_encode(w, tk, tv, cache)
+    torch.cuda.synchronize()
+    kc, vc, mq, ms, sk, sv = gc.oracle_encode_wide(w, ok, ov, cfg.hkv) if wide else gc.oracle_encode(w, ok, ov)
+    got_k, got_v = _np(cache.k_cont), _np(cache.v_cont)
+    if wide:
+        got_k, got_v = gc.from_interleaved(got_k, ok.rec), gc.from_interleaved(got_v, ov.rec)
+    assert np.array_equal(got_k, kc) and np.array_equal(got_v, vc)
+    assert np.array_equal(_np(cache.mean_q), mq) and np.array_equal(_np(cache.mean_scale), ms)
+    assert list(_np(cache.status)[:3]) == [sk[i] + sv[i] for i in range(3)]
+    assert sk[0] + sv[0] > 0 and sk[1] + sv[1] > 0      # both the fallback and the constant path were taken
