@@ -35,7 +35,9 @@
  *
  * Pins (tests/test_oracle_*.py): closed-form storage accounting, the feasibility
  * boundary and NMSE curve of Table 2, rANS round trip, Shannon bound, orthonormal
- * self-inverse Hadamard, brute-force drift optimality, textbook special cases.
+ * self-inverse Hadamard, brute-force drift optimality, textbook special cases; the
+ * Refit of Algorithm 1 against a library least-squares solve rounded once to binary16,
+ * with its summation order shown to change no record (tests/test_oracle_refit.py).
  * PARITY UNPINNED by the paper (defined only by this build's contract): the mean
  * carry-forward rule for appended tokens and the automatic choice of alpha.  (The INT8
  * window-mean quantiser is pinned to a library per-tensor quantiser.)
