@@ -140,8 +140,8 @@ int dq_tables_info(const dq_tables *t, dq_table_info *out);
  * With token-wide tables (heads_per_stream = hs > 1; both tables must agree, Hkv % hs == 0) one
  * CTA of hs warps encodes a stream and the containers use the interleaved layout.
  * Calls with many streams (prefill, bulk encodes) run batch kernels that code 32 streams per CTA;
- * the records are the same.  The environment variable DQ_ENCODE_BATCH_MIN (a stream count, read at
- * every call) moves the size from which they are used.
+ * the records are the same.  The option DQ_OPT_ENCODE_BATCH_MIN (a stream count, dq_set_option)
+ * moves the size from which they are used.
  * Errors: DQ_ERR_ARG for null / negative arguments, DQ_ERR_UNSUPPORTED for mismatched
  * heads_per_stream, DQ_ERR_CUDA on launch failure. */
 int dq_encode_tokens(const dq_tables *tk, const dq_tables *tv, const void *k_bf16,
@@ -220,7 +220,7 @@ int dq_decode_attention_residual(const dq_tables *tk, const dq_tables *tv, const
  * Other arguments as in dq_decode_attention.  Not to be mixed on one stream with work that
  * reads `workspace` concurrently; the first 16 bytes of the workspace carry the hand-over state.
  * The attention CTAs take the hand-over on a flag they poll a bounded number of times (65 536 polls,
- * 64 ns apart; the environment variable DQ_STEP_POLL_LIMIT, read at every call, replaces the count);
+ * 64 ns apart; the option DQ_OPT_STEP_POLL_LIMIT, dq_set_option, replaces the count);
  * a CTA that gives up waits for the preceding kernels instead: same results, no overlap. */
 int dq_decode_step(const dq_tables *tk, const dq_tables *tv, const void *k_new_bf16, const void *v_new_bf16,
                    const int32_t *slot_new, const void *q_bf16, uint8_t *k_cont, uint8_t *v_cont,
@@ -304,6 +304,19 @@ int dq_bf16_decode_attention(const void *q_bf16, const void *k_bf16_pages, const
                              const int32_t *page_table, int max_pages, const int32_t *seq_lens,
                              int B, int Hq, int Hkv, float sm_scale, void *out_bf16,
                              void *workspace, size_t workspace_bytes, void *cuda_stream);
+
+/* Process-wide tuning options (no counterpart in the paper).  value < 0 restores the default.
+ *   DQ_OPT_STEP_POLL_LIMIT    dq_decode_step: polls of the hand-over flag before an attention CTA
+ *                             falls back to waiting for the preceding kernels (0: at once;
+ *                             at most 2^24).  Same results either way.
+ *   DQ_OPT_ENCODE_BATCH_MIN   encoder: number of streams in a call from which the batch kernels
+ *                             are used (0: always).  Same records either way.
+ * Returns DQ_ERR_ARG for an unknown key or an out-of-range value.  dq_get_option returns the value
+ * set (-1: default in force, or unknown key). */
+#define DQ_OPT_STEP_POLL_LIMIT 1
+#define DQ_OPT_ENCODE_BATCH_MIN 2
+int dq_set_option(int key, long long value);
+long long dq_get_option(int key);
 
 /* Measurement aid (no counterpart in the paper): while enabled (on > 0), every on-th
  * dq_decode_attention call records CUDA events on its stream around the fused kernel (up to

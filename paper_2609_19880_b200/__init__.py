@@ -26,8 +26,8 @@ EXPORTS = ["dq_build_tables", "dq_free_tables", "dq_tables_info", "dq_encode_tok
            "dq_decode_workspace_bytes", "dq_decode_attention", "dq_decode_attention_residual",
            "dq_decode_attention_multi", "dq_window_append", "dq_decode_step",
            "dq_decode_attention_static", "dq_decode_tokens",
-           "dq_bf16_decode_attention", "dq_profile_enable", "dq_profile_read", "dq_strerror",
-           "dq_last_cuda_error"]
+           "dq_bf16_decode_attention", "dq_set_option", "dq_get_option", "dq_profile_enable", "dq_profile_read",
+           "dq_strerror", "dq_last_cuda_error"]
 
 
 class DqError(RuntimeError):
@@ -96,6 +96,10 @@ def lib():
         L.dq_decode_tokens.argtypes = [vp, vp, vp, vp, i32, vp, vp, vp, i32, i32, vp, vp, vp]
         L.dq_bf16_decode_attention.restype = i32
         L.dq_bf16_decode_attention.argtypes = [vp, vp, vp, vp, i32, vp, i32, i32, i32, f32, vp, vp, sz, vp]
+        L.dq_set_option.restype = i32
+        L.dq_set_option.argtypes = [i32, C.c_longlong]
+        L.dq_get_option.restype = C.c_longlong
+        L.dq_get_option.argtypes = [i32]
         L.dq_profile_enable.restype = None
         L.dq_profile_enable.argtypes = [i32]
         L.dq_profile_read.restype = i32
@@ -291,6 +295,19 @@ def dq_bf16_decode_attention(q_bf16, k_pages, v_pages, page_table, seq_lens, Hkv
                                         _ptr(out_bf16), _ptr(workspace),
                                         int(workspace.numel() * workspace.element_size()), _stream(stream))
     _check(rc, "dq_bf16_decode_attention")
+
+
+OPT_STEP_POLL_LIMIT = 1
+OPT_ENCODE_BATCH_MIN = 2
+
+
+def dq_set_option(key: int, value: int):
+    """Process-wide tuning option (OPT_*); a negative value restores the library default."""
+    _check(lib().dq_set_option(int(key), int(value)), "dq_set_option")
+
+
+def dq_get_option(key: int) -> int:
+    return int(lib().dq_get_option(int(key)))
 
 
 def dq_profile_enable(on):

@@ -1,4 +1,5 @@
 // C ABI of the library: argument validation and kernel launches (see include/dq.h).
+#include <atomic>
 #include <cstdio>
 #include <cstring>
 #include <new>
@@ -16,7 +17,40 @@ int cuda_fail(cudaError_t e, const char* where) {
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
+// Process-wide options (dq_set_option); a negative value means "library default".
+std::atomic<long long> g_opt_step_poll_limit{-1};
+std::atomic<long long> g_opt_encode_batch_min{-1};
+
+// Checks every attention entry point makes on the tables and the arrays they describe: values carry
+// no window mean, both tables group heads the same way and Hkv is a whole number of groups (the
+// kernels derive the container layout from them), the mean arrays cover every addressable
+// position, and the alignments the 16-byte copies need.
+int check_attn_tables(const dq_tables* tk, const dq_tables* tv, int Hkv, const uint8_t* k_cont, const uint8_t* v_cont,
+                      const int8_t* k_mean_q, const float* k_mean_scale, int max_windows, int max_pages,
+                      const void* out_bf16, const float* out_f32) {
+    if (!tk || !tv || !k_cont || !v_cont) return DQ_ERR_ARG;
+    if (tv->info.has_mean) return DQ_ERR_UNSUPPORTED;
+    if (tk->info.heads_per_stream != tv->info.heads_per_stream) return DQ_ERR_UNSUPPORTED;
+    if (Hkv <= 0 || Hkv % tk->info.heads_per_stream != 0) return DQ_ERR_ARG;
+    if (tk->info.has_mean && (!k_mean_q || !k_mean_scale || max_windows <= 0)) return DQ_ERR_ARG;
+    if (tk->info.has_mean && (long long)max_windows * DQ_WINDOW_TOKENS < (long long)max_pages * DQ_PAGE_TOKENS)
+        return DQ_ERR_ARG;  // every addressable position needs a window slot
+    if (!aligned16(k_cont) || !aligned16(v_cont) || (tk->info.has_mean && !aligned16(k_mean_q))) return DQ_ERR_ARG;
+    if ((out_bf16 && (reinterpret_cast<uintptr_t>(out_bf16) & 7u)) || (out_f32 && !aligned16(out_f32)))
+        return DQ_ERR_ARG;
+    return DQ_OK;
+}
+
 }  // namespace
+
+int dq_opt_step_poll_limit(int dflt) {
+    const long long v = g_opt_step_poll_limit.load(std::memory_order_relaxed);
+    return v < 0 ? dflt : (int)v;
+}
+long long dq_opt_encode_batch_min(long long dflt) {
+    const long long v = g_opt_encode_batch_min.load(std::memory_order_relaxed);
+    return v < 0 ? dflt : v;
+}
 
 extern "C" {
 
@@ -134,15 +168,8 @@ int dq_decode_attention_multi(const dq_tables* tk, const dq_tables* tv, const vo
         const int pass_tokens = q_len < per_pass ? q_len : per_pass;
         if (workspace_bytes < dq_attn_workspace_bytes(B, Hq * pass_tokens, max_pages)) return DQ_ERR_WORKSPACE;
     }
-    if (tv->info.has_mean) return DQ_ERR_UNSUPPORTED;
-    if (tk->info.heads_per_stream != tv->info.heads_per_stream) return DQ_ERR_UNSUPPORTED;
-    if (Hkv % tk->info.heads_per_stream != 0) return DQ_ERR_ARG;
-    if (tk->info.has_mean && (!k_mean_q || !k_mean_scale || max_windows <= 0)) return DQ_ERR_ARG;
-    if (tk->info.has_mean && (long long)max_windows * DQ_WINDOW_TOKENS < (long long)max_pages * DQ_PAGE_TOKENS)
-        return DQ_ERR_ARG;  // every addressable position needs a window slot
-    if (!aligned16(k_cont) || !aligned16(v_cont) || (tk->info.has_mean && !aligned16(k_mean_q))) return DQ_ERR_ARG;
-    if ((out_bf16 && (reinterpret_cast<uintptr_t>(out_bf16) & 7u)) || (out_f32 && !aligned16(out_f32)))
-        return DQ_ERR_ARG;
+    rc = check_attn_tables(tk, tv, Hkv, k_cont, v_cont, k_mean_q, k_mean_scale, max_windows, max_pages, out_bf16, out_f32);
+    if (rc != DQ_OK) return rc;
     DqAttnArgs a;
     a.q_bf16 = q_bf16; a.k_cont = k_cont; a.v_cont = v_cont;
     a.mean_q = k_mean_q; a.mean_scale = k_mean_scale;
@@ -188,6 +215,8 @@ int dq_decode_attention_static(const dq_tables* tk, const dq_tables* tv, const v
                                void* out_bf16, float* out_f32, void* cuda_stream) {
     if (!tk || !tv || !k_cont || !v_cont) return DQ_ERR_ARG;
     if (B <= 0 || Hq <= 0 || Hkv <= 0 || max_pages <= 0) return DQ_ERR_ARG;
+    int rc = check_attn_tables(tk, tv, Hkv, k_cont, v_cont, k_mean_q, k_mean_scale, max_windows, max_pages, out_bf16, out_f32);
+    if (rc != DQ_OK) return rc;   // decided on the host, before any CUDA call
     const size_t need = dq_attn_workspace_bytes(B, Hq, max_pages);
     if (need > (size_t)DQ_STATIC_SCRATCH_BYTES) {  // decided on the host, before any CUDA call
         std::snprintf(g_cuda_error, sizeof g_cuda_error,
@@ -199,16 +228,9 @@ int dq_decode_attention_static(const dq_tables* tk, const dq_tables* tv, const v
     void* scratch = nullptr;
     cudaError_t e = dq_attn_static_scratch(&scratch);
     if (e != cudaSuccess) return cuda_fail(e, "static scratch address");
-    int rc = check_attn_common(q_bf16, page_table, max_pages, seq_lens, B, Hq, Hkv, out_bf16, out_f32, scratch,
-                               (size_t)DQ_STATIC_SCRATCH_BYTES);
+    rc = check_attn_common(q_bf16, page_table, max_pages, seq_lens, B, Hq, Hkv, out_bf16, out_f32, scratch,
+                           (size_t)DQ_STATIC_SCRATCH_BYTES);
     if (rc != DQ_OK) return rc;
-    if (tv->info.has_mean) return DQ_ERR_UNSUPPORTED;
-    if (tk->info.has_mean && (!k_mean_q || !k_mean_scale || max_windows <= 0)) return DQ_ERR_ARG;
-    if (tk->info.has_mean && (long long)max_windows * DQ_WINDOW_TOKENS < (long long)max_pages * DQ_PAGE_TOKENS)
-        return DQ_ERR_ARG;
-    if (!aligned16(k_cont) || !aligned16(v_cont) || (tk->info.has_mean && !aligned16(k_mean_q))) return DQ_ERR_ARG;
-    if ((out_bf16 && (reinterpret_cast<uintptr_t>(out_bf16) & 7u)) || (out_f32 && !aligned16(out_f32)))
-        return DQ_ERR_ARG;
     DqAttnArgs a;
     a.q_bf16 = q_bf16; a.k_cont = k_cont; a.v_cont = v_cont;
     a.mean_q = k_mean_q; a.mean_scale = k_mean_scale;
@@ -229,6 +251,7 @@ int dq_decode_tokens(const dq_tables* t, const uint8_t* cont, const int8_t* mean
                      int Hkv, uint8_t* symbols, float* dequant, void* cuda_stream) {
     if (!t || !cont || !slot || T < 0 || Hkv <= 0 || (!symbols && !dequant)) return DQ_ERR_ARG;
     if (t->info.has_mean && mean_q && (!mean_scale || !seq_id || !pos || max_windows <= 0)) return DQ_ERR_ARG;
+    if (Hkv % t->info.heads_per_stream != 0) return DQ_ERR_ARG;   // the container layout has Hkv / hs groups
     if (T == 0) return DQ_OK;
     const cudaError_t e = dq_launch_decode_tokens(t->dev, cont, mean_q, mean_scale, max_windows, seq_id, pos,
                                                   slot, T, Hkv, symbols, dequant,
@@ -268,13 +291,9 @@ int dq_decode_step(const dq_tables* tk, const dq_tables* tv, const void* k_new_b
                                workspace_bytes);
     if (rc != DQ_OK) return rc;
     if (tk->info.heads_per_stream != 1 || tv->info.heads_per_stream != 1) return DQ_ERR_UNSUPPORTED;
-    if (tv->info.has_mean) return DQ_ERR_UNSUPPORTED;
-    if (tk->info.has_mean && (!k_mean_q || !k_mean_scale || max_windows <= 0)) return DQ_ERR_ARG;
-    if (tk->info.has_mean && (long long)max_windows * DQ_WINDOW_TOKENS < (long long)max_pages * DQ_PAGE_TOKENS)
-        return DQ_ERR_ARG;
-    if (!aligned16(k_cont) || !aligned16(v_cont) || (tk->info.has_mean && !aligned16(k_mean_q))) return DQ_ERR_ARG;
+    rc = check_attn_tables(tk, tv, Hkv, k_cont, v_cont, k_mean_q, k_mean_scale, max_windows, max_pages, out_bf16, out_f32);
+    if (rc != DQ_OK) return rc;
     if ((reinterpret_cast<uintptr_t>(k_new_bf16) & 7u) || (reinterpret_cast<uintptr_t>(v_new_bf16) & 7u)) return DQ_ERR_ARG;
-    if ((out_bf16 && (reinterpret_cast<uintptr_t>(out_bf16) & 7u)) || (out_f32 && !aligned16(out_f32))) return DQ_ERR_ARG;
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     DqEncodeArgs e;
     std::memset(&e, 0, sizeof e);
@@ -307,6 +326,28 @@ int dq_window_append(const void* k_bf16, const void* v_bf16, void* resid_k_bf16,
                                                   static_cast<cudaStream_t>(cuda_stream));
     if (e != cudaSuccess) return cuda_fail(e, "window append");
     return DQ_OK;
+}
+
+int dq_set_option(int key, long long value) {
+    if (value < 0) value = -1;
+    switch (key) {
+        case DQ_OPT_STEP_POLL_LIMIT:
+            if (value > (1LL << 24)) return DQ_ERR_ARG;
+            g_opt_step_poll_limit.store(value, std::memory_order_relaxed);
+            return DQ_OK;
+        case DQ_OPT_ENCODE_BATCH_MIN:
+            g_opt_encode_batch_min.store(value, std::memory_order_relaxed);
+            return DQ_OK;
+        default: return DQ_ERR_ARG;
+    }
+}
+
+long long dq_get_option(int key) {
+    switch (key) {
+        case DQ_OPT_STEP_POLL_LIMIT: return g_opt_step_poll_limit.load(std::memory_order_relaxed);
+        case DQ_OPT_ENCODE_BATCH_MIN: return g_opt_encode_batch_min.load(std::memory_order_relaxed);
+        default: return -1;
+    }
 }
 
 void dq_profile_enable(int on) { dq_attn_profile_enable(on); }

@@ -25,8 +25,6 @@
 #include <cuda_bf16.h>
 #include <cuda_fp16.h>
 
-#include <cstdlib>
-
 #include "dq_attention_common.cuh"
 
 using namespace dqdev;
@@ -288,15 +286,9 @@ __device__ __forceinline__ void fused_pass(uint32_t xk, uint32_t ptrk, uint32_t 
 #ifndef DQ_STEP_POLL_LIMIT
 #define DQ_STEP_POLL_LIMIT (1 << 16)   // polls of the ready flag (64 ns apart) before a CTA falls back to the grid wait
 #endif
-// The environment variable DQ_STEP_POLL_LIMIT (read at every call) replaces the default; 0 makes every CTA
-// take the fallback at once, which is how the tests run that path.
-static int step_poll_limit() {
-    const char* e = getenv("DQ_STEP_POLL_LIMIT");
-    if (!e || !*e) return DQ_STEP_POLL_LIMIT;
-    char* end = nullptr;
-    const long v = strtol(e, &end, 10);
-    return (end && *end == 0 && v >= 0 && v <= (1L << 24)) ? (int)v : DQ_STEP_POLL_LIMIT;
-}
+// The option DQ_OPT_STEP_POLL_LIMIT replaces the default; 0 makes every CTA take the fallback at once,
+// which is how the tests run that path.
+static int step_poll_limit() { return dq_opt_step_poll_limit(DQ_STEP_POLL_LIMIT); }
 template <bool FUSED>
 __global__ void __launch_bounds__(kMaxWarps * 32, 1)
 dq_attention_kernel(const __grid_constant__ DqDevTable TK, const __grid_constant__ DqDevTable TV,
@@ -992,17 +984,34 @@ int dq_attn_profile_read(float* ms, int max_records) {
     return n;
 }
 
+// SM count and opt-in shared memory of the current device, looked up once per device.
+static cudaError_t device_limits(int* sm_count, int* smem_max) {
+    constexpr int kDevs = 64;
+    static int s_sm[kDevs], s_smem[kDevs];
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= kDevs) return cudaErrorInvalidDevice;
+    if (s_sm[dev] == 0) {
+        int sm = 0, smem = 0;
+        e = cudaDeviceGetAttribute(&sm, cudaDevAttrMultiProcessorCount, dev);
+        if (e != cudaSuccess) return e;
+        e = cudaDeviceGetAttribute(&smem, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
+        if (e != cudaSuccess) return e;
+        s_smem[dev] = smem;
+        s_sm[dev] = sm;
+    }
+    *sm_count = s_sm[dev];
+    *smem_max = s_smem[dev];
+    return cudaSuccess;
+}
+
 // One pass: query tokens [q_first, q_first + q_len) of the q_total given; q_len * (Hq / Hkv) <= 8.
 static cudaError_t launch_attention_pass(const DqDevTable& tk, const DqDevTable& tv, const DqAttnArgs& a, int q_total,
                                          int q_first, int q_len, cudaStream_t st) {
-    static int sm_count = 0, smem_max = 0;
-    if (sm_count == 0) {
-        int dev = 0;
-        cudaError_t e = cudaGetDevice(&dev);
-        if (e != cudaSuccess) return e;
-        e = cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev);
-        if (e != cudaSuccess) return e;
-        e = cudaDeviceGetAttribute(&smem_max, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
+    int sm_count = 0, smem_max = 0;
+    {
+        const cudaError_t e = device_limits(&sm_count, &smem_max);
         if (e != cudaSuccess) return e;
     }
     int nw = kMaxWarps;

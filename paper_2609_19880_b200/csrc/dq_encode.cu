@@ -995,15 +995,9 @@ cudaError_t dq_launch_means(const DqDevTable& tk, const void* k_bf16, int T, int
     return cudaGetLastError();
 }
 
-// Smallest number of streams for which a call goes to the batch kernels (32 streams per CTA).  The
-// environment variable DQ_ENCODE_BATCH_MIN overrides the default (tuning; 0 sends every call there).
-static long long batch_min_streams(long long dflt) {
-    const char* e = getenv("DQ_ENCODE_BATCH_MIN");
-    if (!e || !*e) return dflt;
-    char* end = nullptr;
-    const long long v = strtoll(e, &end, 10);
-    return (end && *end == 0 && v >= 0) ? v : dflt;
-}
+// Smallest number of streams for which a call goes to the batch kernels (32 streams per CTA); the
+// option DQ_OPT_ENCODE_BATCH_MIN replaces the default (0 sends every call there).
+static long long batch_min_streams(long long dflt) { return dq_opt_encode_batch_min(dflt); }
 
 cudaError_t dq_launch_encode(const DqDevTable& tk, const DqDevTable& tv, const DqEncodeArgs& a, cudaStream_t st) {
     const long long warps = (long long)a.T * a.Hkv;

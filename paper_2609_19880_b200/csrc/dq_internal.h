@@ -23,6 +23,10 @@ struct dq_tables {
     DqDevTable dev;
 };
 
+// dq_api.cu: process-wide options (dq_set_option); `dflt` is returned while an option is unset
+int dq_opt_step_poll_limit(int dflt);
+long long dq_opt_encode_batch_min(long long dflt);
+
 // dq_tables.cu
 int dq_host_build(int levels, double bits_per_elem, const dq_table_opts* opts, dq_tables* out);
 

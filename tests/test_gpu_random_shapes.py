@@ -121,9 +121,12 @@ def test_largest_batch(wide):
 
 
 @pytest.mark.parametrize("seed", range(16, 28))
-def test_random_shape_through_the_batch_encoders(seed, monkeypatch):
+def test_random_shape_through_the_batch_encoders(seed):
     """The same sweep with every encode call sent to the batch kernels (32 streams per CTA, one
     lane per stream in the rANS pass), which calls of this size would not reach on their own:
     ragged last CTAs, empty sequences, both stream groupings, every record against the oracle."""
-    monkeypatch.setenv("DQ_ENCODE_BATCH_MIN", "0")
-    test_random_shape(seed)
+    dq.dq_set_option(dq.OPT_ENCODE_BATCH_MIN, 0)
+    try:
+        test_random_shape(seed)
+    finally:
+        dq.dq_set_option(dq.OPT_ENCODE_BATCH_MIN, -1)

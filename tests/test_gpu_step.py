@@ -110,9 +110,12 @@ def test_step_many_steps_budget_3bits():
     _loop(cfg, steps=20, seed=4, check_every=7)
 
 
-def test_step_when_the_ready_flag_is_never_seen(monkeypatch):
+def test_step_when_the_ready_flag_is_never_seen():
     """Poll limit 0: every attention CTA gives up on the ready flag at once and takes the grid
     dependency wait instead; the step must still equal the two-call sequence and the oracle."""
-    monkeypatch.setenv("DQ_STEP_POLL_LIMIT", "0")
-    cfg = _cfg(2, batch=5, seq_lens=[511, 127, 0, 1023, 300])
-    _loop(cfg, steps=3, seed=5)
+    dq.dq_set_option(dq.OPT_STEP_POLL_LIMIT, 0)
+    try:
+        cfg = _cfg(2, batch=5, seq_lens=[511, 127, 0, 1023, 300])
+        _loop(cfg, steps=3, seed=5)
+    finally:
+        dq.dq_set_option(dq.OPT_STEP_POLL_LIMIT, -1)

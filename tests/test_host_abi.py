@@ -159,7 +159,33 @@ def test_calls_validate_before_launch(L):
     assert L.dq_window_append(fake, fake, fake, fake, fake, 0, 2, 8, n) == -1
     assert L.dq_window_append(fake, fake, C.c_void_p(0x1008), fake, fake, 128, 2, 8, n) == -1
     assert L.dq_decode_tokens(tk.handle, n, n, n, 0, n, n, fake, 4, 8, fake, n, n) == -1
+    assert L.dq_decode_tokens(tw.handle, fake, n, n, 0, n, n, fake, 4, 12, fake, n, n) == -1   # 12 heads, 8 per stream
+    # the entry point with built-in scratch makes the same table / layout checks, all before any CUDA call
+    def call_st(**kw):
+        d = dict(a); d.update(kw)
+        return L.dq_decode_attention_static(*[d[k] for k in ("tk", "tv", "q", "kc", "vc", "mq", "ms", "mw", "pt", "mp",
+                                                             "sl", "B", "Hq", "Hkv", "sm", "ob", "of", "st")])
+
+    assert call_st(tk=n) == -1 and call_st(kc=n) == -1 and call_st(B=0) == -1
+    assert call_st(tk=tw.handle) == -3                               # key and value tables group heads differently
+    assert call_st(tk=tw.handle, tv=twv.handle, Hkv=4, Hq=16) == -1  # 4 KV heads are not a whole 8-head stream
+    assert call_st(tv=tk.handle) == -3                               # values carry no window mean
+    assert call_st(mq=n) == -1 and call_st(mw=0) == -1 and call_st(kc=C.c_void_p(0x1001)) == -1
+    assert call_st(mp=1 << 20) == -1                                 # one window slot cannot cover that many pages
+    assert call_st(mw=1 << 17, mp=1 << 20) == -4                     # and this one exceeds the built-in scratch
     assert L.dq_bf16_decode_attention(fake, n, fake, fake, 8, fake, 2, 32, 8, C.c_float(0.1), fake, fake, ws, n) == -1
+
+
+def test_options_round_trip(L):
+    assert dq.dq_get_option(dq.OPT_STEP_POLL_LIMIT) == -1 and dq.dq_get_option(dq.OPT_ENCODE_BATCH_MIN) == -1
+    dq.dq_set_option(dq.OPT_STEP_POLL_LIMIT, 0)
+    dq.dq_set_option(dq.OPT_ENCODE_BATCH_MIN, 12345)
+    assert dq.dq_get_option(dq.OPT_STEP_POLL_LIMIT) == 0 and dq.dq_get_option(dq.OPT_ENCODE_BATCH_MIN) == 12345
+    dq.dq_set_option(dq.OPT_STEP_POLL_LIMIT, -7)
+    dq.dq_set_option(dq.OPT_ENCODE_BATCH_MIN, -1)
+    assert dq.dq_get_option(dq.OPT_STEP_POLL_LIMIT) == -1 and dq.dq_get_option(dq.OPT_ENCODE_BATCH_MIN) == -1
+    assert L.dq_set_option(99, 1) == -1 and L.dq_set_option(dq.OPT_STEP_POLL_LIMIT, 1 << 30) == -1
+    assert dq.dq_get_option(99) == -1
 
 
 def test_binding_fails_loudly_without_library(monkeypatch, tmp_path):

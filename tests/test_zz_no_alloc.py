@@ -50,6 +50,15 @@ def test_static_scratch_entry_point_matches_workspace_entry_point():
         assert ((out32_b - out32_a).abs() <= 2e-3 * scale).all()          # the tolerance of the parity tests
         assert torch.equal(out32_b, out32_a) and torch.equal(out_b, out_a)  # and in fact the same bits
     assert not out_b[1].any()                                             # empty sequence -> zero row
+    # a warm call leaves the device's memory accounting untouched: neither torch's allocator nor the
+    # driver (cudaMemGetInfo) sees a byte move
+    torch.cuda.synchronize()
+    alloc0, free0 = torch.cuda.memory_allocated(), torch.cuda.mem_get_info()[0]
+    dq.dq_decode_attention_static(tk, tv, w.q, cache.k_cont, cache.v_cont, cache.mean_q, cache.mean_scale,
+                                  w.page_table, second, cfg.hkv, gc.SM_SCALE, out_b, out32_b)
+    torch.cuda.synchronize()
+    assert torch.cuda.memory_allocated() == alloc0 and torch.cuda.mem_get_info()[0] == free0
+    assert torch.equal(out32_b, out32_a)
 
 
 def test_static_scratch_rejects_oversized_calls():
