@@ -32,11 +32,15 @@ if ROOT not in sys.path:
 METRIC = "decode_attention_kv_tokens_per_s"
 UNIT = "KV tokens/s"
 L2_BYTES = 126 * 2 ** 20
-# Algorithmic integer work of Algorithm 2 per decoded symbol (lane operations): slot mask,
-# table address, table read, two field extracts, state shift, multiply-add, compare with L,
-# byte merge, pointer advance.
-ALU_OPS_PER_SYMBOL = 10.0
-SM_COUNT, LANES_PER_SM_CLK = 148, 128
+SM_COUNT, SCHEDULERS_PER_SM = 148, 4
+# Stored ncu captures of the fused kernels (profiles/*.md): DRAM bytes per launch on config 2 and the
+# measured warp instructions per decoded symbol step.  They are constants of this file, not
+# quantities measured by a bench run; the line says so where it uses them.
+NCU_HEAD = {"dram_bytes": 37.62e6, "token_heads": 524288, "bytes_per_token_head": 72.0, "instr_per_symbol": 16.1,
+            "issue_active": 0.637, "source": "profiles/dq_attention_kernel_config2_ncu.md"}
+NCU_WIDE = {"instr_per_symbol": 19.8, "issue_active": None, "source": "profiles/dq_attention_wide_kernel_config2_ncu.md"}
+REGIONS = 21          # the K-step timed region is repeated this many times; ms_per_step is the median
+ORACLE_MAX_TOKENS = 131072   # the oracle legs run whole sequences of the workload up to this many tokens
 
 
 def _peaks():
@@ -116,44 +120,55 @@ def stream_setup(cfg, streams: str):
 
 
 def oracle_step_runner(cfg_idx: int, budget: float, streams: str = "head"):
-    """Builds the bounded oracle sample (sequence 0 of the workload, all KV heads) and returns
-    (step function, KV tokens per step, description).  GPU-free."""
+    """Builds the oracle's workload -- the same seeded configuration the GPU leg runs, all of its
+    sequences while they stay within ORACLE_MAX_TOKENS tokens in total (configs 2, 3 and 5 whole;
+    the first sequences of config 4) -- and returns (step function, KV tokens per step,
+    description, threads, whole workload?).  GPU-free."""
     import numpy as np
     import oracle
     from paper_2609_19880_b200 import workloads
 
     cfg = workloads.make_config(cfg_idx, budget=budget)
-    cfg.batch, cfg.seq_lens = 1, [min(cfg.seq_lens[0], 8192)]
+    full_batch = cfg.batch
+    keep, tot = 0, 0
+    for ln in cfg.seq_lens:
+        if keep and tot + ln > ORACLE_MAX_TOKENS:
+            break
+        keep, tot = keep + 1, tot + ln
+    cfg.batch, cfg.seq_lens = keep, list(cfg.seq_lens[:keep])
     w = workloads.generate(cfg, device="cpu")
     st = stream_setup(cfg, streams)
     ok = oracle.build_table(st["k_levels"], 128 * st["hs"], st["k_rec"], st["alpha"], has_mean=True, rotate=True)
     ov = oracle.build_table(st["v_levels"], 128 * st["hs"], st["v_rec"], st["alpha"], has_mean=False, rotate=True)
     kb, vb, qb = workloads.bf16_bits(w.k), workloads.bf16_bits(w.v), workloads.bf16_bits(w.q)
     seq_id, pos, slot = (t.numpy() for t in (w.seq_id, w.pos, w.slot))
-    mq = np.zeros((1, w.max_windows, cfg.hkv, 128), np.int8)
-    ms = np.zeros((1, w.max_windows, cfg.hkv), np.float32)
+    mq = np.zeros((cfg.batch, w.max_windows, cfg.hkv, 128), np.int8)
+    ms = np.zeros((cfg.batch, w.max_windows, cfg.hkv), np.float32)
     oracle.window_means(kb, seq_id, pos, mq, ms, 0)
     kc = np.zeros((w.num_pages, cfg.hkv // st["hs"], 16, ok.rec), np.uint8)
     vc = np.zeros((w.num_pages, cfg.hkv // st["hs"], 16, ov.rec), np.uint8)
     oracle.encode_tokens(ok, kb, seq_id, pos, slot, kc, mq, ms)
     oracle.encode_tokens(ov, vb, seq_id, pos, slot, vc)
-    last = slice(cfg.total_tokens - 1, cfg.total_tokens)
+    last = np.cumsum(np.asarray(cfg.seq_lens, dtype=np.int64)) - 1          # the newest token of every sequence
+    kl, vl = np.ascontiguousarray(kb[last]), np.ascontiguousarray(vb[last])
+    sl_, pl_, tl_ = (np.ascontiguousarray(a[last]) for a in (seq_id, pos, slot))
     pt, sl = w.page_table.numpy(), w.seq_lens.numpy()
     sm = 1.0 / math.sqrt(128.0)
 
     def step():
-        oracle.window_means(kb[last], seq_id[last], pos[last], mq, ms, 1)
-        oracle.encode_tokens(ok, kb[last], seq_id[last], pos[last], slot[last], kc, mq, ms)
-        oracle.encode_tokens(ov, vb[last], seq_id[last], pos[last], slot[last], vc)
+        oracle.window_means(kl, sl_, pl_, mq, ms, 1)
+        oracle.encode_tokens(ok, kl, sl_, pl_, tl_, kc, mq, ms)
+        oracle.encode_tokens(ov, vl, sl_, pl_, tl_, vc)
         return oracle.attention(ok, ov, qb, kc, vc, mq, ms, pt, sl, cfg.hkv, sm)
 
-    desc = (f"sequence 0 of {cfg.name}: {cfg.seq_lens[0]} tokens x {cfg.hkv} KV heads x {cfg.hq} query heads, "
-            f"encode 1 token + fp64 attention per step")
-    return step, cfg.seq_lens[0], desc, oracle.num_threads()
+    whole = keep == full_batch
+    desc = ((f"the whole workload {cfg.name}" if whole else f"the first {keep} of {full_batch} sequences of {cfg.name}") +
+            f": {tot} tokens x {cfg.hkv} KV heads x {cfg.hq} query heads, encode 1 token per sequence + fp64 attention per step")
+    return step, tot, desc, oracle.num_threads(), whole
 
 
 def time_oracle(cfg_idx, budget, budget_s=10.0, max_steps=1000, warmup=1, streams="head"):
-    step, toks, desc, cores = oracle_step_runner(cfg_idx, budget, streams)
+    step, toks, desc, cores, _ = oracle_step_runner(cfg_idx, budget, streams)
     for _ in range(warmup):
         step()
     n, t0 = 0, time.perf_counter()
@@ -171,7 +186,7 @@ def run_reference(args):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
-    step, toks, desc, cores = oracle_step_runner(args.config, args.budget, args.streams)
+    step, toks, desc, cores, whole = oracle_step_runner(args.config, args.budget, args.streams)
     for _ in range(max(args.warmup, 1)):
         step()
     t0 = time.perf_counter()
@@ -182,7 +197,8 @@ def run_reference(args):
     line = {"impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * dt / args.steps,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-            "config": {"workload": f"config {args.config} at {args.budget} bits/elem, bounded sample: {desc}"},
+            "config": {"workload": f"config {args.config} at {args.budget} bits/elem, " +
+                       ("" if whole else "bounded sample: ") + desc},
             "cpu_baseline": {"value": val, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": desc},
             "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
             "gpu_launches": 0}
@@ -344,32 +360,40 @@ def run_ours(args):
         step(i)
     barrier()
 
-    # ---- timed region: exactly K steps, CUDA events on the launch stream
-    # CUDA events around the fused kernel of every prof_period-th step (the events serialise that step's
-    # kernels, ~20 us each time, so they are kept sparse; at least 4 samples)
-    prof_period = max(1, min(int(os.environ.get("DQ_BENCH_PROFILE_PERIOD", "16")), args.steps // 4))
-    dq.dq_profile_enable(prof_period)
+    # ---- timed region: exactly K steps between a barrier + synchronize on both sides, CUDA events on the
+    # launch stream, nothing else enabled.  The region is repeated REGIONS times back to back (the rotating
+    # cache copies keep every step out of L2); ms_per_step is the median region, min / max beside it.
     t_wall0 = time.time()
     closes0 = state["closes"]
-    e0.record()
-    for i in range(args.steps):
-        step(i)
-    e1.record()
+    region_ms = []
+    n_regions = 1 if args.profile_only else REGIONS
+    for r in range(n_regions):
+        barrier()
+        e0.record()
+        for i in range(args.steps):
+            step(r * args.steps + i)
+        e1.record()
+        barrier()
+        region_ms.append(max_over_ranks(e0.elapsed_time(e1), world, dev) / args.steps)
     closes_timed = state["closes"] - closes0
-    barrier()
     t_wall1 = time.time()
-    total_ms = e0.elapsed_time(e1)
+    ms_per_step = statistics.median(region_ms)
+    value = job_throughput(kv_tokens, ms_per_step * 1e-3, world)
+
+    # ---- separate pass: CUDA events around the fused kernel of every step (they serialise the step's
+    # kernels, which is why this is not done inside the timed region)
+    dq.dq_profile_enable(1)
+    for i in range(max(16, min(args.steps, 64))):
+        step(i)
+    torch.cuda.synchronize()
     kern_ms = dq.dq_profile_read(4096)
     dq.dq_profile_enable(False)
-    total_ms = max_over_ranks(total_ms, world, dev)
-    ms_per_step = total_ms / args.steps
-    value = job_throughput(kv_tokens, ms_per_step * 1e-3, world)
 
     if args.profile_only:   # short run for an ncu capture: no soak, no e2e, no baselines
         sampler.stop()
         if rank == 0:
             print(json.dumps({"profile_only": True, "ms_per_step": ms_per_step,
-                              "kernel_ms": statistics.mean(kern_ms) if kern_ms else None}), flush=True)
+                              "kernel_ms": statistics.median(kern_ms) if kern_ms else None}), flush=True)
         if world > 1:
             dist.destroy_process_group()
         return
@@ -434,13 +458,15 @@ def run_ours(args):
 
     for i in range(3):
         e2e_step(i)
-    barrier()
-    t0 = time.perf_counter()
-    for i in range(args.steps):
-        e2e_step(i)
-    barrier()
-    e2e_s = time.perf_counter() - t0
-    e2e_s = max_over_ranks(e2e_s, world, dev)
+    e2e_regions = []
+    for r in range(5):                      # median of 5 regions of K steps, wall clock around each
+        barrier()
+        t0 = time.perf_counter()
+        for i in range(args.steps):
+            e2e_step(r * args.steps + i)
+        barrier()
+        e2e_regions.append(max_over_ranks(time.perf_counter() - t0, world, dev))
+    e2e_s = statistics.median(e2e_regions)
     e2e_value = job_throughput(kv_tokens, e2e_s / args.steps, world)
     # what came back to the host must be what a direct call computes (same inputs, same cache contents)
     e2e_check = None
@@ -454,28 +480,41 @@ def run_ours(args):
             dist.destroy_process_group()
         return
 
-    # ---- roofline of the dominant kernel (fused decode attention)
-    k_ms = statistics.mean(kern_ms) if kern_ms else None
+    # ---- roofline of the dominant kernel (fused decode attention): the metric's own quantity, compressed
+    # cache bytes per second against the measured copy bandwidth; beside it the issue-slot figures that
+    # say why the fraction is what it is (the kernel is bound by instruction issue, not by HBM)
+    k_ms = statistics.median(kern_ms) if kern_ms else None
     symbols = token_heads * 256.0
     comp_bytes = token_heads * (k_b + v_b + 1.0)   # records + amortised INT8 mean byte
     roofline = None
     extra = {}
+    ncu = NCU_HEAD if hs == 1 else NCU_WIDE
     if args.traffic_bytes is None:
-        # ncu, config 2: dram__bytes_read + write = 37.62 MB for 524288 token-heads at 42 + 29 byte records;
-        # the kernel reads every record once, so traffic grows with the records' bytes
-        args.traffic_bytes = 37.62e6 * (token_heads * (k_b + v_b + 1.0)) / (524288 * 72.0)
+        # every record is read once, so the captured config-2 figure scales with the records' bytes
+        args.traffic_bytes = NCU_HEAD["dram_bytes"] * comp_bytes / (NCU_HEAD["token_heads"] * NCU_HEAD["bytes_per_token_head"])
+        traffic_src = (f"scaled from the stored ncu capture {NCU_HEAD['source']} (dram__bytes_read + write of one launch "
+                       "on config 2); not measured in this run")
+    else:
+        traffic_src = "given on the command line (--traffic-bytes)"
     if k_ms:
-        alu_peak = SM_COUNT * LANES_PER_SM_CLK * sm_max_mhz * 1e6 / 1e9          # G lane-ops / s
-        alu_ach = symbols * ALU_OPS_PER_SYMBOL / (k_ms * 1e-3) / 1e9
         gbs = comp_bytes / (k_ms * 1e-3) / 1e9
-        roofline = {"bound": "alu", "achieved": alu_ach, "peak": alu_peak, "unit": "Gop/s (int32 lane ops)",
-                    "frac": alu_ach / alu_peak, "traffic": args.traffic_bytes,
-                    "kernel": "dq_attention_kernel" if hs == 1 else "dq_attention_wide_kernel", "kernel_ms": k_ms, "launches_timed": len(kern_ms),
-                    "peak_source": f"148 SM x 128 lanes x {sm_max_mhz:.0f} MHz ({peak_kind} clocks)",
-                    "ops_per_symbol": ALU_OPS_PER_SYMBOL}
-        extra = {"hbm": {"bound": "hbm", "achieved": gbs, "peak": hbm_peak, "unit": "GB/s", "frac": gbs / hbm_peak,
-                         "frac_of_8TBps": gbs / 8000.0, "peak_source": peak_kind,
-                         "bytes_per_token_head": k_b + v_b + 1},
+        mhz = sm_max_mhz
+        roofline = {"bound": "hbm", "achieved": gbs, "peak": hbm_peak, "unit": "GB/s", "frac": gbs / hbm_peak,
+                    "frac_of_8TBps": gbs / 8000.0, "peak_source": f"MEASURED_PEAKS.json hbm_gbs ({peak_kind})",
+                    "traffic": args.traffic_bytes, "traffic_source": traffic_src,
+                    "algorithmic_bytes_per_launch": comp_bytes, "bytes_per_token_head": k_b + v_b + 1,
+                    "kernel": "dq_attention_kernel" if hs == 1 else "dq_attention_wide_kernel",
+                    "kernel_ms": k_ms, "kernel_ms_min": min(kern_ms), "kernel_ms_max": max(kern_ms),
+                    "launches_timed": len(kern_ms),
+                    "timed": "CUDA events around the kernel on its launch stream, in a pass of its own after the timed region"}
+        warp_instr = symbols / 32.0 * ncu["instr_per_symbol"]
+        issue_peak = SM_COUNT * SCHEDULERS_PER_SM * mhz * 1e6     # warp instructions per second at max clock
+        extra = {"issue_slots": {"bound": "alu", "unit": "warp instructions/s",
+                                 "achieved": warp_instr / (k_ms * 1e-3), "peak": issue_peak,
+                                 "frac": warp_instr / (k_ms * 1e-3) / issue_peak,
+                                 "peak_source": f"148 SMs x 4 schedulers x {mhz:.0f} MHz, one warp instruction per clock each",
+                                 "instr_per_symbol": ncu["instr_per_symbol"], "ncu_issue_active": ncu["issue_active"],
+                                 "instr_source": f"stored ncu capture {ncu['source']}; not measured in this run"},
                  "kernel_token_heads_per_s": token_heads / (k_ms * 1e-3),
                  "kernel_symbols_per_s": symbols / (k_ms * 1e-3)}
 
@@ -514,7 +553,11 @@ def run_ours(args):
 
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
-        "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "ms_per_step": ms_per_step,
+        "timing": {"regions": len(region_ms), "steps_per_region": args.steps, "ms_per_step_median": ms_per_step,
+                   "ms_per_step_min": min(region_ms), "ms_per_step_max": max(region_ms),
+                   "ms_per_step_x_sm_mhz": (ms_per_step * clocks["sm_mhz"]) if clocks.get("sm_mhz") else None},
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "u32 rANS state / f16 mma, f32 accumulate", "data": "synthetic",
         "config": {"workload": cfg.name + ("" if hs == 1 else "_tokenwide"), "batch": B, "q_heads": Hq, "kv_heads": Hkv, "head_dim": 128,
                    "context": cfg.seq_lens if len(set(cfg.seq_lens)) > 1 and B <= 8 else
@@ -529,7 +572,8 @@ def run_ours(args):
         "roofline": roofline, "cpu_baseline": cpu,
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                 "launch": graph_note, "output_equals_direct_call": e2e_check},
-        "gpu_launches": int(round(launches_per_step * args.steps)), "clocks": clocks,
+        "gpu_launches": int(round(launches_per_step * args.steps)), "gpu_launches_note": "per timed region of K steps",
+        "clocks": clocks,
         "encoder": {"token_heads_per_s": 2 * token_heads / (enc_ms * 1e-3), "prefill_ms": enc_ms,
                     "streams": 2 * token_heads // hs},
         "bf16_baseline": bf16,
@@ -538,6 +582,47 @@ def run_ours(args):
     print(json.dumps(line), flush=True)
     if world > 1:
         dist.destroy_process_group()
+
+
+def run_decode_loop(args):
+    """`--decode-loop`: the bare rANS symbol step of the fused kernel (dq_microbench_decode_loop) on 148 CTAs,
+    timed with CUDA events; one JSON line per (threads, chains) with clocks per symbol per SM sub-partition."""
+    import torch
+    import paper_2609_19880_b200 as dq
+    from paper_2609_19880_b200 import _build
+    if not os.path.exists(dq.LIB_PATH):
+        _build.build()
+    dev = torch.device("cuda", 0)
+    tk = dq.dq_build_tables(5, 42 * 8 / 128, alpha=1.4, has_mean=True, rotate=True)
+    g = torch.Generator(device="cpu").manual_seed(1)
+    data = torch.randint(0, 256, (1 << 20,), dtype=torch.uint8, generator=g).to(dev)
+    out = torch.zeros(SM_COUNT * 1024, dtype=torch.int32, device=dev)
+    sampler = ClockSampler(0, period_s=0.005)
+    sampler.start()
+    reps = 400
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    rows = []
+    for threads in (512, 1024):
+        for chains in (1, 2):
+            dq.dq_microbench_decode_loop(tk, data, SM_COUNT, threads, chains, 8, out)
+            torch.cuda.synchronize()
+            best, t0 = None, time.time()
+            for _ in range(5):
+                e0.record()
+                dq.dq_microbench_decode_loop(tk, data, SM_COUNT, threads, chains, reps, out)
+                e1.record()
+                torch.cuda.synchronize()
+                ms = e0.elapsed_time(e1)
+                best = ms if best is None else min(best, ms)
+            mhz = sampler.summary(t0, time.time()).get("sm_mhz") or _peaks()[1]
+            symbols = SM_COUNT * threads * chains * 128.0 * reps
+            steps_per_smsp = symbols / 32.0 / (SM_COUNT * SCHEDULERS_PER_SM)
+            rows.append({"decode_loop": True, "threads_per_cta": threads, "chains_per_lane": chains, "ms": best,
+                         "symbols_per_s": symbols / (best * 1e-3), "sm_mhz": mhz,
+                         "clk_per_symbol_per_smsp": best * 1e-3 * mhz * 1e6 / steps_per_smsp})
+    sampler.stop()
+    for r in rows:
+        print(json.dumps(r), flush=True)
 
 
 def main():
@@ -560,8 +645,12 @@ def main():
     ap.add_argument("--traffic-bytes", type=float, default=None,
                     help="DRAM bytes per launch of the fused kernel from an ncu capture; default: the captured "
                          "figure of profiles/dq_attention_kernel_config2_ncu.md scaled by the token-heads processed")
+    ap.add_argument("--decode-loop", action="store_true",
+                    help="micro-benchmark of the bare rANS decode loop (no tiles, no contractions) instead of the step")
     args = ap.parse_args()
-    if args.impl == "reference":
+    if args.decode_loop:
+        run_decode_loop(args)
+    elif args.impl == "reference":
         run_reference(args)
     else:
         run_ours(args)

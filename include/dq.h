@@ -326,6 +326,17 @@ long long dq_get_option(int key);
 void dq_profile_enable(int on);
 int dq_profile_read(float *ms_out, int max_records);
 
+/* Measurement aid (no counterpart in the paper): the bare symbol step of Algorithm 2 as the fused
+ * kernel executes it, on byte streams held in shared memory -- no tiles, contractions, softmax or
+ * global traffic.  `ctas` CTAs of `threads` threads (a multiple of 32, <= 1024) each make `reps`
+ * passes of 128 symbols per chain with `chains` (1 or 2) independent chains per lane; the caller
+ * times the launch with events on its stream.  Symbols decoded = ctas * threads * chains * 128 * reps.
+ *   t       any per token-head table (its 256-entry table is the one looked up)
+ *   bytes   device, nbytes >= 4096 arbitrary bytes the streams are filled from
+ *   out     device uint32 [ctas * threads]: a checksum per thread (keeps the loop alive) */
+int dq_microbench_decode_loop(const dq_tables *t, const uint8_t *bytes, size_t nbytes, int ctas,
+                              int threads, int chains, int reps, uint32_t *out, void *cuda_stream);
+
 const char *dq_strerror(int code);
 /* Text of the last CUDA error seen by this thread's calls ("" if none). */
 const char *dq_last_cuda_error(void);

@@ -26,7 +26,7 @@ EXPORTS = ["dq_build_tables", "dq_free_tables", "dq_tables_info", "dq_encode_tok
            "dq_decode_workspace_bytes", "dq_decode_attention", "dq_decode_attention_residual",
            "dq_decode_attention_multi", "dq_window_append", "dq_decode_step",
            "dq_decode_attention_static", "dq_decode_tokens",
-           "dq_bf16_decode_attention", "dq_set_option", "dq_get_option", "dq_profile_enable", "dq_profile_read",
+           "dq_bf16_decode_attention", "dq_microbench_decode_loop", "dq_set_option", "dq_get_option", "dq_profile_enable", "dq_profile_read",
            "dq_strerror", "dq_last_cuda_error"]
 
 
@@ -96,6 +96,8 @@ def lib():
         L.dq_decode_tokens.argtypes = [vp, vp, vp, vp, i32, vp, vp, vp, i32, i32, vp, vp, vp]
         L.dq_bf16_decode_attention.restype = i32
         L.dq_bf16_decode_attention.argtypes = [vp, vp, vp, vp, i32, vp, i32, i32, i32, f32, vp, vp, sz, vp]
+        L.dq_microbench_decode_loop.restype = i32
+        L.dq_microbench_decode_loop.argtypes = [vp, vp, sz, i32, i32, i32, i32, vp, vp]
         L.dq_set_option.restype = i32
         L.dq_set_option.argtypes = [i32, C.c_longlong]
         L.dq_get_option.restype = C.c_longlong
@@ -295,6 +297,13 @@ def dq_bf16_decode_attention(q_bf16, k_pages, v_pages, page_table, seq_lens, Hkv
                                         _ptr(out_bf16), _ptr(workspace),
                                         int(workspace.numel() * workspace.element_size()), _stream(stream))
     _check(rc, "dq_bf16_decode_attention")
+
+
+def dq_microbench_decode_loop(table, bytes_u8, ctas: int, threads: int, chains: int, reps: int, out_u32, stream=None):
+    """Bare rANS decode loop (measurement aid); time it with CUDA events on the stream."""
+    rc = lib().dq_microbench_decode_loop(table.handle, _ptr(bytes_u8), int(bytes_u8.numel()), int(ctas), int(threads),
+                                         int(chains), int(reps), _ptr(out_u32), _stream(stream))
+    _check(rc, "dq_microbench_decode_loop")
 
 
 OPT_STEP_POLL_LIMIT = 1

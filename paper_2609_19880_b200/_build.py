@@ -19,6 +19,7 @@ _SOURCES = [
     ("dq_decode_tokens.cu", []),
     ("dq_attention.cu", []),
     ("dq_attention_wide.cu", []),
+    ("dq_microbench.cu", []),
     ("dq_encode.cu", ["-fmad=false"]),
 ]
 _COMMON = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",

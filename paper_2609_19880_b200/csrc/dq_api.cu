@@ -350,6 +350,17 @@ long long dq_get_option(int key) {
     }
 }
 
+int dq_microbench_decode_loop(const dq_tables* t, const uint8_t* bytes, size_t nbytes, int ctas, int threads, int chains,
+                              int reps, uint32_t* out, void* cuda_stream) {
+    if (!t || !bytes || !out || nbytes < 4096 || nbytes > 0xffffffffull) return DQ_ERR_ARG;
+    if (ctas <= 0 || reps <= 0 || (chains != 1 && chains != 2)) return DQ_ERR_ARG;
+    if (threads < 32 || threads > 1024 || threads % 32 != 0) return DQ_ERR_ARG;
+    const cudaError_t e = dq_launch_microbench_decode_loop(t->dev, bytes, nbytes, ctas, threads, chains, reps, out,
+                                                           static_cast<cudaStream_t>(cuda_stream));
+    if (e != cudaSuccess) return cuda_fail(e, "decode-loop microbenchmark");
+    return DQ_OK;
+}
+
 void dq_profile_enable(int on) { dq_attn_profile_enable(on); }
 
 int dq_profile_read(float* ms_out, int max_records) {

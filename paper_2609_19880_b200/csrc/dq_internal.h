@@ -97,3 +97,7 @@ void dq_attn_profile_enable(int on);
 int dq_attn_profile_read(float* ms, int max_records);
 cudaError_t dq_launch_bf16_attention(const DqAttnArgs& a, const void* k_pages, const void* v_pages,
                                      cudaStream_t st);
+
+// dq_microbench.cu: bare decode loop (measurement aid)
+cudaError_t dq_launch_microbench_decode_loop(const DqDevTable& t, const uint8_t* bytes, size_t nbytes, int ctas, int threads,
+                                             int chains, int reps, uint32_t* out, cudaStream_t st);
