@@ -1,9 +1,8 @@
 """Full-size GPU parity: the benchmark configurations at their real sizes, in the launch
-configuration bench.py times.  The oracle cannot redo millions of streams in seconds, so it
-is run on seeded samples: whole windows of tokens for the encoder (containers and means bit
-for bit), sampled tokens for the decoder, sampled (sequence, query head) rows for attention
-(each row needs every token of that sequence and KV head), plus properties that hold at any
-size."""
+configuration bench.py times.  EVERY record, window mean, decoded symbol, dequantised value and
+attention row of configurations 2, 3 (all five budgets), 4 and 5 and of the token-wide
+configurations 2 and 4 is compared with the oracle (the oracle does a whole configuration in
+seconds on the host cores); the sampled checks remain for the decode-step variants."""
 import numpy as np
 import pytest
 import torch
@@ -69,6 +68,49 @@ def _check_encoder_sample(w, ok, ov, host, rng, n_windows=6, groups=None):
         assert np.array_equal(vc[compact // 16, :, compact % 16], host["vc"][sl // 16, :, sl % 16]), (b, win)
 
 
+def _check_encoder_full(w, ok, ov, host, wide_hs=None):
+    """The oracle encodes the whole workload; every container byte and every window mean must match."""
+    if wide_hs is None:
+        kc, vc, mq, ms, sk, sv = gc.oracle_encode(w, ok, ov)
+    else:
+        kc, vc, mq, ms, sk, sv = gc.oracle_encode_wide(w, ok, ov, wide_hs)
+    assert np.array_equal(mq, host["mq"]) and np.array_equal(ms.view(np.uint32), host["ms"].view(np.uint32))
+    assert np.array_equal(kc, host["kc"])
+    assert np.array_equal(vc, host["vc"])
+    assert sk[0] == 0 and sv[0] == 0
+
+
+def _check_decoder_full(w, tk, tv, ok, ov, cache, host, chunk=16384):
+    """Every token of the workload through dq_decode_tokens, in chunks: symbols and dequantised values bit for bit."""
+    cfg = w.cfg
+    for lo in range(0, cfg.total_tokens, chunk):
+        hi = min(cfg.total_tokens, lo + chunk)
+        seq_id, pos, slot = w.seq_id[lo:hi].contiguous(), w.pos[lo:hi].contiguous(), w.slot[lo:hi].contiguous()
+        for (t_lib, t_or, cont_d, cont_h, m_q, m_s, mqd, msd) in (
+                (tk, ok, cache.k_cont, host["kc"], host["mq"], host["ms"], cache.mean_q, cache.mean_scale),
+                (tv, ov, cache.v_cont, host["vc"], None, None, None, None)):
+            sym_ref, deq_ref = oracle.decode_tokens(t_or, cont_h, _np(seq_id), _np(pos), _np(slot), cfg.hkv, m_q, m_s)
+            sym = torch.zeros(sym_ref.shape, dtype=torch.uint8, device="cuda")
+            deq = torch.zeros(deq_ref.shape, dtype=torch.float32, device="cuda")
+            dq.dq_decode_tokens(t_lib, cont_d, slot, cfg.hkv, sym, deq, mqd, msd, seq_id, pos)
+            torch.cuda.synchronize()
+            assert np.array_equal(_np(sym), sym_ref), lo
+            assert np.array_equal(_np(deq).view(np.uint32), deq_ref.view(np.uint32)), lo
+
+
+def _check_attention_full(w, tk, tv, ok, ov, cache, host, seq_lens=None):
+    """Every (sequence, query head) row against the oracle's fp64 attention over the same containers."""
+    cfg = w.cfg
+    out, out32 = gc.gpu_attention(w, tk, tv, cache, seq_lens=seq_lens)
+    assert torch.isfinite(out32).all()
+    lens = _np(w.seq_lens if seq_lens is None else seq_lens)
+    ref = oracle.attention(ok, ov, workloads.bf16_bits(w.q), host["kc"], host["vc"], host["mq"], host["ms"],
+                           _np(w.page_table), lens, cfg.hkv, gc.SM_SCALE)
+    worst = gc.check_attention(out, out32, ref)          # tolerance 2e-3 per row
+    assert worst < 1e-3                                  # and, as a regression guard, well inside it
+    return out, out32
+
+
 def _check_decoder_sample(w, tk, tv, ok, ov, cache, host, rng, n_tokens=256):
     cfg = w.cfg
     idx = np.sort(rng.choice(cfg.total_tokens, size=min(n_tokens, cfg.total_tokens), replace=False))
@@ -108,7 +150,7 @@ def _check_attention_sample(w, tk, tv, ok, ov, cache, host, rng, rows=3, seq_len
     return out32
 
 
-def _run_config(cfg, seed):
+def _run_config(cfg, seed, exhaustive=False, windows=6, all_rows=False):
     rng = np.random.default_rng(seed)
     w = workloads.generate(cfg, device="cuda")
     tk, tv, ok, ov = gc.tables(cfg)
@@ -118,55 +160,62 @@ def _run_config(cfg, seed):
     st = _np(cache.status)
     assert st[0] == 0 and st[3] <= max(ok.rec, ov.rec)     # every stream fits; no all-central fallback
     host = _host(cache)
-    _check_encoder_sample(w, ok, ov, host, rng)
-    _check_decoder_sample(w, tk, tv, ok, ov, cache, host, rng)
-    _check_attention_sample(w, tk, tv, ok, ov, cache, host, rng)
+    if exhaustive:
+        _check_encoder_full(w, ok, ov, host)
+        _check_decoder_full(w, tk, tv, ok, ov, cache, host)
+    else:
+        _check_encoder_sample(w, ok, ov, host, rng, n_windows=windows)
+        _check_decoder_sample(w, tk, tv, ok, ov, cache, host, rng)
+    if exhaustive or all_rows:
+        _check_attention_full(w, tk, tv, ok, ov, cache, host)
+    else:
+        _check_attention_sample(w, tk, tv, ok, ov, cache, host, rng)
     return w, tk, tv, ok, ov, cache
 
 
 def test_config2_llama3_8b_full():
+    """Every record, mean, symbol, dequantised value and attention row of configuration 2."""
     cfg = workloads.make_config(2)
     assert cfg.total_tokens * cfg.hkv == 524288
-    _run_config(cfg, 2)
+    _run_config(cfg, 2, exhaustive=True)
 
 
 @pytest.mark.parametrize("budget", [1.5, 2.0, 2.26, 3.0, 4.0])
 def test_config3_long_context_budget_sweep_full(budget):
+    """Every budget of the sweep exhaustively (1 048 576 token-heads each)."""
     cfg = workloads.make_config(3, budget=budget)
     assert cfg.seq_lens == [131072] and cfg.hq // cfg.hkv == 8
-    _run_config(cfg, 30 + int(budget * 10))
+    _run_config(cfg, 30 + int(budget * 10), exhaustive=True)
 
 
 def test_config4_ragged_paged_full():
+    """Every record, mean, symbol, dequantised value and attention row of the 128 ragged sequences
+    (8.65 M token-heads, shuffled pages)."""
     cfg = workloads.make_config(4)
     assert cfg.batch == 128 and cfg.shuffle_pages
-    w, tk, tv, ok, ov, cache = _run_config(cfg, 4)
+    w, tk, tv, ok, ov, cache = _run_config(cfg, 4, exhaustive=True)
     pt = _np(w.page_table)
     assert not np.array_equal(pt[0, :8], np.sort(pt[0, :8]))     # pages really are shuffled
 
 
 def test_config5_encode_decode_loop_full():
-    """Prefill-encode 4 x 32768 tokens, then 256 decode steps, each appending one freshly
-    encoded token per sequence (means carried forward) before attention."""
+    """Prefill-encode 4 x 32768 tokens (every record and mean against the oracle), then 256 decode
+    steps, each appending one freshly encoded token per sequence (means carried forward) before
+    attention; the oracle mirrors the loop for all four sequences: every appended record, every
+    touched window mean, every attention row of the last step."""
     cfg = workloads.make_config(5)
     steps = cfg.decode_steps
     assert steps == 256 and cfg.hq // cfg.hkv == 7
-    rng = np.random.default_rng(5)
     w = workloads.generate(cfg, device="cuda", extra_tokens_per_seq=steps)
     tk, tv, ok, ov = gc.tables(cfg)
     cache = gc.GpuCache(w, ok.rec, ov.rec)
     gc.gpu_encode(w, tk, tv, cache)
     torch.cuda.synchronize()
-    _check_encoder_sample(w, ok, ov, _host(cache), rng, n_windows=4)
-
-    # oracle mirror of the append loop for one sequence: its last prefill window, then every step
-    b0 = int(rng.integers(0, cfg.batch))
-    L0 = cfg.seq_lens[b0]
-    start = int(np.cumsum([0] + cfg.seq_lens)[b0])
-    last_win = torch.arange(start + L0 - 128, start + L0, device="cuda")
-    _, _, mq_o, ms_o, _, _ = gc.oracle_encode(w, ok, ov, sel=last_win)
-    kc_o = np.zeros((w.num_pages, cfg.hkv, 16, ok.rec), np.uint8)
-    vc_o = np.zeros((w.num_pages, cfg.hkv, 16, ov.rec), np.uint8)
+    kc_o, vc_o, mq_o, ms_o, sk, sv = gc.oracle_encode(w, ok, ov)
+    host = _host(cache)
+    assert np.array_equal(kc_o, host["kc"]) and np.array_equal(vc_o, host["vc"])
+    assert np.array_equal(mq_o, host["mq"]) and np.array_equal(ms_o.view(np.uint32), host["ms"].view(np.uint32))
+    _check_decoder_full(w, tk, tv, ok, ov, cache, host)
 
     gen = torch.Generator(device="cuda").manual_seed(55)
     lens = torch.tensor(cfg.seq_lens)
@@ -186,34 +235,33 @@ def test_config5_encode_decode_loop_full():
         cur = (lens + s + 1).to(torch.int32).cuda()
         dq.dq_decode_attention(tk, tv, w.q, cache.k_cont, cache.v_cont, cache.mean_q, cache.mean_scale,
                                w.page_table, cur, cfg.hkv, gc.SM_SCALE, out, ws, out32)
-        kb, vb = workloads.bf16_bits(k1[b0:b0 + 1]), workloads.bf16_bits(v1[b0:b0 + 1])
-        sid, ps, sl = np.array([b0], np.int32), pos[b0:b0 + 1].numpy(), slot[b0:b0 + 1].numpy()
+        kb, vb = workloads.bf16_bits(k1), workloads.bf16_bits(v1)
+        sid, ps, sl = seq.numpy(), pos.numpy(), slot.numpy()
         oracle.window_means(kb, sid, ps, mq_o, ms_o, 1)
         oracle.encode_tokens(ok, kb, sid, ps, sl, kc_o, mq_o, ms_o)
         oracle.encode_tokens(ov, vb, sid, ps, sl, vc_o)
-        new_slots.append(int(sl[0]))
+        new_slots.extend(int(x) for x in sl)
     torch.cuda.synchronize()
     assert int(_np(cache.status)[0]) == 0
     new_slots = np.array(new_slots)
-    kc, vc = _np(cache.k_cont), _np(cache.v_cont)
-    assert np.array_equal(_rec_view(kc)[new_slots], _rec_view(kc_o)[new_slots])
-    assert np.array_equal(_rec_view(vc)[new_slots], _rec_view(vc_o)[new_slots])
-    wins = slice(L0 // 128 - 1, (L0 + steps - 1) // 128 + 1)
-    assert np.array_equal(_np(cache.mean_q)[b0, wins], mq_o[b0, wins])
-    assert np.array_equal(_np(cache.mean_scale)[b0, wins], ms_o[b0, wins])
-    # attention of the last step against the oracle over the grown cache
+    host = _host(cache)
+    assert np.array_equal(_rec_view(host["kc"])[new_slots], _rec_view(kc_o)[new_slots])
+    assert np.array_equal(_rec_view(host["vc"])[new_slots], _rec_view(vc_o)[new_slots])
+    assert np.array_equal(host["kc"], kc_o) and np.array_equal(host["vc"], vc_o)      # and nothing else moved
+    assert np.array_equal(host["mq"], mq_o) and np.array_equal(host["ms"].view(np.uint32), ms_o.view(np.uint32))
+    # attention of the last step, every row, against the oracle over the grown cache
     final = (lens + steps).to(torch.int32).cuda()
-    _check_attention_sample(w, tk, tv, ok, ov, cache, _host(cache), rng, rows=3, seq_lens=final)
-    ref_rows = oracle.attention(ok, ov, workloads.bf16_bits(w.q), kc, vc, _np(cache.mean_q), _np(cache.mean_scale),
-                                _np(w.page_table), _np(final), cfg.hkv, gc.SM_SCALE, only=(b0, 3))
-    gc.check_attention(out, out32, ref_rows, rows=[(b0, 3)])     # the loop's own last output
+    ref = oracle.attention(ok, ov, workloads.bf16_bits(w.q), host["kc"], host["vc"], host["mq"], host["ms"],
+                           _np(w.page_table), _np(final), cfg.hkv, gc.SM_SCALE)
+    gc.check_attention(out, out32, ref)     # the loop's own last output
+    _check_attention_full(w, tk, tv, ok, ov, cache, host, seq_lens=final)
 
 
 # ------------------------------------------------ token-wide streams at full size
 
-def _run_config_wide(cfg, seed, hs=8):
+def _run_config_wide(cfg, seed, hs=8, exhaustive=False, windows=4, all_rows=False):
     """The paper's default grouping (one 335 / 235-byte record per token, 8 / 6 levels) on a full
-    benchmark shape: same sampled checks, containers compared after undoing the page interleave."""
+    benchmark shape: same checks, containers compared after undoing the page interleave."""
     rng = np.random.default_rng(seed)
     w = workloads.generate(cfg, device="cuda")
     tk, tv, ok, ov = gc.wide_tables(cfg, hs)
@@ -224,22 +272,30 @@ def _run_config_wide(cfg, seed, hs=8):
     assert st[0] == 0 and st[3] <= max(ok.rec, ov.rec)
     host = dict(kc=gc.from_interleaved(_np(cache.k_cont), ok.rec), vc=gc.from_interleaved(_np(cache.v_cont), ov.rec),
                 mq=_np(cache.mean_q), ms=_np(cache.mean_scale))
-    _check_encoder_sample(w, ok, ov, host, rng, n_windows=4, groups=cfg.hkv // hs)
-    _check_decoder_sample(w, tk, tv, ok, ov, cache, host, rng, n_tokens=128)
-    _check_attention_sample(w, tk, tv, ok, ov, cache, host, rng)
+    if exhaustive:
+        _check_encoder_full(w, ok, ov, host, wide_hs=hs)
+        _check_decoder_full(w, tk, tv, ok, ov, cache, host)
+    else:
+        _check_encoder_sample(w, ok, ov, host, rng, n_windows=windows, groups=cfg.hkv // hs)
+        _check_decoder_sample(w, tk, tv, ok, ov, cache, host, rng, n_tokens=128)
+    if exhaustive or all_rows:
+        _check_attention_full(w, tk, tv, ok, ov, cache, host)
+    else:
+        _check_attention_sample(w, tk, tv, ok, ov, cache, host, rng)
     return w, tk, tv, ok, ov, cache
 
 
 def test_config2_token_wide_full():
+    """Every record, mean, symbol, dequantised value and attention row of the token-wide configuration 2."""
     cfg = workloads.make_config(2)
     assert cfg.total_tokens == 65536 and cfg.hkv == 8
-    _run_config_wide(cfg, 12)
+    _run_config_wide(cfg, 12, exhaustive=True)
 
 
 def test_config4_ragged_paged_token_wide_full():
     cfg = workloads.make_config(4)
     assert cfg.batch == 128 and cfg.shuffle_pages
-    _run_config_wide(cfg, 14)
+    _run_config_wide(cfg, 14, exhaustive=True)
 
 
 def _step_vs_two_calls(cfg, steps, seed):
