@@ -44,7 +44,17 @@ class Table(C.Structure):
         ("f", C.c_int32 * MAX_LEVELS), ("c", C.c_int32 * (MAX_LEVELS + 1)),
         ("r", C.c_float * MAX_LEVELS), ("R", C.c_uint32 * MAX_LEVELS),
         ("lut_m", C.c_uint8 * 256), ("lut_f", C.c_uint8 * 256), ("lut_d", C.c_uint8 * 256),
+        ("sigma", C.c_int), ("early_exit", C.c_int),
     ]
+
+    @property
+    def L(self):
+        """Lower bound of the state interval: 2^23 (sigma = 32) or 2^15 (sigma = 24)."""
+        return 1 << (self.sigma - 9)
+
+    @property
+    def state_bytes(self):
+        return self.sigma // 8
 
     def freqs(self):
         return [int(self.f[m]) for m in range(self.M)]
@@ -78,6 +88,9 @@ def lib():
             L.dqo_build_table.restype = C.c_int
             L.dqo_build_table.argtypes = [C.c_int, C.c_int, C.c_int, C.c_double, C.c_int, C.c_int,
                                           C.POINTER(Table)]
+            L.dqo_build_table_ex.restype = C.c_int
+            L.dqo_build_table_ex.argtypes = [C.c_int, C.c_int, C.c_int, C.c_double, C.c_int, C.c_int,
+                                             C.c_int, C.c_int, C.POINTER(Table)]
             _lib = L
     return _lib
 
@@ -111,9 +124,15 @@ def rec_bytes(bits_per_elem: float, n: int) -> int:
 
 
 def build_table(levels: int, n: int, rec: int, alpha: float = 1.4, has_mean: bool = False,
-                rotate: bool = True, allow_infeasible: bool = False) -> Table:
+                rotate: bool = True, allow_infeasible: bool = False, sigma: int = 32,
+                early_exit: bool = False) -> Table:
+    """sigma / early_exit select the opt-in codec variants (defaults: the paper's codec)."""
     T = Table()
-    rc = lib().dqo_build_table(levels, n, rec, float(alpha), int(has_mean), int(rotate), C.byref(T))
+    if sigma == 32 and not early_exit:
+        rc = lib().dqo_build_table(levels, n, rec, float(alpha), int(has_mean), int(rotate), C.byref(T))
+    else:
+        rc = lib().dqo_build_table_ex(levels, n, rec, float(alpha), int(has_mean), int(rotate), int(sigma),
+                                      int(early_exit), C.byref(T))
     if rc == -1 or (rc != 0 and not allow_infeasible):
         raise ValueError(f"oracle table build failed rc={rc} (M={levels}, n={n}, rec={rec})")
     return T

@@ -32,6 +32,15 @@
  *     spans +-E[max of n normals], cells clipped to that span;
  *   - the bisection of log2(lambda) is done as a geometric mean sqrt(lo*hi);
  *   - code length is summed in 1/65536-bit fixed point, rounded up per symbol.
+ * Opt-in variants of the codec (off unless a table asks for them; the defaults above are
+ * untouched by them):
+ *   - early exit of Drift (table field early_exit): Algorithm 1's bisection ends at a known
+ *     multiplier when every one of its 12 tests passes; that assignment is evaluated first
+ *     and returned if it meets the budget, else the full bisection runs (App. C: most
+ *     streams have budget to spare, so most take the short path);
+ *   - sigma = 24 (table field sigma): the state lives in [2^15, 2^23) and its final value
+ *     takes 3 bytes of the container instead of 4 (Eq. budget: B = 8C - sigma), one byte
+ *     per stream back for symbols; streams of at most 640 values (five heads) only.
  *
  * Pins (tests/test_oracle_*.py): closed-form storage accounting, the feasibility
  * boundary and NMSE curve of Table 2, rANS round trip, Shannon bound, orthonormal
@@ -55,8 +64,7 @@
 #define DQO_MAX_N 1024
 #define DQO_P 8            /* rANS precision: sum f = 2^p (Sec. 3.1)              */
 #define DQO_TOT 256
-#define DQO_L (1u << 23)   /* lower bound of the normalised state interval         */
-#define DQO_SIGMA 32       /* bits of final state stored in the record             */
+#define DQO_SIGMA 32       /* bits of final state stored in the record (default)   */
 #define DQO_WINDOW 128     /* tokens per channel-mean window                       */
 #define DQO_PAGE 16        /* tokens per physical page                             */
 #define DQO_HEAD 128       /* head dimension of the token-level entry points       */
@@ -72,7 +80,12 @@ typedef struct {
     float r[DQO_MAX_LEVELS];       /* ideal cost -log2(f/256) in bits (Alg. 1)      */
     uint32_t R[DQO_MAX_LEVELS];    /* ceil(r * 65536)                               */
     uint8_t lut_m[DQO_TOT], lut_f[DQO_TOT], lut_d[DQO_TOT]; /* T[z] = (m, f_m, z - c_m) */
+    int sigma;                     /* bits of final state in the record: 32 (default) or 24  */
+    int early_exit;                /* 1: Drift first tries the multiplier the bisection ends at when all tests pass */
 } dqo_table;
+
+/* lower bound L of the normalised state interval [L, 2^8 L): 2^23 for sigma = 32, 2^15 for 24 */
+static uint32_t dqo_L(const dqo_table *T) { return 1u << (T->sigma - 9); }
 
 /* ------------------------------------------------------------------ numbers */
 
@@ -198,13 +211,21 @@ static double dqo_entropy256(const dqo_table *T)
  * alpha >= 0: used as given.  alpha < 0: smallest alpha in {1.4, 1.5, ..., 32.0}
  * whose table has entropy <= B/n and lets the all-central stream fit.
  * Returns 0, or -1 for bad arguments, -2 when no feasible table exists. */
-int dqo_build_table(int M, int n, int rec_bytes, double alpha, int has_mean, int rotate,
-                    dqo_table *T)
+int dqo_build_table_ex(int M, int n, int rec_bytes, double alpha, int has_mean, int rotate,
+                       int sigma, int early_exit, dqo_table *T)
 {
     if (M < 2 || M > DQO_MAX_LEVELS || n < 1 || n > DQO_MAX_N || rec_bytes < 9) return -1;
+    if (sigma != 32 && sigma != 24) return -1;
+    /* With the 24-bit state an encode step may lose up to log2(1 + 2^-7) bits to floor(x / f)
+     * (x >= 2^15, f < 2^8).  The budget test keeps sum r <= B = 8(C - 3); the stream then fits
+     * its C bytes as long as the accumulated loss stays below one byte: n log2(1 + 2^-7) < 8,
+     * i.e. n <= 712.  Longer streams would need a byte of margin, which is the byte the
+     * variant saves, so they are not offered. */
+    if (sigma == 24 && n > 640) return -1;
     memset(T, 0, sizeof *T);
     T->M = M; T->n = n; T->rec = rec_bytes; T->C = rec_bytes - 4;
-    T->B = 8 * T->C - DQO_SIGMA;
+    T->sigma = sigma; T->early_exit = early_exit ? 1 : 0;
+    T->B = 8 * T->C - sigma;                           /* Eq. (budget) */
     T->has_mean = has_mean; T->rotate = rotate;
     T->E = dqo_expected_max(n);
     double E = T->E, delta = 2.0 * E / (M - 1), ps = 0.0;
@@ -227,6 +248,13 @@ int dqo_build_table(int M, int n, int rec_bytes, double alpha, int has_mean, int
         if (T->feasible && dqo_entropy256(T) <= (double)T->B / n) return 0;
     }
     return -2;
+}
+
+/* The paper's codec: sigma = 32, no early exit. */
+int dqo_build_table(int M, int n, int rec_bytes, double alpha, int has_mean, int rotate,
+                    dqo_table *T)
+{
+    return dqo_build_table_ex(M, n, rec_bytes, alpha, has_mean, rotate, DQO_SIGMA, 0, T);
 }
 
 int dqo_table_size(void) { return (int)sizeof(dqo_table); }
@@ -285,6 +313,27 @@ int64_t dqo_drift(const float *z, int n, float s, float o, const dqo_table *T, u
     float lam_hi = 8.0f * (maxD - minD);
     float lam_lo = lam_hi * 0x1p-40f;
     int64_t len = 0;
+    if (T->early_exit) {
+        /* When each of the 12 tests passes, the bracket's upper end walks hi <- sqrt(lo * hi)
+         * twelve times with lo fixed; the assignment at that multiplier is what the loop below
+         * would return.  Evaluate it first and stop if it meets the budget. */
+        float lam_e = lam_hi;
+        for (int it = 0; it < 12; ++it) lam_e = sqrtf(lam_lo * lam_e);
+        len = 0;
+        for (int j = 0; j < n; ++j) {
+            int best = 0;
+            float bestc = 0.0f;
+            for (int m = 0; m < M; ++m) {
+                float d = z[j] - t[m];
+                float D = d * d;
+                float cost = fmaf(lam_e, T->r[m], D);
+                if (m == 0 || cost < bestc) { bestc = cost; best = m; }
+            }
+            m_out[j] = (uint8_t)best;
+            len += T->R[best];
+        }
+        if (len <= budget) return len;
+    }
     for (int it = 0; it <= 12; ++it) {
         float lam = (it < 12) ? sqrtf(lam_lo * lam_hi) : lam_hi;
         len = 0;
@@ -310,24 +359,23 @@ int64_t dqo_drift(const float *z, int n, float s, float o, const dqo_table *T, u
 /* -------------------------------------------------------------------- rANS */
 
 /* Eq. (rans) Enc applied to symbols n-1 ... 0 (so that decoding runs forward),
- * byte-wise renormalisation.  Writes the final state (4 bytes LE) followed by the
+ * byte-wise renormalisation.  Writes the final state (sigma / 8 bytes LE) followed by the
  * emitted bytes in reverse order of emission into `payload` (capacity cap bytes).
- * Returns the number of renormalisation bytes k, or -1 if 4 + k > cap. */
+ * Returns the number of renormalisation bytes k, or -1 if sigma / 8 + k > cap. */
 int dqo_rans_encode(const uint8_t *sym, int n, const dqo_table *T, uint8_t *payload, int cap)
 {
     uint8_t tmp[2 * DQO_MAX_N];
-    int k = 0;
-    uint32_t x = DQO_L;
+    int k = 0, sb = T->sigma / 8;                      /* bytes of final state */
+    uint32_t L = dqo_L(T), x = L;
     for (int j = n - 1; j >= 0; --j) {
         uint32_t f = (uint32_t)T->f[sym[j]], c = (uint32_t)T->c[sym[j]];
-        while (x >= (f << 23)) { tmp[k++] = (uint8_t)(x & 255u); x >>= 8; }
+        while (x >= f * L) { tmp[k++] = (uint8_t)(x & 255u); x >>= 8; }   /* x_max = f (L / 2^p) 2^8 */
         x = (x / f) * DQO_TOT + (x % f) + c;
     }
-    if (4 + k > cap) return -1;
-    payload[0] = (uint8_t)x; payload[1] = (uint8_t)(x >> 8);
-    payload[2] = (uint8_t)(x >> 16); payload[3] = (uint8_t)(x >> 24);
-    for (int i = 0; i < k; ++i) payload[4 + i] = tmp[k - 1 - i];
-    for (int i = 4 + k; i < cap; ++i) payload[i] = 0;
+    if (sb + k > cap) return -1;
+    for (int i = 0; i < sb; ++i) payload[i] = (uint8_t)(x >> (8 * i));
+    for (int i = 0; i < k; ++i) payload[sb + i] = tmp[k - 1 - i];
+    for (int i = sb + k; i < cap; ++i) payload[i] = 0;
     return k;
 }
 
@@ -337,15 +385,15 @@ int dqo_rans_encode(const uint8_t *sym, int n, const dqo_table *T, uint8_t *payl
 void dqo_rans_decode(const uint8_t *payload, int cap, int n, const dqo_table *T, uint8_t *sym,
                      uint32_t *end)
 {
-    uint32_t x = (uint32_t)payload[0] | ((uint32_t)payload[1] << 8) |
-                 ((uint32_t)payload[2] << 16) | ((uint32_t)payload[3] << 24);
-    int ptr = DQO_SIGMA / 8;
+    uint32_t x = 0, L = dqo_L(T);
+    int ptr = T->sigma / 8;
+    for (int i = 0; i < ptr; ++i) x |= (uint32_t)payload[i] << (8 * i);
     for (int i = 0; i < n; ++i) {
         uint32_t z = x & (DQO_TOT - 1);
         uint32_t f = T->lut_f[z], d = T->lut_d[z];
         sym[i] = T->lut_m[z];
         x = f * (x >> DQO_P) + d;
-        while (x < DQO_L && ptr < cap) { x = (x << 8) | payload[ptr]; ptr += 1; }
+        while (x < L && ptr < cap) { x = (x << 8) | payload[ptr]; ptr += 1; }
     }
     if (end) { end[0] = x; end[1] = (uint32_t)ptr; }
 }
@@ -432,7 +480,7 @@ void dqo_encode_stream(const float *z, const dqo_table *T, uint8_t *rec, uint32_
     rec[2] = (uint8_t)o16; rec[3] = (uint8_t)(o16 >> 8);
     int k = dqo_rans_encode(m, n, T, rec + 4, T->C);
     if (k < 0) { memset(rec + 4, 0, (size_t)T->C); k = 0; } /* excluded by the budget test */
-    if (stats && (uint32_t)(8 + k) > stats[3]) stats[3] = (uint32_t)(8 + k);
+    if (stats && (uint32_t)(4 + T->sigma / 8 + k) > stats[3]) stats[3] = (uint32_t)(4 + T->sigma / 8 + k);
     if (sym_out) memcpy(sym_out, m, (size_t)n);
 }
 
