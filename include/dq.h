@@ -50,6 +50,14 @@
  *     given stream and return; 0 means "validated and enqueued".
  *   - Errors are returned, never thrown; nothing is launched when validation fails;
  *     no kernel traps or spins.
+ *   - Codec variants (opt-in per table, dq_table_opts; the defaults are the paper's codec):
+ *     * drift_early_exit: Algorithm 1's Drift bisects log2(lambda) in 12 steps; when every test
+ *       passes it ends at a multiplier known beforehand.  The variant evaluates that multiplier
+ *       first and returns its assignment when it meets the budget, otherwise runs the bisection
+ *       (App. C: most streams have budget to spare).  Same record format.
+ *     * sigma_bits = 24: records are [s fp16][o fp16][final state, 3 bytes LE][bytes ...]; the state
+ *       lives in [2^15, 2^23) and B = 8C - 24 (Eq. budget), one more byte for symbols.  Key and
+ *       value tables of one cache must agree on sigma_bits.  Per token-head streams only.
  */
 #ifndef DQ_H_
 #define DQ_H_
@@ -95,6 +103,12 @@ typedef struct {
     int heads_per_stream; /* 0 or 1: one stream per (token, KV head); hs in 2..8: one stream per
                        hs consecutive KV heads of a token (hs = Hkv: the paper's token-wide
                        default, Sec. 5.1).  The model's n is then hs * 128. */
+    /* Opt-in codec variants (0 = the paper's codec; see "Codec variants" below) */
+    int drift_early_exit; /* 1: Drift first evaluates the multiplier its bisection ends at when every
+                       test passes and stops there if the budget is met (encoder only; records
+                       are read by the same decoder) */
+    int sigma_bits;  /* 0 or 32: 32-bit final state, state in [2^23, 2^31).  24: 24-bit final state,
+                       state in [2^15, 2^23), B = 8C - 24; per token-head streams only */
 } dq_table_opts;
 
 typedef struct {
@@ -107,6 +121,8 @@ typedef struct {
     uint32_t lut[256];             /* f << 24 | (fp16 bits of level) << 8 | (z - c) */
     int heads_per_stream;          /* >= 1                                           */
     int rec_words;                 /* ceil(rec_bytes / 4): words per record in the interleaved layout */
+    int sigma_bits;                /* 32 or 24: bits of final rANS state in a record    */
+    int drift_early_exit;          /* 0 / 1                                             */
 } dq_table_info;
 
 /* Probability model and rANS tables of one tensor kind (Sec. 3.1 "Entropy Coding",

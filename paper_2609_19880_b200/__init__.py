@@ -38,7 +38,7 @@ class DqError(RuntimeError):
 
 class TableOpts(C.Structure):
     _fields_ = [("head_dim", C.c_int), ("alpha", C.c_double), ("has_mean", C.c_int), ("rotate", C.c_int),
-                ("heads_per_stream", C.c_int)]
+                ("heads_per_stream", C.c_int), ("drift_early_exit", C.c_int), ("sigma_bits", C.c_int)]
 
 
 class TableInfo(C.Structure):
@@ -47,7 +47,8 @@ class TableInfo(C.Structure):
                 ("has_mean", C.c_int), ("rotate", C.c_int), ("alpha", C.c_double),
                 ("f", C.c_int32 * MAX_LEVELS), ("c", C.c_int32 * (MAX_LEVELS + 1)),
                 ("r", C.c_float * MAX_LEVELS), ("R", C.c_uint32 * MAX_LEVELS), ("lut", C.c_uint32 * 256),
-                ("heads_per_stream", C.c_int), ("rec_words", C.c_int)]
+                ("heads_per_stream", C.c_int), ("rec_words", C.c_int), ("sigma_bits", C.c_int),
+                ("drift_early_exit", C.c_int)]
 
 
 _lib = None
@@ -157,10 +158,13 @@ class Tables:
 
 
 def dq_build_tables(levels: int, bits_per_elem: float, *, alpha: float = 1.4, has_mean: bool = False,
-                    rotate: bool = True, head_dim: int = HEAD_DIM, heads_per_stream: int = 1) -> Tables:
+                    rotate: bool = True, head_dim: int = HEAD_DIM, heads_per_stream: int = 1,
+                    drift_early_exit: bool = False, sigma_bits: int = 32) -> Tables:
     """``heads_per_stream`` = hs > 1 builds tables for streams that span hs KV heads of a token
-    (hs = Hkv: the paper's token-wide default); bits_per_elem then refers to hs * 128 values."""
-    opts = TableOpts(head_dim, float(alpha), int(has_mean), int(rotate), int(heads_per_stream))
+    (hs = Hkv: the paper's token-wide default); bits_per_elem then refers to hs * 128 values.
+    ``drift_early_exit`` / ``sigma_bits`` select the opt-in codec variants."""
+    opts = TableOpts(head_dim, float(alpha), int(has_mean), int(rotate), int(heads_per_stream),
+                     int(drift_early_exit), int(sigma_bits))
     h = C.c_void_p()
     _check(lib().dq_build_tables(int(levels), float(bits_per_elem), C.byref(opts), C.byref(h)), "dq_build_tables")
     return Tables(h.value)

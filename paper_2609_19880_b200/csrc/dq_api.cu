@@ -31,6 +31,7 @@ int check_attn_tables(const dq_tables* tk, const dq_tables* tv, int Hkv, const u
     if (!tk || !tv || !k_cont || !v_cont) return DQ_ERR_ARG;
     if (tv->info.has_mean) return DQ_ERR_UNSUPPORTED;
     if (tk->info.heads_per_stream != tv->info.heads_per_stream) return DQ_ERR_UNSUPPORTED;
+    if (tk->info.sigma_bits != tv->info.sigma_bits) return DQ_ERR_UNSUPPORTED;   // one state width per cache
     if (Hkv <= 0 || Hkv % tk->info.heads_per_stream != 0) return DQ_ERR_ARG;
     if (tk->info.has_mean && (!k_mean_q || !k_mean_scale || max_windows <= 0)) return DQ_ERR_ARG;
     if (tk->info.has_mean && (long long)max_windows * DQ_WINDOW_TOKENS < (long long)max_pages * DQ_PAGE_TOKENS)

@@ -204,6 +204,8 @@ dq_attn_prepare_kernel(AttnParams p) {
 // + (z - c) (f by dp4a, product by mad, addend by dp4a); if x < L one byte is appended with a
 // byte-permute from a 4-byte window that is reloaded every 4 symbols (a symbol takes at most
 // one byte because the state stays >= 2^15).
+// LBITS: log2 of the lower bound L of the state interval, 23 (32-bit final state) or 15 (24-bit).
+template <int LBITS>
 __device__ __forceinline__ void decode16(uint32_t& x, uint32_t& ptr, uint32_t lut, uint32_t one,
                                          uint32_t (&packed)[8]) {
 #pragma unroll
@@ -218,9 +220,9 @@ __device__ __forceinline__ void decode16(uint32_t& x, uint32_t& ptr, uint32_t lu
             const uint32_t f = dp4a_u32(e[i], 0x01000000u, 0u);
             const uint32_t t = f * (x >> 8);
             x = dp4a_u32(e[i], 1u, t);
-            asm("{.reg .pred p; setp.lt.u32 p, %0, 0x800000; @p prmt.b32 %0, %0, %2, %1; "
+            asm("{.reg .pred p; setp.lt.u32 p, %0, %4; @p prmt.b32 %0, %0, %2, %1; "
                 "@p mad.lo.u32 %1, %3, %3, %1;}"
-                : "+r"(x), "+r"(sel) : "r"(win), "r"(one));
+                : "+r"(x), "+r"(sel) : "r"(win), "r"(one), "n"(1u << LBITS));
         }
         ptr += sel - 0x2104u;
         packed[2 * q4] = __byte_perm(e[0], e[1], 0x6521u);
@@ -233,7 +235,7 @@ __device__ __forceinline__ void decode16(uint32_t& x, uint32_t& ptr, uint32_t lu
 // DO_V the V streams of the previous item are decoded and each finished 16-channel tile of
 // O[j][g] = sum_t (a_t s_t) level_tj (Eq. fold-value, first sum) goes to this warp's output
 // slot in shared memory.  Both decodes are interleaved in one instruction stream.
-template <bool DO_K, bool DO_V>
+template <bool DO_K, bool DO_V, int LBITS>
 __device__ __forceinline__ void fused_pass(uint32_t xk, uint32_t ptrk, uint32_t xv, uint32_t ptrv, uint32_t lutk,
                                            uint32_t lutv, uint32_t one, uint32_t ktile, uint32_t vtile, uint32_t q16,
                                            uint32_t obuf, int lane, int G, float (&sacc)[4][4],
@@ -246,8 +248,8 @@ __device__ __forceinline__ void fused_pass(uint32_t xk, uint32_t ptrk, uint32_t 
 #pragma unroll 1
     for (int cg = 0; cg < 8; ++cg) {
         uint32_t pk[8], pv[8];
-        if (DO_K) decode16(xk, ptrk, lutk, one, pk);
-        if (DO_V) decode16(xv, ptrv, lutv, one, pv);
+        if (DO_K) decode16<LBITS>(xk, ptrk, lutk, one, pk);
+        if (DO_V) decode16<LBITS>(xv, ptrv, lutv, one, pv);
         if (DO_K) { sts128(ktile + lane * kTileStride, pk); sts128(ktile + lane * kTileStride + 16, pk + 4); }
         if (DO_V) { sts128(vtile + lane * kTileStride, pv); sts128(vtile + lane * kTileStride + 16, pv + 4); }
         __syncwarp();
@@ -289,7 +291,7 @@ __device__ __forceinline__ void fused_pass(uint32_t xk, uint32_t ptrk, uint32_t 
 // The option DQ_OPT_STEP_POLL_LIMIT replaces the default; 0 makes every CTA take the fallback at once,
 // which is how the tests run that path.
 static int step_poll_limit() { return dq_opt_step_poll_limit(DQ_STEP_POLL_LIMIT); }
-template <bool FUSED>
+template <bool FUSED, int LBITS>
 __global__ void __launch_bounds__(kMaxWarps * 32, 1)
 dq_attention_kernel(const __grid_constant__ DqDevTable TK, const __grid_constant__ DqDevTable TV,
                     const AttnParams p) {
@@ -514,16 +516,19 @@ dq_attention_kernel(const __grid_constant__ DqDevTable TK, const __grid_constant
 #pragma unroll
         for (int i = 0; i < 4; ++i) { sacc[i][0] = sacc[i][1] = sacc[i][2] = sacc[i][3] = 0.f; }
         {
-            const uint32_t xk = lds32_unaligned(rk + 4), xv = lds32_unaligned(rvp + 4);
+            // final state: 4 bytes (LBITS 23) or 3 bytes (LBITS 15) after the two fp16 grid parameters
+            constexpr uint32_t kStateMask = LBITS == 23 ? 0xffffffffu : 0x00ffffffu;
+            constexpr uint32_t kPay = LBITS == 23 ? 8u : 7u;
+            const uint32_t xk = lds32_unaligned(rk + 4) & kStateMask, xv = lds32_unaligned(rvp + 4) & kStateMask;
             if (cur.valid && have_prev)
-                fused_pass<true, true>(xk, rk + 8, xv, rvp + 8, my_lutk, my_lutv, one, ktile, vtile, q16, my_obuf, lane, G,
-                                       sacc, pb_hi, pb_lo);
+                fused_pass<true, true, LBITS>(xk, rk + kPay, xv, rvp + kPay, my_lutk, my_lutv, one, ktile, vtile, q16, my_obuf,
+                                              lane, G, sacc, pb_hi, pb_lo);
             else if (cur.valid)
-                fused_pass<true, false>(xk, rk + 8, xv, rvp + 8, my_lutk, my_lutv, one, ktile, vtile, q16, my_obuf, lane, G,
-                                        sacc, pb_hi, pb_lo);
+                fused_pass<true, false, LBITS>(xk, rk + kPay, xv, rvp + kPay, my_lutk, my_lutv, one, ktile, vtile, q16, my_obuf,
+                                               lane, G, sacc, pb_hi, pb_lo);
             else
-                fused_pass<false, true>(xk, rk + 8, xv, rvp + 8, my_lutk, my_lutv, one, ktile, vtile, q16, my_obuf, lane, G,
-                                        sacc, pb_hi, pb_lo);
+                fused_pass<false, true, LBITS>(xk, rk + kPay, xv, rvp + kPay, my_lutk, my_lutv, one, ktile, vtile, q16, my_obuf,
+                                               lane, G, sacc, pb_hi, pb_lo);
         }
 
         // ------------------------------------------ logits of `cur` and this warp's maximum (base 2)
@@ -1067,9 +1072,12 @@ static cudaError_t launch_attention_pass(const DqDevTable& tk, const DqDevTable&
     const long long prep_warps = (long long)heads * (1 + (p.has_mean ? (p.windows + kPrepWindows - 1) / kPrepWindows : 0));
     cudaError_t e = dq_launch_pdl(dq_attn_prepare_kernel, dim3((unsigned)((prep_warps + 7) / 8)), dim3(256), 0, st, p);
     if (e != cudaSuccess) return e;
+    // the four instantiations of the main kernel: decode-step mode or not, 32- or 24-bit final state
+    void (*main_kernel)(DqDevTable, DqDevTable, AttnParams) =
+        tk.sigma == 24 ? (p.fused ? dq_attention_kernel<true, 15> : dq_attention_kernel<false, 15>)
+                       : (p.fused ? dq_attention_kernel<true, 23> : dq_attention_kernel<false, 23>);
     if (!wide) {
-        e = p.fused ? cudaFuncSetAttribute(dq_attention_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, L.total)
-                    : cudaFuncSetAttribute(dq_attention_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, L.total);
+        e = cudaFuncSetAttribute(main_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, L.total);
         if (e != cudaSuccess) return e;
     }
     const bool prof = g_prof_on && g_prof_count < kProfRing && (g_prof_calls++ % g_prof_period) == 0;
@@ -1082,8 +1090,7 @@ static cudaError_t launch_attention_pass(const DqDevTable& tk, const DqDevTable&
         cudaEventRecord(g_prof_ev[g_prof_count][0], st);
     }
     if (wide) e = dq_launch_attention_wide_main(tk, tv, p, nw, sm_count, st);
-    else if (p.fused) e = dq_launch_pdl(dq_attention_kernel<true>, dim3(sm_count), dim3(nw * 32), (size_t)L.total, st, tk, tv, p);
-    else e = dq_launch_pdl(dq_attention_kernel<false>, dim3(sm_count), dim3(nw * 32), (size_t)L.total, st, tk, tv, p);
+    else e = dq_launch_pdl(main_kernel, dim3(sm_count), dim3(nw * 32), (size_t)L.total, st, tk, tv, p);
     if (e != cudaSuccess) return e;
     if (prof) cudaEventRecord(g_prof_ev[g_prof_count++][1], st);
     return dq_launch_pdl(dq_attn_combine_kernel, dim3(heads), dim3(256), 0, st, p);

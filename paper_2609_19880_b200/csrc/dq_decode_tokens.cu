@@ -21,9 +21,11 @@ dq_decode_tokens_kernel(const __grid_constant__ DqDevTable T, const uint8_t* __r
                                  (size_t)(sl % DQ_PAGE_TOKENS)) * T.rec;
     const float s = __half2float(__ushort_as_half((unsigned short)(rec[0] | (rec[1] << 8))));
     const float o = __half2float(__ushort_as_half((unsigned short)(rec[2] | (rec[3] << 8))));
-    uint32_t x = (uint32_t)rec[4] | ((uint32_t)rec[5] << 8) | ((uint32_t)rec[6] << 16) |
-                 ((uint32_t)rec[7] << 24);
-    int ptr = 8;
+    // final state: sigma / 8 bytes, little-endian; the state interval starts at L = 2^(sigma - 9)
+    uint32_t x = (uint32_t)rec[4] | ((uint32_t)rec[5] << 8) | ((uint32_t)rec[6] << 16);
+    if (T.sigma == 32) x |= (uint32_t)rec[7] << 24;
+    int ptr = 4 + (T.sigma >> 3);
+    const uint32_t L = 1u << (T.sigma - 9);
     const int8_t* mq = nullptr;
     float msc = 0.f;
     if (T.has_mean && mean_q) {
@@ -34,7 +36,7 @@ dq_decode_tokens_kernel(const __grid_constant__ DqDevTable T, const uint8_t* __r
     for (int j = 0; j < DQ_HEAD_DIM; ++j) {
         const uint32_t e = T.lut[x & 255u];
         x = (e >> 24) * (x >> 8) + (e & 255u);
-        if (x < (1u << 23) && ptr < T.rec) x = (x << 8) | rec[ptr++];  // at most one byte
+        if (x < L && ptr < T.rec) x = (x << 8) | rec[ptr++];  // at most one byte
         const float lvl = __half2float(__ushort_as_half((unsigned short)((e >> 8) & 0xffffu)));
         if (symbols) symbols[sid * DQ_HEAD_DIM + j] = (uint8_t)(int)lvl;
         if (dequant) {

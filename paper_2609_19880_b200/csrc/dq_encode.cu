@@ -14,7 +14,7 @@ namespace {
 
 constexpr unsigned kFull = dqdev::kFullMask;
 constexpr int kN = DQ_HEAD_DIM;
-constexpr uint32_t kL = 1u << 23;  // lower bound of the rANS state interval
+constexpr uint32_t kL = 1u << 23;  // lower bound of the rANS state interval (sigma = 32; token-wide streams always)
 
 using dqdev::bf16_bits_to_float;
 using dqdev::warp_fwht128;  // per-head Hadamard rotation (Sec. 4.2), 4 values per lane
@@ -145,8 +145,9 @@ struct EncTable {
     uint32_t rsh[DQ_MAX_LEVELS];
     uint32_t bias[DQ_MAX_LEVELS];  // c (+ 255 when f = 1)
     uint32_t cmpl[DQ_MAX_LEVELS];  // 2^p - f
-    uint32_t thr[DQ_MAX_LEVELS];   // f << 23: renormalise while the state is not below it
+    uint32_t thr[DQ_MAX_LEVELS];   // f << (sigma - 9) = f L: renormalise while the state is not below it
     int M, rec, mstar, budget_bits, has_mean, rotate;
+    int early_exit, sigma;         // codec variants: Drift tries its end multiplier first; bits of final state (32 / 24)
 };
 
 // Function Drift of Algorithm 1 on a stream held 4 values per lane.  The bisection of
@@ -189,9 +190,14 @@ __device__ __noinline__ uint32_t drift_m(const EncTable& T, float z0, float z1, 
     float lam_hi = __fmul_rn(8.0f, __fsub_rn(maxD, minD));
     float lam_lo = __fmul_rn(lam_hi, 0x1p-40f);
     uint32_t len = 0, sym[4] = {0u, 0u, 0u, 0u};
+    // Early-exit variant: when each of the 12 tests passes, the upper end walks hi <- sqrt(lo hi) twelve
+    // times with lo fixed; sweep -1 evaluates that multiplier and ends the search if its assignment fits.
+    float lam_e = lam_hi;
+    if (T.early_exit)
+        for (int i = 0; i < 12; ++i) lam_e = __fsqrt_rn(__fmul_rn(lam_lo, lam_e));
 #pragma unroll 1
-    for (int it = 0; it <= 12; ++it) {
-        const float lam = (it < 12) ? __fsqrt_rn(__fmul_rn(lam_lo, lam_hi)) : lam_hi;
+    for (int it = T.early_exit ? -1 : 0; it <= 12; ++it) {
+        const float lam = (it < 0) ? lam_e : (it < 12) ? __fsqrt_rn(__fmul_rn(lam_lo, lam_hi)) : lam_hi;
         uint32_t cost_sum = 0;
 #pragma unroll
         for (int e = 0; e < 4; ++e) {
@@ -209,7 +215,9 @@ __device__ __noinline__ uint32_t drift_m(const EncTable& T, float z0, float z1, 
             cost_sum += key[0];
         }
         len = __reduce_add_sync(kFull, cost_sum >> 8);   // four indices (< 16 each) stay below bit 8
-        if (it < 12) {
+        if (it < 0) {
+            if (len <= budget) break;
+        } else if (it < 12) {
             if (len <= budget) lam_hi = lam; else lam_lo = lam;
         }
     }
@@ -389,12 +397,13 @@ dq_encode_kernel(const __grid_constant__ DqDevTable TK, const __grid_constant__ 
         T.bias[i] = aux & 1023u;
         T.cmpl[i] = (aux >> 10) & 511u;
         T.rsh[i] = aux >> 19;
-        T.thr[i] = (256u - ((aux >> 10) & 511u)) << 23;
+        T.thr[i] = (256u - ((aux >> 10) & 511u)) << ((is_v ? TV.sigma : TK.sigma) - 9);
     }
     if (threadIdx.x == 0) {
         T.M = is_v ? TV.M : TK.M; T.rec = is_v ? TV.rec : TK.rec; T.mstar = is_v ? TV.mstar : TK.mstar;
         T.budget_bits = is_v ? TV.budget_bits : TK.budget_bits;
         T.has_mean = is_v ? TV.has_mean : TK.has_mean; T.rotate = is_v ? TV.rotate : TK.rotate;
+        T.early_exit = is_v ? TV.early_exit : TK.early_exit; T.sigma = is_v ? TV.sigma : TK.sigma;
     }
     __syncthreads();
     dqdev::pdl_wait_prior_grid();   // inputs and the cache may be written / read by the previous kernel
@@ -418,7 +427,7 @@ dq_encode_kernel(const __grid_constant__ DqDevTable TK, const __grid_constant__ 
     // carries the same state (the symbols come from shared memory); lane 0 records the bytes.
     *reinterpret_cast<uint32_t*>(&s_sym[wib][4 * lane]) = sq.sym;
     __syncwarp();
-    uint32_t xs = kL;
+    uint32_t xs = 1u << (T.sigma - 9);   // L: 2^23, or 2^15 with the 24-bit state
     int k = 0;
     // emitted bytes go to shared memory through stores the compiler does not treat as aliasing
     // the symbol / table loads, so those loads are issued ahead of the serial state chain
@@ -427,7 +436,7 @@ dq_encode_kernel(const __grid_constant__ DqDevTable TK, const __grid_constant__ 
     for (int j = kN - 1; j >= 0; --j) {
         const uint32_t m = s_sym[wib][j];
         const uint32_t rcp = T.rcp[m], rsh = T.rsh[m], bias = T.bias[m], cmpl = T.cmpl[m], thr = T.thr[m];
-        if (xs >= thr) {  // at most once: xs < 2^31 <= 2^8 * (f << 23)
+        if (xs >= thr) {  // at most once: xs < 2^8 L <= 2^8 * (f L)
             if (lane == 0) asm volatile("st.shared.u8 [%0], %1;" ::"r"(bytes_addr + k), "r"(xs & 0xffu));
             ++k;
             xs >>= 8;
@@ -440,19 +449,20 @@ dq_encode_kernel(const __grid_constant__ DqDevTable TK, const __grid_constant__ 
     const int sl = a.slot[t];
     uint8_t* rec = cont + (((size_t)(sl / DQ_PAGE_TOKENS) * Hkv + h) * DQ_PAGE_TOKENS +
                            (size_t)(sl % DQ_PAGE_TOKENS)) * T.rec;
-    const int used = min(8 + k, T.rec);  // the budget test keeps 8 + k <= rec
+    const int pay = 4 + (T.sigma >> 3);              // first payload byte: after (s, o) and the final state
+    const int used = min(pay + k, T.rec);            // the budget test keeps pay + k <= rec
     for (int i = lane; i < T.rec; i += 32) {
         uint8_t v = 0;
         if (i < 4) v = (uint8_t)(hdr0 >> (8 * i));
-        else if (i < 8) v = (uint8_t)(xs >> (8 * (i - 4)));
-        else if (i < used) v = s_bytes[wib][k - 1 - (i - 8)];
+        else if (i < pay) v = (uint8_t)(xs >> (8 * (i - 4)));
+        else if (i < used) v = s_bytes[wib][k - 1 - (i - pay)];
         rec[i] = v;
     }
     if (a.status && lane == 0) {
         if (sq.flags & 1u) atomicAdd(a.status + 0, 1u);
         if (sq.flags & 2u) atomicAdd(a.status + 1, 1u);
         if (sq.flags & 4u) atomicAdd(a.status + 2, 1u);
-        atomicMax(a.status + 3, (uint32_t)(8 + k));
+        atomicMax(a.status + 3, (uint32_t)(pay + k));
     }
 }
 
@@ -493,12 +503,13 @@ dq_encode_batch32_kernel(const __grid_constant__ DqDevTable TK, const __grid_con
         T.bias[i] = aux & 1023u;
         T.cmpl[i] = (aux >> 10) & 511u;
         T.rsh[i] = aux >> 19;
-        T.thr[i] = (256u - ((aux >> 10) & 511u)) << 23;
+        T.thr[i] = (256u - ((aux >> 10) & 511u)) << ((is_v ? TV.sigma : TK.sigma) - 9);
     }
     if (threadIdx.x == 0) {
         T.M = is_v ? TV.M : TK.M; T.rec = is_v ? TV.rec : TK.rec; T.mstar = is_v ? TV.mstar : TK.mstar;
         T.budget_bits = is_v ? TV.budget_bits : TK.budget_bits;
         T.has_mean = is_v ? TV.has_mean : TK.has_mean; T.rotate = is_v ? TV.rotate : TK.rotate;
+        T.early_exit = is_v ? TV.early_exit : TK.early_exit; T.sigma = is_v ? TV.sigma : TK.sigma;
     }
     __syncthreads();
     dqdev::pdl_wait_prior_grid();
@@ -528,12 +539,12 @@ dq_encode_batch32_kernel(const __grid_constant__ DqDevTable TK, const __grid_con
     }
     __syncthreads();
     if (wib == 0 && lane < ns) {   // rANS, Eq. (rans) Enc on symbols 127 .. 0; lane = stream
-        uint32_t xs = kL, k = 0;
+        uint32_t xs = 1u << (T.sigma - 9), k = 0;
 #pragma unroll 4
         for (int j = kN - 1; j >= 0; --j) {
             const uint32_t m = s_symT[j * kB32SymStride + lane];
             const uint32_t rcp = T.rcp[m], rsh = T.rsh[m], bias = T.bias[m], cmpl = T.cmpl[m], thr = T.thr[m];
-            if (xs >= thr) {   // at most once: xs < 2^31 <= 2^8 * (f << 23)
+            if (xs >= thr) {   // at most once: xs < 2^8 L <= 2^8 * (f L)
                 if (k < DQ_MAX_REC_BYTES) s_bytesT[k * kB32 + lane] = (uint8_t)xs;   // the budget test keeps k < rec - 8
                 ++k;
                 xs >>= 8;
@@ -542,17 +553,17 @@ dq_encode_batch32_kernel(const __grid_constant__ DqDevTable TK, const __grid_con
         }
         s_xs[lane] = xs;
         s_k[lane] = k;
-        if (a.status) atomicMax(a.status + 3, 8u + k);
+        if (a.status) atomicMax(a.status + 3, 4u + (uint32_t)(T.sigma >> 3) + k);
     }
     __syncthreads();
-    const int rec = T.rec;
-    for (int idx = threadIdx.x; idx < ns * rec; idx += blockDim.x) {   // records out: 8 + k bytes, then zeros
+    const int rec = T.rec, pay = 4 + (T.sigma >> 3);
+    for (int idx = threadIdx.x; idx < ns * rec; idx += blockDim.x) {   // records out: header, state, k bytes, then zeros
         const int si = idx / rec, i = idx - si * rec;
-        const int k = (int)s_k[si], used = min(8 + k, rec);
+        const int k = (int)s_k[si], used = min(pay + k, rec);
         uint8_t v = 0;
         if (i < 4) v = (uint8_t)(s_hdr[si] >> (8 * i));
-        else if (i < 8) v = (uint8_t)(s_xs[si] >> (8 * (i - 4)));
-        else if (i < used) v = s_bytesT[(k - 1 - (i - 8)) * kB32 + si];   // emitted last = read first
+        else if (i < pay) v = (uint8_t)(s_xs[si] >> (8 * (i - 4)));
+        else if (i < used) v = s_bytesT[(k - 1 - (i - pay)) * kB32 + si];   // emitted last = read first
         reinterpret_cast<uint8_t*>(s_rec[si])[i] = v;
     }
 }
@@ -649,9 +660,14 @@ __device__ __noinline__ uint32_t drift_wide_m(const EncTable& T, WideShared& W, 
     float lam_hi = __fmul_rn(8.0f, __fsub_rn(maxD, minD));
     float lam_lo = __fmul_rn(lam_hi, 0x1p-40f);
     uint32_t len = 0, sym[4] = {0u, 0u, 0u, 0u};
+    // Early-exit variant: when each of the 12 tests passes, the upper end walks hi <- sqrt(lo hi) twelve
+    // times with lo fixed; sweep -1 evaluates that multiplier and ends the search if its assignment fits.
+    float lam_e = lam_hi;
+    if (T.early_exit)
+        for (int i = 0; i < 12; ++i) lam_e = __fsqrt_rn(__fmul_rn(lam_lo, lam_e));
 #pragma unroll 1
-    for (int it = 0; it <= 12; ++it) {
-        const float lam = (it < 12) ? __fsqrt_rn(__fmul_rn(lam_lo, lam_hi)) : lam_hi;
+    for (int it = T.early_exit ? -1 : 0; it <= 12; ++it) {
+        const float lam = (it < 0) ? lam_e : (it < 12) ? __fsqrt_rn(__fmul_rn(lam_lo, lam_hi)) : lam_hi;
         uint32_t cost_sum = 0;
 #pragma unroll
         for (int e = 0; e < 4; ++e) {
@@ -673,7 +689,9 @@ __device__ __noinline__ uint32_t drift_wide_m(const EncTable& T, WideShared& W, 
         len = 0;
         for (int w = 0; w < hs; ++w) len += W.len[parity][w];
         parity ^= 1u;
-        if (it < 12) {
+        if (it < 0) {
+            if (len <= budget) break;   // uniform across the CTA: every warp sees the same stream-wide length
+        } else if (it < 12) {
             if (len <= budget) lam_hi = lam; else lam_lo = lam;
         }
     }
@@ -710,6 +728,7 @@ __device__ __forceinline__ void load_wide_table(EncTable& T, WideShared& W, cons
         T.M = is_v ? TV.M : TK.M; T.rec = is_v ? TV.rec : TK.rec; T.mstar = is_v ? TV.mstar : TK.mstar;
         T.budget_bits = is_v ? TV.budget_bits : TK.budget_bits;
         T.has_mean = is_v ? TV.has_mean : TK.has_mean; T.rotate = is_v ? TV.rotate : TK.rotate;
+        T.early_exit = is_v ? TV.early_exit : TK.early_exit; T.sigma = 32;   // token-wide streams keep the 32-bit state
     }
 }
 

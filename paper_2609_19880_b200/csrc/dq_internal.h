@@ -11,6 +11,7 @@ struct DqDevTable {
     int M, rec, mstar, budget_bits;
     int has_mean, rotate;
     int hs, rec_words;           // heads per stream (>= 1); words per record (interleaved layout, hs > 1)
+    int sigma, early_exit;       // bits of final state in a record (32 / 24); Drift tries its end multiplier first
     uint32_t enc_rcp[DQ_MAX_LEVELS];  // encoder, Eq. rans Enc by reciprocal: floor(x / f) = umulhi(x, rcp) >> rsh
     uint32_t enc_aux[DQ_MAX_LEVELS];  // bias | (256 - f) << 10 | rsh << 19, bias = c (+ 255 when f = 1)
     float r[DQ_MAX_LEVELS];      // ideal cost in bits     (Algorithm 1)

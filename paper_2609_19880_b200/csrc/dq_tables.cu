@@ -124,6 +124,9 @@ int dq_host_build(int levels, double bits_per_elem, const dq_table_opts* opts, d
     if (rec_d > (hs > 1 ? DQ_MAX_WIDE_REC_BYTES : DQ_MAX_REC_BYTES)) return DQ_ERR_UNSUPPORTED;
     const int rec = (int)rec_d;
     if (rec < 9) return DQ_ERR_INFEASIBLE;  // header alone is 8 bytes
+    const int sigma = opts->sigma_bits == 0 ? 32 : opts->sigma_bits;
+    if (sigma != 32 && sigma != 24) return DQ_ERR_ARG;
+    if (sigma == 24 && hs > 1) return DQ_ERR_UNSUPPORTED;   // the short state is offered for 128-value streams
 
     dq_table_info& t = out->info;
     std::memset(out, 0, sizeof *out);
@@ -133,7 +136,9 @@ int dq_host_build(int levels, double bits_per_elem, const dq_table_opts* opts, d
     t.rec_words = (rec + 3) / 4;
     t.rec_bytes = rec;
     t.container_bytes = rec - 4;              // Eq. (budget): C bytes hold state + payload
-    t.budget_bits = 8 * t.container_bytes - 32;  // B = 8C - sigma, sigma = 32
+    t.budget_bits = 8 * t.container_bytes - sigma;  // B = 8C - sigma
+    t.sigma_bits = sigma;
+    t.drift_early_exit = opts->drift_early_exit ? 1 : 0;
     t.has_mean = opts->has_mean ? 1 : 0;
     t.rotate = opts->rotate ? 1 : 0;
 
@@ -163,6 +168,8 @@ int dq_host_build(int levels, double bits_per_elem, const dq_table_opts* opts, d
     d.rotate = t.rotate;
     d.hs = hs;
     d.rec_words = t.rec_words;
+    d.sigma = sigma;
+    d.early_exit = t.drift_early_exit;
     for (int m = 0; m < levels; ++m) {
         // Enc(x, m) = floor(x / f) 2^p + x mod f + c = x + c + floor(x / f) (2^p - f); the quotient of a
         // 31-bit x by f comes from one high multiply with rcp = ceil(2^(31 + s) / f), s = ceil(log2 f),

@@ -14,12 +14,17 @@ from paper_2609_19880_b200 import workloads
 SM_SCALE = 1.0 / math.sqrt(128.0)
 
 
-def tables(cfg, rotate_v=True):
-    """(library K, library V, oracle K, oracle V) tables of a configuration."""
-    tk = dq.dq_build_tables(cfg.k_levels, cfg.bits_k, alpha=cfg.alpha, has_mean=True, rotate=True)
-    tv = dq.dq_build_tables(cfg.v_levels, cfg.bits_v, alpha=cfg.alpha, has_mean=False, rotate=rotate_v)
-    ok = oracle.build_table(cfg.k_levels, 128, cfg.k_rec, cfg.alpha, has_mean=True, rotate=True)
-    ov = oracle.build_table(cfg.v_levels, 128, cfg.v_rec, cfg.alpha, has_mean=False, rotate=rotate_v)
+def tables(cfg, rotate_v=True, early_exit=False, sigma=32):
+    """(library K, library V, oracle K, oracle V) tables of a configuration; early_exit / sigma select
+    the opt-in codec variants on both sides."""
+    tk = dq.dq_build_tables(cfg.k_levels, cfg.bits_k, alpha=cfg.alpha, has_mean=True, rotate=True,
+                            drift_early_exit=early_exit, sigma_bits=sigma)
+    tv = dq.dq_build_tables(cfg.v_levels, cfg.bits_v, alpha=cfg.alpha, has_mean=False, rotate=rotate_v,
+                            drift_early_exit=early_exit, sigma_bits=sigma)
+    ok = oracle.build_table(cfg.k_levels, 128, cfg.k_rec, cfg.alpha, has_mean=True, rotate=True,
+                            early_exit=early_exit, sigma=sigma)
+    ov = oracle.build_table(cfg.v_levels, 128, cfg.v_rec, cfg.alpha, has_mean=False, rotate=rotate_v,
+                            early_exit=early_exit, sigma=sigma)
     return tk, tv, ok, ov
 
 
@@ -102,12 +107,14 @@ def check_attention(out_bf16, out_f32, ref, rows=None):
 # ---- token-wide streams (heads_per_stream = hs > 1): the library stores records word-interleaved
 # per page, uint8 [pages][groups][rec_words][16][4]; the oracle keeps [pages][groups][16][rec].
 
-def wide_tables(cfg, hs, k_rec=335, v_rec=235, k_levels=8, v_levels=6, alpha=1.4):
+def wide_tables(cfg, hs, k_rec=335, v_rec=235, k_levels=8, v_levels=6, alpha=1.4, early_exit=False):
     n = 128 * hs
-    tk = dq.dq_build_tables(k_levels, k_rec * 8 / n, alpha=alpha, has_mean=True, rotate=True, heads_per_stream=hs)
-    tv = dq.dq_build_tables(v_levels, v_rec * 8 / n, alpha=alpha, has_mean=False, rotate=True, heads_per_stream=hs)
-    ok = oracle.build_table(k_levels, n, k_rec, alpha, has_mean=True, rotate=True)
-    ov = oracle.build_table(v_levels, n, v_rec, alpha, has_mean=False, rotate=True)
+    tk = dq.dq_build_tables(k_levels, k_rec * 8 / n, alpha=alpha, has_mean=True, rotate=True, heads_per_stream=hs,
+                            drift_early_exit=early_exit)
+    tv = dq.dq_build_tables(v_levels, v_rec * 8 / n, alpha=alpha, has_mean=False, rotate=True, heads_per_stream=hs,
+                            drift_early_exit=early_exit)
+    ok = oracle.build_table(k_levels, n, k_rec, alpha, has_mean=True, rotate=True, early_exit=early_exit)
+    ov = oracle.build_table(v_levels, n, v_rec, alpha, has_mean=False, rotate=True, early_exit=early_exit)
     assert tk.info().rec_bytes == k_rec and tv.info().rec_bytes == v_rec
     return tk, tv, ok, ov
 
