@@ -779,12 +779,27 @@ dq_attn_combine_kernel(AttnParams p) {
 }
 
 // ------------------------------------------------- bf16-cache comparison baseline
+//
+// Plain split-K decode attention over an un-quantised bf16 cache [page][Hkv][16][128], written to be
+// bound by HBM: every warp streams a contiguous token range of one (sequence, KV head) on its own --
+// its own cp.async ring of 32-token K and V tiles, the query fragments, online softmax and the output
+// accumulator in registers, no CTA barrier in the loop -- and leaves one partial per range.  The
+// ranges ("splits") are sized on the device from the sequence lengths so that the whole cache is cut
+// into about two ranges per resident warp.
 
-constexpr int kBfWarps = 4;
+#ifndef DQ_BF_WARPS
+#define DQ_BF_WARPS 5
+#endif
+#ifndef DQ_BF_STAGES
+#define DQ_BF_STAGES 2
+#endif
+constexpr int kBfWarps = DQ_BF_WARPS;
+constexpr int kBfStages = DQ_BF_STAGES;                 // 32-token (K, V) tile pairs in flight per warp
 constexpr int kBfRowStride = 272;                       // 128 bf16 + 16 bytes pad
-constexpr int kBfTileBytes = kChunk * kBfRowStride;     // one warp's K (or V) tile
-constexpr int kBfSmem = 16 * kBfRowStride + kBfWarps * 2 * kBfTileBytes + 3 * kBfWarps * 8 * 4 +
-                        kBfWarps * 8 * kORow * 4;
+constexpr int kBfTileBytes = kChunk * kBfRowStride;     // one 32-token K (or V) tile
+constexpr int kBfWarpBytes = kBfStages * 2 * kBfTileBytes;
+constexpr int kBfSmem = kBfWarps * kBfWarpBytes;
+constexpr int kBfMinSplitTokens = 128;                  // a split never covers fewer tokens (bounds the partial count)
 
 __device__ __forceinline__ void mma_bf16_16816(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
     asm volatile(
@@ -794,138 +809,181 @@ __device__ __forceinline__ void mma_bf16_16816(float (&d)[4], const uint32_t (&a
         : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
 }
 
-// Plain split-K decode attention over an un-quantised bf16 cache [page][Hkv][16][128].
-// One CTA per (block of 128 tokens, KV head, sequence); each warp owns 32 tokens.
-__global__ void __launch_bounds__(kBfWarps * 32)
-dq_bf16_attention_kernel(const AttnParams p, const uint16_t* __restrict__ kp, const uint16_t* __restrict__ vp) {
+__global__ void __launch_bounds__(kBfWarps * 32, 1)
+dq_bf16_attention_kernel(const AttnParams p, const uint16_t* __restrict__ kp, const uint16_t* __restrict__ vp,
+                         int units_target) {
     extern __shared__ __align__(128) uint8_t smem[];
+    __shared__ int s_prefix[4096 + 1];   // splits before each sequence (B <= 4096)
+    __shared__ long long s_tot[kBfWarps];
     pdl_launch_dependents();
-    pdl_wait_prior_grid();
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int b = blockIdx.z, h = blockIdx.y, blk = blockIdx.x, G = p.G;
-    const int bg0 = p.prefix[b];
-    if (blk >= p.prefix[b + 1] - bg0) return;
-    const int len = min(p.seq_lens[b], p.max_pages * DQ_PAGE_TOKENS);
-    const uint32_t sbase = smem_addr(smem);
-    const uint32_t q16 = sbase;
-    const uint32_t kt = sbase + 16 * kBfRowStride + warp * 2 * kBfTileBytes, vt = kt + kBfTileBytes;
-    float* red_m = reinterpret_cast<float*>(smem + 16 * kBfRowStride + kBfWarps * 2 * kBfTileBytes);
-    float* red_l = red_m + kBfWarps * 8;
-    float* mbuf = red_l + 2 * kBfWarps * 8;
-
-    const int tok0 = (blk * kBfWarps + warp) * kChunk;
-    if (tok0 < len) {
-        const int npg = (tok0 + 16 < len) ? 2 : 1;
-        for (int pg = 0; pg < npg; ++pg) {
-            const size_t page = (size_t)p.page_table[(size_t)b * p.max_pages + (tok0 >> 4) + pg] * p.Hkv + h;
-            const uint8_t* ks = reinterpret_cast<const uint8_t*>(kp) + page * (16 * kN * 2);
-            const uint8_t* vs = reinterpret_cast<const uint8_t*>(vp) + page * (16 * kN * 2);
-            for (int i = lane; i < 256; i += 32) {   // 16 rows x 16 chunks of 16 bytes
-                const int r = i >> 4, c = i & 15;
-                cp_async16(kt + (pg * 16 + r) * kBfRowStride + c * 16, ks + i * 16);
-                cp_async16(vt + (pg * 16 + r) * kBfRowStride + c * 16, vs + i * 16);
+    pdl_wait_prior_grid();   // the previous call's merge kernel still reads the arrays written here
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, G = p.G;
+    // Every CTA sizes the splits itself (the lengths live on the device): tokens per split = a multiple of
+    // 32, >= kBfMinSplitTokens, about total token-heads / units_target; then the exclusive scan of the splits
+    // per sequence.  CTA 0 leaves the scan in global memory for the merge kernel.
+    int split_tokens;
+    {
+        long long tot = 0;
+        for (int b = threadIdx.x; b < p.B; b += blockDim.x) tot += min(max(p.seq_lens[b], 0), p.max_pages * DQ_PAGE_TOKENS);
+#pragma unroll
+        for (int d = 16; d >= 1; d >>= 1) tot += __shfl_xor_sync(kFullMask, tot, d);
+        if (lane == 0) s_tot[warp] = tot;
+        __syncthreads();
+        tot = 0;
+        for (int i = 0; i < kBfWarps; ++i) tot += s_tot[i];
+        long long per = (tot * p.Hkv + units_target - 1) / units_target;
+        per = max((long long)kBfMinSplitTokens, (per + kChunk - 1) / kChunk * kChunk);
+        split_tokens = (int)min(per, (long long)p.max_pages * DQ_PAGE_TOKENS + kChunk);
+        if (warp == 0) {
+            int carry = 0;
+            for (int base = 0; base < p.B; base += 32) {
+                const int b = base + lane;
+                int nb = 0;
+                if (b < p.B) nb = (min(max(p.seq_lens[b], 0), p.max_pages * DQ_PAGE_TOKENS) + split_tokens - 1) / split_tokens;
+                int incl = nb;
+#pragma unroll
+                for (int d = 1; d < 32; d <<= 1) {
+                    const int o = __shfl_up_sync(kFullMask, incl, d);
+                    if (lane >= d) incl += o;
+                }
+                if (b < p.B) { s_prefix[b] = carry + incl - nb; if (blockIdx.x == 0) p.prefix[b] = carry + incl - nb; }
+                carry += __shfl_sync(kFullMask, incl, 31);
             }
+            if (lane == 0) { s_prefix[p.B] = carry; if (blockIdx.x == 0) p.prefix[p.B] = carry; }
         }
+        __syncthreads();
     }
-    cp_async_commit();
-    for (int i = tid; i < 16 * 64; i += blockDim.x) {   // q rows (bf16 pairs), zero beyond G
-        const int g = i >> 6, c = i & 63;
-        uint32_t v = 0;
-        if (g < G) v = *reinterpret_cast<const uint32_t*>(p.q + ((size_t)b * p.Hq + (size_t)h * G + g) * kN + 2 * c);
-        *reinterpret_cast<uint32_t*>(smem + g * kBfRowStride + c * 4) = v;
-    }
-    cp_async_wait<0>();
-    __syncthreads();
-
+    const uint32_t ring = smem_addr(smem) + warp * kBfWarpBytes;   // stage s: K at ring + s * 2 tiles, V one tile later
+    const int units = s_prefix[p.B] * p.Hkv;
     const int g_row = lane >> 2, qd = lane & 3;
-    float oacc[16][4];
-#pragma unroll
-    for (int i = 0; i < 16; ++i) { oacc[i][0] = oacc[i][1] = oacc[i][2] = oacc[i][3] = 0.f; }
-    float m_run = -INFINITY, l_run = 0.f;
-    if (tok0 < len) {
-        float sacc[4][4];
-#pragma unroll
-        for (int i = 0; i < 4; ++i) { sacc[i][0] = sacc[i][1] = sacc[i][2] = sacc[i][3] = 0.f; }
-        const uint32_t a_addr = q16 + ((lane & 7) + ((lane >> 3) & 1) * 8) * kBfRowStride + (lane >> 4) * 16;
-        const uint32_t b_addr = kt + ((lane & 7) + (lane >> 4) * 8) * kBfRowStride + ((lane >> 3) & 1) * 16;
-#pragma unroll
-        for (int cg = 0; cg < 8; ++cg) {
-            uint32_t a[4], b0[4], b1[4];
-            ldmatrix_x4(a, a_addr + cg * 32);
-            ldmatrix_x4(b0, b_addr + cg * 32);
-            ldmatrix_x4(b1, b_addr + cg * 32 + 16 * kBfRowStride);
-            mma_bf16_16816(sacc[0], a, b0[0], b0[1]);
-            mma_bf16_16816(sacc[1], a, b0[2], b0[3]);
-            mma_bf16_16816(sacc[2], a, b1[0], b1[1]);
-            mma_bf16_16816(sacc[3], a, b1[2], b1[3]);
+    const uint32_t frag = ((lane & 7) + (lane >> 4) * 8) * kBfRowStride + ((lane >> 3) & 1) * 16;        // K tile, B operand
+    const uint32_t fragv = ((lane & 7) + ((lane >> 3) & 1) * 8) * kBfRowStride + (lane >> 4) * 16;       // V tile, transposed
+
+    for (int u = blockIdx.x * kBfWarps + warp; u < units; u += gridDim.x * kBfWarps) {
+        const int bg = u / p.Hkv, h = u - bg * p.Hkv;
+        int lo = 0, hi = p.B;                     // largest b with prefix[b] <= bg
+        while (hi - lo > 1) {
+            const int mid = (lo + hi) >> 1;
+            if (s_prefix[mid] <= bg) lo = mid; else hi = mid;
         }
-        float mx = -INFINITY;
+        const int b = lo, split = bg - s_prefix[b];
+        const int len = min(p.seq_lens[b], p.max_pages * DQ_PAGE_TOKENS);
+        const int tok_lo = split * split_tokens, tok_hi = min(len, tok_lo + split_tokens);
+        const int32_t* pt = p.page_table + (size_t)b * p.max_pages;
+        __syncwarp();
+        // A fragments of q for the 8 channel groups, straight from global memory: row g = lane / 4 holds head g of
+        // this KV head (rows beyond G, and the upper 8 rows of the tile, are zero)
+        uint32_t qa[8][2];
+        {
+            const uint32_t* qrow = reinterpret_cast<const uint32_t*>(p.q + ((size_t)b * p.Hq + (size_t)h * G + min(g_row, G - 1)) * kN);
 #pragma unroll
-        for (int i = 0; i < 4; ++i)
-#pragma unroll
-            for (int u = 0; u < 2; ++u) {
-                const bool ok = tok0 + 8 * i + 2 * qd + u < len;
-                sacc[i][u] = ok ? sacc[i][u] * p.scale_log2 : -INFINITY;
-                mx = fmaxf(mx, sacc[i][u]);
+            for (int cg = 0; cg < 8; ++cg) {
+                qa[cg][0] = g_row < G ? qrow[cg * 8 + qd] : 0u;
+                qa[cg][1] = g_row < G ? qrow[cg * 8 + 4 + qd] : 0u;
             }
-        mx = fmaxf(mx, __shfl_xor_sync(kFullMask, mx, 1));
-        mx = fmaxf(mx, __shfl_xor_sync(kFullMask, mx, 2));
-        m_run = mx;
-        const float m_use = (mx == -INFINITY) ? 0.f : mx;
-        uint32_t pa[2][4];
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            const float p0 = exp2f(sacc[i][0] - m_use), p1 = exp2f(sacc[i][1] - m_use);
-            l_run += p0 + p1;
-            const __nv_bfloat162 pk = __floats2bfloat162_rn(p0, p1);
-            pa[i >> 1][(i & 1) * 2] = *reinterpret_cast<const uint32_t*>(&pk);
-            pa[i >> 1][(i & 1) * 2 + 1] = 0u;
         }
-        // rows beyond the sequence end hold stale shared memory: zero weights times NaN must not
-        // leak, so clear the unused V rows of the last chunk
-        if (tok0 + kChunk > len) {
-            for (int r = len - tok0; r < kChunk; ++r)
-                for (int c = lane; c < 64; c += 32) *reinterpret_cast<uint32_t*>(smem + (vt - sbase) + r * kBfRowStride + c * 4) = 0u;
+        auto load_chunk = [&](int tok0, int stage) {
+            const uint32_t kt = ring + stage * 2 * kBfTileBytes, vt = kt + kBfTileBytes;
+            const int npg = (tok0 + 16 < len) ? 2 : 1;
+            for (int pg = 0; pg < npg; ++pg) {
+                const size_t page = ((size_t)pt[(tok0 >> 4) + pg] * p.Hkv + h) * (size_t)(16 * kN * 2);
+                const uint8_t* ks = reinterpret_cast<const uint8_t*>(kp) + page;
+                const uint8_t* vs = reinterpret_cast<const uint8_t*>(vp) + page;
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {   // 16 rows x 16 pieces of 16 bytes
+                    const int i = lane + 32 * j, r = i >> 4, c = i & 15;
+                    cp_async16(kt + (pg * 16 + r) * kBfRowStride + c * 16, ks + i * 16);
+                    cp_async16(vt + (pg * 16 + r) * kBfRowStride + c * 16, vs + i * 16);
+                }
+            }
+        };
+        float oacc[16][4];
+#pragma unroll
+        for (int i = 0; i < 16; ++i) { oacc[i][0] = oacc[i][1] = oacc[i][2] = oacc[i][3] = 0.f; }
+        float m_run = -INFINITY, l_run = 0.f;
+#pragma unroll
+        for (int s0 = 0; s0 < kBfStages - 1; ++s0) {   // prologue: the first stages - 1 chunks
+            if (tok_lo + s0 * kChunk < tok_hi) load_chunk(tok_lo + s0 * kChunk, s0);
+            cp_async_commit();
+        }
+        int stage = 0;
+        for (int tok0 = tok_lo; tok0 < tok_hi; tok0 += kChunk, stage = (stage + 1 == kBfStages) ? 0 : stage + 1) {
+            {
+                const int ahead = tok0 + (kBfStages - 1) * kChunk;
+                if (ahead < tok_hi) load_chunk(ahead, (stage + kBfStages - 1) % kBfStages);
+                cp_async_commit();
+            }
+            cp_async_wait<kBfStages - 1>();
             __syncwarp();
-        }
-        const uint32_t v_addr = vt + ((lane & 7) + ((lane >> 3) & 1) * 8) * kBfRowStride + (lane >> 4) * 16;
+            const uint32_t kt = ring + stage * 2 * kBfTileBytes, vt = kt + kBfTileBytes;
+            float sacc[4][4];
 #pragma unroll
-        for (int cg = 0; cg < 8; ++cg) {
-            uint32_t b0[4], b1[4];
-            ldmatrix_x4_trans(b0, v_addr + cg * 32);
-            ldmatrix_x4_trans(b1, v_addr + cg * 32 + 16 * kBfRowStride);
-            mma_bf16_16816(oacc[2 * cg], pa[0], b0[0], b0[1]);
-            mma_bf16_16816(oacc[2 * cg + 1], pa[0], b0[2], b0[3]);
-            mma_bf16_16816(oacc[2 * cg], pa[1], b1[0], b1[1]);
-            mma_bf16_16816(oacc[2 * cg + 1], pa[1], b1[2], b1[3]);
-        }
-    }
-    l_run += __shfl_xor_sync(kFullMask, l_run, 1);
-    l_run += __shfl_xor_sync(kFullMask, l_run, 2);
-    if (qd == 0) { red_m[warp * 8 + g_row] = m_run; red_l[warp * 8 + g_row] = l_run; }
-    __syncthreads();
-    float m_all = -INFINITY;
-    for (int w = 0; w < kBfWarps; ++w) m_all = fmaxf(m_all, red_m[w * 8 + g_row]);
-    const float my_scale = exp2f(m_run - ((m_all == -INFINITY) ? 0.f : m_all));
-    if (g_row < G) {
-        float* dst = mbuf + (warp * G + g_row) * kORow + 2 * qd;
+            for (int i = 0; i < 4; ++i) { sacc[i][0] = sacc[i][1] = sacc[i][2] = sacc[i][3] = 0.f; }
 #pragma unroll
-        for (int nt = 0; nt < 16; ++nt)
-            *reinterpret_cast<float2*>(dst + 8 * nt) = make_float2(oacc[nt][0] * my_scale, oacc[nt][1] * my_scale);
-    }
-    __syncthreads();
-    for (int e = tid; e < G * kN; e += blockDim.x) {
-        const int g = e >> 7, ch = e & (kN - 1);
-        float mg = -INFINITY, s = 0.f, lsum = 0.f;
-        for (int w = 0; w < kBfWarps; ++w) mg = fmaxf(mg, red_m[w * 8 + g]);
-        const float mb = (mg == -INFINITY) ? 0.f : mg;
-        for (int w = 0; w < kBfWarps; ++w) {
-            s += mbuf[(w * G + g) * kORow + ch];
-            lsum = fmaf(red_l[w * 8 + g], exp2f(red_m[w * 8 + g] - mb), lsum);
+            for (int cg = 0; cg < 8; ++cg) {
+                uint32_t b0[4], b1[4];
+                const uint32_t a[4] = {qa[cg][0], 0u, qa[cg][1], 0u};
+                ldmatrix_x4(b0, kt + frag + cg * 32);
+                ldmatrix_x4(b1, kt + frag + cg * 32 + 16 * kBfRowStride);
+                mma_bf16_16816(sacc[0], a, b0[0], b0[1]);
+                mma_bf16_16816(sacc[1], a, b0[2], b0[3]);
+                mma_bf16_16816(sacc[2], a, b1[0], b1[1]);
+                mma_bf16_16816(sacc[3], a, b1[2], b1[3]);
+            }
+            float mx = -INFINITY;
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+#pragma unroll
+                for (int uu = 0; uu < 2; ++uu) {
+                    const bool ok = tok0 + 8 * i + 2 * qd + uu < tok_hi;
+                    sacc[i][uu] = ok ? sacc[i][uu] * p.scale_log2 : -INFINITY;
+                    mx = fmaxf(mx, sacc[i][uu]);
+                }
+            mx = fmaxf(mx, __shfl_xor_sync(kFullMask, mx, 1));
+            mx = fmaxf(mx, __shfl_xor_sync(kFullMask, mx, 2));
+            const float m_new = fmaxf(m_run, mx);           // finite: the chunk holds at least one token of the range
+            const float keep = exp2f(m_run - m_new);        // 0 on the first chunk
+            m_run = m_new;
+            l_run *= keep;
+#pragma unroll
+            for (int i = 0; i < 16; ++i) { oacc[i][0] *= keep; oacc[i][1] *= keep; }
+            uint32_t pa[2][4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const float p0 = exp2f(sacc[i][0] - m_new), p1 = exp2f(sacc[i][1] - m_new);
+                l_run += p0 + p1;
+                const __nv_bfloat162 pk = __floats2bfloat162_rn(p0, p1);
+                pa[i >> 1][(i & 1) * 2] = *reinterpret_cast<const uint32_t*>(&pk);
+                pa[i >> 1][(i & 1) * 2 + 1] = 0u;
+            }
+            // rows beyond the range end hold stale shared memory: zero weights times NaN must not
+            // leak, so clear the unused V rows of the last chunk
+            if (tok0 + kChunk > tok_hi) {
+                for (int r = tok_hi - tok0; r < kChunk; ++r)
+                    for (int c = lane; c < 64; c += 32) *reinterpret_cast<uint32_t*>(smem + (vt - smem_addr(smem)) + r * kBfRowStride + c * 4) = 0u;
+                __syncwarp();
+            }
+#pragma unroll
+            for (int cg = 0; cg < 8; ++cg) {
+                uint32_t b0[4], b1[4];
+                ldmatrix_x4_trans(b0, vt + fragv + cg * 32);
+                ldmatrix_x4_trans(b1, vt + fragv + cg * 32 + 16 * kBfRowStride);
+                mma_bf16_16816(oacc[2 * cg], pa[0], b0[0], b0[1]);
+                mma_bf16_16816(oacc[2 * cg + 1], pa[0], b0[2], b0[3]);
+                mma_bf16_16816(oacc[2 * cg], pa[1], b1[0], b1[1]);
+                mma_bf16_16816(oacc[2 * cg + 1], pa[1], b1[2], b1[3]);
+            }
+            __syncwarp();   // the tiles of this stage are free for the load issued next iteration
         }
-        float* dst = p.partial + ((size_t)(bg0 + blk) * p.Hq + (size_t)h * G + g) * kPartial;
-        dst[ch] = s;
-        if (ch == 0) { dst[kN] = mg; dst[kN + 1] = lsum; dst[kN + 2] = 0.f; }
+        cp_async_wait<0>();
+        l_run += __shfl_xor_sync(kFullMask, l_run, 1);
+        l_run += __shfl_xor_sync(kFullMask, l_run, 2);
+        if (g_row < G) {
+            float* dst = p.partial + ((size_t)bg * p.Hq + (size_t)h * G + g_row) * kPartial;
+#pragma unroll
+            for (int nt = 0; nt < 16; ++nt) *reinterpret_cast<float2*>(dst + 8 * nt + 2 * qd) = make_float2(oacc[nt][0], oacc[nt][1]);
+            if (qd == 0) { dst[kN] = m_run; dst[kN + 1] = l_run; dst[kN + 2] = 0.f; }
+        }
     }
 }
 
@@ -1140,7 +1198,7 @@ cudaError_t dq_launch_bf16_attention(const DqAttnArgs& a, const void* k_pages, c
     p.out_bf16 = a.out_bf16; p.out_f32 = nullptr;
     p.max_windows = 0; p.windows = 0; p.has_mean = 0; p.max_pages = a.max_pages;
     p.B = a.B; p.Hq = a.Hq; p.Hkv = a.Hkv; p.G = a.Hq / a.Hkv;
-    p.item_tokens = kBfWarps * kChunk;
+    p.item_tokens = kBfMinSplitTokens;
     p.rotate_q = 0; p.rotate_out = 0;
     p.scale_log2 = a.sm_scale * 1.4426950408889634f;
     p.hkv_magic = 0;
@@ -1149,15 +1207,15 @@ cudaError_t dq_launch_bf16_attention(const DqAttnArgs& a, const void* k_pages, c
     p.fused = 0; p.attn_grid = 0; p.poll_limit = 0; p.flags = p.counter; p.ne_before = p.prefix + (a.B + 1);
     p.resid_k = nullptr; p.resid_v = nullptr; p.resid_lens = nullptr; p.resid_cap = 0;
     const int heads = a.B * a.Hq;
-    dq_attn_prepare_kernel<<<(heads + 7) / 8, 256, 0, st>>>(p);
-    cudaError_t e = cudaGetLastError();
+    int sm_count = 0, smem_max = 0;
+    cudaError_t e = device_limits(&sm_count, &smem_max);
     if (e != cudaSuccess) return e;
+    if (kBfSmem + 17 * 1024 > smem_max) return cudaErrorInvalidConfiguration;   // ring + the static scan arrays
     e = cudaFuncSetAttribute(dq_bf16_attention_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kBfSmem);
     if (e != cudaSuccess) return e;
-    const int max_blocks = (a.max_pages * DQ_PAGE_TOKENS + p.item_tokens - 1) / p.item_tokens;
-    dq_bf16_attention_kernel<<<dim3(max_blocks, a.Hkv, a.B), kBfWarps * 32, kBfSmem, st>>>(
-        p, static_cast<const uint16_t*>(k_pages), static_cast<const uint16_t*>(v_pages));
-    e = cudaGetLastError();
+    e = dq_launch_pdl(dq_bf16_attention_kernel, dim3(sm_count), dim3(kBfWarps * 32), (size_t)kBfSmem, st, p,
+                      static_cast<const uint16_t*>(k_pages), static_cast<const uint16_t*>(v_pages),
+                      2 * sm_count * kBfWarps);
     if (e != cudaSuccess) return e;
     return dq_launch_pdl(dq_attn_combine_kernel, dim3(heads), dim3(256), 0, st, p);
 }

@@ -349,3 +349,28 @@ def test_config4_decode_step_full():
     cfg = workloads.make_config(4)
     assert sum((l + 511) // 512 for l in cfg.seq_lens) * cfg.hkv > 32 * 148
     _step_vs_two_calls(cfg, steps=3, seed=44)
+
+
+def test_bf16_baseline_config2_full():
+    """The bf16-cache comparison kernel at the benchmark's size (splits of several 32-token chunks per warp,
+    online softmax across them) against a binary32 torch reference."""
+    cfg = workloads.make_config(2)
+    w = workloads.generate(cfg, device="cuda")
+    kp = torch.zeros((w.num_pages * 16, cfg.hkv, 128), dtype=torch.bfloat16, device="cuda")
+    vp = torch.zeros_like(kp)
+    kp[w.slot.long()] = w.k
+    vp[w.slot.long()] = w.v
+    kp = kp.view(w.num_pages, 16, cfg.hkv, 128).transpose(1, 2).contiguous()
+    vp = vp.view(w.num_pages, 16, cfg.hkv, 128).transpose(1, 2).contiguous()
+    out = torch.empty((cfg.batch, cfg.hq, 128), dtype=torch.bfloat16, device="cuda")
+    ws = torch.empty(dq.dq_decode_workspace_bytes(cfg.batch, cfg.hq, w.page_table.shape[1]), dtype=torch.uint8, device="cuda")
+    dq.dq_bf16_decode_attention(w.q, kp, vp, w.page_table, w.seq_lens, cfg.hkv, gc.SM_SCALE, out, ws)
+    torch.cuda.synchronize()
+    start = 0
+    for b, n in enumerate(cfg.seq_lens):
+        k = w.k[start:start + n].float().repeat_interleave(cfg.hq // cfg.hkv, dim=1)
+        v = w.v[start:start + n].float().repeat_interleave(cfg.hq // cfg.hkv, dim=1)
+        a = torch.softmax(gc.SM_SCALE * torch.einsum("hd,thd->ht", w.q[b].float(), k), -1)
+        ref = torch.einsum("ht,thd->hd", a, v)
+        assert (out[b].float() - ref).abs().max() <= 6e-3 * ref.abs().max()
+        start += n

@@ -231,7 +231,8 @@ def test_bf16_baseline_against_torch():
         v = w.v[start:start + n].float().repeat_interleave(cfg.hq // cfg.hkv, dim=1)
         a = torch.softmax(gc.SM_SCALE * torch.einsum("hd,thd->ht", w.q[b].float(), k), -1)
         ref = torch.einsum("ht,thd->hd", a, v)
-        assert (out[b].float() - ref).abs().max() <= 0.02 * ref.abs().max()
+        # bf16 softmax weights and a bf16 result: a few half-ulps of 2^-9 against the fp32 reference
+        assert (out[b].float() - ref).abs().max() <= 6e-3 * ref.abs().max()
         start += n
 
 
