@@ -245,8 +245,11 @@ __device__ __forceinline__ void fused_pass(uint32_t xk, uint32_t ptrk, uint32_t 
     const uint32_t av_addr = vtile + ((lane & 7) + (lane >> 4) * 8) * kTileStride + ((lane >> 3) & 1) * 16;
     // output slot: thread holds channels (lane/4, lane/4 + 8) of heads (2 qd, 2 qd + 1)
     const uint32_t o_addr = obuf + ((2 * (lane & 3)) * kORow + (lane >> 2)) * 4;
+#ifndef DQ_EXP_CG
+#define DQ_EXP_CG 8   // channel groups per pass (only ever changed to count the pass's instructions)
+#endif
 #pragma unroll 1
-    for (int cg = 0; cg < 8; ++cg) {
+    for (int cg = 0; cg < DQ_EXP_CG; ++cg) {
         uint32_t pk[8], pv[8];
         if (DO_K) decode16<LBITS>(xk, ptrk, lutk, one, pk);
         if (DO_V) decode16<LBITS>(xv, ptrv, lutv, one, pv);
@@ -418,37 +421,41 @@ dq_attention_kernel(const __grid_constant__ DqDevTable TK, const __grid_constant
             cp_async4(smem_addr(my_pages + (n % 3) * 2 + lane),
                       p.page_table + (size_t)it.b * p.max_pages + (tok0 >> 4) + lane);
     };
-    // cp.async of the K records, q'.mean values and q' operand of item n_k, V records of item n_v
+    // cp.async of the K records, q'.mean values and q' operand of item n_k, V records of item n_v.
+    // A warp's 32 tokens are two pages whose (page, head) blocks land back to back in its buffer, so
+    // piece i of the 2 * rec 16-byte pieces goes to buffer offset 16 i and comes from page i / rec.
     auto issue_loads = [&](int nk, const Item& ik, int nv, const Item& iv) {
         if (ik.valid) {
-            const uint32_t kst = sbase + L.off_kst + ((nk & 1) * nw + warp) * L.stage_k;
             const int tok0 = (ik.blk * nw + warp) * kChunk;
             if (tok0 < ik.len) {
-                const int npg = (tok0 + 16 < ik.len) ? 2 : 1;
-                for (int pg = 0; pg < npg; ++pg) {
-                    const uint8_t* ks = p.k_cont + ((size_t)my_pages[(nk % 3) * 2 + pg] * p.Hkv + ik.h) * (size_t)(16 * TK.rec);
-                    for (int i = lane; i < TK.rec; i += 32) cp_async16(kst + pg * 16 * TK.rec + i * 16, ks + i * 16);
-                }
+                const uint32_t kst = sbase + L.off_kst + ((nk & 1) * nw + warp) * L.stage_k;
+                const int rec = TK.rec, np = (tok0 + 16 < ik.len) ? 2 * rec : rec;
+                const uint32_t blk = 16u * (uint32_t)rec;
+                const uint8_t* s0 = p.k_cont + ((size_t)my_pages[(nk % 3) * 2] * p.Hkv + ik.h) * blk;
+                const uint8_t* s1 = p.k_cont + ((size_t)my_pages[(nk % 3) * 2 + 1] * p.Hkv + ik.h) * blk - blk;
+                for (int i = lane; i < np; i += 32) cp_async16(kst + i * 16, (i < rec ? s0 : s1) + i * 16);
                 if (p.has_mean && lane < G)
                     cp_async4(kst + L.stage_k - kKTail + lane * 4,
                               p.qmu + ((size_t)ik.b * p.Hq + (size_t)ik.h * G + lane) * p.windows + tok0 / DQ_WINDOW_TOKENS);
             }
-            const uint16_t* qsrc = p.q16 + ((size_t)ik.b * p.Hkv + ik.h) * 16 * kN;
-            for (int i = tid; i < 16 * 16; i += nthreads)  // 16 rows x 16 chunks of 16 bytes
-                cp_async16(sbase + L.off_q16 + (nk & 1) * kQ16Bytes + (i >> 4) * kQ16Stride + (i & 15) * 16, qsrc + i * 8);
-            if (tid < G)
-                cp_async4(sbase + L.off_qsum + ((nk & 1) * DQ_MAX_GROUP + tid) * 4,
-                          p.qsum + (size_t)ik.b * p.Hq + (size_t)ik.h * G + tid);
+            if (tid < 16 * 16) {   // q' operand: 16 rows x 16 pieces of 16 bytes
+                const uint16_t* qsrc = p.q16 + ((size_t)ik.b * p.Hkv + ik.h) * 16 * kN;
+                for (int i = tid; i < 16 * 16; i += nthreads)
+                    cp_async16(sbase + L.off_q16 + (nk & 1) * kQ16Bytes + (i >> 4) * kQ16Stride + (i & 15) * 16, qsrc + i * 8);
+                if (tid < G)
+                    cp_async4(sbase + L.off_qsum + ((nk & 1) * DQ_MAX_GROUP + tid) * 4,
+                              p.qsum + (size_t)ik.b * p.Hq + (size_t)ik.h * G + tid);
+            }
         }
         if (iv.valid) {
-            const uint32_t vst = sbase + L.off_vst + ((nv & 1) * nw + warp) * L.stage_v;
             const int tok0 = (iv.blk * nw + warp) * kChunk;
             if (tok0 < iv.len) {
-                const int npg = (tok0 + 16 < iv.len) ? 2 : 1;
-                for (int pg = 0; pg < npg; ++pg) {
-                    const uint8_t* vs = p.v_cont + ((size_t)my_pages[(nv % 3) * 2 + pg] * p.Hkv + iv.h) * (size_t)(16 * TV.rec);
-                    for (int i = lane; i < TV.rec; i += 32) cp_async16(vst + pg * 16 * TV.rec + i * 16, vs + i * 16);
-                }
+                const uint32_t vst = sbase + L.off_vst + ((nv & 1) * nw + warp) * L.stage_v;
+                const int rec = TV.rec, np = (tok0 + 16 < iv.len) ? 2 * rec : rec;
+                const uint32_t blk = 16u * (uint32_t)rec;
+                const uint8_t* s0 = p.v_cont + ((size_t)my_pages[(nv % 3) * 2] * p.Hkv + iv.h) * blk;
+                const uint8_t* s1 = p.v_cont + ((size_t)my_pages[(nv % 3) * 2 + 1] * p.Hkv + iv.h) * blk - blk;
+                for (int i = lane; i < np; i += 32) cp_async16(vst + i * 16, (i < rec ? s0 : s1) + i * 16);
             }
         }
     };
@@ -547,35 +554,51 @@ dq_attention_kernel(const __grid_constant__ DqDevTable TK, const __grid_constant
                 const float oK = __half2float(__ushort_as_half((unsigned short)(hk >> 16)));
                 const float sV = __half2float(__ushort_as_half((unsigned short)(hv & 0xffffu)));
                 const float oV = __half2float(__ushort_as_half((unsigned short)(hv >> 16)));
-                asm volatile("st.shared.v4.f32 [%0], {%1,%2,%3,%4};\n" ::"r"(ktile + lane * kTileStride + 32), "f"(sK),
-                             "f"(oK), "f"(sV), "f"(oV) : "memory");
+                // the key scale carries the logit scale (sm_scale * log2 e): logits come out in base-2 units
+                asm volatile("st.shared.v4.f32 [%0], {%1,%2,%3,%4};\n" ::"r"(ktile + lane * kTileStride + 32),
+                             "f"(sK * p.scale_log2), "f"(oK), "f"(sV), "f"(oV) : "memory");
             }
             // tokens this thread's row may see: a query token that is not the last one stops earlier; tokens
             // of a BF16 residual window come after the compressed ones and absorb the offset first
             int row_len = cur.len;
             if (p.q_total > 1) row_len -= max(0, row_offset(p, g_row) - (p.resid_lens ? max(p.resid_lens[cur.b], 0) : 0));
-            float qmu = 0.f, qs = 0.f;   // q' . window mean and sum of q', for the head row this thread owns
+            float qmu = 0.f, qs = 0.f;   // q' . window mean and sum of q' (both times the logit scale), for this thread's head row
             if (g_row < G) {
-                qs = qsum[(n & 1) * DQ_MAX_GROUP + g_row];
-                if (p.has_mean && tok0 < cur.len) qmu = __uint_as_float(lds32(kst + L.stage_k - kKTail + g_row * 4));
+                qs = qsum[(n & 1) * DQ_MAX_GROUP + g_row] * p.scale_log2;
+                if (p.has_mean && tok0 < cur.len) qmu = __uint_as_float(lds32(kst + L.stage_k - kKTail + g_row * 4)) * p.scale_log2;
             }
             __syncwarp();
             float mx = -INFINITY;
+            const uint32_t meta = ktile + 2 * qd * kTileStride + 32;
+            if (tok0 + kChunk <= row_len) {   // every token of the chunk is visible: no masks
 #pragma unroll
-            for (int i = 0; i < 4; ++i)
+                for (int i = 0; i < 4; ++i)
 #pragma unroll
-                for (int u = 0; u < 2; ++u) {
-                    const int tk = 8 * i + 2 * qd + u;
-                    float4 m4;
-                    asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4];\n"
-                                 : "=f"(m4.x), "=f"(m4.y), "=f"(m4.z), "=f"(m4.w) : "r"(ktile + tk * kTileStride + 32));
-                    const float S = sacc[i][u] + sacc[i][2 + u];
-                    const bool ok = tok0 + tk < row_len;
-                    lg[i][u] = ok ? p.scale_log2 * fmaf(m4.x, S, fmaf(m4.y, qs, qmu)) : -INFINITY;
-                    sv_t[i][u] = ok ? m4.z : 0.f;
-                    ov_t[i][u] = ok ? m4.w : 0.f;
-                    mx = fmaxf(mx, lg[i][u]);
-                }
+                    for (int u = 0; u < 2; ++u) {
+                        float4 m4;
+                        asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4];\n"
+                                     : "=f"(m4.x), "=f"(m4.y), "=f"(m4.z), "=f"(m4.w) : "r"(meta + (8 * i + u) * kTileStride));
+                        lg[i][u] = fmaf(m4.x, sacc[i][u] + sacc[i][2 + u], fmaf(m4.y, qs, qmu));
+                        sv_t[i][u] = m4.z;
+                        ov_t[i][u] = m4.w;
+                        mx = fmaxf(mx, lg[i][u]);
+                    }
+            } else {
+                const int lim = row_len - tok0 - 2 * qd;   // token 8 i + 2 qd + u is visible iff 8 i + u < lim
+#pragma unroll
+                for (int i = 0; i < 4; ++i)
+#pragma unroll
+                    for (int u = 0; u < 2; ++u) {
+                        float4 m4;
+                        asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4];\n"
+                                     : "=f"(m4.x), "=f"(m4.y), "=f"(m4.z), "=f"(m4.w) : "r"(meta + (8 * i + u) * kTileStride));
+                        const bool ok = 8 * i + u < lim;
+                        lg[i][u] = ok ? fmaf(m4.x, sacc[i][u] + sacc[i][2 + u], fmaf(m4.y, qs, qmu)) : -INFINITY;
+                        sv_t[i][u] = ok ? m4.z : 0.f;
+                        ov_t[i][u] = ok ? m4.w : 0.f;
+                        mx = fmaxf(mx, lg[i][u]);
+                    }
+            }
             mx = fmaxf(mx, __shfl_xor_sync(kFullMask, mx, 1));
             mx = fmaxf(mx, __shfl_xor_sync(kFullMask, mx, 2));
             if (qd == 0) red_m[warp * DQ_MAX_GROUP + g_row] = mx;
@@ -584,41 +607,57 @@ dq_attention_kernel(const __grid_constant__ DqDevTable TK, const __grid_constant
 
         // ------------------------------------------ finish `prev`: sum its warps' slots, write the partial
         if (have_prev) {
-            const int lcol = kN + 2 * ((n + 1) & 1);   // l, off columns written when `prev` was `cur`
-            for (int e = tid; e < G * 130; e += nthreads) {
-                const int g = e / 130, col = e - g * 130;
-                const int src = col < kN ? col : lcol + (col - kN);
-                float s = 0.f;
-                for (int w = 0; w < nw; ++w) s += obuf_all[(w * G + g) * kORow + src];
-                float* dst = p.partial + ((size_t)s_prev_row[(n + 1) & 1] + g) * kPartial;
-                if (col < kN) dst[col] = s;
-                else dst[col + 1] = s;                       // l at 129, off at 130
-                if (col == 0) dst[kN] = red_M[((n + 1) & 1) * DQ_MAX_GROUP + g];
+            // G x 32 threads add the channel sums four at a time, 2 G more the (l, off) columns written when
+            // `prev` was `cur` (by item parity); the item maximum goes along
+            const int par = (n + 1) & 1;
+            const int wstride = G * kORow;   // floats between the slots of neighbouring warps
+            for (int e = tid; e < G * 34; e += nthreads) {
+                if (e < G * 32) {
+                    const int g = e >> 5, c4 = e & 31;
+                    const float* src = obuf_all + g * kORow + 4 * c4;
+                    float4 acc = *reinterpret_cast<const float4*>(src);
+                    for (int w = 1; w < nw; ++w) {
+                        const float4 v = *reinterpret_cast<const float4*>(src + w * wstride);
+                        acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
+                    }
+                    *reinterpret_cast<float4*>(p.partial + ((size_t)s_prev_row[par] + g) * kPartial + 4 * c4) = acc;
+                } else {
+                    const int e2 = e - G * 32, g = e2 >> 1, which = e2 & 1;
+                    const float* src = obuf_all + g * kORow + kN + 2 * par + which;
+                    float acc = 0.f;
+                    for (int w = 0; w < nw; ++w) acc += src[w * wstride];
+                    float* dst = p.partial + ((size_t)s_prev_row[par] + g) * kPartial;
+                    dst[kN + 1 + which] = acc;                   // l at 129, off at 130
+                    if (which == 0) dst[kN] = red_M[par * DQ_MAX_GROUP + g];
+                }
             }
         }
 
         // ------------------------------------------ softmax weights of `cur`, scaled by the item maximum
         have_prev = cur.valid;
         if (cur.valid) {
-            float m_item = -INFINITY;
-            for (int w = 0; w < nw; ++w) m_item = fmaxf(m_item, red_m[w * DQ_MAX_GROUP + g_row]);
+            float m_item = -INFINITY;   // the four threads of a head row share the warps' maxima
+            for (int w = qd; w < nw; w += 4) m_item = fmaxf(m_item, red_m[w * DQ_MAX_GROUP + g_row]);
+            m_item = fmaxf(m_item, __shfl_xor_sync(kFullMask, m_item, 1));
+            m_item = fmaxf(m_item, __shfl_xor_sync(kFullMask, m_item, 2));
             if (warp == 0 && qd == 0) red_M[(n & 1) * DQ_MAX_GROUP + g_row] = m_item;
             const float m_use = (m_item == -INFINITY) ? 0.f : m_item;
             float lsum = 0.f, osum = 0.f;
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
-                float hi[2], lo[2];
+                float ps[2];
 #pragma unroll
                 for (int u = 0; u < 2; ++u) {
-                    const float pr = exp2f(lg[i][u] - m_use);
+                    const float pr = ex2_approx(lg[i][u] - m_use);   // <= 1; exp2(-inf) = 0
                     lsum += pr;
                     osum = fmaf(pr, ov_t[i][u], osum);
-                    const float ps = pr * sv_t[i][u];
-                    hi[u] = __half2float(__float2half_rn(ps));
-                    lo[u] = ps - hi[u];
+                    ps[u] = pr * sv_t[i][u];
                 }
-                pb_hi[i >> 1][i & 1] = pack_half2(hi[0], hi[1]);
-                pb_lo[i >> 1][i & 1] = pack_half2(lo[0], lo[1]);
+                // fp16 hi + lo pair of each weight: hi = rn(ps), lo = rn(ps - hi)
+                const __half2 h2 = __floats2half2_rn(ps[0], ps[1]);
+                const float2 hf = __half22float2(h2);
+                pb_hi[i >> 1][i & 1] = *reinterpret_cast<const uint32_t*>(&h2);
+                pb_lo[i >> 1][i & 1] = pack_half2(ps[0] - hf.x, ps[1] - hf.y);
             }
             lsum += __shfl_xor_sync(kFullMask, lsum, 1);
             lsum += __shfl_xor_sync(kFullMask, lsum, 2);
