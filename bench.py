@@ -36,8 +36,8 @@ SM_COUNT, SCHEDULERS_PER_SM = 148, 4
 # Stored ncu captures of the fused kernels (profiles/*.md): DRAM bytes per launch on config 2 and the
 # measured warp instructions per decoded symbol step.  They are constants of this file, not
 # quantities measured by a bench run; the line says so where it uses them.
-NCU_HEAD = {"dram_bytes": 37.62e6, "token_heads": 524288, "bytes_per_token_head": 72.0, "instr_per_symbol": 16.1,
-            "issue_active": 0.637, "source": "profiles/dq_attention_kernel_config2_ncu.md"}
+NCU_HEAD = {"dram_bytes": 37.62e6, "token_heads": 524288, "bytes_per_token_head": 72.0, "instr_per_symbol": 15.2,
+            "issue_active": 0.622, "source": "profiles/dq_attention_kernel_config2_ncu.md"}
 NCU_WIDE = {"instr_per_symbol": 19.8, "issue_active": None, "source": "profiles/dq_attention_wide_kernel_config2_ncu.md"}
 REGIONS = 21          # the K-step timed region is repeated this many times; ms_per_step is the median
 ORACLE_MAX_TOKENS = 131072   # the oracle legs run whole sequences of the workload up to this many tokens
