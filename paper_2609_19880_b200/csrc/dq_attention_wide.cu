@@ -431,33 +431,49 @@ dq_attention_wide_kernel(const __grid_constant__ DqDevTable TK, const __grid_con
                 const float oK = __half2float(__ushort_as_half((unsigned short)(hk >> 16)));
                 const float sV = __half2float(__ushort_as_half((unsigned short)(hv & 0xffffu)));
                 const float oV = __half2float(__ushort_as_half((unsigned short)(hv >> 16)));
-                asm volatile("st.shared.v4.f32 [%0], {%1,%2,%3,%4};\n" ::"r"(ktile + lane * 16), "f"(sK), "f"(oK), "f"(sV),
-                             "f"(oV) : "memory");
+                // the key scale carries the logit scale (sm_scale * log2 e): logits come out in base-2 units
+                asm volatile("st.shared.v4.f32 [%0], {%1,%2,%3,%4};\n" ::"r"(ktile + lane * 16), "f"(sK * p.scale_log2), "f"(oK),
+                             "f"(sV), "f"(oV) : "memory");
             }
             int row_len = cur.len;   // tokens this thread's row may see (earlier query tokens stop earlier)
             if (p.q_total > 1) row_len -= max(0, row_offset(p, g_row) - (p.resid_lens ? max(p.resid_lens[cur.b], 0) : 0));
-            float qmu = 0.f, qs = 0.f;
+            float qmu = 0.f, qs = 0.f;   // both times the logit scale
             if (g_row < G) {
-                qs = qsum[(s & 1) * DQ_MAX_GROUP + g_row];
-                if (p.has_mean && tok0 < cur.len) qmu = __uint_as_float(lds32(my_qmu + ((s & 1) * DQ_MAX_GROUP + g_row) * 4));
+                qs = qsum[(s & 1) * DQ_MAX_GROUP + g_row] * p.scale_log2;
+                if (p.has_mean && tok0 < cur.len) qmu = __uint_as_float(lds32(my_qmu + ((s & 1) * DQ_MAX_GROUP + g_row) * 4)) * p.scale_log2;
             }
             __syncwarp();
             float mx = -INFINITY;
+            const uint32_t meta = ktile + 2 * qd * 16;
+            if (tok0 + kChunk <= row_len) {   // every token of the chunk is visible: no masks
 #pragma unroll
-            for (int i = 0; i < 4; ++i)
+                for (int i = 0; i < 4; ++i)
 #pragma unroll
-                for (int u = 0; u < 2; ++u) {
-                    const int tk = 8 * i + 2 * qd + u;
-                    float4 m4;
-                    asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4];\n"
-                                 : "=f"(m4.x), "=f"(m4.y), "=f"(m4.z), "=f"(m4.w) : "r"(ktile + tk * 16));
-                    const float S = sacc[i][u] + sacc[i][2 + u];
-                    const bool ok = tok0 + tk < row_len;
-                    lg[i][u] = ok ? p.scale_log2 * fmaf(m4.x, S, fmaf(m4.y, qs, qmu)) : -INFINITY;
-                    sv_t[i][u] = ok ? m4.z : 0.f;
-                    ov_t[i][u] = ok ? m4.w : 0.f;
-                    mx = fmaxf(mx, lg[i][u]);
-                }
+                    for (int u = 0; u < 2; ++u) {
+                        float4 m4;
+                        asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4];\n"
+                                     : "=f"(m4.x), "=f"(m4.y), "=f"(m4.z), "=f"(m4.w) : "r"(meta + (8 * i + u) * 16));
+                        lg[i][u] = fmaf(m4.x, sacc[i][u] + sacc[i][2 + u], fmaf(m4.y, qs, qmu));
+                        sv_t[i][u] = m4.z;
+                        ov_t[i][u] = m4.w;
+                        mx = fmaxf(mx, lg[i][u]);
+                    }
+            } else {
+                const int lim = row_len - tok0 - 2 * qd;   // token 8 i + 2 qd + u is visible iff 8 i + u < lim
+#pragma unroll
+                for (int i = 0; i < 4; ++i)
+#pragma unroll
+                    for (int u = 0; u < 2; ++u) {
+                        float4 m4;
+                        asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4];\n"
+                                     : "=f"(m4.x), "=f"(m4.y), "=f"(m4.z), "=f"(m4.w) : "r"(meta + (8 * i + u) * 16));
+                        const bool ok = 8 * i + u < lim;
+                        lg[i][u] = ok ? fmaf(m4.x, sacc[i][u] + sacc[i][2 + u], fmaf(m4.y, qs, qmu)) : -INFINITY;
+                        sv_t[i][u] = ok ? m4.z : 0.f;
+                        ov_t[i][u] = ok ? m4.w : 0.f;
+                        mx = fmaxf(mx, lg[i][u]);
+                    }
+            }
             mx = fmaxf(mx, __shfl_xor_sync(kFullMask, mx, 1));
             mx = fmaxf(mx, __shfl_xor_sync(kFullMask, mx, 2));
             if (qd == 0) red_m[warp * DQ_MAX_GROUP + g_row] = mx;
@@ -466,17 +482,29 @@ dq_attention_wide_kernel(const __grid_constant__ DqDevTable TK, const __grid_con
 
         // ------------------------------------------ finish the V step: sum the warps' slots, write the partial
         if (have_prev) {
-            const int lcol = kN + 2 * ((s + 1) & 1);
-            for (int e = tid; e < G * 130; e += nthreads) {
-                const int g = e / 130, col = e - g * 130;
-                const int src = col < kN ? col : lcol + (col - kN);
-                float sum = 0.f;
-                for (int w = 0; w < nwv; ++w)
-                    sum += reinterpret_cast<const float*>(smem + kOffWarp + w * wstride + kWObuf)[g * kORow + src];
-                float* dst = p.partial + ((size_t)s_prev_row[(s + 1) & 1] + g) * kPartial;
-                if (col < kN) dst[col] = sum;
-                else dst[col + 1] = sum;
-                if (col == 0) dst[kN] = red_M[((s + 1) & 1) * DQ_MAX_GROUP + g];
+            // G x 32 threads add the channel sums four at a time, 2 G more the (l, off) columns (by step parity)
+            const int par = (s + 1) & 1;
+            const float* slots = reinterpret_cast<const float*>(smem + kOffWarp + kWObuf);
+            const int wfl = wstride / 4;   // floats between the slots of neighbouring warps
+            for (int e = tid; e < G * 34; e += nthreads) {
+                if (e < G * 32) {
+                    const int g = e >> 5, c4 = e & 31;
+                    const float* src = slots + g * kORow + 4 * c4;
+                    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+                    for (int w = 0; w < nwv; ++w) {
+                        const float4 v = *reinterpret_cast<const float4*>(src + w * wfl);
+                        acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
+                    }
+                    *reinterpret_cast<float4*>(p.partial + ((size_t)s_prev_row[par] + g) * kPartial + 4 * c4) = acc;
+                } else {
+                    const int e2 = e - G * 32, g = e2 >> 1, which = e2 & 1;
+                    const float* src = slots + g * kORow + kN + 2 * par + which;
+                    float acc = 0.f;
+                    for (int w = 0; w < nwv; ++w) acc += src[w * wfl];
+                    float* dst = p.partial + ((size_t)s_prev_row[par] + g) * kPartial;
+                    dst[kN + 1 + which] = acc;
+                    if (which == 0) dst[kN] = red_M[par * DQ_MAX_GROUP + g];
+                }
             }
         }
 
@@ -486,25 +514,27 @@ dq_attention_wide_kernel(const __grid_constant__ DqDevTable TK, const __grid_con
         wv = wk;
         nwv = min(nw, (cur.len - cur.blk * nw * kChunk + kChunk - 1) / kChunk);
         if (cur.valid) {
-            float m_item = -INFINITY;
-            for (int w = 0; w < nw; ++w) m_item = fmaxf(m_item, red_m[w * DQ_MAX_GROUP + g_row]);
+            float m_item = -INFINITY;   // the four threads of a head row share the warps' maxima
+            for (int w = qd; w < nw; w += 4) m_item = fmaxf(m_item, red_m[w * DQ_MAX_GROUP + g_row]);
+            m_item = fmaxf(m_item, __shfl_xor_sync(kFullMask, m_item, 1));
+            m_item = fmaxf(m_item, __shfl_xor_sync(kFullMask, m_item, 2));
             if (warp == 0 && qd == 0) red_M[(s & 1) * DQ_MAX_GROUP + g_row] = m_item;
             const float m_use = (m_item == -INFINITY) ? 0.f : m_item;
             float lsum = 0.f, osum = 0.f;
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
-                float hi[2], lo[2];
+                float ps[2];
 #pragma unroll
                 for (int u = 0; u < 2; ++u) {
-                    const float pr = exp2f(lg[i][u] - m_use);
+                    const float pr = ex2_approx(lg[i][u] - m_use);
                     lsum += pr;
                     osum = fmaf(pr, ov_t[i][u], osum);
-                    const float ps = pr * sv_t[i][u];
-                    hi[u] = __half2float(__float2half_rn(ps));
-                    lo[u] = ps - hi[u];
+                    ps[u] = pr * sv_t[i][u];
                 }
-                pb_hi[i >> 1][i & 1] = pack_half2(hi[0], hi[1]);
-                pb_lo[i >> 1][i & 1] = pack_half2(lo[0], lo[1]);
+                const __half2 h2 = __floats2half2_rn(ps[0], ps[1]);   // fp16 hi + lo pair of each weight
+                const float2 hf = __half22float2(h2);
+                pb_hi[i >> 1][i & 1] = *reinterpret_cast<const uint32_t*>(&h2);
+                pb_lo[i >> 1][i & 1] = pack_half2(ps[0] - hf.x, ps[1] - hf.y);
             }
             lsum += __shfl_xor_sync(kFullMask, lsum, 1);
             lsum += __shfl_xor_sync(kFullMask, lsum, 2);

@@ -262,3 +262,23 @@ def test_encoder_extreme_finite_values(wide):
     assert np.array_equal(_np(cache.mean_q), mq) and np.array_equal(_np(cache.mean_scale), ms)
     assert list(_np(cache.status)[:3]) == [sk[i] + sv[i] for i in range(3)]
     assert sk[0] + sv[0] > 0 and sk[1] + sv[1] > 0      # both the fallback and the constant path were taken
+
+
+def test_decode_loop_microbenchmark_runs():
+    """The bare decode-loop measurement aid: launches for both chain counts, fills every thread's checksum slot,
+    is deterministic, and refuses shapes it cannot run."""
+    tk = dq.dq_build_tables(5, 42 * 8 / 128, has_mean=True)
+    g = torch.Generator(device="cpu").manual_seed(3)
+    data = torch.randint(0, 256, (1 << 16,), dtype=torch.uint8, generator=g).cuda()
+    for threads, chains in ((512, 2), (1024, 1), (64, 2)):
+        a = torch.zeros(4 * threads, dtype=torch.int32, device="cuda")
+        b = torch.zeros_like(a)
+        dq.dq_microbench_decode_loop(tk, data, 4, threads, chains, 3, a)
+        dq.dq_microbench_decode_loop(tk, data, 4, threads, chains, 3, b)
+        torch.cuda.synchronize()
+        assert torch.equal(a, b) and int((a != 0).sum()) > a.numel() // 2
+    out = torch.zeros(1024, dtype=torch.int32, device="cuda")
+    for bad in (dict(threads=48), dict(threads=2048), dict(chains=3), dict(reps=0), dict(ctas=0)):
+        kw = dict(ctas=1, threads=256, chains=1, reps=1); kw.update(bad)
+        with pytest.raises(dq.DqError):
+            dq.dq_microbench_decode_loop(tk, data, kw["ctas"], kw["threads"], kw["chains"], kw["reps"], out)
