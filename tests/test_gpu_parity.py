@@ -282,3 +282,36 @@ def test_decode_loop_microbenchmark_runs():
         kw = dict(ctas=1, threads=256, chains=1, reps=1); kw.update(bad)
         with pytest.raises(dq.DqError):
             dq.dq_microbench_decode_loop(tk, data, kw["ctas"], kw["threads"], kw["chains"], kw["reps"], out)
+
+
+@pytest.mark.parametrize("lens", [[0, 0, 1], [1, 0, 17, 16, 33], [5] * 300, [2047, 1, 0, 129, 640]])
+def test_bf16_baseline_edge_shapes(lens):
+    """Empty batches, empty and one-token sequences, hundreds of tiny sequences, ragged lengths: the split sizing on
+    the device, ranges that end inside a chunk, zero rows for empty sequences."""
+    cfg = _small(4, batch=len(lens), seq_lens=lens)
+    w = workloads.generate(cfg, device="cuda")
+    kp = torch.zeros((max(w.num_pages, 1) * 16, cfg.hkv, 128), dtype=torch.bfloat16, device="cuda")
+    vp = torch.zeros_like(kp)
+    if cfg.total_tokens:
+        kp[w.slot.long()] = w.k
+        vp[w.slot.long()] = w.v
+    kp = kp.view(-1, 16, cfg.hkv, 128).transpose(1, 2).contiguous()
+    vp = vp.view(-1, 16, cfg.hkv, 128).transpose(1, 2).contiguous()
+    out = torch.full((cfg.batch, cfg.hq, 128), float("nan"), dtype=torch.bfloat16, device="cuda")
+    ws = torch.empty(dq.dq_decode_workspace_bytes(cfg.batch, cfg.hq, w.page_table.shape[1]), dtype=torch.uint8,
+                     device="cuda")
+    for _ in range(2):   # twice: nothing of the first call may linger in the workspace
+        dq.dq_bf16_decode_attention(w.q, kp, vp, w.page_table, w.seq_lens, cfg.hkv, gc.SM_SCALE, out, ws)
+    torch.cuda.synchronize()
+    assert torch.isfinite(out.float()).all()
+    start = 0
+    for b, n in enumerate(cfg.seq_lens):
+        if n == 0:
+            assert not out[b].any()
+            continue
+        k = w.k[start:start + n].float().repeat_interleave(cfg.hq // cfg.hkv, dim=1)
+        v = w.v[start:start + n].float().repeat_interleave(cfg.hq // cfg.hkv, dim=1)
+        a = torch.softmax(gc.SM_SCALE * torch.einsum("hd,thd->ht", w.q[b].float(), k), -1)
+        ref = torch.einsum("ht,thd->hd", a, v)
+        assert (out[b].float() - ref).abs().max() <= 6e-3 * ref.abs().max()
+        start += n
