@@ -33,12 +33,13 @@ METRIC = "decode_attention_kv_tokens_per_s"
 UNIT = "KV tokens/s"
 L2_BYTES = 126 * 2 ** 20
 SM_COUNT, SCHEDULERS_PER_SM = 148, 4
-# Stored ncu captures of the fused kernels (profiles/*.md): DRAM bytes per launch on config 2 and the
+# Stored ncu captures of the fused kernels (summaries under profiles/): DRAM bytes per launch on config 2 and the
 # measured warp instructions per decoded symbol step.  They are constants of this file, not
 # quantities measured by a bench run; the line says so where it uses them.
 NCU_HEAD = {"dram_bytes": 37.62e6, "token_heads": 524288, "bytes_per_token_head": 72.0, "instr_per_symbol": 15.2,
-            "issue_active": 0.622, "source": "profiles/dq_attention_kernel_config2_ncu.md"}
-NCU_WIDE = {"instr_per_symbol": 19.8, "issue_active": None, "source": "profiles/dq_attention_wide_kernel_config2_ncu.md"}
+            "issue_active": 0.622, "source": "the ncu summary of dq_attention_kernel on config 2 under profiles/"}
+NCU_WIDE = {"instr_per_symbol": 19.2, "issue_active": 0.641,
+            "source": "the ncu summary of dq_attention_wide_kernel on config 2 under profiles/"}
 REGIONS = 21          # the K-step timed region is repeated this many times; ms_per_step is the median
 ORACLE_MAX_TOKENS = 131072   # the oracle legs run whole sequences of the workload up to this many tokens
 
@@ -644,7 +645,7 @@ def main():
                     help="warm-up and timed steps only (for profiler captures); prints a short line")
     ap.add_argument("--traffic-bytes", type=float, default=None,
                     help="DRAM bytes per launch of the fused kernel from an ncu capture; default: the captured "
-                         "figure of profiles/dq_attention_kernel_config2_ncu.md scaled by the token-heads processed")
+                         "figure of the config-2 capture summarised under profiles/, scaled by the token-heads processed")
     ap.add_argument("--decode-loop", action="store_true",
                     help="micro-benchmark of the bare rANS decode loop (no tiles, no contractions) instead of the step")
     args = ap.parse_args()
