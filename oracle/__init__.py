@@ -45,6 +45,9 @@ class Table(C.Structure):
         ("r", C.c_float * MAX_LEVELS), ("R", C.c_uint32 * MAX_LEVELS),
         ("lut_m", C.c_uint8 * 256), ("lut_f", C.c_uint8 * 256), ("lut_d", C.c_uint8 * 256),
         ("sigma", C.c_int), ("early_exit", C.c_int),
+        ("pair", C.c_int), ("ustar", C.c_int),
+        ("pf", C.c_int32 * 256), ("pc", C.c_int32 * 257), ("pr", C.c_float * 256), ("pR", C.c_uint32 * 256),
+        ("plut_u", C.c_uint8 * 256), ("plut_f", C.c_uint8 * 256), ("plut_d", C.c_uint8 * 256),
     ]
 
     @property
@@ -58,6 +61,16 @@ class Table(C.Structure):
 
     def freqs(self):
         return [int(self.f[m]) for m in range(self.M)]
+
+    def pair_freqs(self):
+        """Frequencies of the pair alphabet, index u = a * M + b (paired-symbol variant)."""
+        return [int(self.pf[u]) for u in range(self.M * self.M)]
+
+    def code_length(self, sym) -> int:
+        """Fixed-point code length (1/65536 bit) of a symbol sequence under this table's alphabet."""
+        if self.pair:
+            return sum(int(self.pR[int(sym[j]) * self.M + int(sym[j + 1])]) for j in range(0, len(sym), 2))
+        return sum(int(self.R[int(m)]) for m in sym)
 
     def cum(self):
         return [int(self.c[m]) for m in range(self.M + 1)]
@@ -90,7 +103,7 @@ def lib():
                                           C.POINTER(Table)]
             L.dqo_build_table_ex.restype = C.c_int
             L.dqo_build_table_ex.argtypes = [C.c_int, C.c_int, C.c_int, C.c_double, C.c_int, C.c_int,
-                                             C.c_int, C.c_int, C.POINTER(Table)]
+                                             C.c_int, C.c_int, C.c_int, C.POINTER(Table)]
             _lib = L
     return _lib
 
@@ -125,14 +138,14 @@ def rec_bytes(bits_per_elem: float, n: int) -> int:
 
 def build_table(levels: int, n: int, rec: int, alpha: float = 1.4, has_mean: bool = False,
                 rotate: bool = True, allow_infeasible: bool = False, sigma: int = 32,
-                early_exit: bool = False) -> Table:
-    """sigma / early_exit select the opt-in codec variants (defaults: the paper's codec)."""
+                early_exit: bool = False, pair: bool = False) -> Table:
+    """sigma / early_exit / pair select the opt-in codec variants (defaults: the paper's codec)."""
     T = Table()
-    if sigma == 32 and not early_exit:
+    if sigma == 32 and not early_exit and not pair:
         rc = lib().dqo_build_table(levels, n, rec, float(alpha), int(has_mean), int(rotate), C.byref(T))
     else:
         rc = lib().dqo_build_table_ex(levels, n, rec, float(alpha), int(has_mean), int(rotate), int(sigma),
-                                      int(early_exit), C.byref(T))
+                                      int(early_exit), int(pair), C.byref(T))
     if rc == -1 or (rc != 0 and not allow_infeasible):
         raise ValueError(f"oracle table build failed rc={rc} (M={levels}, n={n}, rec={rec})")
     return T

@@ -40,7 +40,13 @@
  *     streams have budget to spare, so most take the short path);
  *   - sigma = 24 (table field sigma): the state lives in [2^15, 2^23) and its final value
  *     takes 3 bytes of the container instead of 4 (Eq. budget: B = 8C - sigma), one byte
- *     per stream back for symbols; streams of at most 640 values (five heads) only.
+ *     per stream back for symbols; streams of at most 640 values (five heads) only;
+ *   - paired symbols (table field pair): one rANS symbol is the pair of levels of two
+ *     consecutive values (2i, 2i + 1), u = m_2i M + m_2i+1, over an alphabet of M^2 <= 256
+ *     pairs whose model is the product of the sharpened level model with itself, made
+ *     integer by the same rule as the level table (Sec. 3.1: the coder is the same Eq. rans
+ *     on a larger alphabet; a decoder then takes n / 2 steps for n values).  Drift assigns
+ *     a pair at a time: argmin over the M^2 pairs of D_a + D_b + lambda r_ab.
  *
  * Pins (tests/test_oracle_*.py): closed-form storage accounting, the feasibility
  * boundary and NMSE curve of Table 2, rANS round trip, Shannon bound, orthonormal
@@ -82,6 +88,13 @@ typedef struct {
     uint8_t lut_m[DQO_TOT], lut_f[DQO_TOT], lut_d[DQO_TOT]; /* T[z] = (m, f_m, z - c_m) */
     int sigma;                     /* bits of final state in the record: 32 (default) or 24  */
     int early_exit;                /* 1: Drift first tries the multiplier the bisection ends at when all tests pass */
+    /* paired-symbol variant: alphabet of the pairs u = a M + b (a: value 2i, b: value 2i + 1) */
+    int pair, ustar;               /* 1: rANS symbols are pairs; most probable pair                    */
+    int32_t pf[DQO_TOT];           /* integer pair frequencies, sum 256                               */
+    int32_t pc[DQO_TOT + 1];       /* cumulative                                                      */
+    float pr[DQO_TOT];             /* ideal cost of a pair, -log2(pf/256) bits                        */
+    uint32_t pR[DQO_TOT];          /* ceil(pr * 65536)                                                */
+    uint8_t plut_u[DQO_TOT], plut_f[DQO_TOT], plut_d[DQO_TOT]; /* T[z] = (u, pf_u, z - pc_u)          */
 } dqo_table;
 
 /* lower bound L of the normalised state interval [L, 2^8 L): 2^23 for sigma = 32, 2^15 for 24 */
@@ -154,31 +167,66 @@ float dqo_f16_to_f32(uint16_t h)
 
 /* ------------------------------------------------------------------- tables */
 
+/* Integer frequencies of a K-symbol alphabet with targets t[k] = 256 * probability: floor, at
+ * least 1, then adjusted to sum 256. */
+static void dqo_integer_freqs(const double *t, int K, int32_t *f)
+{
+    int tot = 0;
+    for (int k = 0; k < K; ++k) {
+        int fl = (int)floor(t[k]);
+        f[k] = fl < 1 ? 1 : fl;
+        tot += f[k];
+    }
+    while (tot < DQO_TOT) { /* largest remainder; tie -> lowest index */
+        int best = 0;
+        for (int k = 1; k < K; ++k)
+            if (t[k] - f[k] > t[best] - f[best]) best = k;
+        f[best] += 1; tot += 1;
+    }
+    while (tot > DQO_TOT) { /* largest excess among f > 1; tie -> highest index */
+        int best = -1;
+        for (int k = 0; k < K; ++k)
+            if (f[k] > 1 && (best < 0 || f[k] - t[k] >= f[best] - t[best])) best = k;
+        f[best] -= 1; tot -= 1;
+    }
+}
+
+/* Pair alphabet of the paired-symbol variant: probability of the pair (a, b) = q_a q_b. */
+static void dqo_fill_pair_freqs(dqo_table *T)
+{
+    int M = T->M, K = M * M;
+    double t[DQO_TOT];
+    for (int a = 0; a < M; ++a)
+        for (int b = 0; b < M; ++b) t[a * M + b] = DQO_TOT * (T->q[a] * T->q[b]);
+    dqo_integer_freqs(t, K, T->pf);
+    T->pc[0] = 0;
+    T->ustar = 0;
+    for (int u = 0; u < K; ++u) {
+        T->pc[u + 1] = T->pc[u] + T->pf[u];
+        double r = (double)DQO_P - log2((double)T->pf[u]);
+        T->pr[u] = (float)r;
+        T->pR[u] = (uint32_t)ceil(r * 65536.0);
+        if (T->pf[u] > T->pf[T->ustar]) T->ustar = u;
+    }
+    for (int u = 0; u < K; ++u)
+        for (int z = T->pc[u]; z < T->pc[u + 1]; ++z) {
+            T->plut_u[z] = (uint8_t)u;
+            T->plut_f[z] = (uint8_t)T->pf[u];
+            T->plut_d[z] = (uint8_t)(z - T->pc[u]);
+        }
+    T->feasible = ((int64_t)(T->n / 2) * T->pR[T->ustar] <= (int64_t)T->B * 65536);
+}
+
 static void dqo_fill_freqs(dqo_table *T)
 {
     int M = T->M;
     double qs = 0.0, t[DQO_MAX_LEVELS];
     for (int m = 0; m < M; ++m) { T->q[m] = pow(T->p[m], T->alpha); qs += T->q[m]; }
-    int tot = 0;
     for (int m = 0; m < M; ++m) {
         T->q[m] /= qs;
         t[m] = DQO_TOT * T->q[m];
-        int fl = (int)floor(t[m]);
-        T->f[m] = fl < 1 ? 1 : fl;
-        tot += T->f[m];
     }
-    while (tot < DQO_TOT) { /* largest remainder; tie -> lowest index */
-        int best = 0;
-        for (int m = 1; m < M; ++m)
-            if (t[m] - T->f[m] > t[best] - T->f[best]) best = m;
-        T->f[best] += 1; tot += 1;
-    }
-    while (tot > DQO_TOT) { /* largest excess among f > 1; tie -> highest index */
-        int best = -1;
-        for (int m = 0; m < M; ++m)
-            if (T->f[m] > 1 && (best < 0 || T->f[m] - t[m] >= T->f[best] - t[best])) best = m;
-        T->f[best] -= 1; tot -= 1;
-    }
+    dqo_integer_freqs(t, M, T->f);
     T->c[0] = 0;
     T->mstar = 0;
     for (int m = 0; m < M; ++m) {
@@ -195,11 +243,20 @@ static void dqo_fill_freqs(dqo_table *T)
             T->lut_d[z] = (uint8_t)(z - T->c[m]);
         }
     T->feasible = ((int64_t)T->n * T->R[T->mstar] <= (int64_t)T->B * 65536);
+    if (T->pair) dqo_fill_pair_freqs(T);
 }
 
+/* entropy of the integer table in bits per value */
 static double dqo_entropy256(const dqo_table *T)
 {
     double H = 0.0;
+    if (T->pair) {
+        for (int u = 0; u < T->M * T->M; ++u) {
+            double pu = T->pf[u] / 256.0;
+            H -= pu * log2(pu);
+        }
+        return H / 2.0;
+    }
     for (int m = 0; m < T->M; ++m) {
         double pm = T->f[m] / 256.0;
         H -= pm * log2(pm);
@@ -212,10 +269,11 @@ static double dqo_entropy256(const dqo_table *T)
  * whose table has entropy <= B/n and lets the all-central stream fit.
  * Returns 0, or -1 for bad arguments, -2 when no feasible table exists. */
 int dqo_build_table_ex(int M, int n, int rec_bytes, double alpha, int has_mean, int rotate,
-                       int sigma, int early_exit, dqo_table *T)
+                       int sigma, int early_exit, int pair, dqo_table *T)
 {
     if (M < 2 || M > DQO_MAX_LEVELS || n < 1 || n > DQO_MAX_N || rec_bytes < 9) return -1;
     if (sigma != 32 && sigma != 24) return -1;
+    if (pair && (n % 2)) return -1;                    /* M <= 16 keeps the pair alphabet within 2^p */
     /* With the 24-bit state an encode step may lose up to log2(1 + 2^-7) bits to floor(x / f)
      * (x >= 2^15, f < 2^8).  The budget test keeps sum r <= B = 8(C - 3); the stream then fits
      * its C bytes as long as the accumulated loss stays below one byte: n log2(1 + 2^-7) < 8,
@@ -224,7 +282,7 @@ int dqo_build_table_ex(int M, int n, int rec_bytes, double alpha, int has_mean, 
     if (sigma == 24 && n > 640) return -1;
     memset(T, 0, sizeof *T);
     T->M = M; T->n = n; T->rec = rec_bytes; T->C = rec_bytes - 4;
-    T->sigma = sigma; T->early_exit = early_exit ? 1 : 0;
+    T->sigma = sigma; T->early_exit = early_exit ? 1 : 0; T->pair = pair ? 1 : 0;
     T->B = 8 * T->C - sigma;                           /* Eq. (budget) */
     T->has_mean = has_mean; T->rotate = rotate;
     T->E = dqo_expected_max(n);
@@ -254,7 +312,7 @@ int dqo_build_table_ex(int M, int n, int rec_bytes, double alpha, int has_mean, 
 int dqo_build_table(int M, int n, int rec_bytes, double alpha, int has_mean, int rotate,
                     dqo_table *T)
 {
-    return dqo_build_table_ex(M, n, rec_bytes, alpha, has_mean, rotate, DQO_SIGMA, 0, T);
+    return dqo_build_table_ex(M, n, rec_bytes, alpha, has_mean, rotate, DQO_SIGMA, 0, 0, T);
 }
 
 int dqo_table_size(void) { return (int)sizeof(dqo_table); }
@@ -292,6 +350,48 @@ void dqo_fwht_f64(double *x, int n)
 
 /* ------------------------------------------------------------------- drift */
 
+/* One sweep of Drift at the multiplier lam: every rANS symbol takes the candidate that minimises
+ * distortion + lam * ideal cost (the lowest index among equal costs); returns the fixed-point code
+ * length of the assignment.  t[m] = grid level m.  A symbol is one value, or with the paired-symbol
+ * variant the values (2i, 2i + 1) with the M^2 candidates u = a M + b taken in ascending u. */
+static int64_t dqo_assign(const float *z, int n, const float *t, float lam, const dqo_table *T,
+                          uint8_t *m_out)
+{
+    int M = T->M;
+    int64_t len = 0;
+    if (T->pair) {
+        for (int i = 0; i < n / 2; ++i) {
+            int best = 0;
+            float bestc = 0.0f;
+            for (int a = 0; a < M; ++a)
+                for (int b = 0; b < M; ++b) {
+                    float da = z[2 * i] - t[a], db = z[2 * i + 1] - t[b];
+                    float Da = da * da, Db = db * db;
+                    float D = Da + Db;
+                    float cost = fmaf(lam, T->pr[a * M + b], D);
+                    if ((a == 0 && b == 0) || cost < bestc) { bestc = cost; best = a * M + b; }
+                }
+            m_out[2 * i] = (uint8_t)(best / M);
+            m_out[2 * i + 1] = (uint8_t)(best % M);
+            len += T->pR[best];
+        }
+        return len;
+    }
+    for (int j = 0; j < n; ++j) {
+        int best = 0;
+        float bestc = 0.0f;
+        for (int m = 0; m < M; ++m) {
+            float d = z[j] - t[m];
+            float D = d * d;
+            float cost = fmaf(lam, T->r[m], D);
+            if (m == 0 || cost < bestc) { bestc = cost; best = m; }
+        }
+        m_out[j] = (uint8_t)best;
+        len += T->R[best];
+    }
+    return len;
+}
+
 /* Function Drift of Algorithm 1: Lagrangian bisection (T = 12) on log2(lambda),
  * realised as the geometric mean of the bracket; returns argmin at `hi`.
  * z: stream values, (s, o): grid.  Writes symbols to m_out and returns the
@@ -310,7 +410,9 @@ int64_t dqo_drift(const float *z, int n, float s, float o, const dqo_table *T, u
             if (D < minD) minD = D;
         }
     const int64_t budget = (int64_t)T->B * 65536;
-    float lam_hi = 8.0f * (maxD - minD);
+    /* upper end of the bracket: a multiplier at which 1/8 bit outweighs any difference in
+     * distortion between two candidates (a pair's distortion is the sum of two values') */
+    float lam_hi = (T->pair ? 16.0f : 8.0f) * (maxD - minD);
     float lam_lo = lam_hi * 0x1p-40f;
     int64_t len = 0;
     if (T->early_exit) {
@@ -319,36 +421,12 @@ int64_t dqo_drift(const float *z, int n, float s, float o, const dqo_table *T, u
          * would return.  Evaluate it first and stop if it meets the budget. */
         float lam_e = lam_hi;
         for (int it = 0; it < 12; ++it) lam_e = sqrtf(lam_lo * lam_e);
-        len = 0;
-        for (int j = 0; j < n; ++j) {
-            int best = 0;
-            float bestc = 0.0f;
-            for (int m = 0; m < M; ++m) {
-                float d = z[j] - t[m];
-                float D = d * d;
-                float cost = fmaf(lam_e, T->r[m], D);
-                if (m == 0 || cost < bestc) { bestc = cost; best = m; }
-            }
-            m_out[j] = (uint8_t)best;
-            len += T->R[best];
-        }
+        len = dqo_assign(z, n, t, lam_e, T, m_out);
         if (len <= budget) return len;
     }
     for (int it = 0; it <= 12; ++it) {
         float lam = (it < 12) ? sqrtf(lam_lo * lam_hi) : lam_hi;
-        len = 0;
-        for (int j = 0; j < n; ++j) {
-            int best = 0;
-            float bestc = 0.0f;
-            for (int m = 0; m < M; ++m) {
-                float d = z[j] - t[m];
-                float D = d * d;
-                float cost = fmaf(lam, T->r[m], D);
-                if (m == 0 || cost < bestc) { bestc = cost; best = m; }
-            }
-            m_out[j] = (uint8_t)best;
-            len += T->R[best];
-        }
+        len = dqo_assign(z, n, t, lam, T, m_out);
         if (it < 12) {
             if (len <= budget) lam_hi = lam; else lam_lo = lam;
         }
@@ -367,8 +445,11 @@ int dqo_rans_encode(const uint8_t *sym, int n, const dqo_table *T, uint8_t *payl
     uint8_t tmp[2 * DQO_MAX_N];
     int k = 0, sb = T->sigma / 8;                      /* bytes of final state */
     uint32_t L = dqo_L(T), x = L;
-    for (int j = n - 1; j >= 0; --j) {
-        uint32_t f = (uint32_t)T->f[sym[j]], c = (uint32_t)T->c[sym[j]];
+    int step = T->pair ? 2 : 1;                        /* values per rANS symbol */
+    for (int j = n - step; j >= 0; j -= step) {
+        uint32_t f, c;
+        if (T->pair) { int u = sym[j] * T->M + sym[j + 1]; f = (uint32_t)T->pf[u]; c = (uint32_t)T->pc[u]; }
+        else { f = (uint32_t)T->f[sym[j]]; c = (uint32_t)T->c[sym[j]]; }
         while (x >= f * L) { tmp[k++] = (uint8_t)(x & 255u); x >>= 8; }   /* x_max = f (L / 2^p) 2^8 */
         x = (x / f) * DQO_TOT + (x % f) + c;
     }
@@ -388,10 +469,18 @@ void dqo_rans_decode(const uint8_t *payload, int cap, int n, const dqo_table *T,
     uint32_t x = 0, L = dqo_L(T);
     int ptr = T->sigma / 8;
     for (int i = 0; i < ptr; ++i) x |= (uint32_t)payload[i] << (8 * i);
-    for (int i = 0; i < n; ++i) {
+    int step = T->pair ? 2 : 1;
+    for (int i = 0; i + step <= n; i += step) {
         uint32_t z = x & (DQO_TOT - 1);
-        uint32_t f = T->lut_f[z], d = T->lut_d[z];
-        sym[i] = T->lut_m[z];
+        uint32_t f, d;
+        if (T->pair) {
+            f = T->plut_f[z]; d = T->plut_d[z];
+            sym[i] = (uint8_t)(T->plut_u[z] / T->M);
+            sym[i + 1] = (uint8_t)(T->plut_u[z] % T->M);
+        } else {
+            f = T->lut_f[z]; d = T->lut_d[z];
+            sym[i] = T->lut_m[z];
+        }
         x = f * (x >> DQO_P) + d;
         while (x < L && ptr < cap) { x = (x << 8) | payload[ptr]; ptr += 1; }
     }
@@ -405,6 +494,13 @@ void dqo_rans_decode(const uint8_t *payload, int cap, int n, const dqo_table *T,
  * [0] += streams that fell back to the all-central assignment, [1] += degenerate
  * (constant) streams, [2] += streams whose refit was rejected, [3] = max bytes used.
  * sym_out (nullable) receives the final symbols. */
+/* the most probable symbol everywhere (a pair's two levels with the paired-symbol variant) */
+static void dqo_all_central(const dqo_table *T, uint8_t *m)
+{
+    for (int j = 0; j < T->n; ++j)
+        m[j] = (uint8_t)(!T->pair ? T->mstar : (j % 2 == 0 ? T->ustar / T->M : T->ustar % T->M));
+}
+
 void dqo_encode_stream(const float *z, const dqo_table *T, uint8_t *rec, uint32_t *stats,
                        uint8_t *sym_out)
 {
@@ -465,7 +561,7 @@ void dqo_encode_stream(const float *z, const dqo_table *T, uint8_t *rec, uint32_
         else {
             int64_t len = dqo_drift(z, n, sf, of, T, m); /* second Drift on the fp16 grid */
             if (len > budget) {
-                for (int j = 0; j < n; ++j) m[j] = (uint8_t)T->mstar;
+                dqo_all_central(T, m);
                 if (stats) stats[0] += 1;
             }
         }
@@ -473,7 +569,7 @@ void dqo_encode_stream(const float *z, const dqo_table *T, uint8_t *rec, uint32_
     if (degenerate) {
         s16 = 0;
         o16 = dqo_f64_to_f16((double)mn);
-        for (int j = 0; j < n; ++j) m[j] = (uint8_t)T->mstar;
+        dqo_all_central(T, m);
         if (stats) stats[1] += 1;
     }
     rec[0] = (uint8_t)s16; rec[1] = (uint8_t)(s16 >> 8);
