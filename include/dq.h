@@ -58,6 +58,14 @@
  *     * sigma_bits = 24: records are [s fp16][o fp16][final state, 3 bytes LE][bytes ...]; the state
  *       lives in [2^15, 2^23) and B = 8C - 24 (Eq. budget), one more byte for symbols.  Key and
  *       value tables of one cache must agree on sigma_bits.  Per token-head streams only.
+ *     * pair_symbols: one rANS symbol is the pair of levels of two consecutive values (2i, 2i + 1),
+ *       u = m_2i M + m_2i+1, over the alphabet of M^2 pairs (Sec. 3.1: Eq. rans unchanged on a larger
+ *       alphabet; the pair model is the product of the sharpened level model with itself, made
+ *       integer by the same rule).  Algorithm 2 then takes 64 steps for 128 values, which is what
+ *       halves the decode cost of the attention kernel; Algorithm 1's Drift assigns a pair at a
+ *       time (argmin over the M^2 pairs of D_a + D_b + lambda r_ab, lowest u among equals; bracket
+ *       16 (max D - min D)).  Same record layout and sizes.  At most 9 levels; per token-head
+ *       streams only; key and value tables of one cache must agree.
  */
 #ifndef DQ_H_
 #define DQ_H_
@@ -77,6 +85,8 @@ extern "C" {
 #define DQ_ERR_CUDA (-5)         /* a CUDA runtime call failed (see dq_last_cuda_error) */
 
 #define DQ_MAX_LEVELS 16
+#define DQ_MAX_PAIR_LEVELS 9      /* paired-symbol variant: levels 0..8 (their fp16 codes fit one byte) */
+#define DQ_MAX_PAIRS 81
 #define DQ_HEAD_DIM 128
 #define DQ_PAGE_TOKENS 16
 #define DQ_WINDOW_TOKENS 128
@@ -109,6 +119,7 @@ typedef struct {
                        are read by the same decoder) */
     int sigma_bits;  /* 0 or 32: 32-bit final state, state in [2^23, 2^31).  24: 24-bit final state,
                        state in [2^15, 2^23), B = 8C - 24; per token-head streams only */
+    int pair_symbols; /* 1: rANS symbols are pairs of levels (levels <= 9, per token-head streams only) */
 } dq_table_opts;
 
 typedef struct {
@@ -123,13 +134,19 @@ typedef struct {
     int rec_words;                 /* ceil(rec_bytes / 4): words per record in the interleaved layout */
     int sigma_bits;                /* 32 or 24: bits of final rANS state in a record    */
     int drift_early_exit;          /* 0 / 1                                             */
+    /* paired-symbol variant (pair_symbols = 1); pair index u = a * levels + b, a = the even value's level.
+       `lut` then holds  code(b) << 24 | f_u << 16 | code(a) << 8 | (z - c_u),  code(m) = high byte of fp16(m) */
+    int pair_symbols, ustar;       /* 0 / 1; most probable pair                          */
+    int32_t pair_f[DQ_MAX_PAIRS];  /* pair frequencies, sum 256                          */
+    uint32_t pair_R[DQ_MAX_PAIRS]; /* ceil(65536 * -log2(pair_f / 256))                  */
 } dq_table_info;
 
 /* Probability model and rANS tables of one tensor kind (Sec. 3.1 "Entropy Coding",
  * Sec. 4.2 last paragraph, Sec. 4.4 "Distribution sharpening").  The probability of level
  * m is the N(0,1) mass of its cell on an M-level grid spanning +-E[max of n normals], n the
  * stream length (128, or hs * 128); frequencies are integers summing to 256.  Host only; needs
- * no GPU.  Returns DQ_ERR_INFEASIBLE when n * R[mstar] > 65536 * B.  *out is set only on DQ_OK. */
+ * no GPU.  Returns DQ_ERR_INFEASIBLE when n * R[mstar] > 65536 * B (paired symbols: when
+ * (n / 2) * pair_R[ustar] > 65536 * B).  *out is set only on DQ_OK. */
 int dq_build_tables(int levels, double bits_per_elem, const dq_table_opts *opts, dq_tables **out);
 void dq_free_tables(dq_tables *t);
 int dq_tables_info(const dq_tables *t, dq_table_info *out);

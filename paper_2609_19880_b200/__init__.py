@@ -13,6 +13,7 @@ _PKG = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_PKG, "libdquant.so")
 
 MAX_LEVELS = 16
+MAX_PAIRS = 81
 HEAD_DIM = 128
 PAGE_TOKENS = 16
 WINDOW_TOKENS = 128
@@ -38,7 +39,8 @@ class DqError(RuntimeError):
 
 class TableOpts(C.Structure):
     _fields_ = [("head_dim", C.c_int), ("alpha", C.c_double), ("has_mean", C.c_int), ("rotate", C.c_int),
-                ("heads_per_stream", C.c_int), ("drift_early_exit", C.c_int), ("sigma_bits", C.c_int)]
+                ("heads_per_stream", C.c_int), ("drift_early_exit", C.c_int), ("sigma_bits", C.c_int),
+                ("pair_symbols", C.c_int)]
 
 
 class TableInfo(C.Structure):
@@ -48,7 +50,8 @@ class TableInfo(C.Structure):
                 ("f", C.c_int32 * MAX_LEVELS), ("c", C.c_int32 * (MAX_LEVELS + 1)),
                 ("r", C.c_float * MAX_LEVELS), ("R", C.c_uint32 * MAX_LEVELS), ("lut", C.c_uint32 * 256),
                 ("heads_per_stream", C.c_int), ("rec_words", C.c_int), ("sigma_bits", C.c_int),
-                ("drift_early_exit", C.c_int)]
+                ("drift_early_exit", C.c_int), ("pair_symbols", C.c_int), ("ustar", C.c_int),
+                ("pair_f", C.c_int32 * MAX_PAIRS), ("pair_R", C.c_uint32 * MAX_PAIRS)]
 
 
 _lib = None
@@ -159,12 +162,12 @@ class Tables:
 
 def dq_build_tables(levels: int, bits_per_elem: float, *, alpha: float = 1.4, has_mean: bool = False,
                     rotate: bool = True, head_dim: int = HEAD_DIM, heads_per_stream: int = 1,
-                    drift_early_exit: bool = False, sigma_bits: int = 32) -> Tables:
+                    drift_early_exit: bool = False, sigma_bits: int = 32, pair_symbols: bool = False) -> Tables:
     """``heads_per_stream`` = hs > 1 builds tables for streams that span hs KV heads of a token
     (hs = Hkv: the paper's token-wide default); bits_per_elem then refers to hs * 128 values.
-    ``drift_early_exit`` / ``sigma_bits`` select the opt-in codec variants."""
+    ``drift_early_exit`` / ``sigma_bits`` / ``pair_symbols`` select the opt-in codec variants."""
     opts = TableOpts(head_dim, float(alpha), int(has_mean), int(rotate), int(heads_per_stream),
-                     int(drift_early_exit), int(sigma_bits))
+                     int(drift_early_exit), int(sigma_bits), int(pair_symbols))
     h = C.c_void_p()
     _check(lib().dq_build_tables(int(levels), float(bits_per_elem), C.byref(opts), C.byref(h)), "dq_build_tables")
     return Tables(h.value)

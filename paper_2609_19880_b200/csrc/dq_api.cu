@@ -32,6 +32,7 @@ int check_attn_tables(const dq_tables* tk, const dq_tables* tv, int Hkv, const u
     if (tv->info.has_mean) return DQ_ERR_UNSUPPORTED;
     if (tk->info.heads_per_stream != tv->info.heads_per_stream) return DQ_ERR_UNSUPPORTED;
     if (tk->info.sigma_bits != tv->info.sigma_bits) return DQ_ERR_UNSUPPORTED;   // one state width per cache
+    if (tk->info.pair_symbols != tv->info.pair_symbols) return DQ_ERR_UNSUPPORTED;   // one symbol alphabet kind per cache
     if (Hkv <= 0 || Hkv % tk->info.heads_per_stream != 0) return DQ_ERR_ARG;
     if (tk->info.has_mean && (!k_mean_q || !k_mean_scale || max_windows <= 0)) return DQ_ERR_ARG;
     if (tk->info.has_mean && (long long)max_windows * DQ_WINDOW_TOKENS < (long long)max_pages * DQ_PAGE_TOKENS)
@@ -94,6 +95,7 @@ int dq_encode_tokens_rope(const dq_tables* tk, const dq_tables* tv, const void* 
     {
         const int hs = tk ? tk->info.heads_per_stream : tv->info.heads_per_stream;
         if (tk && tv && tk->info.heads_per_stream != tv->info.heads_per_stream) return DQ_ERR_UNSUPPORTED;
+        if (tk && tv && tk->info.pair_symbols != tv->info.pair_symbols) return DQ_ERR_UNSUPPORTED;
         if (Hkv % hs != 0) return DQ_ERR_ARG;
     }
     if ((k_bf16 && (reinterpret_cast<uintptr_t>(k_bf16) & 7u)) ||
@@ -117,7 +119,7 @@ int dq_encode_tokens_rope(const dq_tables* tk, const dq_tables* tv, const void* 
     a.do_k = tk ? 1 : 0; a.do_v = tv ? 1 : 0;
     a.rope_cos = rope_cos; a.rope_sin = rope_sin; a.rope_style = rope_style;
     a.step_seq_lens = nullptr; a.step_flags = nullptr;
-    e = dq_launch_encode(tk ? tk->dev : tv->dev, tv ? tv->dev : tk->dev, a, st);
+    e = dq_launch_encode(tk ? tk->dev : tv->dev, tv ? tv->dev : tk->dev, tk ? tk->penc : tv->penc, tv ? tv->penc : tk->penc, a, st);
     if (e != cudaSuccess) return cuda_fail(e, "encode");
     return DQ_OK;
 }
@@ -303,7 +305,7 @@ int dq_decode_step(const dq_tables* tk, const dq_tables* tv, const void* k_new_b
     e.status = status; e.T = B; e.Hkv = Hkv; e.max_windows = max_windows; e.mean_mode = DQ_MEAN_REUSE;
     e.do_k = 1; e.do_v = 1;
     e.step_seq_lens = seq_lens; e.step_flags = dq_attn_workspace_flags(workspace);
-    cudaError_t ce = dq_launch_encode(tk->dev, tv->dev, e, st);
+    cudaError_t ce = dq_launch_encode(tk->dev, tv->dev, tk->penc, tv->penc, e, st);
     if (ce != cudaSuccess) return cuda_fail(ce, "decode step: encode");
     DqAttnArgs a;
     std::memset(&a, 0, sizeof a);

@@ -230,12 +230,39 @@ __device__ __forceinline__ void decode16(uint32_t& x, uint32_t& ptr, uint32_t lu
     }
 }
 
+// Paired-symbol variant: one step decodes the levels of two consecutive channels, 8 steps the 16.  A table
+// entry is code(b) << 24 | f << 16 | code(a) << 8 | (z - c) with code(m) the high byte of the fp16
+// pattern of level m (levels 0..8 have a zero low byte), so a step's fp16x2 word (level a, level b) is the
+// entry with its f and (z - c) bytes cleared.
+template <int LBITS>
+__device__ __forceinline__ void decode16_pairs(uint32_t& x, uint32_t& ptr, uint32_t lut, uint32_t one,
+                                               uint32_t (&packed)[8]) {
+#pragma unroll
+    for (int q4 = 0; q4 < 2; ++q4) {
+        const uint32_t base = ptr & ~3u;
+        const uint32_t win = __funnelshift_r(lds32(base), lds32(base + 4), ptr << 3);
+        uint32_t sel = 0x2104u;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const uint32_t e = lds32(dp4a_u32(x, 0x80u, lut));
+            const uint32_t f = dp4a_u32(e, 0x00010000u, 0u);
+            const uint32_t t = f * (x >> 8);
+            x = dp4a_u32(e, 1u, t);
+            asm("{.reg .pred p; setp.lt.u32 p, %0, %4; @p prmt.b32 %0, %0, %2, %1; "
+                "@p mad.lo.u32 %1, %3, %3, %1;}"
+                : "+r"(x), "+r"(sel) : "r"(win), "r"(one), "n"(1u << LBITS));
+            packed[4 * q4 + i] = e & 0xff00ff00u;
+        }
+        ptr += sel - 0x2104u;
+    }
+}
+
 // One pass over the 128 channels, 16 at a time.  With DO_K the K streams of the current item
 // are decoded and S[g][t] = sum_j q'_gj level_tj accumulated (Eq. fold-key, inner sum).  With
 // DO_V the V streams of the previous item are decoded and each finished 16-channel tile of
 // O[j][g] = sum_t (a_t s_t) level_tj (Eq. fold-value, first sum) goes to this warp's output
 // slot in shared memory.  Both decodes are interleaved in one instruction stream.
-template <bool DO_K, bool DO_V, int LBITS>
+template <bool DO_K, bool DO_V, int LBITS, bool PAIRS>
 __device__ __forceinline__ void fused_pass(uint32_t xk, uint32_t ptrk, uint32_t xv, uint32_t ptrv, uint32_t lutk,
                                            uint32_t lutv, uint32_t one, uint32_t ktile, uint32_t vtile, uint32_t q16,
                                            uint32_t obuf, int lane, int G, float (&sacc)[4][4],
@@ -251,8 +278,8 @@ __device__ __forceinline__ void fused_pass(uint32_t xk, uint32_t ptrk, uint32_t 
 #pragma unroll 1
     for (int cg = 0; cg < DQ_EXP_CG; ++cg) {
         uint32_t pk[8], pv[8];
-        if (DO_K) decode16<LBITS>(xk, ptrk, lutk, one, pk);
-        if (DO_V) decode16<LBITS>(xv, ptrv, lutv, one, pv);
+        if (DO_K) { if (PAIRS) decode16_pairs<LBITS>(xk, ptrk, lutk, one, pk); else decode16<LBITS>(xk, ptrk, lutk, one, pk); }
+        if (DO_V) { if (PAIRS) decode16_pairs<LBITS>(xv, ptrv, lutv, one, pv); else decode16<LBITS>(xv, ptrv, lutv, one, pv); }
         if (DO_K) { sts128(ktile + lane * kTileStride, pk); sts128(ktile + lane * kTileStride + 16, pk + 4); }
         if (DO_V) { sts128(vtile + lane * kTileStride, pv); sts128(vtile + lane * kTileStride + 16, pv + 4); }
         __syncwarp();
@@ -294,7 +321,8 @@ __device__ __forceinline__ void fused_pass(uint32_t xk, uint32_t ptrk, uint32_t 
 // The option DQ_OPT_STEP_POLL_LIMIT replaces the default; 0 makes every CTA take the fallback at once,
 // which is how the tests run that path.
 static int step_poll_limit() { return dq_opt_step_poll_limit(DQ_STEP_POLL_LIMIT); }
-template <bool FUSED, int LBITS>
+// PAIRS: the tables' rANS symbols are pairs of levels (64 steps per stream instead of 128).
+template <bool FUSED, int LBITS, bool PAIRS>
 __global__ void __launch_bounds__(kMaxWarps * 32, 1)
 dq_attention_kernel(const __grid_constant__ DqDevTable TK, const __grid_constant__ DqDevTable TV,
                     const AttnParams p) {
@@ -528,13 +556,13 @@ dq_attention_kernel(const __grid_constant__ DqDevTable TK, const __grid_constant
             constexpr uint32_t kPay = LBITS == 23 ? 8u : 7u;
             const uint32_t xk = lds32_unaligned(rk + 4) & kStateMask, xv = lds32_unaligned(rvp + 4) & kStateMask;
             if (cur.valid && have_prev)
-                fused_pass<true, true, LBITS>(xk, rk + kPay, xv, rvp + kPay, my_lutk, my_lutv, one, ktile, vtile, q16, my_obuf,
+                fused_pass<true, true, LBITS, PAIRS>(xk, rk + kPay, xv, rvp + kPay, my_lutk, my_lutv, one, ktile, vtile, q16, my_obuf,
                                               lane, G, sacc, pb_hi, pb_lo);
             else if (cur.valid)
-                fused_pass<true, false, LBITS>(xk, rk + kPay, xv, rvp + kPay, my_lutk, my_lutv, one, ktile, vtile, q16, my_obuf,
+                fused_pass<true, false, LBITS, PAIRS>(xk, rk + kPay, xv, rvp + kPay, my_lutk, my_lutv, one, ktile, vtile, q16, my_obuf,
                                                lane, G, sacc, pb_hi, pb_lo);
             else
-                fused_pass<false, true, LBITS>(xk, rk + kPay, xv, rvp + kPay, my_lutk, my_lutv, one, ktile, vtile, q16, my_obuf,
+                fused_pass<false, true, LBITS, PAIRS>(xk, rk + kPay, xv, rvp + kPay, my_lutk, my_lutv, one, ktile, vtile, q16, my_obuf,
                                                lane, G, sacc, pb_hi, pb_lo);
         }
 
@@ -1171,8 +1199,10 @@ static cudaError_t launch_attention_pass(const DqDevTable& tk, const DqDevTable&
     if (e != cudaSuccess) return e;
     // the four instantiations of the main kernel: decode-step mode or not, 32- or 24-bit final state
     void (*main_kernel)(DqDevTable, DqDevTable, AttnParams) =
-        tk.sigma == 24 ? (p.fused ? dq_attention_kernel<true, 15> : dq_attention_kernel<false, 15>)
-                       : (p.fused ? dq_attention_kernel<true, 23> : dq_attention_kernel<false, 23>);
+        tk.pair ? (tk.sigma == 24 ? (p.fused ? dq_attention_kernel<true, 15, true> : dq_attention_kernel<false, 15, true>)
+                                  : (p.fused ? dq_attention_kernel<true, 23, true> : dq_attention_kernel<false, 23, true>))
+                : (tk.sigma == 24 ? (p.fused ? dq_attention_kernel<true, 15, false> : dq_attention_kernel<false, 15, false>)
+                                  : (p.fused ? dq_attention_kernel<true, 23, false> : dq_attention_kernel<false, 23, false>));
     if (!wide) {
         e = cudaFuncSetAttribute(main_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, L.total);
         if (e != cudaSuccess) return e;

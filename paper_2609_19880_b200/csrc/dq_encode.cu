@@ -138,17 +138,57 @@ dq_means_compute_kernel(const uint16_t* __restrict__ k, int T, int Hkv, int rota
 // ------------------------------------------------------------------------ drift
 
 // Per-CTA copy of the table fields the encoder touches (a CTA encodes one tensor kind).
+// With the paired-symbol variant the rANS alphabet is the M^2 pairs u = a M + b: the coder's arrays
+// (rcp .. thr) and prk then hold the pair alphabet, r / R are not used.
 struct EncTable {
     float r[DQ_MAX_LEVELS];
     uint32_t R[DQ_MAX_LEVELS];
-    uint32_t rcp[DQ_MAX_LEVELS];   // Eq. rans Enc by reciprocal: floor(x / f) = umulhi(x, rcp) >> rsh
-    uint32_t rsh[DQ_MAX_LEVELS];
-    uint32_t bias[DQ_MAX_LEVELS];  // c (+ 255 when f = 1)
-    uint32_t cmpl[DQ_MAX_LEVELS];  // 2^p - f
-    uint32_t thr[DQ_MAX_LEVELS];   // f << (sigma - 9) = f L: renormalise while the state is not below it
+    uint32_t rcp[DQ_MAX_PAIRS];    // Eq. rans Enc by reciprocal: floor(x / f) = umulhi(x, rcp) >> rsh
+    uint32_t rsh[DQ_MAX_PAIRS];
+    uint32_t bias[DQ_MAX_PAIRS];   // c (+ 255 when f = 1)
+    uint32_t cmpl[DQ_MAX_PAIRS];   // 2^p - f
+    uint32_t thr[DQ_MAX_PAIRS];    // f << (sigma - 9) = f L: renormalise while the state is not below it
+    uint2 prk[DQ_MAX_PAIRS];       // pairs: {bits of r_u, ceil(65536 r_u) << 8 | u}
     int M, rec, mstar, budget_bits, has_mean, rotate;
     int early_exit, sigma;         // codec variants: Drift tries its end multiplier first; bits of final state (32 / 24)
+    int pair;                      // paired symbols
+    uint32_t central;              // the all-central stream's four levels of a lane, one per byte
 };
+
+// Table of one tensor kind into shared memory (threads 0 .. DQ_MAX_PAIRS - 1 and thread 0).
+__device__ __forceinline__ void load_enc_table(EncTable& T, const DqDevTable& TK, const DqDevTable& TV,
+                                               const DqPairEnc& PK, const DqPairEnc& PV, bool is_v) {
+    const int pair = is_v ? TV.pair : TK.pair, sigma = is_v ? TV.sigma : TK.sigma;
+    const int i = threadIdx.x;
+    if (i < DQ_MAX_LEVELS) {
+        T.r[i] = is_v ? TV.r[i] : TK.r[i];
+        T.R[i] = is_v ? TV.R[i] : TK.R[i];
+    }
+    if (i < (pair ? DQ_MAX_PAIRS : DQ_MAX_LEVELS)) {
+        uint32_t aux;
+        if (pair) {
+            T.rcp[i] = is_v ? PV.enc_rcp[i] : PK.enc_rcp[i];
+            aux = is_v ? PV.enc_aux[i] : PK.enc_aux[i];
+            T.prk[i] = make_uint2(__float_as_uint(is_v ? PV.r[i] : PK.r[i]), ((is_v ? PV.R[i] : PK.R[i]) << 8) | (uint32_t)i);
+        } else {
+            T.rcp[i] = is_v ? TV.enc_rcp[i] : TK.enc_rcp[i];
+            aux = is_v ? TV.enc_aux[i] : TK.enc_aux[i];
+        }
+        T.bias[i] = aux & 1023u;
+        T.cmpl[i] = (aux >> 10) & 511u;
+        T.rsh[i] = aux >> 19;
+        T.thr[i] = (256u - ((aux >> 10) & 511u)) << (sigma - 9);
+    }
+    if (i == 0) {
+        T.M = is_v ? TV.M : TK.M; T.rec = is_v ? TV.rec : TK.rec; T.mstar = is_v ? TV.mstar : TK.mstar;
+        T.budget_bits = is_v ? TV.budget_bits : TK.budget_bits;
+        T.has_mean = is_v ? TV.has_mean : TK.has_mean; T.rotate = is_v ? TV.rotate : TK.rotate;
+        T.early_exit = is_v ? TV.early_exit : TK.early_exit; T.sigma = sigma;
+        T.pair = pair;
+        const uint32_t ms = (uint32_t)T.mstar, us = (uint32_t)(is_v ? TV.ustar : TK.ustar), M = (uint32_t)T.M;
+        T.central = pair ? (us / M) * 0x00010001u + (us % M) * 0x01000100u : ms * 0x01010101u;
+    }
+}
 
 // Function Drift of Algorithm 1 on a stream held 4 values per lane.  The bisection of
 // log2(lambda) over T = 12 steps is carried out as the geometric mean of the bracket
@@ -241,6 +281,100 @@ __device__ __forceinline__ uint32_t drift(const EncTable& T, const float (&z)[4]
     return len;
 }
 
+// Drift for the paired-symbol variant: a lane's values (0, 1) and (2, 3) are two rANS symbols; each takes
+// the pair u = a M + b that minimises (D_a + D_b) + lambda r_u, the lowest u among equal costs (rows a in
+// ascending order, each reduced left to right, then the row winners: the same winner as an ascending scan
+// with a strict comparison).  Bracket: hi = 16 (max D - min D), D over single values as above.
+template <int M>
+__device__ __noinline__ uint32_t drift_pair_m(const EncTable& T, float z0, float z1, float z2, float z3, float s, float o,
+                                              uint32_t& sym_packed) {
+    const float z[4] = {z0, z1, z2, z3};
+    float D[4][M];
+    float maxD = -INFINITY, minD = INFINITY;
+#pragma unroll
+    for (int m = 0; m < M; ++m) {
+        const float tm = __fmaf_rn((float)m, s, o);
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            const float d = __fsub_rn(z[e], tm);
+            D[e][m] = __fmul_rn(d, d);
+            maxD = fmaxf(maxD, D[e][m]);
+            minD = fminf(minD, D[e][m]);
+        }
+    }
+#pragma unroll
+    for (int d = 16; d >= 1; d >>= 1) {
+        maxD = fmaxf(maxD, __shfl_xor_sync(kFull, maxD, d));
+        minD = fminf(minD, __shfl_xor_sync(kFull, minD, d));
+    }
+    const uint32_t budget = (uint32_t)T.budget_bits << 16;
+    float lam_hi = __fmul_rn(16.0f, __fsub_rn(maxD, minD));
+    float lam_lo = __fmul_rn(lam_hi, 0x1p-40f);
+    uint32_t len = 0, psym[2] = {0u, 0u};
+    float lam_e = lam_hi;
+    if (T.early_exit)
+        for (int i = 0; i < 12; ++i) lam_e = __fsqrt_rn(__fmul_rn(lam_lo, lam_e));
+#pragma unroll 1
+    for (int it = T.early_exit ? -1 : 0; it <= 12; ++it) {
+        const float lam = (it < 0) ? lam_e : (it < 12) ? __fsqrt_rn(__fmul_rn(lam_lo, lam_hi)) : lam_hi;
+        uint32_t cost_sum = 0;
+#pragma unroll
+        for (int p = 0; p < 2; ++p) {
+            float rc[M];
+            uint32_t rkey[M];
+#pragma unroll
+            for (int a = 0; a < M; ++a) {
+                float c[M];
+                uint32_t key[M];
+#pragma unroll
+                for (int b = 0; b < M; ++b) {
+                    const uint2 e = T.prk[a * M + b];
+                    c[b] = __fmaf_rn(lam, __uint_as_float(e.x), __fadd_rn(D[2 * p][a], D[2 * p + 1][b]));
+                    key[b] = e.y;
+                }
+#pragma unroll
+                for (int w = 1; w < M; w <<= 1)
+#pragma unroll
+                    for (int b = 0; b + w < M; b += 2 * w)
+                        if (c[b + w] < c[b]) { c[b] = c[b + w]; key[b] = key[b + w]; }
+                rc[a] = c[0];
+                rkey[a] = key[0];
+            }
+#pragma unroll
+            for (int w = 1; w < M; w <<= 1)
+#pragma unroll
+                for (int a = 0; a + w < M; a += 2 * w)
+                    if (rc[a + w] < rc[a]) { rc[a] = rc[a + w]; rkey[a] = rkey[a + w]; }
+            psym[p] = rkey[0];
+            cost_sum += rkey[0];
+        }
+        len = __reduce_add_sync(kFull, cost_sum >> 8);   // two pair indices (< 81 each) stay below bit 8
+        if (it < 0) {
+            if (len <= budget) break;
+        } else if (it < 12) {
+            if (len <= budget) lam_hi = lam; else lam_lo = lam;
+        }
+    }
+    const uint32_t u0 = psym[0] & 0xffu, u1 = psym[1] & 0xffu;
+    sym_packed = (u0 / M) | ((u0 % M) << 8) | ((u1 / M) << 16) | ((u1 % M) << 24);
+    return len;
+}
+
+__device__ __forceinline__ uint32_t drift_pair(const EncTable& T, const float (&z)[4], float s, float o,
+                                               uint32_t (&sym)[4]) {
+    uint32_t packed = 0, len = 0;
+    switch (T.M) {   // uniform across the CTA
+#define DQ_DRIFT_CASE(M_) case M_: len = drift_pair_m<M_>(T, z[0], z[1], z[2], z[3], s, o, packed); break;
+        DQ_DRIFT_CASE(2) DQ_DRIFT_CASE(3) DQ_DRIFT_CASE(4) DQ_DRIFT_CASE(5) DQ_DRIFT_CASE(6) DQ_DRIFT_CASE(7)
+        DQ_DRIFT_CASE(8) DQ_DRIFT_CASE(9)
+#undef DQ_DRIFT_CASE
+        default: break;
+    }
+#pragma unroll
+    for (int e = 0; e < 4; ++e) sym[e] = (packed >> (8 * e)) & 0xffu;
+    return len;
+}
+
 // ---------------------------------------------------------------------- encoder
 
 constexpr int kEncWarps = 8;
@@ -260,6 +394,9 @@ struct StreamQuantised {
 
 // Steps 1-6 of Algorithm 1 for the stream (token t, KV head h) by one warp: rotation (and rotary
 // embedding when asked), mean removal, min-max grid, drift, refit, fp16 metadata, second drift.
+// PAIR: the table's rANS symbols are pairs of levels (a kernel instantiation of its own, so that the
+// single-level kernels carry none of its code).
+template <bool PAIR>
 __device__ __forceinline__ StreamQuantised quantise_stream(const EncTable& T, const DqEncodeArgs& a, bool is_v, int t, int h,
                                                            int lane) {
     const int Hkv = a.Hkv;
@@ -314,7 +451,7 @@ __device__ __forceinline__ StreamQuantised quantise_stream(const EncTable& T, co
     if (!degenerate) {
         const float o = mn;                                         // FitMinMax, Eq. (affine_token)
         const float s = __fdiv_rn(__fsub_rn(mx, mn), (float)(T.M - 1));
-        drift(T, z, s, o, sym);
+        if (PAIR) drift_pair(T, z, s, o, sym); else drift(T, z, s, o, sym);
         // Refit: least squares of z on the symbols; binary64 sums in a fixed order
         double sa = (double)z[0], sb = __dmul_rn((double)sym[0], (double)z[0]);
         int sm = (int)sym[0], smm = (int)(sym[0] * sym[0]);
@@ -348,10 +485,10 @@ __device__ __forceinline__ StreamQuantised quantise_stream(const EncTable& T, co
         }
         if (!(sf > 0.0f)) degenerate = true;
         else {
-            const uint32_t len = drift(T, z, sf, of, sym);          // second Drift, fp16 grid
+            const uint32_t len = PAIR ? drift_pair(T, z, sf, of, sym) : drift(T, z, sf, of, sym);   // second Drift, fp16 grid
             if (len > ((uint32_t)T.budget_bits << 16)) {
 #pragma unroll
-                for (int e = 0; e < 4; ++e) sym[e] = (uint32_t)T.mstar;
+                for (int e = 0; e < 4; ++e) sym[e] = (T.central >> (8 * e)) & 0xffu;
                 st_fallback = 1;
             }
         }
@@ -360,7 +497,7 @@ __device__ __forceinline__ StreamQuantised quantise_stream(const EncTable& T, co
         s16 = __ushort_as_half(0);
         o16 = __float2half_rn(mn);
 #pragma unroll
-        for (int e = 0; e < 4; ++e) sym[e] = (uint32_t)T.mstar;
+        for (int e = 0; e < 4; ++e) sym[e] = (T.central >> (8 * e)) & 0xffu;
     }
 
     StreamQuantised r;
@@ -376,10 +513,10 @@ __device__ __forceinline__ StreamQuantised quantise_stream(const EncTable& T, co
 // few spills for twice the resident warps (throughput: prefill, bulk encodes).
 // WARPS streams per CTA: 8 normally; the decode step uses 16 (512 threads at full register budget) so that its
 // 2 B Hkv streams occupy few SMs while the attention kernel runs on all the others.
-template <int MINB, int WARPS>
+template <int MINB, int WARPS, bool PAIR>
 __global__ void __launch_bounds__(WARPS * 32, MINB)
 dq_encode_kernel(const __grid_constant__ DqDevTable TK, const __grid_constant__ DqDevTable TV,
-                 const DqEncodeArgs a) {
+                 const __grid_constant__ DqPairEnc PK, const __grid_constant__ DqPairEnc PV, const DqEncodeArgs a) {
     __shared__ EncTable T;
     __shared__ uint8_t s_bytes[WARPS][DQ_MAX_REC_BYTES];
     __shared__ __align__(4) uint8_t s_sym[WARPS][kN];
@@ -388,23 +525,7 @@ dq_encode_kernel(const __grid_constant__ DqDevTable TK, const __grid_constant__ 
     // hand-over words are cleared).  Otherwise: trigger first, so that the next kernel's launch overlaps this one.
     if (!a.step_flags) dqdev::pdl_launch_dependents();
     const bool is_v = a.do_k ? (blockIdx.y == 1) : true;
-    if (threadIdx.x < DQ_MAX_LEVELS) {
-        const int i = threadIdx.x;
-        T.r[i] = is_v ? TV.r[i] : TK.r[i];
-        T.R[i] = is_v ? TV.R[i] : TK.R[i];
-        T.rcp[i] = is_v ? TV.enc_rcp[i] : TK.enc_rcp[i];
-        const uint32_t aux = is_v ? TV.enc_aux[i] : TK.enc_aux[i];
-        T.bias[i] = aux & 1023u;
-        T.cmpl[i] = (aux >> 10) & 511u;
-        T.rsh[i] = aux >> 19;
-        T.thr[i] = (256u - ((aux >> 10) & 511u)) << ((is_v ? TV.sigma : TK.sigma) - 9);
-    }
-    if (threadIdx.x == 0) {
-        T.M = is_v ? TV.M : TK.M; T.rec = is_v ? TV.rec : TK.rec; T.mstar = is_v ? TV.mstar : TK.mstar;
-        T.budget_bits = is_v ? TV.budget_bits : TK.budget_bits;
-        T.has_mean = is_v ? TV.has_mean : TK.has_mean; T.rotate = is_v ? TV.rotate : TK.rotate;
-        T.early_exit = is_v ? TV.early_exit : TK.early_exit; T.sigma = is_v ? TV.sigma : TK.sigma;
-    }
+    load_enc_table(T, TK, TV, PK, PV, is_v);
     __syncthreads();
     dqdev::pdl_wait_prior_grid();   // inputs and the cache may be written / read by the previous kernel
     if (a.step_flags) {
@@ -422,10 +543,17 @@ dq_encode_kernel(const __grid_constant__ DqDevTable TK, const __grid_constant__ 
     const int t = (int)(wid / a.Hkv), h = (int)(wid % a.Hkv), Hkv = a.Hkv;
     uint8_t* cont = is_v ? a.v_cont : a.k_cont;
 
-    const StreamQuantised sq = quantise_stream(T, a, is_v, t, h, lane);
+    const StreamQuantised sq = quantise_stream<PAIR>(T, a, is_v, t, h, lane);
     // rANS, Eq. (rans) Enc on symbols 127 .. 0 so that decoding runs forward.  Every lane
     // carries the same state (the symbols come from shared memory); lane 0 records the bytes.
-    *reinterpret_cast<uint32_t*>(&s_sym[wib][4 * lane]) = sq.sym;
+    // (paired symbols: the lane's two pair indices u = a M + b; the coder then runs over 64 symbols)
+    if (PAIR) {
+        const uint32_t M = (uint32_t)T.M;
+        const uint32_t u0 = (sq.sym & 0xffu) * M + ((sq.sym >> 8) & 0xffu), u1 = ((sq.sym >> 16) & 0xffu) * M + (sq.sym >> 24);
+        *reinterpret_cast<uint16_t*>(&s_sym[wib][2 * lane]) = (uint16_t)(u0 | (u1 << 8));
+    } else {
+        *reinterpret_cast<uint32_t*>(&s_sym[wib][4 * lane]) = sq.sym;
+    }
     __syncwarp();
     uint32_t xs = 1u << (T.sigma - 9);   // L: 2^23, or 2^15 with the 24-bit state
     int k = 0;
@@ -433,7 +561,7 @@ dq_encode_kernel(const __grid_constant__ DqDevTable TK, const __grid_constant__ 
     // the symbol / table loads, so those loads are issued ahead of the serial state chain
     const uint32_t bytes_addr = dqdev::smem_addr(s_bytes[wib]);
 #pragma unroll 8
-    for (int j = kN - 1; j >= 0; --j) {
+    for (int j = (PAIR ? kN / 2 : kN) - 1; j >= 0; --j) {
         const uint32_t m = s_sym[wib][j];
         const uint32_t rcp = T.rcp[m], rsh = T.rsh[m], bias = T.bias[m], cmpl = T.cmpl[m], thr = T.thr[m];
         if (xs >= thr) {  // at most once: xs < 2^8 L <= 2^8 * (f L)
@@ -483,10 +611,10 @@ dq_encode_kernel(const __grid_constant__ DqDevTable TK, const __grid_constant__ 
 constexpr int kB32 = 32;                 // streams per CTA
 constexpr int kB32SymStride = 36;        // bytes per position row (32 streams + pad against bank conflicts)
 constexpr int kB32Warps = DQ_B32_WARPS;
-template <int MINB>
+template <int MINB, bool PAIR>
 __global__ void __launch_bounds__(kB32Warps * 32, MINB)
 dq_encode_batch32_kernel(const __grid_constant__ DqDevTable TK, const __grid_constant__ DqDevTable TV,
-                         const DqEncodeArgs a) {
+                         const __grid_constant__ DqPairEnc PK, const __grid_constant__ DqPairEnc PV, const DqEncodeArgs a) {
     __shared__ EncTable T;
     __shared__ __align__(4) uint8_t s_symT[kN * kB32SymStride];
     __shared__ uint8_t s_bytesT[DQ_MAX_REC_BYTES * kB32];
@@ -494,23 +622,7 @@ dq_encode_batch32_kernel(const __grid_constant__ DqDevTable TK, const __grid_con
     __shared__ unsigned long long s_rec[kB32];   // record addresses
     dqdev::pdl_launch_dependents();
     const bool is_v = a.do_k ? (blockIdx.y == 1) : true;
-    if (threadIdx.x < DQ_MAX_LEVELS) {
-        const int i = threadIdx.x;
-        T.r[i] = is_v ? TV.r[i] : TK.r[i];
-        T.R[i] = is_v ? TV.R[i] : TK.R[i];
-        T.rcp[i] = is_v ? TV.enc_rcp[i] : TK.enc_rcp[i];
-        const uint32_t aux = is_v ? TV.enc_aux[i] : TK.enc_aux[i];
-        T.bias[i] = aux & 1023u;
-        T.cmpl[i] = (aux >> 10) & 511u;
-        T.rsh[i] = aux >> 19;
-        T.thr[i] = (256u - ((aux >> 10) & 511u)) << ((is_v ? TV.sigma : TK.sigma) - 9);
-    }
-    if (threadIdx.x == 0) {
-        T.M = is_v ? TV.M : TK.M; T.rec = is_v ? TV.rec : TK.rec; T.mstar = is_v ? TV.mstar : TK.mstar;
-        T.budget_bits = is_v ? TV.budget_bits : TK.budget_bits;
-        T.has_mean = is_v ? TV.has_mean : TK.has_mean; T.rotate = is_v ? TV.rotate : TK.rotate;
-        T.early_exit = is_v ? TV.early_exit : TK.early_exit; T.sigma = is_v ? TV.sigma : TK.sigma;
-    }
+    load_enc_table(T, TK, TV, PK, PV, is_v);
     __syncthreads();
     dqdev::pdl_wait_prior_grid();
     const int lane = threadIdx.x & 31, wib = threadIdx.x >> 5;
@@ -522,9 +634,15 @@ dq_encode_batch32_kernel(const __grid_constant__ DqDevTable TK, const __grid_con
     for (int i = wib; i < ns; i += kB32Warps) {   // quantise: warp w takes streams w, w + warps, ...
         const long long wid = first + i;
         const int t = (int)(wid / a.Hkv), h = (int)(wid % a.Hkv);
-        const StreamQuantised sq = quantise_stream(T, a, is_v, t, h, lane);
+        const StreamQuantised sq = quantise_stream<PAIR>(T, a, is_v, t, h, lane);
+        if (PAIR) {   // the lane's two pair indices u = a M + b at positions 2 lane, 2 lane + 1
+            const uint32_t M = (uint32_t)T.M;
+            s_symT[(2 * lane) * kB32SymStride + i] = (uint8_t)((sq.sym & 0xffu) * M + ((sq.sym >> 8) & 0xffu));
+            s_symT[(2 * lane + 1) * kB32SymStride + i] = (uint8_t)(((sq.sym >> 16) & 0xffu) * M + (sq.sym >> 24));
+        } else {
 #pragma unroll
-        for (int e = 0; e < 4; ++e) s_symT[(4 * lane + e) * kB32SymStride + i] = (uint8_t)(sq.sym >> (8 * e));
+            for (int e = 0; e < 4; ++e) s_symT[(4 * lane + e) * kB32SymStride + i] = (uint8_t)(sq.sym >> (8 * e));
+        }
         if (lane == 0) {
             s_hdr[i] = sq.hdr0;
             const int sl = a.slot[t];
@@ -541,7 +659,7 @@ dq_encode_batch32_kernel(const __grid_constant__ DqDevTable TK, const __grid_con
     if (wib == 0 && lane < ns) {   // rANS, Eq. (rans) Enc on symbols 127 .. 0; lane = stream
         uint32_t xs = 1u << (T.sigma - 9), k = 0;
 #pragma unroll 4
-        for (int j = kN - 1; j >= 0; --j) {
+        for (int j = (PAIR ? kN / 2 : kN) - 1; j >= 0; --j) {
             const uint32_t m = s_symT[j * kB32SymStride + lane];
             const uint32_t rcp = T.rcp[m], rsh = T.rsh[m], bias = T.bias[m], cmpl = T.cmpl[m], thr = T.thr[m];
             if (xs >= thr) {   // at most once: xs < 2^8 L <= 2^8 * (f L)
@@ -729,6 +847,7 @@ __device__ __forceinline__ void load_wide_table(EncTable& T, WideShared& W, cons
         T.budget_bits = is_v ? TV.budget_bits : TK.budget_bits;
         T.has_mean = is_v ? TV.has_mean : TK.has_mean; T.rotate = is_v ? TV.rotate : TK.rotate;
         T.early_exit = is_v ? TV.early_exit : TK.early_exit; T.sigma = 32;   // token-wide streams keep the 32-bit state
+        T.pair = 0; T.central = (uint32_t)T.mstar * 0x01010101u;   // and single levels as symbols
     }
 }
 
@@ -1018,7 +1137,8 @@ cudaError_t dq_launch_means(const DqDevTable& tk, const void* k_bf16, int T, int
 // option DQ_OPT_ENCODE_BATCH_MIN replaces the default (0 sends every call there).
 static long long batch_min_streams(long long dflt) { return dq_opt_encode_batch_min(dflt); }
 
-cudaError_t dq_launch_encode(const DqDevTable& tk, const DqDevTable& tv, const DqEncodeArgs& a, cudaStream_t st) {
+cudaError_t dq_launch_encode(const DqDevTable& tk, const DqDevTable& tv, const DqPairEnc& pk, const DqPairEnc& pv,
+                             const DqEncodeArgs& a, cudaStream_t st) {
     const long long warps = (long long)a.T * a.Hkv;
     if (warps == 0 || (!a.do_k && !a.do_v)) return cudaSuccess;
     if (tk.hs > 1) {   // token-wide streams: CTAs of hs warps; few streams: one per CTA, many: 32 per CTA
@@ -1033,13 +1153,16 @@ cudaError_t dq_launch_encode(const DqDevTable& tk, const DqDevTable& tv, const D
                              dim3(tk.hs * 32), (size_t)smem, st, tk, tv, a);
     }
     const unsigned blocks = (unsigned)((warps + kEncWarps - 1) / kEncWarps);
+    const bool pair = tk.pair != 0;   // the caller has checked that both tables agree
+    const dim3 kinds(1, (a.do_k && a.do_v) ? 2 : 1);
     if (!a.step_flags && warps >= batch_min_streams(4LL * 148 * kB32 * 4))   // enough streams to fill the GPU several times
-        return dq_launch_pdl(dq_encode_batch32_kernel<DQ_B32_MINB>, dim3((unsigned)((warps + kB32 - 1) / kB32), (a.do_k && a.do_v) ? 2 : 1),
-                             dim3(kB32Warps * 32), 0, st, tk, tv, a);
+        return dq_launch_pdl(pair ? dq_encode_batch32_kernel<DQ_B32_MINB, true> : dq_encode_batch32_kernel<DQ_B32_MINB, false>,
+                             dim3((unsigned)((warps + kB32 - 1) / kB32), kinds.y), dim3(kB32Warps * 32), 0, st, tk, tv, pk, pv, a);
     if (a.step_flags) {   // decode step: big CTAs, so that few SMs are kept from the attention kernel
         constexpr int kStepWarps = DQ_STEP_ENC_WARPS;
-        return dq_launch_pdl(dq_encode_kernel<1, kStepWarps>, dim3((unsigned)((warps + kStepWarps - 1) / kStepWarps), (a.do_k && a.do_v) ? 2 : 1),
-                             dim3(kStepWarps * 32), 0, st, tk, tv, a);
+        return dq_launch_pdl(pair ? dq_encode_kernel<1, kStepWarps, true> : dq_encode_kernel<1, kStepWarps, false>,
+                             dim3((unsigned)((warps + kStepWarps - 1) / kStepWarps), kinds.y), dim3(kStepWarps * 32), 0, st, tk, tv, pk, pv, a);
     }
-    return dq_launch_pdl(dq_encode_kernel<2, kEncWarps>, dim3(blocks, (a.do_k && a.do_v) ? 2 : 1), dim3(kEncWarps * 32), 0, st, tk, tv, a);
+    return dq_launch_pdl(pair ? dq_encode_kernel<2, kEncWarps, true> : dq_encode_kernel<2, kEncWarps, false>, dim3(blocks, kinds.y),
+                         dim3(kEncWarps * 32), 0, st, tk, tv, pk, pv, a);
 }

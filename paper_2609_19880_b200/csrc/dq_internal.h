@@ -12,16 +12,27 @@ struct DqDevTable {
     int has_mean, rotate;
     int hs, rec_words;           // heads per stream (>= 1); words per record (interleaved layout, hs > 1)
     int sigma, early_exit;       // bits of final state in a record (32 / 24); Drift tries its end multiplier first
+    int pair, ustar;             // paired-symbol variant: rANS symbols are pairs u = a M + b; most probable pair
     uint32_t enc_rcp[DQ_MAX_LEVELS];  // encoder, Eq. rans Enc by reciprocal: floor(x / f) = umulhi(x, rcp) >> rsh
     uint32_t enc_aux[DQ_MAX_LEVELS];  // bias | (256 - f) << 10 | rsh << 19, bias = c (+ 255 when f = 1)
     float r[DQ_MAX_LEVELS];      // ideal cost in bits     (Algorithm 1)
     uint32_t R[DQ_MAX_LEVELS];   // ceil(r * 65536)
     uint32_t lut[256];           // f << 24 | fp16(level) << 8 | (z - c)   (Algorithm 2)
+                                 // pair: code(b) << 24 | f << 16 | code(a) << 8 | (z - c), code = high byte of fp16(level)
+};
+
+// Encoder-side tables of the pair alphabet (paired-symbol variant); same packing as DqDevTable's.
+struct DqPairEnc {
+    uint32_t enc_rcp[DQ_MAX_PAIRS];
+    uint32_t enc_aux[DQ_MAX_PAIRS];
+    float r[DQ_MAX_PAIRS];
+    uint32_t R[DQ_MAX_PAIRS];
 };
 
 struct dq_tables {
     dq_table_info info;
     DqDevTable dev;
+    DqPairEnc penc;              // zero unless dev.pair
 };
 
 // dq_api.cu: process-wide options (dq_set_option); `dflt` is returned while an option is unset
@@ -56,7 +67,9 @@ struct DqEncodeArgs {
     const int32_t* step_seq_lens;
     int* step_flags;         // decode-step mode: 4 hand-over words this kernel clears for the kernels after it
 };
-cudaError_t dq_launch_encode(const DqDevTable& tk, const DqDevTable& tv, const DqEncodeArgs& a, cudaStream_t st);
+// pk / pv: pair alphabets of the key / value table (read only when that table has dev.pair set)
+cudaError_t dq_launch_encode(const DqDevTable& tk, const DqDevTable& tv, const DqPairEnc& pk, const DqPairEnc& pv,
+                             const DqEncodeArgs& a, cudaStream_t st);
 cudaError_t dq_launch_decode_tokens(const DqDevTable& t, const uint8_t* cont, const int8_t* mean_q,
                                     const float* mean_scale, int max_windows, const int32_t* seq_id,
                                     const int32_t* pos, const int32_t* slot, int T, int Hkv,

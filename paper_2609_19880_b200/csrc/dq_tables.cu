@@ -52,17 +52,22 @@ Model cell_masses(int M, int n) {
     return mod;
 }
 
-// Integer frequencies summing to 256: floor with a floor of 1, then largest remainders up
-// (ties to the lowest index) or largest excesses down among f > 1 (ties to the highest index).
-void integer_frequencies(const Model& mod, double alpha, int32_t* f) {
-    const int M = (int)mod.cell.size();
-    std::vector<double> target(M);
+// Sharpened model p' ~ p^alpha, normalised (Sec. 4.4).
+std::vector<double> sharpened(const Model& mod, double alpha) {
+    std::vector<double> q(mod.cell.size());
     double norm = 0.0;
-    for (int m = 0; m < M; ++m) norm += (target[m] = std::pow(mod.cell[m], alpha));
+    for (size_t m = 0; m < q.size(); ++m) norm += (q[m] = std::pow(mod.cell[m], alpha));
+    for (double& v : q) v = v / norm;
+    return q;
+}
+
+// Integer frequencies summing to 256 for targets 256 * probability: floor with a floor of 1, then
+// largest remainders up (ties to the lowest index) or largest excesses down among f > 1 (ties to
+// the highest index).
+void integer_frequencies(const std::vector<double>& target, int32_t* f) {
+    const int M = (int)target.size();
     int sum = 0;
     for (int m = 0; m < M; ++m) {
-        target[m] = target[m] / norm;
-        target[m] = kTotal * target[m];
         f[m] = std::max(1, (int)std::floor(target[m]));
         sum += f[m];
     }
@@ -77,6 +82,41 @@ void integer_frequencies(const Model& mod, double alpha, int32_t* f) {
         for (int m = 0; m < M; ++m)
             if (f[m] > 1 && (pick < 0 || f[m] - target[m] >= f[pick] - target[pick])) pick = m;
         --f[pick];
+    }
+}
+
+// Level table: 256 * q_m.  Pair table (paired-symbol variant): 256 * (q_a q_b), u = a M + b.
+void level_frequencies(const Model& mod, double alpha, int32_t* f) {
+    std::vector<double> target = sharpened(mod, alpha);
+    for (double& v : target) v = kTotal * v;
+    integer_frequencies(target, f);
+}
+
+void pair_frequencies(const Model& mod, double alpha, int32_t* f) {
+    const std::vector<double> q = sharpened(mod, alpha);
+    const int M = (int)q.size();
+    std::vector<double> target((size_t)M * M);
+    for (int a = 0; a < M; ++a)
+        for (int b = 0; b < M; ++b) target[(size_t)a * M + b] = kTotal * (q[a] * q[b]);
+    integer_frequencies(target, f);
+}
+
+// High byte of the binary16 pattern of a level 0..8 (their low byte is zero).
+uint32_t level_code(int m) { return (uint32_t)__half_as_ushort(__float2half((float)m)) >> 8; }
+
+// Pair alphabet: costs, most probable pair and the decode table
+//   lut[z] = code(b) << 24 | f_u << 16 | code(a) << 8 | (z - c_u).
+void finish_pairs(dq_table_info& t) {
+    const int M = t.levels, K = M * M;
+    t.ustar = 0;
+    int c = 0;
+    for (int u = 0; u < K; ++u) {
+        const double bits = 8.0 - std::log2((double)t.pair_f[u]);
+        t.pair_R[u] = (uint32_t)std::ceil(bits * 65536.0);
+        if (t.pair_f[u] > t.pair_f[t.ustar]) t.ustar = u;
+        for (int z = c; z < c + t.pair_f[u]; ++z)
+            t.lut[z] = (level_code(u % M) << 24) | ((uint32_t)t.pair_f[u] << 16) | (level_code(u / M) << 8) | (uint32_t)(z - c);
+        c += t.pair_f[u];
     }
 }
 
@@ -95,14 +135,25 @@ void finish(dq_table_info& t) {
         for (int z = t.c[m]; z < t.c[m + 1]; ++z)
             t.lut[z] = ((uint32_t)t.f[m] << 24) | (level_bits << 8) | (uint32_t)(z - t.c[m]);
     }
+    if (t.pair_symbols) finish_pairs(t);
 }
 
 bool all_central_fits(const dq_table_info& t) {
-    return (int64_t)t.head_dim * t.heads_per_stream * t.R[t.mstar] <= (int64_t)t.budget_bits * 65536;
+    const int64_t n = (int64_t)t.head_dim * t.heads_per_stream;
+    if (t.pair_symbols) return (n / 2) * t.pair_R[t.ustar] <= (int64_t)t.budget_bits * 65536;
+    return n * t.R[t.mstar] <= (int64_t)t.budget_bits * 65536;
 }
 
+// bits per value
 double table_entropy(const dq_table_info& t) {
     double h = 0.0;
+    if (t.pair_symbols) {
+        for (int u = 0; u < t.levels * t.levels; ++u) {
+            const double p = t.pair_f[u] / (double)kTotal;
+            h -= p * std::log2(p);
+        }
+        return 0.5 * h;
+    }
     for (int m = 0; m < t.levels; ++m) {
         const double p = t.f[m] / (double)kTotal;
         h -= p * std::log2(p);
@@ -127,6 +178,8 @@ int dq_host_build(int levels, double bits_per_elem, const dq_table_opts* opts, d
     const int sigma = opts->sigma_bits == 0 ? 32 : opts->sigma_bits;
     if (sigma != 32 && sigma != 24) return DQ_ERR_ARG;
     if (sigma == 24 && hs > 1) return DQ_ERR_UNSUPPORTED;   // the short state is offered for 128-value streams
+    const bool pair = opts->pair_symbols != 0;
+    if (pair && (hs > 1 || levels > DQ_MAX_PAIR_LEVELS)) return DQ_ERR_UNSUPPORTED;
 
     dq_table_info& t = out->info;
     std::memset(out, 0, sizeof *out);
@@ -139,6 +192,7 @@ int dq_host_build(int levels, double bits_per_elem, const dq_table_opts* opts, d
     t.budget_bits = 8 * t.container_bytes - sigma;  // B = 8C - sigma
     t.sigma_bits = sigma;
     t.drift_early_exit = opts->drift_early_exit ? 1 : 0;
+    t.pair_symbols = pair ? 1 : 0;
     t.has_mean = opts->has_mean ? 1 : 0;
     t.rotate = opts->rotate ? 1 : 0;
 
@@ -146,13 +200,15 @@ int dq_host_build(int levels, double bits_per_elem, const dq_table_opts* opts, d
     bool ok = false;
     if (opts->alpha >= 0.0) {
         t.alpha = opts->alpha;
-        integer_frequencies(mod, t.alpha, t.f);
+        level_frequencies(mod, t.alpha, t.f);
+        if (pair) pair_frequencies(mod, t.alpha, t.pair_f);
         finish(t);
         ok = all_central_fits(t);
     } else {
         for (int tenth = 14; tenth <= 320 && !ok; ++tenth) {
             t.alpha = tenth / 10.0;
-            integer_frequencies(mod, t.alpha, t.f);
+            level_frequencies(mod, t.alpha, t.f);
+            if (pair) pair_frequencies(mod, t.alpha, t.pair_f);
             finish(t);
             ok = all_central_fits(t) && table_entropy(t) <= (double)t.budget_bits / n;
         }
@@ -170,23 +226,36 @@ int dq_host_build(int levels, double bits_per_elem, const dq_table_opts* opts, d
     d.rec_words = t.rec_words;
     d.sigma = sigma;
     d.early_exit = t.drift_early_exit;
-    for (int m = 0; m < levels; ++m) {
-        // Enc(x, m) = floor(x / f) 2^p + x mod f + c = x + c + floor(x / f) (2^p - f); the quotient of a
-        // 31-bit x by f comes from one high multiply with rcp = ceil(2^(31 + s) / f), s = ceil(log2 f),
-        // followed by a shift of s - 1.  f = 1: rcp = 2^32 - 1 gives x - 1 and the bias absorbs it.
-        const uint32_t f = (uint32_t)t.f[m];
-        uint32_t rcp = 0xffffffffu, rsh = 0, bias = (uint32_t)t.c[m] + 255u;
+    d.pair = t.pair_symbols;
+    d.ustar = t.ustar;
+    // Enc(x, m) = floor(x / f) 2^p + x mod f + c = x + c + floor(x / f) (2^p - f); the quotient of a
+    // 31-bit x by f comes from one high multiply with rcp = ceil(2^(31 + s) / f), s = ceil(log2 f),
+    // followed by a shift of s - 1.  f = 1: rcp = 2^32 - 1 gives x - 1 and the bias absorbs it.
+    auto enc_entry = [](uint32_t f, uint32_t c, uint32_t& rcp_out, uint32_t& aux_out) {
+        uint32_t rcp = 0xffffffffu, rsh = 0, bias = c + 255u;
         if (f > 1) {
             uint32_t s = 0;
             while ((1u << s) < f) ++s;
             rcp = (uint32_t)((((uint64_t)1 << (s + 31)) + f - 1) / f);
             rsh = s - 1;
-            bias = (uint32_t)t.c[m];
+            bias = c;
         }
-        d.enc_rcp[m] = rcp;
-        d.enc_aux[m] = bias | ((256u - f) << 10) | (rsh << 19);
+        rcp_out = rcp;
+        aux_out = bias | ((256u - f) << 10) | (rsh << 19);
+    };
+    for (int m = 0; m < levels; ++m) {
+        enc_entry((uint32_t)t.f[m], (uint32_t)t.c[m], d.enc_rcp[m], d.enc_aux[m]);
         d.r[m] = t.r[m];
         d.R[m] = t.R[m];
+    }
+    if (pair) {
+        uint32_t c = 0;
+        for (int u = 0; u < levels * levels; ++u) {
+            enc_entry((uint32_t)t.pair_f[u], c, out->penc.enc_rcp[u], out->penc.enc_aux[u]);
+            out->penc.r[u] = (float)(8.0 - std::log2((double)t.pair_f[u]));
+            out->penc.R[u] = t.pair_R[u];
+            c += (uint32_t)t.pair_f[u];
+        }
     }
     std::memcpy(d.lut, t.lut, sizeof d.lut);
     return DQ_OK;

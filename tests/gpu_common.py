@@ -14,17 +14,17 @@ from paper_2609_19880_b200 import workloads
 SM_SCALE = 1.0 / math.sqrt(128.0)
 
 
-def tables(cfg, rotate_v=True, early_exit=False, sigma=32):
-    """(library K, library V, oracle K, oracle V) tables of a configuration; early_exit / sigma select
-    the opt-in codec variants on both sides."""
+def tables(cfg, rotate_v=True, early_exit=False, sigma=32, pair=False):
+    """(library K, library V, oracle K, oracle V) tables of a configuration; early_exit / sigma / pair
+    select the opt-in codec variants on both sides."""
     tk = dq.dq_build_tables(cfg.k_levels, cfg.bits_k, alpha=cfg.alpha, has_mean=True, rotate=True,
-                            drift_early_exit=early_exit, sigma_bits=sigma)
+                            drift_early_exit=early_exit, sigma_bits=sigma, pair_symbols=pair)
     tv = dq.dq_build_tables(cfg.v_levels, cfg.bits_v, alpha=cfg.alpha, has_mean=False, rotate=rotate_v,
-                            drift_early_exit=early_exit, sigma_bits=sigma)
+                            drift_early_exit=early_exit, sigma_bits=sigma, pair_symbols=pair)
     ok = oracle.build_table(cfg.k_levels, 128, cfg.k_rec, cfg.alpha, has_mean=True, rotate=True,
-                            early_exit=early_exit, sigma=sigma)
+                            early_exit=early_exit, sigma=sigma, pair=pair)
     ov = oracle.build_table(cfg.v_levels, 128, cfg.v_rec, cfg.alpha, has_mean=False, rotate=rotate_v,
-                            early_exit=early_exit, sigma=sigma)
+                            early_exit=early_exit, sigma=sigma, pair=pair)
     return tk, tv, ok, ov
 
 

@@ -7,7 +7,11 @@ variants are pinned in test_oracle_variants.py):
   configuration 2 at full size, every record;
 * sigma = 24: records, decoded symbols, dequantised values bit for bit, attention within tolerance,
   for the default 5 / 3 levels and for 6 value levels in 29 bytes (a table that only the shorter
-  state makes feasible); the decode step in one call; mixed state widths are refused.
+  state makes feasible); the decode step in one call; mixed state widths are refused;
+* paired symbols: records, decoded symbols, dequantised values bit for bit and attention within
+  tolerance for 5 / 3, 8 / 6 and 9 / 9 levels, alone and together with the other two variants, through
+  both encoder kernels, the check decoder, every attention entry point and the decode step; the
+  whole of configuration 2 at full size; mixed alphabets are refused.
 """
 import numpy as np
 import pytest
@@ -32,9 +36,9 @@ def _np(t):
     return t.cpu().numpy()
 
 
-def _encode_and_compare(cfg, early_exit=False, sigma=32, batch_kernels=False):
+def _encode_and_compare(cfg, early_exit=False, sigma=32, batch_kernels=False, pair=False):
     w = workloads.generate(cfg, device="cuda")
-    tk, tv, ok, ov = gc.tables(cfg, early_exit=early_exit, sigma=sigma)
+    tk, tv, ok, ov = gc.tables(cfg, early_exit=early_exit, sigma=sigma, pair=pair)
     cache = gc.GpuCache(w, ok.rec, ov.rec)
     if batch_kernels:
         dq.dq_set_option(dq.OPT_ENCODE_BATCH_MIN, 0)
@@ -199,3 +203,117 @@ def test_mixed_state_widths_are_refused():
     assert err.value.code == -3
     with pytest.raises(dq.DqError):
         dq.dq_build_tables(8, 335 * 8 / 1024, heads_per_stream=8, sigma_bits=24)   # token-wide streams keep 32 bits
+
+
+# ------------------------------------------------------------------ paired symbols
+
+@pytest.mark.parametrize("batch_kernels", [False, True])
+@pytest.mark.parametrize("cfg_idx,scale,levels", [(1, 1.0, (7, 48, 5, 40)), (2, 1 / 16, None), (4, 1 / 32, None), (5, 1 / 32, None),
+                                                  (2, 1 / 32, (8, 56, 6, 40)), (2, 1 / 32, (9, 60, 9, 60)),
+                                                  (2, 1 / 32, (2, 24, 4, 37))])
+def test_pair_symbols_parity(cfg_idx, scale, levels, batch_kernels):
+    cfg = workloads.make_config(cfg_idx, scale=scale) if cfg_idx > 1 else workloads.make_config(1)
+    if levels:
+        cfg.k_levels, cfg.k_rec, cfg.v_levels, cfg.v_rec = levels
+    w, tk, tv, ok, ov, cache, host = _encode_and_compare(cfg, pair=True, batch_kernels=batch_kernels)
+    assert tk.info().pair_symbols == 1 and tv.info().pair_symbols == 1
+    _decode_and_attend(w, tk, tv, ok, ov, cache, host)
+
+
+@pytest.mark.parametrize("sigma,early_exit", [(24, False), (32, True), (24, True)])
+def test_pair_symbols_with_the_other_variants(sigma, early_exit):
+    cfg = workloads.make_config(2, scale=1 / 16)
+    for batch in (False, True):
+        w, tk, tv, ok, ov, cache, host = _encode_and_compare(cfg, pair=True, sigma=sigma, early_exit=early_exit,
+                                                             batch_kernels=batch)
+        _decode_and_attend(w, tk, tv, ok, ov, cache, host)
+
+
+def test_pair_symbols_decode_step():
+    """dq_decode_step with paired symbols: appended records and attention against the oracle, across a
+    window boundary and a page boundary."""
+    cfg = workloads.make_config(2, scale=1 / 16)
+    cfg.batch, cfg.seq_lens = 4, [300, 127, 512, 15]
+    steps = 4
+    w = workloads.generate(cfg, device="cuda", extra_tokens_per_seq=steps)
+    tk, tv, ok, ov = gc.tables(cfg, pair=True)
+    cache = gc.GpuCache(w, ok.rec, ov.rec)
+    gc.gpu_encode(w, tk, tv, cache)
+    kc, vc, mq, ms, _, _ = gc.oracle_encode(w, ok, ov)
+    gen = torch.Generator(device="cuda").manual_seed(11)
+    lens = torch.tensor(cfg.seq_lens, dtype=torch.int32)
+    seq = np.arange(cfg.batch, dtype=np.int32)
+    pt_cpu = w.page_table.cpu()
+    B, Hq, Hkv = cfg.batch, cfg.hq, cfg.hkv
+    ws = torch.empty(dq.dq_decode_workspace_bytes(B, Hq, w.page_table.shape[1]), dtype=torch.uint8, device="cuda")
+    out = torch.empty((B, Hq, 128), dtype=torch.bfloat16, device="cuda")
+    out32 = torch.empty((B, Hq, 128), dtype=torch.float32, device="cuda")
+    for s in range(steps):
+        k1, v1 = workloads.make_kv(cfg, B, gen, torch.device("cuda"), w.k_offsets, w.k_gain)
+        lens = lens + 1
+        pos = lens - 1
+        slot = (pt_cpu[torch.arange(B), (pos // 16).long()] * 16 + pos % 16).to(torch.int32)
+        dq.dq_decode_step(tk, tv, k1, v1, slot.cuda(), w.q, cache.k_cont, cache.v_cont, cache.mean_q, cache.mean_scale,
+                          w.page_table, lens.cuda(), Hkv, gc.SM_SCALE, out, ws, out32, cache.status)
+        kb, vb = workloads.bf16_bits(k1), workloads.bf16_bits(v1)
+        oracle.window_means(kb, seq, pos.numpy(), mq, ms, 1)
+        oracle.encode_tokens(ok, kb, seq, pos.numpy(), slot.numpy(), kc, mq, ms)
+        oracle.encode_tokens(ov, vb, seq, pos.numpy(), slot.numpy(), vc)
+        torch.cuda.synchronize()
+        assert np.array_equal(_np(cache.k_cont), kc) and np.array_equal(_np(cache.v_cont), vc)
+        ref = oracle.attention(ok, ov, workloads.bf16_bits(w.q), kc, vc, mq, ms, _np(w.page_table), lens.numpy(), Hkv,
+                               gc.SM_SCALE)
+        gc.check_attention(out, out32, ref)
+
+
+def test_pair_symbols_config2_full_size():
+    """Configuration 2 at full size with paired symbols: every record against the oracle, then every
+    attention row; kernel times of both alphabets printed side by side."""
+    cfg = workloads.make_config(2)
+    w, tk, tv, ok, ov, cache, host = _encode_and_compare(cfg, pair=True)
+    out, out32 = gc.gpu_attention(w, tk, tv, cache)
+    ref = oracle.attention(ok, ov, workloads.bf16_bits(w.q), host[0], host[1], host[2], host[3], _np(w.page_table),
+                           _np(w.seq_lens), cfg.hkv, gc.SM_SCALE)
+    worst = gc.check_attention(out, out32, ref)
+    assert worst < 1e-3
+    tk0, tv0, _, _ = gc.tables(cfg)
+    c0 = gc.GpuCache(w, ok.rec, ov.rec)
+    gc.gpu_encode(w, tk0, tv0, c0)
+    times = {}
+    for name, (a, b, c) in {"levels": (tk0, tv0, c0), "pairs": (tk, tv, cache)}.items():
+        for _ in range(3):
+            gc.gpu_attention(w, a, b, c)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(10):
+            gc.gpu_attention(w, a, b, c, want_f32=False)
+        e1.record()
+        torch.cuda.synchronize()
+        times[name] = e0.elapsed_time(e1) / 10
+        gc.gpu_encode(w, a, b, c)
+        torch.cuda.synchronize()
+        e0.record()
+        gc.gpu_encode(w, a, b, c)
+        e1.record()
+        torch.cuda.synchronize()
+        times[name + "_encode"] = e0.elapsed_time(e1)
+    print(f"config 2 attention call incl. host sync: levels {times['levels']:.4f} ms, pairs {times['pairs']:.4f} ms; "
+          f"prefill encode: levels {times['levels_encode']:.3f} ms, pairs {times['pairs_encode']:.3f} ms; worst rel err {worst:.2e}")
+    assert times["pairs"] < times["levels"]
+
+
+def test_mixed_alphabets_are_refused():
+    cfg = workloads.make_config(2, scale=1 / 64)
+    w = workloads.generate(cfg, device="cuda")
+    tk, tv, ok, ov = gc.tables(cfg, pair=True)
+    tk0, tv0, _, _ = gc.tables(cfg)
+    cache = gc.GpuCache(w, ok.rec, ov.rec)
+    out = torch.zeros((cfg.batch, cfg.hq, 128), dtype=torch.bfloat16, device="cuda")
+    ws = torch.empty(dq.dq_decode_workspace_bytes(cfg.batch, cfg.hq, w.page_table.shape[1]), dtype=torch.uint8, device="cuda")
+    with pytest.raises(dq.DqError) as err:
+        dq.dq_decode_attention(tk, tv0, w.q, cache.k_cont, cache.v_cont, cache.mean_q, cache.mean_scale, w.page_table,
+                               w.seq_lens, cfg.hkv, gc.SM_SCALE, out, ws)
+    assert err.value.code == -3
+    with pytest.raises(dq.DqError) as err:
+        gc.gpu_encode(w, tk, tv0, cache)
+    assert err.value.code == -3

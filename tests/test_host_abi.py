@@ -49,6 +49,38 @@ def test_tables_equal_oracle(L, M, rec, alpha):
         assert lvl == float(o.lut_m[z])
 
 
+@pytest.mark.parametrize("M,rec,alpha,sigma", [(5, 42, 1.4, 32), (3, 29, 1.4, 32), (9, 60, 1.4, 32), (8, 56, 1.4, 24),
+                                               (4, 37, 1.4, 32), (2, 24, 0.0, 32), (7, 44, 2.5, 32), (6, 42, -1.0, 32)])
+def test_pair_tables_equal_oracle(L, M, rec, alpha, sigma):
+    """Paired-symbol variant: the pair alphabet's integers and the decode table, entry by entry."""
+    t = dq.dq_build_tables(M, rec * 8 / 128, alpha=alpha, has_mean=True, rotate=True, pair_symbols=True, sigma_bits=sigma)
+    i = t.info()
+    o = oracle.build_table(M, 128, rec, alpha, pair=True, sigma=sigma)
+    assert (i.pair_symbols, i.ustar, i.budget_bits, i.sigma_bits) == (1, o.ustar, o.B, sigma)
+    assert abs(i.alpha - o.alpha) < 1e-12
+    assert [i.f[m] for m in range(M)] == o.freqs()
+    assert [i.pair_f[u] for u in range(M * M)] == o.pair_freqs()
+    assert [i.pair_R[u] for u in range(M * M)] == [o.pR[u] for u in range(M * M)]
+    for z in range(256):
+        e = i.lut[z]
+        u = o.plut_u[z]
+        assert (e >> 16) & 255 == o.plut_f[z] and e & 255 == o.plut_d[z]
+        assert oracle.f16_bits_to_f32(e & 0xFF00) == float(u // M)          # level of the even value
+        assert oracle.f16_bits_to_f32((e >> 16) & 0xFF00) == float(u % M)   # level of the odd value
+
+
+def test_pair_tables_limits(L):
+    with pytest.raises(dq.DqError) as err:
+        dq.dq_build_tables(10, 60 * 8 / 128, pair_symbols=True)            # levels 0..8 only
+    assert err.value.code == -3
+    with pytest.raises(dq.DqError) as err:
+        dq.dq_build_tables(8, 335 * 8 / 1024, heads_per_stream=8, pair_symbols=True)
+    assert err.value.code == -3
+    with pytest.raises(dq.DqError) as err:
+        dq.dq_build_tables(9, 20 * 8 / 128, pair_symbols=True)             # the all-central pairs do not fit
+    assert err.value.code == -2
+
+
 @pytest.mark.parametrize("M,hs,rec,alpha", [(8, 8, 335, 1.4), (6, 8, 235, 1.4), (11, 8, 235, 1.4), (6, 2, 86, 1.4),
                                             (16, 8, 600, -1.0), (4, 4, 150, 0.0)])
 def test_token_wide_tables_equal_oracle(L, M, hs, rec, alpha):
