@@ -38,6 +38,10 @@ SM_COUNT, SCHEDULERS_PER_SM = 148, 4
 # quantities measured by a bench run; the line says so where it uses them.
 NCU_HEAD = {"dram_bytes": 37.62e6, "token_heads": 524288, "bytes_per_token_head": 72.0, "instr_per_symbol": 15.2,
             "issue_active": 0.622, "source": "the ncu summary of dq_attention_kernel on config 2 under profiles/"}
+CODECS = {"paper": "the paper's codec: one level per rANS symbol (Algorithm 2, 128 steps per 128-value stream)",
+          "pairs": "opt-in variant: one rANS symbol = the levels of two consecutive values (64 steps per stream)"}
+NCU_PAIRS = {"instr_per_symbol": 9.96, "issue_active": 0.560,
+             "source": "the ncu summary of dq_attention_kernel with paired-symbol tables on config 2 under profiles/"}
 NCU_WIDE = {"instr_per_symbol": 19.2, "issue_active": 0.641,
             "source": "the ncu summary of dq_attention_wide_kernel on config 2 under profiles/"}
 REGIONS = 21          # the K-step timed region is repeated this many times; ms_per_step is the median
@@ -120,7 +124,7 @@ def stream_setup(cfg, streams: str):
     return dict(hs=1, k_rec=cfg.k_rec, v_rec=cfg.v_rec, k_levels=cfg.k_levels, v_levels=cfg.v_levels, alpha=cfg.alpha)
 
 
-def oracle_step_runner(cfg_idx: int, budget: float, streams: str = "head"):
+def oracle_step_runner(cfg_idx: int, budget: float, streams: str = "head", codec: str = "paper"):
     """Builds the oracle's workload -- the same seeded configuration the GPU leg runs, all of its
     sequences while they stay within ORACLE_MAX_TOKENS tokens in total (configs 2, 3 and 5 whole;
     the first sequences of config 4) -- and returns (step function, KV tokens per step,
@@ -139,8 +143,9 @@ def oracle_step_runner(cfg_idx: int, budget: float, streams: str = "head"):
     cfg.batch, cfg.seq_lens = keep, list(cfg.seq_lens[:keep])
     w = workloads.generate(cfg, device="cpu")
     st = stream_setup(cfg, streams)
-    ok = oracle.build_table(st["k_levels"], 128 * st["hs"], st["k_rec"], st["alpha"], has_mean=True, rotate=True)
-    ov = oracle.build_table(st["v_levels"], 128 * st["hs"], st["v_rec"], st["alpha"], has_mean=False, rotate=True)
+    pair = codec == "pairs"
+    ok = oracle.build_table(st["k_levels"], 128 * st["hs"], st["k_rec"], st["alpha"], has_mean=True, rotate=True, pair=pair)
+    ov = oracle.build_table(st["v_levels"], 128 * st["hs"], st["v_rec"], st["alpha"], has_mean=False, rotate=True, pair=pair)
     kb, vb, qb = workloads.bf16_bits(w.k), workloads.bf16_bits(w.v), workloads.bf16_bits(w.q)
     seq_id, pos, slot = (t.numpy() for t in (w.seq_id, w.pos, w.slot))
     mq = np.zeros((cfg.batch, w.max_windows, cfg.hkv, 128), np.int8)
@@ -168,8 +173,8 @@ def oracle_step_runner(cfg_idx: int, budget: float, streams: str = "head"):
     return step, tot, desc, oracle.num_threads(), whole
 
 
-def time_oracle(cfg_idx, budget, budget_s=10.0, max_steps=1000, warmup=1, streams="head"):
-    step, toks, desc, cores, _ = oracle_step_runner(cfg_idx, budget, streams)
+def time_oracle(cfg_idx, budget, budget_s=10.0, max_steps=1000, warmup=1, streams="head", codec="paper"):
+    step, toks, desc, cores, _ = oracle_step_runner(cfg_idx, budget, streams, codec)
     for _ in range(warmup):
         step()
     n, t0 = 0, time.perf_counter()
@@ -187,7 +192,7 @@ def run_reference(args):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
-    step, toks, desc, cores, whole = oracle_step_runner(args.config, args.budget, args.streams)
+    step, toks, desc, cores, whole = oracle_step_runner(args.config, args.budget, args.streams, args.codec)
     for _ in range(max(args.warmup, 1)):
         step()
     t0 = time.perf_counter()
@@ -199,7 +204,7 @@ def run_reference(args):
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * dt / args.steps,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
             "config": {"workload": f"config {args.config} at {args.budget} bits/elem, " +
-                       ("" if whole else "bounded sample: ") + desc},
+                       ("" if whole else "bounded sample: ") + desc, "codec": CODECS[args.codec]},
             "cpu_baseline": {"value": val, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": desc},
             "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
             "gpu_launches": 0}
@@ -251,10 +256,13 @@ def run_ours(args):
     st = stream_setup(cfg, args.streams)
     hs, k_rec, v_rec = st["hs"], st["k_rec"], st["v_rec"]
     n_stream = 128 * hs
+    if args.codec == "pairs" and hs > 1:
+        raise SystemExit("--codec pairs is offered for per token-head streams (--streams head)")
+    pair = args.codec == "pairs"
     tk = dq.dq_build_tables(st["k_levels"], k_rec * 8 / n_stream, alpha=st["alpha"], has_mean=True, rotate=True,
-                            heads_per_stream=hs)
+                            heads_per_stream=hs, pair_symbols=pair)
     tv = dq.dq_build_tables(st["v_levels"], v_rec * 8 / n_stream, alpha=st["alpha"], has_mean=False, rotate=True,
-                            heads_per_stream=hs)
+                            heads_per_stream=hs, pair_symbols=pair)
     assert tk.info().rec_bytes == k_rec and tv.info().rec_bytes == v_rec
     sm_scale = 1.0 / math.sqrt(128.0)
 
@@ -489,7 +497,7 @@ def run_ours(args):
     comp_bytes = token_heads * (k_b + v_b + 1.0)   # records + amortised INT8 mean byte
     roofline = None
     extra = {}
-    ncu = NCU_HEAD if hs == 1 else NCU_WIDE
+    ncu = (NCU_PAIRS if pair else NCU_HEAD) if hs == 1 else NCU_WIDE
     if args.traffic_bytes is None:
         # every record is read once, so the captured config-2 figure scales with the records' bytes
         args.traffic_bytes = NCU_HEAD["dram_bytes"] * comp_bytes / (NCU_HEAD["token_heads"] * NCU_HEAD["bytes_per_token_head"])
@@ -548,9 +556,58 @@ def run_ours(args):
     except Exception as ex:  # the baseline is context only
         bf16 = {"error": str(ex)}
 
+    # ---- the paired-symbol codec variant on the same workload (context beside the paper codec's line;
+    # `--codec pairs` makes it the line itself): same records' sizes, 64 decode steps per stream instead of 128
+    variants = None
+    if hs == 1 and world == 1 and not pair and not args.no_variants and max(st["k_levels"], st["v_levels"]) <= 9:
+        try:
+            tkp = dq.dq_build_tables(st["k_levels"], k_rec * 8 / 128, alpha=st["alpha"], has_mean=True, rotate=True, pair_symbols=True)
+            tvp = dq.dq_build_tables(st["v_levels"], v_rec * 8 / 128, alpha=st["alpha"], has_mean=False, rotate=True, pair_symbols=True)
+            pc = [new_cache()]
+            for rep_i in range(2):
+                e0.record()
+                dq.dq_encode_tokens(tkp, tvp, w.k, w.v, w.seq_id, w.pos, w.slot, pc[0]["k"], pc[0]["v"], pc[0]["mq"], pc[0]["ms"])
+                e1.record()
+                torch.cuda.synchronize()
+            p_enc_ms = e0.elapsed_time(e1)
+            for _ in range(copies - 1):
+                pc.append({k: v.clone() for k, v in pc[0].items()})
+
+            def pstep(i):
+                c = pc[i % copies]
+                dq.dq_decode_step(tkp, tvp, new_k, new_v, new_slot, w.q, c["k"], c["v"], c["mq"], c["ms"], w.page_table,
+                                  w.seq_lens, Hkv, sm_scale, out, ws)
+            for i in range(5):
+                pstep(i)
+            p_regions = []
+            for r in range(7):
+                torch.cuda.synchronize()
+                e0.record()
+                for i in range(args.steps):
+                    pstep(r * args.steps + i)
+                e1.record()
+                torch.cuda.synchronize()
+                p_regions.append(e0.elapsed_time(e1) / args.steps)
+            dq.dq_profile_enable(1)
+            for i in range(max(16, min(args.steps, 64))):
+                pstep(i)
+            torch.cuda.synchronize()
+            p_kern = dq.dq_profile_read(4096)
+            dq.dq_profile_enable(False)
+            p_ms, p_k = statistics.median(p_regions), statistics.median(p_kern)
+            variants = {"paired_symbols": {
+                "ms_per_step": p_ms, "value": kv_tokens / (p_ms * 1e-3), "unit": UNIT, "kernel_ms": p_k,
+                "compressed_gb_per_s": comp_bytes / (p_k * 1e-3) / 1e9, "frac_of_measured_hbm": comp_bytes / (p_k * 1e-3) / 1e9 / hbm_peak,
+                "prefill_ms": p_enc_ms, "regions": len(p_regions),
+                "note": "opt-in table option pair_symbols: one rANS symbol = the levels of two consecutive values; same record "
+                        "sizes and level counts; parity against the oracle's same variant in tests/test_gpu_variants.py"}}
+            del pc
+        except Exception as ex:   # context only
+            variants = {"paired_symbols": {"error": f"{type(ex).__name__}: {ex}"}}
+
     cpu = None
     if world == 1 and not args.no_cpu_baseline:
-        cpu = time_oracle(args.config, args.budget, streams=args.streams)
+        cpu = time_oracle(args.config, args.budget, streams=args.streams, codec=args.codec)
 
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
@@ -565,6 +622,7 @@ def run_ours(args):
                    {"min": min(cfg.seq_lens), "max": max(cfg.seq_lens), "sum": kv_tokens},
                    "bits_per_elem": args.budget if hs == 1 else round((k_b + v_b + 1.0) * 8 / 256, 3),
                    "streams": "per token-head (128 values)" if hs == 1 else f"per token ({n_stream} values)",
+                   "codec": CODECS[args.codec],
                    "k_rec_bytes": k_rec, "v_rec_bytes": v_rec,
                    "k_levels": st["k_levels"], "v_levels": st["v_levels"],
                    "step": step_desc, **({} if hs == 1 else {"window_closes_in_timed_region": closes_timed}),
@@ -578,6 +636,7 @@ def run_ours(args):
         "encoder": {"token_heads_per_s": 2 * token_heads / (enc_ms * 1e-3), "prefill_ms": enc_ms,
                     "streams": 2 * token_heads // hs},
         "bf16_baseline": bf16,
+        "codec_variants": variants,
     }
     line.update(extra)
     print(json.dumps(line), flush=True)
@@ -637,6 +696,9 @@ def main():
     ap.add_argument("--streams", default="head", choices=["head", "token"],
                     help="head: one stream per (token, KV head), the benchmark's configuration; token: the paper's "
                          "default grouping, one 335 / 235-byte record per token, 8 / 6 levels")
+    ap.add_argument("--codec", default="paper", choices=sorted(CODECS),
+                    help="paper: one level per rANS symbol (Algorithm 2); pairs: the opt-in paired-symbol variant")
+    ap.add_argument("--no-variants", action="store_true", help="skip the codec-variant context measurement")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--separate-calls", action="store_true",
                     help="per token-head streams: dq_encode_tokens + dq_decode_attention instead of dq_decode_step")
