@@ -611,6 +611,7 @@ dq_encode_kernel(const __grid_constant__ DqDevTable TK, const __grid_constant__ 
 constexpr int kB32 = 32;                 // streams per CTA
 constexpr int kB32SymStride = 36;        // bytes per position row (32 streams + pad against bank conflicts)
 constexpr int kB32Warps = DQ_B32_WARPS;
+constexpr int kB32PairMinBlocks = 4;   // paired symbols: the pair search wants 128 registers (7.9 ms against 12.5 ms at 8 CTAs per SM, config 2 prefill)
 template <int MINB, bool PAIR>
 __global__ void __launch_bounds__(kB32Warps * 32, MINB)
 dq_encode_batch32_kernel(const __grid_constant__ DqDevTable TK, const __grid_constant__ DqDevTable TV,
@@ -1156,7 +1157,7 @@ cudaError_t dq_launch_encode(const DqDevTable& tk, const DqDevTable& tv, const D
     const bool pair = tk.pair != 0;   // the caller has checked that both tables agree
     const dim3 kinds(1, (a.do_k && a.do_v) ? 2 : 1);
     if (!a.step_flags && warps >= batch_min_streams(4LL * 148 * kB32 * 4))   // enough streams to fill the GPU several times
-        return dq_launch_pdl(pair ? dq_encode_batch32_kernel<DQ_B32_MINB, true> : dq_encode_batch32_kernel<DQ_B32_MINB, false>,
+        return dq_launch_pdl(pair ? dq_encode_batch32_kernel<kB32PairMinBlocks, true> : dq_encode_batch32_kernel<DQ_B32_MINB, false>,
                              dim3((unsigned)((warps + kB32 - 1) / kB32), kinds.y), dim3(kB32Warps * 32), 0, st, tk, tv, pk, pv, a);
     if (a.step_flags) {   // decode step: big CTAs, so that few SMs are kept from the attention kernel
         constexpr int kStepWarps = DQ_STEP_ENC_WARPS;
