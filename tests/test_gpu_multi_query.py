@@ -25,13 +25,13 @@ def _np(t):
     return t.cpu().numpy()
 
 
-def _run(cfg, q_len, wide_hs=0, resid=None, seed=0):
+def _run(cfg, q_len, wide_hs=0, resid=None, seed=0, pair=False):
     w = workloads.generate(cfg, device="cuda")
     if wide_hs:
         tk, tv, ok, ov = gc.wide_tables(cfg, wide_hs)
         cache = gc.WideGpuCache(w, tk, tv, wide_hs)
     else:
-        tk, tv, ok, ov = gc.tables(cfg)
+        tk, tv, ok, ov = gc.tables(cfg, pair=pair)
         cache = gc.GpuCache(w, ok.rec, ov.rec)
     gc.gpu_encode(w, tk, tv, cache)
     B, Hq, Hkv = cfg.batch, cfg.hq, cfg.hkv
@@ -97,6 +97,13 @@ def test_with_residual_window_gqa2(wide_hs):
     from the compressed tokens (window shorter than q_len, empty window)."""
     cfg = _cfg(2, batch=4, seq_lens=[512, 130, 64, 1000], hq=16)
     _run(cfg, 4, wide_hs=wide_hs, resid=[128, 2, 0, 37])
+
+
+def test_paired_symbols_with_window_and_several_tokens():
+    """The paired-symbol codec variant through the same entry point: several query tokens and a BF16 window."""
+    cfg = _cfg(2, batch=4, seq_lens=[512, 130, 64, 1000], hq=16)
+    _run(cfg, 4, resid=[128, 2, 0, 37], pair=True)
+    _run(_cfg(2, batch=4, seq_lens=[513, 300, 77, 2]), 2, pair=True)
 
 
 def test_single_token_equals_plain_call():
