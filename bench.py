@@ -256,8 +256,6 @@ def run_ours(args):
     st = stream_setup(cfg, args.streams)
     hs, k_rec, v_rec = st["hs"], st["k_rec"], st["v_rec"]
     n_stream = 128 * hs
-    if args.codec == "pairs" and hs > 1:
-        raise SystemExit("--codec pairs is offered for per token-head streams (--streams head)")
     pair = args.codec == "pairs"
     tk = dq.dq_build_tables(st["k_levels"], k_rec * 8 / n_stream, alpha=st["alpha"], has_mean=True, rotate=True,
                             heads_per_stream=hs, pair_symbols=pair)

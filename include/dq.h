@@ -64,8 +64,8 @@
  *       integer by the same rule).  Algorithm 2 then takes 64 steps for 128 values, which is what
  *       halves the decode cost of the attention kernel; Algorithm 1's Drift assigns a pair at a
  *       time (argmin over the M^2 pairs of D_a + D_b + lambda r_ab, lowest u among equals; bracket
- *       16 (max D - min D)).  Same record layout and sizes.  At most 9 levels; per token-head
- *       streams only; key and value tables of one cache must agree.
+ *       16 (max D - min D)).  Same record layout and sizes.  At most 9 levels; key and value tables
+ *       of one cache must agree.
  */
 #ifndef DQ_H_
 #define DQ_H_
@@ -119,7 +119,7 @@ typedef struct {
                        are read by the same decoder) */
     int sigma_bits;  /* 0 or 32: 32-bit final state, state in [2^23, 2^31).  24: 24-bit final state,
                        state in [2^15, 2^23), B = 8C - 24; per token-head streams only */
-    int pair_symbols; /* 1: rANS symbols are pairs of levels (levels <= 9, per token-head streams only) */
+    int pair_symbols; /* 1: rANS symbols are pairs of levels (levels <= 9) */
 } dq_table_opts;
 
 typedef struct {

@@ -86,6 +86,35 @@ __device__ __forceinline__ void decode16_ring(uint32_t& x, uint32_t& ptr, uint32
     }
 }
 
+// Paired-symbol tables: one step decodes the levels of two consecutive channels, 8 steps the 16; an entry is
+// code(b) << 24 | f << 16 | code(a) << 8 | (z - c), code(m) the high byte of fp16(m), so the step's fp16x2 word is
+// the entry with its f and (z - c) bytes cleared.
+template <int ROWS>
+__device__ __forceinline__ void decode16_ring_pairs(uint32_t& x, uint32_t& ptr, uint32_t ring_lane, uint32_t lut, uint32_t one,
+                                                    uint32_t (&packed)[8]) {
+    constexpr uint32_t kMask = (uint32_t)(ROWS - 1) << 7;
+#pragma unroll
+    for (int q4 = 0; q4 < 2; ++q4) {
+        const uint32_t t = ptr << 5;
+        const uint32_t lo = lds32(ring_lane + (t & kMask));
+        const uint32_t hi = lds32(ring_lane + ((t + 128u) & kMask));
+        const uint32_t win = __funnelshift_r(lo, hi, ptr << 3);
+        uint32_t sel = 0x2104u;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const uint32_t e = lds32(dp4a_u32(x, 0x80u, lut));
+            const uint32_t f = dp4a_u32(e, 0x00010000u, 0u);
+            const uint32_t tt = f * (x >> 8);
+            x = dp4a_u32(e, 1u, tt);
+            asm("{.reg .pred p; setp.lt.u32 p, %0, 0x800000; @p prmt.b32 %0, %0, %2, %1; "
+                "@p mad.lo.u32 %1, %3, %3, %1;}"
+                : "+r"(x), "+r"(sel) : "r"(win), "r"(one));
+            packed[4 * q4 + i] = e & 0xff00ff00u;
+        }
+        ptr += sel - 0x2104u;
+    }
+}
+
 // The same 16 symbols for a warp in which some lane lags too far behind the ring: such a lane
 // (`fast` false) takes its window words from the record in global memory (col: its word 0;
 // consecutive words are 16 words apart).  Rare, kept out of line.
@@ -94,9 +123,9 @@ struct Decoded16 {
     uint32_t x, ptr;
 };
 __device__ __noinline__ Decoded16 decode16_mixed(uint32_t x, uint32_t ptr, uint32_t ring_lane, uint32_t ring_mask,
-                                                 uint32_t lut, bool fast, const uint32_t* col, int rec_words) {
+                                                 uint32_t lut, bool fast, const uint32_t* col, int rec_words, bool pairs) {
     Decoded16 r;
-    for (int q4 = 0; q4 < 4; ++q4) {
+    for (int q4 = 0; q4 < (pairs ? 2 : 4); ++q4) {
         const uint32_t t = ptr << 5;
         uint32_t lo, hi;
         if (fast) {
@@ -111,15 +140,19 @@ __device__ __noinline__ Decoded16 decode16_mixed(uint32_t x, uint32_t ptr, uint3
         uint32_t e[4];
         for (int i = 0; i < 4; ++i) {
             e[i] = lds32(lut + ((x & 255u) << 7));
-            x = (e[i] >> 24) * (x >> 8) + (e[i] & 255u);
+            x = (pairs ? (e[i] >> 16) & 255u : e[i] >> 24) * (x >> 8) + (e[i] & 255u);
             if (x < (1u << 23)) {   // at most one byte per symbol
                 x = (x << 8) | (win & 255u);
                 win >>= 8;
                 ++ptr;
             }
         }
-        r.packed[2 * q4] = __byte_perm(e[0], e[1], 0x6521u);
-        r.packed[2 * q4 + 1] = __byte_perm(e[2], e[3], 0x6521u);
+        if (pairs) {
+            for (int i = 0; i < 4; ++i) r.packed[4 * q4 + i] = e[i] & 0xff00ff00u;
+        } else {
+            r.packed[2 * q4] = __byte_perm(e[0], e[1], 0x6521u);
+            r.packed[2 * q4 + 1] = __byte_perm(e[2], e[3], 0x6521u);
+        }
     }
     r.x = x; r.ptr = ptr;
     return r;
@@ -162,7 +195,7 @@ __device__ __forceinline__ const uint32_t* own_column(const Chain& c, const uint
 // One step: 128 channels (one head), 16 at a time; K streams of the current step's head and V
 // streams of the previous step's head decoded in one instruction stream (as in the per-head
 // kernel), each out of its ring.
-template <bool DO_K, bool DO_V>
+template <bool DO_K, bool DO_V, bool PAIRS>
 __device__ __forceinline__ void wide_pass(Chain& ck, Chain& cv, uint32_t ringk, uint32_t ringv, const uint8_t* k_cont,
                                           const uint8_t* v_cont, int rwk, int rwv, uint32_t lutk, uint32_t lutv,
                                           uint32_t one, uint32_t ktile, uint32_t vtile, uint32_t q16, uint32_t obuf,
@@ -186,19 +219,19 @@ __device__ __forceinline__ void wide_pass(Chain& ck, Chain& cv, uint32_t ringk, 
         cp_async_commit();
         uint32_t pk[8], pv[8];
         if (__all_sync(kFullMask, fk && fv)) {
-            if (DO_K) decode16_ring<kRowsK>(ck.x, ck.ptr, ringk_lane, lutk, one, pk);
-            if (DO_V) decode16_ring<kRowsV>(cv.x, cv.ptr, ringv_lane, lutv, one, pv);
+            if (DO_K) { if (PAIRS) decode16_ring_pairs<kRowsK>(ck.x, ck.ptr, ringk_lane, lutk, one, pk); else decode16_ring<kRowsK>(ck.x, ck.ptr, ringk_lane, lutk, one, pk); }
+            if (DO_V) { if (PAIRS) decode16_ring_pairs<kRowsV>(cv.x, cv.ptr, ringv_lane, lutv, one, pv); else decode16_ring<kRowsV>(cv.x, cv.ptr, ringv_lane, lutv, one, pv); }
         } else {   // some lane lags behind its ring: that lane reads global memory (rare, out of line)
             if (DO_K) {
                 const Decoded16 r = decode16_mixed(ck.x, ck.ptr, ringk_lane, (uint32_t)(kRowsK - 1) << 7, lutk, fk,
-                                                   own_column(ck, k_cont, lane), rwk);
+                                                   own_column(ck, k_cont, lane), rwk, PAIRS);
 #pragma unroll
                 for (int i = 0; i < 8; ++i) pk[i] = r.packed[i];
                 ck.x = r.x; ck.ptr = r.ptr;
             }
             if (DO_V) {
                 const Decoded16 r = decode16_mixed(cv.x, cv.ptr, ringv_lane, (uint32_t)(kRowsV - 1) << 7, lutv, fv,
-                                                   own_column(cv, v_cont, lane), rwv);
+                                                   own_column(cv, v_cont, lane), rwv, PAIRS);
 #pragma unroll
                 for (int i = 0; i < 8; ++i) pv[i] = r.packed[i];
                 cv.x = r.x; cv.ptr = r.ptr;
@@ -234,6 +267,7 @@ __device__ __forceinline__ void wide_pass(Chain& ck, Chain& cv, uint32_t ringk, 
     }
 }
 
+template <bool PAIRS>
 __global__ void __launch_bounds__(kWideWarps * 32, 1)
 dq_attention_wide_kernel(const __grid_constant__ DqDevTable TK, const __grid_constant__ DqDevTable TV,
                          const AttnParams p) {
@@ -399,13 +433,13 @@ dq_attention_wide_kernel(const __grid_constant__ DqDevTable TK, const __grid_con
         // its output slot is left out of the merge)
         bool wk = cur.valid && tok0 < cur.len;
         if (wk && wv)
-            wide_pass<true, true>(ck, cv, ringk, ringv, p.k_cont, p.v_cont, rwk, rwv, my_lutk, my_lutv, one, ktile, vtile, q16,
+            wide_pass<true, true, PAIRS>(ck, cv, ringk, ringv, p.k_cont, p.v_cont, rwk, rwv, my_lutk, my_lutv, one, ktile, vtile, q16,
                                   my_obuf, lane, G, sacc, pb_hi, pb_lo);
         else if (wk)
-            wide_pass<true, false>(ck, cv, ringk, ringv, p.k_cont, p.v_cont, rwk, rwv, my_lutk, my_lutv, one, ktile, vtile, q16,
+            wide_pass<true, false, PAIRS>(ck, cv, ringk, ringv, p.k_cont, p.v_cont, rwk, rwv, my_lutk, my_lutv, one, ktile, vtile, q16,
                                    my_obuf, lane, G, sacc, pb_hi, pb_lo);
         else if (wv)
-            wide_pass<false, true>(ck, cv, ringk, ringv, p.k_cont, p.v_cont, rwk, rwv, my_lutk, my_lutv, one, ktile, vtile, q16,
+            wide_pass<false, true, PAIRS>(ck, cv, ringk, ringv, p.k_cont, p.v_cont, rwk, rwv, my_lutk, my_lutv, one, ktile, vtile, q16,
                                    my_obuf, lane, G, sacc, pb_hi, pb_lo);
 
         // The item descriptors are derived again rather than kept in registers across the pass.
@@ -569,7 +603,8 @@ int dq_attn_wide_pick_warps(const DqDevTable& tk, const DqDevTable& tv, int B, i
 cudaError_t dq_launch_attention_wide_main(const DqDevTable& tk, const DqDevTable& tv, const AttnParams& p, int nw,
                                           int sm_count, cudaStream_t st) {
     const int smem_bytes = wide_smem_bytes(nw, p.B, p.G);
-    cudaError_t e = cudaFuncSetAttribute(dq_attention_wide_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes);
+    auto kernel = tk.pair ? dq_attention_wide_kernel<true> : dq_attention_wide_kernel<false>;
+    cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes);
     if (e != cudaSuccess) return e;
-    return dq_launch_pdl(dq_attention_wide_kernel, dim3(sm_count), dim3(nw * 32), (size_t)smem_bytes, st, tk, tv, p);
+    return dq_launch_pdl(kernel, dim3(sm_count), dim3(nw * 32), (size_t)smem_bytes, st, tk, tv, p);
 }

@@ -89,17 +89,29 @@ dq_decode_tokens_wide_kernel(const __grid_constant__ DqDevTable T, const uint8_t
             msc = mean_scale[mi];
         }
         const size_t dst = ((size_t)t * Hkv + h) * DQ_HEAD_DIM;
-        for (int j = 0; j < DQ_HEAD_DIM; ++j) {
-            const uint32_t e = T.lut[x & 255u];
-            x = (e >> 24) * (x >> 8) + (e & 255u);
-            if (x < (1u << 23) && ptr < T.rec) x = (x << 8) | byte_at(ptr++);
-            const float lvl = __half2float(__ushort_as_half((unsigned short)((e >> 8) & 0xffffu)));
+        auto emit = [&](int j, float lvl) {
             if (symbols) symbols[dst + j] = (uint8_t)(int)lvl;
             if (dequant) {
                 float v = __fmaf_rn(lvl, s, o);
                 if (mq) v = __fadd_rn(v, __fmul_rn(msc, (float)mq[j]));
                 dequant[dst + j] = v;
             }
+        };
+        if (T.pair) {   // one step per pair of values: entry = code(b) << 24 | f << 16 | code(a) << 8 | (z - c)
+            for (int j = 0; j < DQ_HEAD_DIM; j += 2) {
+                const uint32_t e = T.lut[x & 255u];
+                x = ((e >> 16) & 255u) * (x >> 8) + (e & 255u);
+                if (x < (1u << 23) && ptr < T.rec) x = (x << 8) | byte_at(ptr++);
+                emit(j, __half2float(__ushort_as_half((unsigned short)(e & 0xff00u))));
+                emit(j + 1, __half2float(__ushort_as_half((unsigned short)((e >> 16) & 0xff00u))));
+            }
+            continue;
+        }
+        for (int j = 0; j < DQ_HEAD_DIM; ++j) {
+            const uint32_t e = T.lut[x & 255u];
+            x = (e >> 24) * (x >> 8) + (e & 255u);
+            if (x < (1u << 23) && ptr < T.rec) x = (x << 8) | byte_at(ptr++);
+            emit(j, __half2float(__ushort_as_half((unsigned short)((e >> 8) & 0xffffu))));
         }
     }
 }

@@ -736,7 +736,7 @@ struct WideShared {
     uint32_t len[2][DQ_MAX_STREAM_HEADS];
     double sa[DQ_MAX_STREAM_HEADS], sb[DQ_MAX_STREAM_HEADS];
     int sm[DQ_MAX_STREAM_HEADS], smm[DQ_MAX_STREAM_HEADS];
-    uint2 ent[DQ_MAX_LEVELS];   // rANS encode entries {rcp, bias | (256 - f) << 10 | rsh << 19}
+    uint2 ent[DQ_MAX_PAIRS];    // rANS encode entries {rcp, bias | (256 - f) << 10 | rsh << 19} (levels, or pairs u = a M + b)
 };
 
 // Function Drift of Algorithm 1 for a stream held by hs warps; same arithmetic as drift_m, with
@@ -834,21 +834,133 @@ __device__ __forceinline__ uint32_t drift_wide(const EncTable& T, WideShared& W,
     return len;
 }
 
-// Table fields of one tensor kind into shared memory (first 16 threads + thread 0).
+// Drift for paired symbols on a stream held by hs warps: the pair search of drift_pair_m with the extrema of D
+// and the code length taken over the whole stream, as in drift_wide_m.
+template <int M>
+__device__ __noinline__ uint32_t drift_wide_pair_m(const EncTable& T, WideShared& W, int hs, int wib, uint32_t& parity,
+                                                   float z0, float z1, float z2, float z3, float s, float o,
+                                                   uint32_t& sym_packed) {
+    const float z[4] = {z0, z1, z2, z3};
+    const int lane = threadIdx.x & 31;
+    float D[4][M];
+    float maxD = -INFINITY, minD = INFINITY;
+#pragma unroll
+    for (int m = 0; m < M; ++m) {
+        const float tm = __fmaf_rn((float)m, s, o);
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            const float d = __fsub_rn(z[e], tm);
+            D[e][m] = __fmul_rn(d, d);
+            maxD = fmaxf(maxD, D[e][m]);
+            minD = fminf(minD, D[e][m]);
+        }
+    }
+#pragma unroll
+    for (int d = 16; d >= 1; d >>= 1) {
+        maxD = fmaxf(maxD, __shfl_xor_sync(kFull, maxD, d));
+        minD = fminf(minD, __shfl_xor_sync(kFull, minD, d));
+    }
+    if (lane == 0) { W.fmax[parity][wib] = maxD; W.fmin[parity][wib] = minD; }
+    __syncthreads();
+    for (int w = 0; w < hs; ++w) { maxD = fmaxf(maxD, W.fmax[parity][w]); minD = fminf(minD, W.fmin[parity][w]); }
+    parity ^= 1u;
+    const uint32_t budget = (uint32_t)T.budget_bits << 16;
+    float lam_hi = __fmul_rn(16.0f, __fsub_rn(maxD, minD));
+    float lam_lo = __fmul_rn(lam_hi, 0x1p-40f);
+    uint32_t len = 0, psym[2] = {0u, 0u};
+    float lam_e = lam_hi;
+    if (T.early_exit)
+        for (int i = 0; i < 12; ++i) lam_e = __fsqrt_rn(__fmul_rn(lam_lo, lam_e));
+#pragma unroll 1
+    for (int it = T.early_exit ? -1 : 0; it <= 12; ++it) {
+        const float lam = (it < 0) ? lam_e : (it < 12) ? __fsqrt_rn(__fmul_rn(lam_lo, lam_hi)) : lam_hi;
+        uint32_t cost_sum = 0;
+#pragma unroll
+        for (int p = 0; p < 2; ++p) {
+            float rc[M];
+            uint32_t rkey[M];
+#pragma unroll
+            for (int a = 0; a < M; ++a) {
+                float c[M];
+                uint32_t key[M];
+#pragma unroll
+                for (int b = 0; b < M; ++b) {
+                    const uint2 e = T.prk[a * M + b];
+                    c[b] = __fmaf_rn(lam, __uint_as_float(e.x), __fadd_rn(D[2 * p][a], D[2 * p + 1][b]));
+                    key[b] = e.y;
+                }
+#pragma unroll
+                for (int w = 1; w < M; w <<= 1)
+#pragma unroll
+                    for (int b = 0; b + w < M; b += 2 * w)
+                        if (c[b + w] < c[b]) { c[b] = c[b + w]; key[b] = key[b + w]; }
+                rc[a] = c[0];
+                rkey[a] = key[0];
+            }
+#pragma unroll
+            for (int w = 1; w < M; w <<= 1)
+#pragma unroll
+                for (int a = 0; a + w < M; a += 2 * w)
+                    if (rc[a + w] < rc[a]) { rc[a] = rc[a + w]; rkey[a] = rkey[a + w]; }
+            psym[p] = rkey[0];
+            cost_sum += rkey[0];
+        }
+        const uint32_t wl = __reduce_add_sync(kFull, cost_sum >> 8);
+        if (lane == 0) W.len[parity][wib] = wl;
+        __syncthreads();
+        len = 0;
+        for (int w = 0; w < hs; ++w) len += W.len[parity][w];
+        parity ^= 1u;
+        if (it < 0) {
+            if (len <= budget) break;   // uniform across the CTA
+        } else if (it < 12) {
+            if (len <= budget) lam_hi = lam; else lam_lo = lam;
+        }
+    }
+    const uint32_t u0 = psym[0] & 0xffu, u1 = psym[1] & 0xffu;
+    sym_packed = (u0 / M) | ((u0 % M) << 8) | ((u1 / M) << 16) | ((u1 % M) << 24);
+    return len;
+}
+
+__device__ __forceinline__ uint32_t drift_wide_pair(const EncTable& T, WideShared& W, int hs, int wib, uint32_t& parity,
+                                                    const float (&z)[4], float s, float o, uint32_t (&sym)[4]) {
+    uint32_t packed = 0, len = 0;
+    switch (T.M) {   // uniform across the CTA
+#define DQ_DRIFT_CASE(M_) case M_: len = drift_wide_pair_m<M_>(T, W, hs, wib, parity, z[0], z[1], z[2], z[3], s, o, packed); break;
+        DQ_DRIFT_CASE(2) DQ_DRIFT_CASE(3) DQ_DRIFT_CASE(4) DQ_DRIFT_CASE(5) DQ_DRIFT_CASE(6) DQ_DRIFT_CASE(7)
+        DQ_DRIFT_CASE(8) DQ_DRIFT_CASE(9)
+#undef DQ_DRIFT_CASE
+        default: break;
+    }
+#pragma unroll
+    for (int e = 0; e < 4; ++e) sym[e] = (packed >> (8 * e)) & 0xffu;
+    return len;
+}
+
+// Table fields of one tensor kind into shared memory (threads 0 .. DQ_MAX_PAIRS - 1 of 3 rounds of 32 + thread 0;
+// a CTA has at least 64 threads).
 __device__ __forceinline__ void load_wide_table(EncTable& T, WideShared& W, const DqDevTable& TK, const DqDevTable& TV,
-                                                bool is_v) {
+                                                const DqPairEnc& PK, const DqPairEnc& PV, bool is_v) {
+    const int pair = is_v ? TV.pair : TK.pair;
     if (threadIdx.x < DQ_MAX_LEVELS) {
         const int i = threadIdx.x;
         T.r[i] = is_v ? TV.r[i] : TK.r[i];
         T.R[i] = is_v ? TV.R[i] : TK.R[i];
-        W.ent[i] = make_uint2(is_v ? TV.enc_rcp[i] : TK.enc_rcp[i], is_v ? TV.enc_aux[i] : TK.enc_aux[i]);
+        if (!pair) W.ent[i] = make_uint2(is_v ? TV.enc_rcp[i] : TK.enc_rcp[i], is_v ? TV.enc_aux[i] : TK.enc_aux[i]);
     }
+    if (pair)
+        for (int i = threadIdx.x; i < DQ_MAX_PAIRS; i += blockDim.x) {
+            W.ent[i] = make_uint2(is_v ? PV.enc_rcp[i] : PK.enc_rcp[i], is_v ? PV.enc_aux[i] : PK.enc_aux[i]);
+            T.prk[i] = make_uint2(__float_as_uint(is_v ? PV.r[i] : PK.r[i]), ((is_v ? PV.R[i] : PK.R[i]) << 8) | (uint32_t)i);
+        }
     if (threadIdx.x == 0) {
         T.M = is_v ? TV.M : TK.M; T.rec = is_v ? TV.rec : TK.rec; T.mstar = is_v ? TV.mstar : TK.mstar;
         T.budget_bits = is_v ? TV.budget_bits : TK.budget_bits;
         T.has_mean = is_v ? TV.has_mean : TK.has_mean; T.rotate = is_v ? TV.rotate : TK.rotate;
         T.early_exit = is_v ? TV.early_exit : TK.early_exit; T.sigma = 32;   // token-wide streams keep the 32-bit state
-        T.pair = 0; T.central = (uint32_t)T.mstar * 0x01010101u;   // and single levels as symbols
+        T.pair = pair;
+        const uint32_t ms = (uint32_t)T.mstar, us = (uint32_t)(is_v ? TV.ustar : TK.ustar), M = (uint32_t)T.M;
+        T.central = pair ? (us / M) * 0x00010001u + (us % M) * 0x01000100u : ms * 0x01010101u;
     }
 }
 
@@ -861,6 +973,9 @@ struct WideQuantised {
 // (warp w owns head grp * hs + w, lane l its elements 4l .. 4l+3 = stream positions
 // 128 w + 4 l + e): rotation, mean removal, min-max grid, drift, refit, fp16 metadata, second
 // drift.  The final symbols go to s_sym (visible to the whole CTA on return).
+// PAIR: rANS symbols are pairs of levels; s_sym then receives the pair index u = a M + b of the values
+// (2i, 2i + 1) at symbol position i (n / 2 positions).
+template <bool PAIR>
 __device__ __forceinline__ WideQuantised wide_quantise(const EncTable& T, WideShared& W, const DqEncodeArgs& a,
                                                        bool is_v, int t, int grp, uint8_t* s_sym, int sym_stride,
                                                        uint32_t& parity) {
@@ -920,7 +1035,7 @@ __device__ __forceinline__ WideQuantised wide_quantise(const EncTable& T, WideSh
     if (!degenerate) {   // uniform across the CTA: mx and mn are stream-wide
         const float o = mn;                                         // FitMinMax, Eq. (affine_token)
         const float s = __fdiv_rn(__fsub_rn(mx, mn), (float)(T.M - 1));
-        drift_wide(T, W, hs, wib, parity, z, s, o, sym);
+        if (PAIR) drift_wide_pair(T, W, hs, wib, parity, z, s, o, sym); else drift_wide(T, W, hs, wib, parity, z, s, o, sym);
         // Refit: head sums as in the per-head encoder (lane order, then xor butterfly), added in head order
         double sa = (double)z[0], sb = __dmul_rn((double)sym[0], (double)z[0]);
         int sm = (int)sym[0], smm = (int)(sym[0] * sym[0]);
@@ -965,10 +1080,11 @@ __device__ __forceinline__ WideQuantised wide_quantise(const EncTable& T, WideSh
         }
         if (!(sf > 0.0f)) degenerate = true;
         else {
-            const uint32_t len = drift_wide(T, W, hs, wib, parity, z, sf, of, sym);   // second Drift, fp16 grid
+            const uint32_t len = PAIR ? drift_wide_pair(T, W, hs, wib, parity, z, sf, of, sym)
+                                      : drift_wide(T, W, hs, wib, parity, z, sf, of, sym);   // second Drift, fp16 grid
             if (len > ((uint32_t)T.budget_bits << 16)) {
 #pragma unroll
-                for (int e = 0; e < 4; ++e) sym[e] = (uint32_t)T.mstar;
+                for (int e = 0; e < 4; ++e) sym[e] = (T.central >> (8 * e)) & 0xffu;
                 flags |= 1u;
             }
         }
@@ -977,12 +1093,18 @@ __device__ __forceinline__ WideQuantised wide_quantise(const EncTable& T, WideSh
         s16 = __ushort_as_half(0);
         o16 = __float2half_rn(mn);
 #pragma unroll
-        for (int e = 0; e < 4; ++e) sym[e] = (uint32_t)T.mstar;
+        for (int e = 0; e < 4; ++e) sym[e] = (T.central >> (8 * e)) & 0xffu;
         flags |= 2u;
     }
     // symbol of stream position j goes to s_sym[j * sym_stride]
+    if (PAIR) {
+        const uint32_t M = (uint32_t)T.M;
+        s_sym[(wib * (kN / 2) + 2 * lane) * sym_stride] = (uint8_t)(sym[0] * M + sym[1]);
+        s_sym[(wib * (kN / 2) + 2 * lane + 1) * sym_stride] = (uint8_t)(sym[2] * M + sym[3]);
+    } else {
 #pragma unroll
-    for (int e = 0; e < 4; ++e) s_sym[(wib * kN + 4 * lane + e) * sym_stride] = (uint8_t)sym[e];
+        for (int e = 0; e < 4; ++e) s_sym[(wib * kN + 4 * lane + e) * sym_stride] = (uint8_t)sym[e];
+    }
     __syncthreads();
     WideQuantised r;
     r.hdr0 = (uint32_t)__half_as_ushort(s16) | ((uint32_t)__half_as_ushort(o16) << 16);
@@ -1016,9 +1138,10 @@ __device__ __forceinline__ void add_status(uint32_t* status, uint32_t flags, int
 
 // One CTA of hs warps per stream (token, group of hs KV heads): lowest latency, used when a
 // call holds few streams (a decode step).  blockIdx.y selects the tensor kind.
+template <bool PAIR>
 __global__ void __launch_bounds__(DQ_MAX_STREAM_HEADS * 32)
 dq_encode_wide_kernel(const __grid_constant__ DqDevTable TK, const __grid_constant__ DqDevTable TV,
-                      const DqEncodeArgs a) {
+                      const __grid_constant__ DqPairEnc PK, const __grid_constant__ DqPairEnc PV, const DqEncodeArgs a) {
     __shared__ EncTable T;
     __shared__ __align__(16) WideShared W;
     __shared__ uint8_t s_bytes[DQ_MAX_WIDE_REC_BYTES];
@@ -1026,18 +1149,18 @@ dq_encode_wide_kernel(const __grid_constant__ DqDevTable TK, const __grid_consta
     __shared__ uint32_t s_final[2];   // final state, bytes emitted
     dqdev::pdl_launch_dependents();
     const bool is_v = a.do_k ? (blockIdx.y == 1) : true;
-    load_wide_table(T, W, TK, TV, is_v);
+    load_wide_table(T, W, TK, TV, PK, PV, is_v);
     __syncthreads();
     dqdev::pdl_wait_prior_grid();
     const int lane = threadIdx.x & 31, wib = threadIdx.x >> 5;
     const int hs = blockDim.x >> 5, groups = a.Hkv / hs;
     const int t = (int)(blockIdx.x / groups), grp = (int)(blockIdx.x % groups);
     uint32_t parity = 0;
-    const WideQuantised q = wide_quantise(T, W, a, is_v, t, grp, s_sym, 1, parity);
+    const WideQuantised q = wide_quantise<PAIR>(T, W, a, is_v, t, grp, s_sym, 1, parity);
     if (wib == 0) {
         uint32_t xs;
         int k;
-        rans_encode_warp(W.ent, s_sym, hs * kN, dqdev::smem_addr(s_bytes), DQ_MAX_WIDE_REC_BYTES, lane, xs, k);
+        rans_encode_warp(W.ent, s_sym, PAIR ? hs * (kN / 2) : hs * kN, dqdev::smem_addr(s_bytes), DQ_MAX_WIDE_REC_BYTES, lane, xs, k);
         if (lane == 0) { s_final[0] = xs; s_final[1] = (uint32_t)k; }
     }
     __syncthreads();
@@ -1057,16 +1180,17 @@ __host__ __device__ inline int wide_batch_smem(int hs, int rec) { return hs * kN
 #ifndef DQ_ENCW_MINB
 #define DQ_ENCW_MINB 3
 #endif
-__global__ void __launch_bounds__(DQ_MAX_STREAM_HEADS * 32, DQ_ENCW_MINB)
+template <bool PAIR>
+__global__ void __launch_bounds__(DQ_MAX_STREAM_HEADS * 32, PAIR ? 2 : DQ_ENCW_MINB)
 dq_encode_wide_batch_kernel(const __grid_constant__ DqDevTable TK, const __grid_constant__ DqDevTable TV,
-                            const DqEncodeArgs a) {
+                            const __grid_constant__ DqPairEnc PK, const __grid_constant__ DqPairEnc PV, const DqEncodeArgs a) {
     extern __shared__ __align__(16) uint8_t dyn[];
     __shared__ EncTable T;
     __shared__ __align__(16) WideShared W;
     __shared__ uint32_t s_hdr[kWB], s_flags[kWB], s_xs[kWB], s_k[kWB];
     dqdev::pdl_launch_dependents();
     const bool is_v = a.do_k ? (blockIdx.y == 1) : true;
-    load_wide_table(T, W, TK, TV, is_v);
+    load_wide_table(T, W, TK, TV, PK, PV, is_v);
     __syncthreads();
     dqdev::pdl_wait_prior_grid();
     const int lane = threadIdx.x & 31, wib = threadIdx.x >> 5;
@@ -1080,14 +1204,14 @@ dq_encode_wide_batch_kernel(const __grid_constant__ DqDevTable TK, const __grid_
     uint32_t parity = 0;
     for (int i = 0; i < ns; ++i) {
         const long long sid = first + i;
-        const WideQuantised q = wide_quantise(T, W, a, is_v, (int)(sid / groups), (int)(sid % groups), s_symT + i,
+        const WideQuantised q = wide_quantise<PAIR>(T, W, a, is_v, (int)(sid / groups), (int)(sid % groups), s_symT + i,
                                               kWBSymStride, parity);
         if (threadIdx.x == 0) { s_hdr[i] = q.hdr0; s_flags[i] = q.flags; }
     }
     if (wib == 0 && lane < ns) {   // rANS, Eq. (rans) Enc on symbols n-1 .. 0; lane = stream
         uint32_t xs = kL, k = 0;
 #pragma unroll 4
-        for (int j = n - 1; j >= 0; --j) {
+        for (int j = (PAIR ? n / 2 : n) - 1; j >= 0; --j) {
             const uint32_t m = s_symT[j * kWBSymStride + lane];
             const uint2 e = W.ent[m];
             const uint32_t cmpl = (e.y >> 10) & 511u;
@@ -1145,13 +1269,16 @@ cudaError_t dq_launch_encode(const DqDevTable& tk, const DqDevTable& tv, const D
     if (tk.hs > 1) {   // token-wide streams: CTAs of hs warps; few streams: one per CTA, many: 32 per CTA
         const long long streams = warps / tk.hs;
         const dim3 kinds_y(1, (a.do_k && a.do_v) ? 2 : 1);
+        const bool wpair = tk.pair != 0;   // the caller has checked that both tables agree
         if (streams < batch_min_streams(3LL * 148 * kWB))
-            return dq_launch_pdl(dq_encode_wide_kernel, dim3((unsigned)streams, kinds_y.y), dim3(tk.hs * 32), 0, st, tk, tv, a);
+            return dq_launch_pdl(wpair ? dq_encode_wide_kernel<true> : dq_encode_wide_kernel<false>, dim3((unsigned)streams, kinds_y.y),
+                                 dim3(tk.hs * 32), 0, st, tk, tv, pk, pv, a);
         const int smem = wide_batch_smem(tk.hs, tk.rec > tv.rec ? tk.rec : tv.rec);
-        const cudaError_t e = cudaFuncSetAttribute(dq_encode_wide_batch_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+        auto batch_kernel = wpair ? dq_encode_wide_batch_kernel<true> : dq_encode_wide_batch_kernel<false>;
+        const cudaError_t e = cudaFuncSetAttribute(batch_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
         if (e != cudaSuccess) return e;
-        return dq_launch_pdl(dq_encode_wide_batch_kernel, dim3((unsigned)((streams + kWB - 1) / kWB), kinds_y.y),
-                             dim3(tk.hs * 32), (size_t)smem, st, tk, tv, a);
+        return dq_launch_pdl(batch_kernel, dim3((unsigned)((streams + kWB - 1) / kWB), kinds_y.y),
+                             dim3(tk.hs * 32), (size_t)smem, st, tk, tv, pk, pv, a);
     }
     const unsigned blocks = (unsigned)((warps + kEncWarps - 1) / kEncWarps);
     const bool pair = tk.pair != 0;   // the caller has checked that both tables agree

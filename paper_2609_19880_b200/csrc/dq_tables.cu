@@ -179,7 +179,7 @@ int dq_host_build(int levels, double bits_per_elem, const dq_table_opts* opts, d
     if (sigma != 32 && sigma != 24) return DQ_ERR_ARG;
     if (sigma == 24 && hs > 1) return DQ_ERR_UNSUPPORTED;   // the short state is offered for 128-value streams
     const bool pair = opts->pair_symbols != 0;
-    if (pair && (hs > 1 || levels > DQ_MAX_PAIR_LEVELS)) return DQ_ERR_UNSUPPORTED;
+    if (pair && levels > DQ_MAX_PAIR_LEVELS) return DQ_ERR_UNSUPPORTED;
 
     dq_table_info& t = out->info;
     std::memset(out, 0, sizeof *out);

@@ -107,14 +107,14 @@ def check_attention(out_bf16, out_f32, ref, rows=None):
 # ---- token-wide streams (heads_per_stream = hs > 1): the library stores records word-interleaved
 # per page, uint8 [pages][groups][rec_words][16][4]; the oracle keeps [pages][groups][16][rec].
 
-def wide_tables(cfg, hs, k_rec=335, v_rec=235, k_levels=8, v_levels=6, alpha=1.4, early_exit=False):
+def wide_tables(cfg, hs, k_rec=335, v_rec=235, k_levels=8, v_levels=6, alpha=1.4, early_exit=False, pair=False):
     n = 128 * hs
     tk = dq.dq_build_tables(k_levels, k_rec * 8 / n, alpha=alpha, has_mean=True, rotate=True, heads_per_stream=hs,
-                            drift_early_exit=early_exit)
+                            drift_early_exit=early_exit, pair_symbols=pair)
     tv = dq.dq_build_tables(v_levels, v_rec * 8 / n, alpha=alpha, has_mean=False, rotate=True, heads_per_stream=hs,
-                            drift_early_exit=early_exit)
-    ok = oracle.build_table(k_levels, n, k_rec, alpha, has_mean=True, rotate=True, early_exit=early_exit)
-    ov = oracle.build_table(v_levels, n, v_rec, alpha, has_mean=False, rotate=True, early_exit=early_exit)
+                            drift_early_exit=early_exit, pair_symbols=pair)
+    ok = oracle.build_table(k_levels, n, k_rec, alpha, has_mean=True, rotate=True, early_exit=early_exit, pair=pair)
+    ov = oracle.build_table(v_levels, n, v_rec, alpha, has_mean=False, rotate=True, early_exit=early_exit, pair=pair)
     assert tk.info().rec_bytes == k_rec and tv.info().rec_bytes == v_rec
     return tk, tv, ok, ov
 

@@ -38,14 +38,19 @@ CASES = {
     "ragged_shuffled": (4, dict(batch=5, seq_lens=[200, 16, 333, 1, 1030]), 8, (335, 235, 8, 6)),
     "pairs_of_heads": (2, dict(batch=2, seq_lens=[130, 64]), 2, (86, 60, 6, 4)),
     "g7_four_heads": (5, dict(batch=2, seq_lens=[640, 129]), 4, (170, 120, 8, 6)),
+    # the paired-symbol codec variant (a sixth field): one rANS symbol = the levels of two consecutive values
+    "paper_default_pairs": (2, dict(batch=3, seq_lens=[512, 300, 77]), 8, (335, 235, 8, 6), True),
+    "ragged_shuffled_pairs": (4, dict(batch=5, seq_lens=[200, 16, 333, 1, 1030]), 8, (335, 235, 8, 6), True),
+    "pairs_of_heads_pairs": (2, dict(batch=2, seq_lens=[130, 64]), 2, (86, 60, 6, 4), True),
+    "g7_four_heads_pairs": (5, dict(batch=2, seq_lens=[640, 129]), 4, (170, 120, 9, 5), True),
 }
 
 
 def _setup(name):
-    idx, over, hs, (kr, vr, mk, mv) = CASES[name]
+    idx, over, hs, (kr, vr, mk, mv) = CASES[name][:4]
     cfg = _cfg(idx, **over)
     w = workloads.generate(cfg, device="cuda")
-    tk, tv, ok, ov = gc.wide_tables(cfg, hs, kr, vr, mk, mv)
+    tk, tv, ok, ov = gc.wide_tables(cfg, hs, kr, vr, mk, mv, pair=len(CASES[name]) > 4)
     return cfg, w, hs, tk, tv, ok, ov
 
 
@@ -140,10 +145,11 @@ def test_attention_edge_lengths():
     assert not out[0].any()
 
 
-def test_lagging_streams_take_the_global_path():
+@pytest.mark.parametrize("name", ["paper_default", "paper_default_pairs"])
+def test_lagging_streams_take_the_global_path(name):
     """Keys whose streams stop consuming bytes early (constant tokens between ordinary ones) fall
     far behind their warp's ring and must be served from global memory with the same result."""
-    cfg, w, hs, tk, tv, ok, ov = _setup("paper_default")
+    cfg, w, hs, tk, tv, ok, ov = _setup(name)
     w.k[5:400:7] = 0.0
     w.v[9:400:11] = 0.0
     cache = gc.WideGpuCache(w, tk, tv, hs)

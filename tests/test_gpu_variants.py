@@ -91,6 +91,31 @@ def test_early_exit_token_wide_records_match_oracle():
         assert np.array_equal(gc.from_interleaved(_np(cache.v_cont), ov.rec), vc)
 
 
+@pytest.mark.parametrize("early_exit", [False, True])
+def test_pair_symbols_token_wide_both_encoders(early_exit):
+    """Token-wide streams (8 heads, 8 / 6 levels) with paired symbols: the one-stream-per-CTA encoder and the
+    batch encoder write the oracle's records; attention over them within tolerance."""
+    cfg = workloads.make_config(2, scale=1 / 16)
+    for batch in (False, True):
+        w = workloads.generate(cfg, device="cuda")
+        tk, tv, ok, ov = gc.wide_tables(cfg, 8, early_exit=early_exit, pair=True)
+        cache = gc.WideGpuCache(w, tk, tv, 8)
+        if batch:
+            dq.dq_set_option(dq.OPT_ENCODE_BATCH_MIN, 0)
+        try:
+            gc.gpu_encode(w, tk, tv, cache)
+            torch.cuda.synchronize()
+        finally:
+            dq.dq_set_option(dq.OPT_ENCODE_BATCH_MIN, -1)
+        kc, vc, mq, ms, sk, sv = gc.oracle_encode_wide(w, ok, ov, 8)
+        assert np.array_equal(gc.from_interleaved(_np(cache.k_cont), ok.rec), kc)
+        assert np.array_equal(gc.from_interleaved(_np(cache.v_cont), ov.rec), vc)
+        out, out32 = gc.gpu_attention(w, tk, tv, cache)
+        ref = oracle.attention(ok, ov, workloads.bf16_bits(w.q), kc, vc, mq, ms, _np(w.page_table), _np(w.seq_lens),
+                               cfg.hkv, gc.SM_SCALE)
+        gc.check_attention(out, out32, ref)
+
+
 def test_early_exit_prefill_config2_full_size():
     """Every record of configuration 2's prefill with the early exit, against the oracle; encoder time beside the default's."""
     cfg = workloads.make_config(2)

@@ -73,8 +73,11 @@ def test_pair_tables_limits(L):
     with pytest.raises(dq.DqError) as err:
         dq.dq_build_tables(10, 60 * 8 / 128, pair_symbols=True)            # levels 0..8 only
     assert err.value.code == -3
+    t = dq.dq_build_tables(8, 335 * 8 / 1024, heads_per_stream=8, pair_symbols=True)   # token-wide streams take pairs too
+    o = oracle.build_table(8, 1024, 335, 1.4, pair=True)
+    assert [t.info().pair_f[u] for u in range(64)] == o.pair_freqs() and t.info().ustar == o.ustar
     with pytest.raises(dq.DqError) as err:
-        dq.dq_build_tables(8, 335 * 8 / 1024, heads_per_stream=8, pair_symbols=True)
+        dq.dq_build_tables(8, 335 * 8 / 1024, heads_per_stream=8, pair_symbols=True, sigma_bits=24)
     assert err.value.code == -3
     with pytest.raises(dq.DqError) as err:
         dq.dq_build_tables(9, 20 * 8 / 128, pair_symbols=True)             # the all-central pairs do not fit
