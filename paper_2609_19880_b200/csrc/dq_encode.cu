@@ -283,8 +283,8 @@ __device__ __forceinline__ uint32_t drift(const EncTable& T, const float (&z)[4]
 
 // Drift for the paired-symbol variant: a lane's values (0, 1) and (2, 3) are two rANS symbols; each takes
 // the pair u = a M + b that minimises (D_a + D_b) + lambda r_u, the lowest u among equal costs (rows a in
-// ascending order, each reduced left to right, then the row winners: the same winner as an ascending scan
-// with a strict comparison).  Bracket: hi = 16 (max D - min D), D over single values as above.
+// ascending order, each reduced pairwise with the left operand winning ties, a later row replacing the best
+// only when strictly cheaper: the same winner as an ascending scan with a strict comparison).  Bracket: hi = 16 (max D - min D), D over single values as above.
 template <int M>
 __device__ __noinline__ uint32_t drift_pair_m(const EncTable& T, float z0, float z1, float z2, float z3, float s, float o,
                                               uint32_t& sym_packed) {
@@ -341,7 +341,7 @@ __device__ __noinline__ uint32_t drift_pair_m(const EncTable& T, float z0, float
                 rkey[a] = key[0];
             }
 #pragma unroll
-            for (int w = 1; w < M; w <<= 1)
+            for (int w = 1; w < M; w <<= 1)   // row winners, the left (lower a) operand wins ties
 #pragma unroll
                 for (int a = 0; a + w < M; a += 2 * w)
                     if (rc[a + w] < rc[a]) { rc[a] = rc[a + w]; rkey[a] = rkey[a + w]; }
@@ -877,8 +877,8 @@ __device__ __noinline__ uint32_t drift_wide_pair_m(const EncTable& T, WideShared
         uint32_t cost_sum = 0;
 #pragma unroll
         for (int p = 0; p < 2; ++p) {
-            float rc[M];
-            uint32_t rkey[M];
+            float best = 0.f;
+            uint32_t bkey = 0u;
 #pragma unroll
             for (int a = 0; a < M; ++a) {
                 float c[M];
@@ -894,16 +894,10 @@ __device__ __noinline__ uint32_t drift_wide_pair_m(const EncTable& T, WideShared
 #pragma unroll
                     for (int b = 0; b + w < M; b += 2 * w)
                         if (c[b + w] < c[b]) { c[b] = c[b + w]; key[b] = key[b + w]; }
-                rc[a] = c[0];
-                rkey[a] = key[0];
+                if (a == 0 || c[0] < best) { best = c[0]; bkey = key[0]; }   // an earlier row keeps equal costs
             }
-#pragma unroll
-            for (int w = 1; w < M; w <<= 1)
-#pragma unroll
-                for (int a = 0; a + w < M; a += 2 * w)
-                    if (rc[a + w] < rc[a]) { rc[a] = rc[a + w]; rkey[a] = rkey[a + w]; }
-            psym[p] = rkey[0];
-            cost_sum += rkey[0];
+            psym[p] = bkey;
+            cost_sum += bkey;
         }
         const uint32_t wl = __reduce_add_sync(kFull, cost_sum >> 8);
         if (lane == 0) W.len[parity][wib] = wl;
