@@ -44,6 +44,8 @@ NCU_PAIRS = {"instr_per_symbol": 9.96, "issue_active": 0.560,
              "source": "the ncu summary of dq_attention_kernel with paired-symbol tables on config 2 under profiles/"}
 NCU_WIDE = {"instr_per_symbol": 19.2, "issue_active": 0.641,
             "source": "the ncu summary of dq_attention_wide_kernel on config 2 under profiles/"}
+NCU_WIDE_PAIRS = {"instr_per_symbol": 13.3, "issue_active": 0.626,
+                  "source": "the ncu summary of dq_attention_wide_kernel (paired-symbol section) on config 2 under profiles/"}
 REGIONS = 21          # the K-step timed region is repeated this many times; ms_per_step is the median
 ORACLE_MAX_TOKENS = 131072   # the oracle legs run whole sequences of the workload up to this many tokens
 
@@ -495,7 +497,7 @@ def run_ours(args):
     comp_bytes = token_heads * (k_b + v_b + 1.0)   # records + amortised INT8 mean byte
     roofline = None
     extra = {}
-    ncu = (NCU_PAIRS if pair else NCU_HEAD) if hs == 1 else NCU_WIDE
+    ncu = (NCU_PAIRS if pair else NCU_HEAD) if hs == 1 else (NCU_WIDE_PAIRS if pair else NCU_WIDE)
     if args.traffic_bytes is None:
         # every record is read once, so the captured config-2 figure scales with the records' bytes
         args.traffic_bytes = NCU_HEAD["dram_bytes"] * comp_bytes / (NCU_HEAD["token_heads"] * NCU_HEAD["bytes_per_token_head"])
