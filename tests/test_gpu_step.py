@@ -31,12 +31,12 @@ def _cfg(idx, **over):
     return cfg
 
 
-def _loop(cfg, steps, seed, check_every=1):
+def _loop(cfg, steps, seed, check_every=1, **table_kw):
     """Prefill `cfg.seq_lens` tokens, then `steps` decode steps through dq_decode_step on one cache and
     through dq_encode_tokens + dq_decode_attention on a second one; both must agree bit for bit at every
     step, and with the oracle's mirror of the loop."""
     w = workloads.generate(cfg, device="cuda", extra_tokens_per_seq=steps)
-    tk, tv, ok, ov = gc.tables(cfg)
+    tk, tv, ok, ov = gc.tables(cfg, **table_kw)   # table_kw: the opt-in codec variants
     ca, cb = gc.GpuCache(w, ok.rec, ov.rec), gc.GpuCache(w, ok.rec, ov.rec)
     B, Hq, Hkv = cfg.batch, cfg.hq, cfg.hkv
     if cfg.total_tokens:
@@ -108,6 +108,16 @@ def test_step_many_steps_budget_3bits():
     cfg = workloads.make_config(3, budget=3.0, scale=1 / 64)      # 64 query / 8 kv heads
     cfg.batch = 2; cfg.seq_lens = [1500, 380]
     _loop(cfg, steps=20, seed=4, check_every=7)
+
+
+@pytest.mark.parametrize("table_kw", [dict(pair=True), dict(pair=True, sigma=24, early_exit=True)])
+def test_step_with_paired_symbols(table_kw):
+    """The paired-symbol codec variant through the one-call step, the two-call sequence and the oracle's mirror:
+    window, block and page openings, an empty sequence; 3-bit budget with 8 / 5 levels."""
+    _loop(_cfg(2, batch=6, seq_lens=[511, 127, 255, 0, 1023, 300]), steps=4, seed=11, **table_kw)
+    cfg = workloads.make_config(3, budget=3.0, scale=1 / 64)
+    cfg.batch = 2; cfg.seq_lens = [1500, 380]
+    _loop(cfg, steps=6, seed=12, check_every=3, **table_kw)
 
 
 def test_step_when_the_ready_flag_is_never_seen():
