@@ -31,8 +31,8 @@ def _angle_tables(positions, base=500000.0):
 
 
 @pytest.mark.parametrize("style", [dq.ROPE_HALF, dq.ROPE_PAIRS])
-@pytest.mark.parametrize("wide_hs", [0, 8])
-def test_rope_encoder_bit_exact(style, wide_hs):
+@pytest.mark.parametrize("wide_hs,pair", [(0, False), (8, False), (0, True), (8, True)])
+def test_rope_encoder_bit_exact(style, wide_hs, pair):
     cfg = workloads.make_config(4, scale=1 / 16)
     cfg.batch = 4; cfg.seq_lens = [300, 16, 129, 1]
     w = workloads.generate(cfg, device="cuda")
@@ -40,10 +40,10 @@ def test_rope_encoder_bit_exact(style, wide_hs):
     rope_o = (cs, sn, style)
     rope_g = (torch.from_numpy(cs).cuda(), torch.from_numpy(sn).cuda(), style)
     if wide_hs:
-        tk, tv, ok, ov = gc.wide_tables(cfg, wide_hs)
+        tk, tv, ok, ov = gc.wide_tables(cfg, wide_hs, pair=pair)   # pair: the paired-symbol codec variant
         cache = gc.WideGpuCache(w, tk, tv, wide_hs)
     else:
-        tk, tv, ok, ov = gc.tables(cfg)
+        tk, tv, ok, ov = gc.tables(cfg, pair=pair)
         cache = gc.GpuCache(w, ok.rec, ov.rec)
     hs = max(1, wide_hs)
     dq.dq_encode_tokens(tk, tv, w.k, w.v, w.seq_id, w.pos, w.slot, cache.k_cont, cache.v_cont, cache.mean_q,
