@@ -44,18 +44,19 @@ def _draw(seed):
 
 
 @pytest.mark.parametrize("seed", range(16))
-def test_random_shape(seed):
+def test_random_shape(seed, pair=False):
     cfg, q_len, wide, resid = _draw(seed)
+    pair = pair and (wide or max(cfg.k_levels, cfg.v_levels) <= 9)   # the pair alphabet holds at most 9 levels
     w = workloads.generate(cfg, device="cuda")
     B, Hq, Hkv = cfg.batch, cfg.hq, cfg.hkv
     if wide:
         hs = Hkv
         n = 128 * hs
-        tk, tv, ok, ov = gc.wide_tables(cfg, hs, k_rec=335 * hs // 8, v_rec=235 * hs // 8)
+        tk, tv, ok, ov = gc.wide_tables(cfg, hs, k_rec=335 * hs // 8, v_rec=235 * hs // 8, pair=pair)
         cache = gc.WideGpuCache(w, tk, tv, hs)
     else:
         hs = 1
-        tk, tv, ok, ov = gc.tables(cfg)
+        tk, tv, ok, ov = gc.tables(cfg, pair=pair)
         cache = gc.GpuCache(w, ok.rec, ov.rec)
     gc.gpu_encode(w, tk, tv, cache)
     torch.cuda.synchronize()
@@ -128,5 +129,16 @@ def test_random_shape_through_the_batch_encoders(seed):
     dq.dq_set_option(dq.OPT_ENCODE_BATCH_MIN, 0)
     try:
         test_random_shape(seed)
+    finally:
+        dq.dq_set_option(dq.OPT_ENCODE_BATCH_MIN, -1)
+
+
+@pytest.mark.parametrize("seed", range(28, 44))
+def test_random_shape_with_paired_symbols(seed):
+    """The same sweep with the paired-symbol codec variant on both sides (the 4-bit budget's 16 key levels keep
+    single levels); odd seeds through the batch encoders."""
+    dq.dq_set_option(dq.OPT_ENCODE_BATCH_MIN, 0 if seed % 2 else -1)
+    try:
+        test_random_shape(seed, pair=True)
     finally:
         dq.dq_set_option(dq.OPT_ENCODE_BATCH_MIN, -1)
