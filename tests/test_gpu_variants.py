@@ -116,6 +116,25 @@ def test_pair_symbols_token_wide_both_encoders(early_exit):
         gc.check_attention(out, out32, ref)
 
 
+def test_pair_symbols_token_wide_config2_full_size():
+    """Token-wide streams with paired symbols on configuration 2 at full size (the batch encoder, 144 attention
+    items): every record and every attention row against the oracle."""
+    cfg = workloads.make_config(2)
+    w = workloads.generate(cfg, device="cuda")
+    tk, tv, ok, ov = gc.wide_tables(cfg, 8, pair=True)
+    cache = gc.WideGpuCache(w, tk, tv, 8)
+    gc.gpu_encode(w, tk, tv, cache)
+    torch.cuda.synchronize()
+    kc, vc, mq, ms, sk, sv = gc.oracle_encode_wide(w, ok, ov, 8)
+    assert np.array_equal(gc.from_interleaved(_np(cache.k_cont), ok.rec), kc)
+    assert np.array_equal(gc.from_interleaved(_np(cache.v_cont), ov.rec), vc)
+    assert int(_np(cache.status)[0]) == sk[0] + sv[0]
+    out, out32 = gc.gpu_attention(w, tk, tv, cache)
+    ref = oracle.attention(ok, ov, workloads.bf16_bits(w.q), kc, vc, mq, ms, _np(w.page_table), _np(w.seq_lens),
+                           cfg.hkv, gc.SM_SCALE)
+    assert gc.check_attention(out, out32, ref) < 1e-3
+
+
 def test_early_exit_prefill_config2_full_size():
     """Every record of configuration 2's prefill with the early exit, against the oracle; encoder time beside the default's."""
     cfg = workloads.make_config(2)
